@@ -1,0 +1,16 @@
+"""Seeded synthetic DETOX workloads (inputs only; none of the aggregation arithmetic lives here).
+
+The CUDA library and the CPU oracle are both fed from this module and from nothing else in common.
+"""
+from .gen import (  # noqa: F401
+    CONFIGS,
+    Workload,
+    WorkloadSpec,
+    expected_byzantine_votes,
+    make_groups,
+    make_sets,
+    make_workload,
+    padded_ld,
+    place_byzantine,
+    sweep_specs,
+)
