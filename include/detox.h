@@ -1,0 +1,163 @@
+/*
+ * libdetox — DETOX parameter-server gradient aggregation for NVIDIA B200 (sm_100a).
+ *
+ * C ABI.  Every entry point enqueues its kernels on the caller's CUDA stream and returns without
+ * synchronising the host.  The library allocates nothing and keeps no state between calls: every
+ * buffer, including scratch ("workspace"), belongs to the caller.
+ *
+ * Notation follows arXiv 1907.12205: n compute nodes (the paper's p) each send a gradient of
+ * dimension d; node groups have size r (odd, r divides n), so there are G = n / r votes; f is the
+ * Byzantine tolerance handed to Multi-Krum / Bulyan.
+ *
+ * Common conventions
+ *   - "dev" pointers are device pointers valid on the current device; "host" pointers are ordinary
+ *     host memory, read before the call returns.
+ *   - Matrices are row-major fp32 with a row stride `ld` in ELEMENTS (ld >= d).  The vectorised paths
+ *     need a 16-byte aligned base and ld % 4 == 0; any other layout takes a slower scalar path with the
+ *     same results.
+ *   - Index outputs are int32.  Limits: n, m <= DETOX_MAX_ROWS; r <= DETOX_MAX_R.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *   - Workspace pointers must be 256-byte aligned; sizes come from the *_workspace_bytes helpers.
+ *   - Errors: argument problems are reported before anything is launched; a failed launch returns
+ *     DETOX_ERR_CUDA.  Nothing aborts or throws.
+ *   - Ranking of values (medians, "closest to the median") uses the total order
+ *     -NaN < -Inf < ... < -0 < +0 < ... < +Inf < +NaN on fp32 bit patterns.
+ */
+#ifndef DETOX_H_
+#define DETOX_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define DETOX_MAX_ROWS 1024
+#define DETOX_MAX_R 15
+
+typedef enum {
+    DETOX_OK = 0,
+    DETOX_ERR_BAD_ARG = 1,      /* null pointer, size out of range, r even or not dividing n, bad partition */
+    DETOX_ERR_UNSUPPORTED = 2,  /* valid request outside the built limits */
+    DETOX_ERR_WORKSPACE = 3,    /* workspace missing, misaligned or too small */
+    DETOX_ERR_CUDA = 4,         /* a CUDA call or launch failed */
+    DETOX_ERR_TIMEOUT = 5       /* a bounded device-side wait ran out (reported through the status word) */
+} detox_status;
+
+typedef enum {
+    DETOX_AGG_NONE = 0,         /* A_0 only: pass the votes through */
+    DETOX_AGG_MEAN = 1,
+    DETOX_AGG_COORD_MEDIAN = 2,
+    DETOX_AGG_MULTIKRUM = 3,
+    DETOX_AGG_BULYAN = 4
+} detox_agg;
+
+const char* detox_status_string(detox_status s);
+
+/* ---------------------------------------------------------------------------------------------
+ * Filtering step (Section 3; Algorithm 1, "Filtering step"): for every node group A_j the majority
+ * vote z_j = maj{ g_i : i in A_j }, and z_j = 0 when no value is sent by more than r/2 members.
+ * Two members agree when their d-vectors are bitwise identical.
+ *
+ *   X        dev, n x ld      the n received gradients (read only)
+ *   members  host, G*r        worker ids; group j owns members[j*r .. j*r+r-1]; a partition of 0..n-1
+ *   Z        dev, G x ldz     out: the votes; may be NULL when only `winner` is wanted
+ *   winner   dev, G           out: lowest worker id of the winning class, or -1 (then Z[j] = 0)
+ *   ws       dev              detox_vote_workspace_bytes(n, r) bytes
+ * ------------------------------------------------------------------------------------------- */
+size_t detox_vote_workspace_bytes(int n, int r);
+detox_status detox_vote(const float* X, int64_t ld, int n, int r, int64_t d, const int32_t* members,
+                        float* Z, int64_t ldz, int32_t* winner, void* ws, size_t ws_bytes, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * A_0 = mean over each vote group (Algorithm 2, step 3, with A_0 the mean as analysed in Section 4):
+ * M[s] = (1/|Z_s|) sum_{j in Z_s} z_j.  A zero vote (no majority) counts as an ordinary member.
+ *
+ *   Z            dev, G x ldz   the votes
+ *   set_offsets  host, S+1      set s owns set_members[set_offsets[s] .. set_offsets[s+1]-1]; sets may be
+ *                               uneven (e.g. 7 and 8 out of 15, Appendix B.1) but not empty
+ *   set_members  host, G        vote indices, a partition of 0..G-1
+ *   M            dev, S x ldm   out
+ * ------------------------------------------------------------------------------------------- */
+detox_status detox_hier_mean(const float* Z, int64_t ldz, int G, int64_t d, const int32_t* set_offsets,
+                             const int32_t* set_members, int S, float* M, int64_t ldm, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * Coordinate-wise median (Section 4; Appendix B.1): out[c] = median_i X[i][c] over the m rows.
+ * Odd m: the middle value, bit for bit one of the inputs.  Even m: fp32 (lo + hi) * 0.5f.
+ *   out  dev, d.   ws: agg_coord_median_workspace_bytes(m, d) bytes (may be 0, then ws may be NULL).
+ * ------------------------------------------------------------------------------------------- */
+size_t agg_coord_median_workspace_bytes(int m, int64_t d);
+detox_status agg_coord_median(const float* X, int64_t ld, int m, int64_t d, float* out, void* ws,
+                              size_t ws_bytes, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * Multi-Krum (cited in Section 4 "Improved speed" as the O(p^2 d) aggregator; requirement
+ * m >= 2f+3 in Appendix B.1).  score_i = sum of the nb smallest squared distances from row i to the
+ * other rows, nb = m - f - 2 clamped to [1, m-1]; the m_sel rows of smallest score (equal scores:
+ * lower index first) are averaged.  m < 2f+3 is accepted (the clamp applies) down to m >= 1.
+ *
+ *   out     dev, d         the average of the selected rows
+ *   sel     dev, m_sel     out, ascending row indices; may be NULL
+ *   scores  dev, m (fp64)  out; may be NULL
+ *   ws      agg_multikrum_workspace_bytes(m, d) bytes
+ * ------------------------------------------------------------------------------------------- */
+size_t agg_multikrum_workspace_bytes(int m, int64_t d);
+detox_status agg_multikrum(const float* X, int64_t ld, int m, int64_t d, int f, int m_sel, float* out,
+                           int32_t* sel, double* scores, void* ws, size_t ws_bytes, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * Bulyan (cited in Section 4; requirement m >= 4f+3 in Appendix B.1, enforced here).  Stage 1:
+ * theta = m - 2f rounds of Krum on the shrinking candidate set (scores recomputed from the cached
+ * distances with nb = |remaining| - f - 2, clamped as above).  Stage 2, per coordinate: the median of
+ * the theta selected values, then the mean of the beta = theta - 2f values closest to it (closeness
+ * |v - median| in fp32; equally close: the smaller value first).
+ *
+ *   out  dev, d
+ *   sel  dev, theta   out, row indices in the order they were selected; may be NULL
+ *   ws   agg_bulyan_workspace_bytes(m, d) bytes
+ * ------------------------------------------------------------------------------------------- */
+size_t agg_bulyan_workspace_bytes(int m, int64_t d);
+detox_status agg_bulyan(const float* X, int64_t ld, int m, int64_t d, int f, float* out, int32_t* sel,
+                        void* ws, size_t ws_bytes, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * The whole parameter-server step (Algorithm 1, filtering + hierarchical aggregation; Algorithm 2):
+ * vote over the node groups, A_0 over each vote group, A_1 over the results.
+ *
+ *   a0 = DETOX_AGG_NONE : the G votes go to A_1 directly (sets are ignored)
+ *   a0 = DETOX_AGG_MEAN : the S set means go to A_1
+ *   a1 = MEAN | COORD_MEDIAN | MULTIKRUM (f, m_sel) | BULYAN (f)
+ *
+ *   out          dev, d
+ *   winner       dev, G        out, as in detox_vote; may be NULL
+ *   sel          dev           out, rows chosen by Multi-Krum (m_sel, ascending) or Bulyan (theta, in
+ *                              selection order) among the rows that entered A_1; may be NULL
+ *   sel_workers  dev           out, the same rows as worker ids (winner[sel[k]]), only meaningful
+ *                              when a0 = DETOX_AGG_NONE; may be NULL
+ *   ws           detox_aggregate_workspace_bytes(desc) bytes (holds the votes and set means too)
+ * ------------------------------------------------------------------------------------------- */
+typedef struct {
+    int32_t n;                   /* compute nodes */
+    int32_t r;                   /* redundancy ratio (odd, divides n) */
+    int64_t d;                   /* gradient dimension */
+    const int32_t* members;      /* host, G*r */
+    int32_t a0;                  /* detox_agg: NONE or MEAN */
+    int32_t n_sets;              /* S, used when a0 = MEAN */
+    const int32_t* set_offsets;  /* host, S+1 */
+    const int32_t* set_members;  /* host, G */
+    int32_t a1;                  /* detox_agg: MEAN, COORD_MEDIAN, MULTIKRUM or BULYAN */
+    int32_t f;                   /* tolerance given to Multi-Krum / Bulyan */
+    int32_t m_sel;               /* rows averaged by Multi-Krum */
+} detox_pipeline_desc;
+
+size_t detox_aggregate_workspace_bytes(const detox_pipeline_desc* desc);
+detox_status detox_aggregate(const detox_pipeline_desc* desc, const float* X, int64_t ld, float* out,
+                             int32_t* winner, int32_t* sel, int32_t* sel_workers, void* ws,
+                             size_t ws_bytes, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DETOX_H_ */

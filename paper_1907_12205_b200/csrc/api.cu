@@ -1,0 +1,306 @@
+// C ABI of libdetox: argument validation, workspace carving and kernel sequencing.
+// Nothing here touches gradient data on the host, allocates, or synchronises.
+#include <string.h>
+
+#include "common.cuh"
+
+using namespace detox;
+
+namespace {
+
+bool ws_ok(const void* ws, size_t have, size_t need) {
+    if (need == 0) return true;
+    return ws != nullptr && (reinterpret_cast<uintptr_t>(ws) & 255u) == 0 && have >= need;
+}
+
+// members must be a partition of 0..n-1 into n/r groups
+detox_status check_groups(int n, int r, const int32_t* members, IdTable* tab) {
+    if (n < 1 || n > kMaxRows || r < 1 || r > kMaxR || (r & 1) == 0 || n % r != 0 || !members)
+        return (n > kMaxRows || r > kMaxR) ? DETOX_ERR_UNSUPPORTED : DETOX_ERR_BAD_ARG;
+    bool seen[kMaxRows];
+    memset(seen, 0, sizeof(seen));
+    for (int k = 0; k < n; ++k) {
+        int32_t id = members[k];
+        if (id < 0 || id >= n || seen[id]) return DETOX_ERR_BAD_ARG;
+        seen[id] = true;
+        tab->id[k] = (uint16_t)id;
+    }
+    return DETOX_OK;
+}
+
+detox_status check_sets(int G, int S, const int32_t* offsets, const int32_t* set_members, SetTable* tab) {
+    if (G < 1 || G > kMaxRows || S < 1 || S > G || !offsets || !set_members) return DETOX_ERR_BAD_ARG;
+    if (offsets[0] != 0 || offsets[S] != G) return DETOX_ERR_BAD_ARG;
+    for (int s = 0; s < S; ++s)
+        if (offsets[s + 1] <= offsets[s]) return DETOX_ERR_BAD_ARG;  // empty or unordered set
+    bool seen[kMaxRows];
+    memset(seen, 0, sizeof(seen));
+    for (int k = 0; k < G; ++k) {
+        int32_t v = set_members[k];
+        if (v < 0 || v >= G || seen[v]) return DETOX_ERR_BAD_ARG;
+        seen[v] = true;
+        tab->member[k] = (uint16_t)v;
+    }
+    for (int s = 0; s <= S; ++s) tab->offset[s] = (uint16_t)offsets[s];
+    return DETOX_OK;
+}
+
+detox_status check_matrix(const float* X, int64_t ld, int m, int64_t d) {
+    if (!X || m < 1 || d < 1 || ld < d) return DETOX_ERR_BAD_ARG;
+    if ((reinterpret_cast<uintptr_t>(X) & 3u) != 0) return DETOX_ERR_BAD_ARG;
+    if (m > kMaxRows) return DETOX_ERR_UNSUPPORTED;
+    return DETOX_OK;
+}
+
+// workspace of the Krum-type aggregators: D | distance scratch | selection scratch | index list
+struct KrumWs {
+    double* D;
+    void* dist;
+    void* select;
+    int32_t* sel;
+    size_t total;
+};
+
+KrumWs krum_ws(void* ws, int m, int64_t d) {
+    KrumWs k;
+    char* p = static_cast<char*>(ws);
+    size_t off = 0;
+    k.D = reinterpret_cast<double*>(p + off);
+    off += align_up((size_t)m * m * sizeof(double));
+    k.dist = p + off;
+    off += dist_ws_bytes(m, d);
+    k.select = p + off;
+    off += select_ws_bytes(m);
+    k.sel = reinterpret_cast<int32_t*>(p + off);
+    off += align_up((size_t)m * sizeof(int32_t));
+    k.total = off;
+    return k;
+}
+
+detox_status run_multikrum(const float* X, int64_t ld, int m, int64_t d, int f, int m_sel, float* out, int32_t* sel,
+                           double* scores, void* ws, cudaStream_t s) {
+    KrumWs k = krum_ws(ws, m, d);
+    int32_t* sel_buf = sel ? sel : k.sel;
+    detox_status st = launch_sqdist(X, ld, m, d, k.D, k.dist, s);
+    if (st != DETOX_OK) return st;
+    st = launch_multikrum_select(k.D, m, f, m_sel, sel_buf, scores, k.select, s);
+    if (st != DETOX_OK) return st;
+    return launch_mean_rows(X, ld, d, sel_buf, m_sel, out, s);
+}
+
+detox_status run_bulyan(const float* X, int64_t ld, int m, int64_t d, int f, float* out, int32_t* sel, void* ws,
+                        cudaStream_t s) {
+    KrumWs k = krum_ws(ws, m, d);
+    int32_t* sel_buf = sel ? sel : k.sel;
+    const int theta = m - 2 * f, beta = theta - 2 * f;
+    detox_status st = launch_sqdist(X, ld, m, d, k.D, k.dist, s);
+    if (st != DETOX_OK) return st;
+    st = launch_bulyan_select(k.D, m, f, sel_buf, k.select, s);
+    if (st != DETOX_OK) return st;
+    return launch_coord_select(X, ld, theta, d, sel_buf, beta, out, s);
+}
+
+detox_status check_multikrum(int m, int f, int m_sel) {
+    if (f < 0 || m_sel < 1 || m_sel > m) return DETOX_ERR_BAD_ARG;
+    return DETOX_OK;
+}
+detox_status check_bulyan(int m, int f) {
+    if (f < 0) return DETOX_ERR_BAD_ARG;
+    if (f == 0) return DETOX_OK;  // theta = beta = m: the plain mean
+    return m >= 4 * f + 3 ? DETOX_OK : DETOX_ERR_BAD_ARG;
+}
+
+int64_t pad_ld(int64_t d) { return (d + 31) / 32 * 32; }
+
+struct PipeWs {
+    void* vote;
+    float* Z;
+    float* M;
+    int32_t* winner;
+    void* agg;
+    size_t total;
+    int64_t ldz;
+};
+
+PipeWs pipe_ws(void* ws, const detox_pipeline_desc* p) {
+    PipeWs w;
+    char* base = static_cast<char*>(ws);
+    const int G = p->n / p->r;
+    const int rows1 = p->a0 == DETOX_AGG_MEAN ? p->n_sets : G;
+    size_t off = 0;
+    w.ldz = pad_ld(p->d);
+    w.vote = base + off;
+    off += vote_ws_bytes(p->n, p->r);
+    w.winner = reinterpret_cast<int32_t*>(base + off);
+    off += align_up((size_t)G * sizeof(int32_t));
+    w.Z = reinterpret_cast<float*>(base + off);
+    off += align_up((size_t)G * w.ldz * sizeof(float));
+    w.M = reinterpret_cast<float*>(base + off);
+    if (p->a0 == DETOX_AGG_MEAN) off += align_up((size_t)p->n_sets * w.ldz * sizeof(float));
+    w.agg = base + off;
+    if (p->a1 == DETOX_AGG_MULTIKRUM || p->a1 == DETOX_AGG_BULYAN) off += krum_ws(nullptr, rows1, p->d).total;
+    w.total = off;
+    return w;
+}
+
+detox_status check_desc(const detox_pipeline_desc* p) {
+    if (!p || p->d < 1) return DETOX_ERR_BAD_ARG;
+    if (p->n < 1 || p->r < 1 || (p->r & 1) == 0 || p->n % p->r != 0) return DETOX_ERR_BAD_ARG;
+    if (p->n > kMaxRows || p->r > kMaxR) return DETOX_ERR_UNSUPPORTED;
+    if (p->a0 != DETOX_AGG_NONE && p->a0 != DETOX_AGG_MEAN) return DETOX_ERR_UNSUPPORTED;
+    const int G = p->n / p->r;
+    if (p->a0 == DETOX_AGG_MEAN && (p->n_sets < 1 || p->n_sets > G)) return DETOX_ERR_BAD_ARG;
+    const int rows1 = p->a0 == DETOX_AGG_MEAN ? p->n_sets : G;
+    switch (p->a1) {
+        case DETOX_AGG_MEAN:
+        case DETOX_AGG_COORD_MEDIAN: return DETOX_OK;
+        case DETOX_AGG_MULTIKRUM: return check_multikrum(rows1, p->f, p->m_sel);
+        case DETOX_AGG_BULYAN: return check_bulyan(rows1, p->f);
+        default: return DETOX_ERR_BAD_ARG;
+    }
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* detox_status_string(detox_status s) {
+    switch (s) {
+        case DETOX_OK: return "ok";
+        case DETOX_ERR_BAD_ARG: return "bad argument";
+        case DETOX_ERR_UNSUPPORTED: return "unsupported size or option";
+        case DETOX_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+        case DETOX_ERR_CUDA: return "CUDA error";
+        case DETOX_ERR_TIMEOUT: return "device-side wait timed out";
+        default: return "unknown status";
+    }
+}
+
+size_t detox_vote_workspace_bytes(int n, int r) {
+    if (n < 1 || r < 1 || n % r != 0) return 0;
+    return vote_ws_bytes(n, r);
+}
+
+detox_status detox_vote(const float* X, int64_t ld, int n, int r, int64_t d, const int32_t* members, float* Z,
+                        int64_t ldz, int32_t* winner, void* ws, size_t ws_bytes, void* stream) {
+    IdTable tab;
+    detox_status st = check_groups(n, r, members, &tab);
+    if (st != DETOX_OK) return st;
+    if ((st = check_matrix(X, ld, n, d)) != DETOX_OK) return st;
+    if (!winner) return DETOX_ERR_BAD_ARG;
+    if (Z && (ldz < d || (reinterpret_cast<uintptr_t>(Z) & 3u))) return DETOX_ERR_BAD_ARG;
+    if (!ws_ok(ws, ws_bytes, vote_ws_bytes(n, r))) return DETOX_ERR_WORKSPACE;
+    return launch_vote(X, ld, n, r, d, tab, Z, ldz, winner, ws, static_cast<cudaStream_t>(stream));
+}
+
+detox_status detox_hier_mean(const float* Z, int64_t ldz, int G, int64_t d, const int32_t* set_offsets,
+                             const int32_t* set_members, int S, float* M, int64_t ldm, void* stream) {
+    SetTable tab;
+    detox_status st = check_sets(G, S, set_offsets, set_members, &tab);
+    if (st != DETOX_OK) return st;
+    if ((st = check_matrix(Z, ldz, G, d)) != DETOX_OK) return st;
+    if (!M || ldm < d || (reinterpret_cast<uintptr_t>(M) & 3u)) return DETOX_ERR_BAD_ARG;
+    return launch_hier_mean(Z, ldz, d, tab, S, M, ldm, static_cast<cudaStream_t>(stream));
+}
+
+size_t agg_coord_median_workspace_bytes(int m, int64_t d) {
+    (void)m;
+    (void)d;
+    return 0;
+}
+
+detox_status agg_coord_median(const float* X, int64_t ld, int m, int64_t d, float* out, void* ws, size_t ws_bytes,
+                              void* stream) {
+    (void)ws;
+    (void)ws_bytes;
+    detox_status st = check_matrix(X, ld, m, d);
+    if (st != DETOX_OK) return st;
+    if (!out || (reinterpret_cast<uintptr_t>(out) & 3u)) return DETOX_ERR_BAD_ARG;
+    return launch_coord_select(X, ld, m, d, nullptr, 0, out, static_cast<cudaStream_t>(stream));
+}
+
+size_t agg_multikrum_workspace_bytes(int m, int64_t d) {
+    if (m < 1 || m > kMaxRows || d < 1) return 0;
+    return krum_ws(nullptr, m, d).total;
+}
+
+detox_status agg_multikrum(const float* X, int64_t ld, int m, int64_t d, int f, int m_sel, float* out, int32_t* sel,
+                           double* scores, void* ws, size_t ws_bytes, void* stream) {
+    detox_status st = check_matrix(X, ld, m, d);
+    if (st != DETOX_OK) return st;
+    if ((st = check_multikrum(m, f, m_sel)) != DETOX_OK) return st;
+    if (!out || (reinterpret_cast<uintptr_t>(out) & 3u)) return DETOX_ERR_BAD_ARG;
+    if (!ws_ok(ws, ws_bytes, krum_ws(nullptr, m, d).total)) return DETOX_ERR_WORKSPACE;
+    return run_multikrum(X, ld, m, d, f, m_sel, out, sel, scores, ws, static_cast<cudaStream_t>(stream));
+}
+
+size_t agg_bulyan_workspace_bytes(int m, int64_t d) {
+    if (m < 1 || m > kMaxRows || d < 1) return 0;
+    return krum_ws(nullptr, m, d).total;
+}
+
+detox_status agg_bulyan(const float* X, int64_t ld, int m, int64_t d, int f, float* out, int32_t* sel, void* ws,
+                        size_t ws_bytes, void* stream) {
+    detox_status st = check_matrix(X, ld, m, d);
+    if (st != DETOX_OK) return st;
+    if ((st = check_bulyan(m, f)) != DETOX_OK) return st;
+    if (!out || (reinterpret_cast<uintptr_t>(out) & 3u)) return DETOX_ERR_BAD_ARG;
+    if (!ws_ok(ws, ws_bytes, krum_ws(nullptr, m, d).total)) return DETOX_ERR_WORKSPACE;
+    return run_bulyan(X, ld, m, d, f, out, sel, ws, static_cast<cudaStream_t>(stream));
+}
+
+size_t detox_aggregate_workspace_bytes(const detox_pipeline_desc* desc) {
+    if (check_desc(desc) != DETOX_OK) return 0;
+    return pipe_ws(nullptr, desc).total;
+}
+
+detox_status detox_aggregate(const detox_pipeline_desc* p, const float* X, int64_t ld, float* out, int32_t* winner,
+                             int32_t* sel, int32_t* sel_workers, void* ws, size_t ws_bytes, void* stream) {
+    detox_status st = check_desc(p);
+    if (st != DETOX_OK) return st;
+    IdTable groups;
+    if ((st = check_groups(p->n, p->r, p->members, &groups)) != DETOX_OK) return st;
+    if ((st = check_matrix(X, ld, p->n, p->d)) != DETOX_OK) return st;
+    if (!out || (reinterpret_cast<uintptr_t>(out) & 3u)) return DETOX_ERR_BAD_ARG;
+    const int G = p->n / p->r;
+    SetTable sets;
+    if (p->a0 == DETOX_AGG_MEAN &&
+        (st = check_sets(G, p->n_sets, p->set_offsets, p->set_members, &sets)) != DETOX_OK)
+        return st;
+    PipeWs w = pipe_ws(ws, p);
+    if (!ws_ok(ws, ws_bytes, w.total)) return DETOX_ERR_WORKSPACE;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    int32_t* win = winner ? winner : w.winner;
+
+    // filtering step, then A_0, then A_1
+    if ((st = launch_vote(X, ld, p->n, p->r, p->d, groups, w.Z, w.ldz, win, w.vote, s)) != DETOX_OK) return st;
+    const float* rows = w.Z;
+    int m = G;
+    if (p->a0 == DETOX_AGG_MEAN) {
+        if ((st = launch_hier_mean(w.Z, w.ldz, p->d, sets, p->n_sets, w.M, w.ldz, s)) != DETOX_OK) return st;
+        rows = w.M;
+        m = p->n_sets;
+    }
+    int cnt = 0;
+    int32_t* sel_buf = nullptr;
+    switch (p->a1) {
+        case DETOX_AGG_MEAN: st = launch_mean_rows(rows, w.ldz, p->d, nullptr, m, out, s); break;
+        case DETOX_AGG_COORD_MEDIAN: st = launch_coord_select(rows, w.ldz, m, p->d, nullptr, 0, out, s); break;
+        case DETOX_AGG_MULTIKRUM:
+            cnt = p->m_sel;
+            sel_buf = sel ? sel : krum_ws(w.agg, m, p->d).sel;
+            st = run_multikrum(rows, w.ldz, m, p->d, p->f, p->m_sel, out, sel_buf, nullptr, w.agg, s);
+            break;
+        case DETOX_AGG_BULYAN:
+            cnt = m - 2 * p->f;
+            sel_buf = sel ? sel : krum_ws(w.agg, m, p->d).sel;
+            st = run_bulyan(rows, w.ldz, m, p->d, p->f, out, sel_buf, w.agg, s);
+            break;
+        default: st = DETOX_ERR_BAD_ARG;
+    }
+    if (st != DETOX_OK) return st;
+    if (sel_workers && sel_buf && p->a0 == DETOX_AGG_NONE) st = launch_map_indices(sel_buf, win, cnt, sel_workers, s);
+    return st;
+}
+
+}  // extern "C"

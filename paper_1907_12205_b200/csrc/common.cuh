@@ -1,0 +1,96 @@
+// Shared device helpers and the launcher declarations of libdetox (internal).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "detox.h"
+
+namespace detox {
+
+constexpr int kSMs = 148;            // B200: 2 dies x 74 SMs; grids are sized in multiples of this
+constexpr int kMaxRows = DETOX_MAX_ROWS;
+constexpr int kMaxR = DETOX_MAX_R;
+
+// Small host-side index tables travel as kernel parameters (no copy, no allocation).
+struct IdTable {
+    uint16_t id[kMaxRows];
+};
+struct SetTable {
+    uint16_t offset[kMaxRows + 1];
+    uint16_t member[kMaxRows];
+};
+
+// ---- order-preserving integer key for fp32 bit patterns -------------------------------------
+// Signed compare on the key gives -NaN < -Inf < ... < -0 < +0 < ... < +Inf < +NaN.
+// The map is its own inverse.
+__device__ __forceinline__ int32_t key_of_bits(uint32_t b) {
+    int32_t s = (int32_t)b;
+    return s ^ ((s >> 31) & 0x7fffffff);
+}
+__device__ __forceinline__ float float_of_key(int32_t k) {
+    return __int_as_float(k ^ ((k >> 31) & 0x7fffffff));
+}
+
+// ---- streaming loads / stores (data is touched once; keep it out of the way in L1) ----------
+__device__ __forceinline__ uint4 ld_stream_u4(const void* p) {
+    return __ldcs(reinterpret_cast<const uint4*>(p));
+}
+__device__ __forceinline__ float4 ld_stream_f4(const void* p) {
+    return __ldcs(reinterpret_cast<const float4*>(p));
+}
+__device__ __forceinline__ uint32_t ld_stream_u1(const void* p) {
+    return __ldcs(reinterpret_cast<const unsigned int*>(p));
+}
+__device__ __forceinline__ void st_stream_u4(void* p, uint4 v) {
+    __stcs(reinterpret_cast<uint4*>(p), v);
+}
+__device__ __forceinline__ void st_stream_f4(void* p, float4 v) {
+    __stcs(reinterpret_cast<float4*>(p), v);
+}
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
+inline size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
+
+inline detox_status launch_status() {
+    return cudaGetLastError() == cudaSuccess ? DETOX_OK : DETOX_ERR_CUDA;
+}
+
+// ---- launchers (each enqueues on `s`; none synchronises) ------------------------------------
+
+// vote.cu
+size_t vote_ws_bytes(int n, int r);
+detox_status launch_vote(const float* X, int64_t ld, int n, int r, int64_t d, const IdTable& members,
+                         float* Z, int64_t ldz, int32_t* winner, void* ws, cudaStream_t s);
+
+// mean.cu
+detox_status launch_hier_mean(const float* Z, int64_t ldz, int64_t d, const SetTable& sets, int S,
+                              float* M, int64_t ldm, cudaStream_t s);
+// mean of k rows of X listed in rows_dev (device int32; NULL = rows 0..k-1)
+detox_status launch_mean_rows(const float* X, int64_t ld, int64_t d, const int32_t* rows_dev, int k,
+                              float* out, cudaStream_t s);
+
+// median.cu: per-coordinate order statistics over m rows (rows_dev: device int32 list or NULL)
+//   beta == 0 : coordinate median;  beta >= 1 : mean of the beta values closest to the median
+detox_status launch_coord_select(const float* X, int64_t ld, int m, int64_t d, const int32_t* rows_dev,
+                                 int beta, float* out, cudaStream_t s);
+
+// dist.cu: squared distances D (m x m, fp64, symmetric, zero diagonal)
+size_t dist_ws_bytes(int m, int64_t d);
+detox_status launch_sqdist(const float* X, int64_t ld, int m, int64_t d, double* D, void* ws,
+                           cudaStream_t s);
+
+// select.cu
+size_t select_ws_bytes(int m);
+// Multi-Krum scoring + selection of the m_sel best rows (ascending indices in sel_dev)
+detox_status launch_multikrum_select(const double* D, int m, int f, int m_sel, int32_t* sel_dev,
+                                     double* scores_dev, void* ws, cudaStream_t s);
+// Bulyan stage 1: theta = m - 2f rounds; sel_dev in selection order
+detox_status launch_bulyan_select(const double* D, int m, int f, int32_t* sel_dev, void* ws,
+                                  cudaStream_t s);
+// out[k] = map[idx[k]] (k < cnt), all device int32
+detox_status launch_map_indices(const int32_t* idx, const int32_t* map, int cnt, int32_t* out,
+                                cudaStream_t s);
+
+}  // namespace detox

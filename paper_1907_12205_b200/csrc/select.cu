@@ -1,0 +1,193 @@
+// Krum scoring and index selection on the m x m distance matrix (Multi-Krum; Bulyan stage 1).
+// All of this is O(m^2 log m) work on at most a few MB: latency-bound, a handful of small kernels.
+//
+// Step 1 (rank_rows): every row's distances are ranked once (ties: lower column index first) and
+//   stored in ascending order together with their column indices.
+// Multi-Krum: score_i = sum of the first nb entries of row i's ascending list, added in that order;
+//   the m_sel smallest scores win (ties: lower index).
+// Bulyan: theta rounds in one CTA; each round sums, per remaining row, the first nb entries of its list
+//   that are still remaining, takes the argmin (ties: lower index) and removes it.
+#include <math_constants.h>
+
+#include "common.cuh"
+
+namespace detox {
+
+namespace {
+
+struct SelectWs {
+    double* sorted_d;    // m x m, row i ascending, self at the end (+inf)
+    int32_t* sorted_j;   // m x m, matching column indices
+    double* score;       // m
+};
+
+SelectWs carve(void* ws, int m) {
+    SelectWs w;
+    char* p = static_cast<char*>(ws);
+    w.sorted_d = reinterpret_cast<double*>(p);
+    p += align_up((size_t)m * m * sizeof(double));
+    w.sorted_j = reinterpret_cast<int32_t*>(p);
+    p += align_up((size_t)m * m * sizeof(int32_t));
+    w.score = reinterpret_cast<double*>(p);
+    return w;
+}
+
+__global__ void __launch_bounds__(256)
+rank_rows_kernel(const double* __restrict__ D, int m, double* __restrict__ sorted_d, int32_t* __restrict__ sorted_j) {
+    extern __shared__ double rowv[];  // m
+    const int i = blockIdx.x;
+    for (int j = threadIdx.x; j < m; j += blockDim.x) rowv[j] = (j == i) ? CUDART_INF : D[(int64_t)i * m + j];
+    __syncthreads();
+    for (int j = threadIdx.x; j < m; j += blockDim.x) {
+        int rank;
+        if (j == i) {
+            rank = m - 1;
+        } else {
+            const double v = rowv[j];
+            rank = 0;
+            for (int k = 0; k < m; ++k) {
+                if (k == i) continue;
+                const double u = rowv[k];
+                rank += (u < v || (u == v && k < j)) ? 1 : 0;
+            }
+        }
+        sorted_d[(int64_t)i * m + rank] = rowv[j];
+        sorted_j[(int64_t)i * m + rank] = j;
+    }
+}
+
+__device__ __forceinline__ int krum_neighbours(int alive, int f) {
+    int nb = alive - f - 2;
+    nb = nb < 1 ? 1 : nb;
+    nb = nb > alive - 1 ? alive - 1 : nb;
+    return nb;
+}
+
+// One CTA, one thread per row (m <= 1024).
+__global__ void __launch_bounds__(1024)
+multikrum_select_kernel(const double* __restrict__ sorted_d, int m, int f, int m_sel, int32_t* __restrict__ sel,
+                        double* __restrict__ scores_out) {
+    __shared__ double score[kMaxRows];
+    __shared__ int chosen[kMaxRows];
+    const int i = threadIdx.x;
+    const int nb = krum_neighbours(m, f);
+    if (i < m) {
+        double s = 0.0;
+        for (int k = 0; k < nb; ++k) s += sorted_d[(int64_t)i * m + k];
+        score[i] = s;
+        if (scores_out) scores_out[i] = s;
+    }
+    __syncthreads();
+    if (i < m) {
+        int rank = 0;
+        const double s = score[i];
+        for (int k = 0; k < m; ++k) rank += (score[k] < s || (score[k] == s && k < i)) ? 1 : 0;
+        chosen[i] = rank < m_sel ? 1 : 0;
+    }
+    __syncthreads();
+    if (i < m && chosen[i] && sel) {
+        int pos = 0;
+        for (int k = 0; k < i; ++k) pos += chosen[k];
+        sel[pos] = i;
+    }
+}
+
+__global__ void __launch_bounds__(1024)
+bulyan_select_kernel(const double* __restrict__ sorted_d, const int32_t* __restrict__ sorted_j, int m, int f,
+                     int32_t* __restrict__ sel) {
+    __shared__ unsigned char alive[kMaxRows];
+    __shared__ double best_s[32];
+    __shared__ int best_i[32];
+    __shared__ int picked;
+    const int i = threadIdx.x;
+    const int lane = i & 31, warp = i >> 5;
+    if (i < kMaxRows) alive[i] = i < m ? 1 : 0;
+    __syncthreads();
+    const int theta = m - 2 * f;
+    for (int round = 0; round < theta; ++round) {
+        const int remaining = m - round;
+        const int nb = krum_neighbours(remaining, f);
+        double s = CUDART_INF;
+        int idx = 0x7fffffff;
+        if (i < m && alive[i]) {
+            s = 0.0;
+            int taken = 0;
+            for (int k = 0; k < m - 1 && taken < nb; ++k) {
+                const int j = sorted_j[(int64_t)i * m + k];
+                if (alive[j]) {
+                    s += sorted_d[(int64_t)i * m + k];
+                    ++taken;
+                }
+            }
+            idx = i;
+        }
+        // argmin over (score, index)
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const double s2 = __shfl_down_sync(0xffffffffu, s, o);
+            const int i2 = __shfl_down_sync(0xffffffffu, idx, o);
+            if (s2 < s || (s2 == s && i2 < idx)) { s = s2; idx = i2; }
+        }
+        if (lane == 0) { best_s[warp] = s; best_i[warp] = idx; }
+        __syncthreads();
+        if (warp == 0) {
+            s = lane < (int)(blockDim.x >> 5) ? best_s[lane] : CUDART_INF;
+            idx = lane < (int)(blockDim.x >> 5) ? best_i[lane] : 0x7fffffff;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                const double s2 = __shfl_down_sync(0xffffffffu, s, o);
+                const int i2 = __shfl_down_sync(0xffffffffu, idx, o);
+                if (s2 < s || (s2 == s && i2 < idx)) { s = s2; idx = i2; }
+            }
+            if (lane == 0) {
+                picked = idx;
+                sel[round] = idx;
+                alive[idx] = 0;
+            }
+        }
+        __syncthreads();
+    }
+    (void)picked;
+}
+
+__global__ void map_indices_kernel(const int32_t* __restrict__ idx, const int32_t* __restrict__ map, int cnt,
+                                   int32_t* __restrict__ out) {
+    int k = blockIdx.x * blockDim.x + threadIdx.x;
+    if (k < cnt) out[k] = map[idx[k]];
+}
+
+int round_up_warp(int m) { return (m + 31) / 32 * 32; }
+
+}  // namespace
+
+size_t select_ws_bytes(int m) {
+    return align_up((size_t)m * m * sizeof(double)) + align_up((size_t)m * m * sizeof(int32_t)) +
+           align_up((size_t)m * sizeof(double));
+}
+
+detox_status launch_multikrum_select(const double* D, int m, int f, int m_sel, int32_t* sel_dev, double* scores_dev,
+                                     void* ws, cudaStream_t s) {
+    SelectWs w = carve(ws, m);
+    rank_rows_kernel<<<m, 256, (size_t)m * sizeof(double), s>>>(D, m, w.sorted_d, w.sorted_j);
+    detox_status st = launch_status();
+    if (st != DETOX_OK) return st;
+    multikrum_select_kernel<<<1, round_up_warp(m), 0, s>>>(w.sorted_d, m, f, m_sel, sel_dev, scores_dev);
+    return launch_status();
+}
+
+detox_status launch_bulyan_select(const double* D, int m, int f, int32_t* sel_dev, void* ws, cudaStream_t s) {
+    SelectWs w = carve(ws, m);
+    rank_rows_kernel<<<m, 256, (size_t)m * sizeof(double), s>>>(D, m, w.sorted_d, w.sorted_j);
+    detox_status st = launch_status();
+    if (st != DETOX_OK) return st;
+    bulyan_select_kernel<<<1, round_up_warp(m), 0, s>>>(w.sorted_d, w.sorted_j, m, f, sel_dev);
+    return launch_status();
+}
+
+detox_status launch_map_indices(const int32_t* idx, const int32_t* map, int cnt, int32_t* out, cudaStream_t s) {
+    if (cnt <= 0) return DETOX_OK;
+    map_indices_kernel<<<(cnt + 127) / 128, 128, 0, s>>>(idx, map, cnt, out);
+    return launch_status();
+}
+
+}  // namespace detox

@@ -1,0 +1,249 @@
+// Filtering step of DETOX (Section 3; Algorithm 1, "Filtering step"): majority vote inside each node
+// group, on bitwise equality of whole d-vectors.
+//
+// One streaming pass.  A strict majority of the whole vectors, when it exists, is also a strict
+// majority on every 16-byte piece, and it is then the only one there.  So each thread compares the
+// r members on its own piece, writes that piece's local majority value (or zeros) to Z at once, and
+// ORs "member a differs from member b" bits into a per-group word.  After the pass the bits tell
+// whether a global majority exists; only groups without one have their Z row cleared again.
+// Traffic: n*d*4 bytes read, G*d*4 bytes written, once.
+#include "common.cuh"
+
+namespace detox {
+
+namespace {
+
+constexpr int kVoteThreads = 256;
+constexpr int kPairWords = 4;  // r <= 15 -> at most 105 member pairs -> 4 words per group
+
+template <int R>
+struct VoteShape {
+    static constexpr int kPairs = R * (R - 1) / 2;
+    static constexpr int kWords = kPairs == 0 ? 1 : (kPairs + 31) / 32;
+    // pieces per thread and item: enough independent 16-byte loads in flight per thread
+    static constexpr int kUnroll = R <= 3 ? 4 : (R <= 7 ? 2 : 1);
+};
+
+__host__ __device__ constexpr int pair_index(int r, int a, int b) {  // a < b
+    return a * (2 * r - a - 1) / 2 + (b - a - 1);
+}
+
+template <int VEC>
+struct Piece;
+template <>
+struct Piece<4> {
+    uint4 v;
+    __device__ __forceinline__ bool differs(const Piece& o) const {
+        return ((v.x ^ o.v.x) | (v.y ^ o.v.y) | (v.z ^ o.v.z) | (v.w ^ o.v.w)) != 0u;
+    }
+    __device__ __forceinline__ void clear() { v = make_uint4(0u, 0u, 0u, 0u); }
+    __device__ __forceinline__ void load(const float* p, int valid) {
+        if (valid >= 4) {
+            v = ld_stream_u4(p);
+        } else {
+            v.x = valid > 0 ? ld_stream_u1(p) : 0u;
+            v.y = valid > 1 ? ld_stream_u1(p + 1) : 0u;
+            v.z = valid > 2 ? ld_stream_u1(p + 2) : 0u;
+            v.w = 0u;
+        }
+    }
+    __device__ __forceinline__ void store(float* p, int valid) const {
+        if (valid >= 4) {
+            st_stream_u4(p, v);
+        } else {
+            uint32_t* q = reinterpret_cast<uint32_t*>(p);
+            if (valid > 0) q[0] = v.x;
+            if (valid > 1) q[1] = v.y;
+            if (valid > 2) q[2] = v.z;
+        }
+    }
+};
+template <>
+struct Piece<1> {
+    uint32_t v;
+    __device__ __forceinline__ bool differs(const Piece& o) const { return v != o.v; }
+    __device__ __forceinline__ void clear() { v = 0u; }
+    __device__ __forceinline__ void load(const float* p, int valid) { v = valid > 0 ? ld_stream_u1(p) : 0u; }
+    __device__ __forceinline__ void store(float* p, int valid) const {
+        if (valid > 0) *reinterpret_cast<uint32_t*>(p) = v;
+    }
+};
+
+template <int R, int VEC, bool WRITE_Z>
+__global__ void __launch_bounds__(kVoteThreads)
+vote_kernel(const float* __restrict__ X, int64_t ld, int64_t d, int64_t tiles_per_group,
+            const __grid_constant__ IdTable members, float* __restrict__ Z, int64_t ldz,
+            uint32_t* __restrict__ pairdiff) {
+    using Shape = VoteShape<R>;
+    constexpr int U = Shape::kUnroll;
+    constexpr int64_t kTile = (int64_t)kVoteThreads * VEC * U;
+
+    const int64_t item = blockIdx.x;
+    const int g = (int)(item / tiles_per_group);
+    const int64_t tile = item - (int64_t)g * tiles_per_group;
+
+    const float* row[R];
+#pragma unroll
+    for (int a = 0; a < R; ++a) row[a] = X + (int64_t)members.id[g * R + a] * ld;
+
+    Piece<VEC> v[U][R];
+    int valid[U];
+    int64_t col[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        col[u] = tile * kTile + ((int64_t)u * kVoteThreads + threadIdx.x) * VEC;
+        int64_t left = d - col[u];
+        valid[u] = left >= VEC ? VEC : (left > 0 ? (int)left : 0);
+    }
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+#pragma unroll
+        for (int a = 0; a < R; ++a) {
+            if (valid[u] > 0) v[u][a].load(row[a] + col[u], valid[u]);
+            else v[u][a].clear();
+        }
+    }
+
+    uint32_t diff[Shape::kWords];
+#pragma unroll
+    for (int w = 0; w < Shape::kWords; ++w) diff[w] = 0u;
+
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        uint32_t loc[Shape::kWords];
+#pragma unroll
+        for (int w = 0; w < Shape::kWords; ++w) loc[w] = 0u;
+#pragma unroll
+        for (int a = 0; a < R; ++a) {
+#pragma unroll
+            for (int b = a + 1; b < R; ++b) {
+                const int p = pair_index(R, a, b);
+                if (v[u][a].differs(v[u][b])) loc[p >> 5] |= 1u << (p & 31);
+            }
+        }
+#pragma unroll
+        for (int w = 0; w < Shape::kWords; ++w) diff[w] |= loc[w];
+
+        if (WRITE_Z) {
+            // local majority: the first member that agrees with more than r/2 members (itself included)
+            Piece<VEC> pick;
+            pick.clear();
+#pragma unroll
+            for (int a = R - 1; a >= 0; --a) {
+                int agree = 1;
+#pragma unroll
+                for (int b = 0; b < R; ++b) {
+                    if (b == a) continue;
+                    const int p = a < b ? pair_index(R, a, b) : pair_index(R, b, a);
+                    agree += ((loc[p >> 5] >> (p & 31)) & 1u) ? 0 : 1;
+                }
+                if (2 * agree > R) pick = v[u][a];
+            }
+            if (valid[u] > 0) pick.store(Z + (int64_t)g * ldz + col[u], valid[u]);
+        }
+    }
+
+    // one OR per warp and word, and only when it would set a new bit
+#pragma unroll
+    for (int w = 0; w < Shape::kWords; ++w) {
+        uint32_t bits = __reduce_or_sync(0xffffffffu, diff[w]);
+        if ((threadIdx.x & 31) == 0 && bits != 0u) {
+            uint32_t* word = pairdiff + (int64_t)g * kPairWords + w;
+            uint32_t seen = *reinterpret_cast<volatile uint32_t*>(word);
+            if (bits & ~seen) atomicOr(word, bits);
+        }
+    }
+}
+
+// One thread per group: read the "differs" bits, find the class with more than r/2 members.
+__global__ void vote_finalize_kernel(int G, int r, const __grid_constant__ IdTable members,
+                                     const uint32_t* __restrict__ pairdiff, int32_t* __restrict__ winner) {
+    int g = blockIdx.x * blockDim.x + threadIdx.x;
+    if (g >= G) return;
+    const uint32_t* bits = pairdiff + (int64_t)g * kPairWords;
+    int win = -1;
+    for (int a = 0; a < r && win < 0; ++a) {
+        int agree = 1;
+        int lowest = members.id[g * r + a];
+        for (int b = 0; b < r; ++b) {
+            if (b == a) continue;
+            int p = a < b ? pair_index(r, a, b) : pair_index(r, b, a);
+            if (((bits[p >> 5] >> (p & 31)) & 1u) == 0u) {
+                ++agree;
+                int idb = members.id[g * r + b];
+                lowest = idb < lowest ? idb : lowest;
+            }
+        }
+        if (2 * agree > r) win = lowest;
+    }
+    winner[g] = win;
+}
+
+// Clears the vote of every group that turned out to have no majority (rare).
+__global__ void vote_clear_kernel(const int32_t* __restrict__ winner, float* __restrict__ Z, int64_t ldz,
+                                  int64_t d) {
+    int g = blockIdx.y;
+    if (winner[g] >= 0) return;
+    float* z = Z + (int64_t)g * ldz;
+    for (int64_t c = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; c < d; c += (int64_t)gridDim.x * blockDim.x)
+        z[c] = 0.0f;
+}
+
+template <int R, int VEC>
+detox_status launch_vote_r(const float* X, int64_t ld, int G, int64_t d, const IdTable& members, float* Z,
+                           int64_t ldz, uint32_t* pairdiff, cudaStream_t s) {
+    constexpr int64_t kTile = (int64_t)kVoteThreads * VEC * VoteShape<R>::kUnroll;
+    int64_t tiles = ceil_div(d, kTile);
+    int64_t items = tiles * G;
+    if (items > 0x7fffffffLL) return DETOX_ERR_UNSUPPORTED;
+    if (Z)
+        vote_kernel<R, VEC, true><<<(unsigned)items, kVoteThreads, 0, s>>>(X, ld, d, tiles, members, Z, ldz, pairdiff);
+    else
+        vote_kernel<R, VEC, false><<<(unsigned)items, kVoteThreads, 0, s>>>(X, ld, d, tiles, members, Z, ldz, pairdiff);
+    return launch_status();
+}
+
+template <int VEC>
+detox_status launch_vote_vec(const float* X, int64_t ld, int G, int r, int64_t d, const IdTable& members,
+                             float* Z, int64_t ldz, uint32_t* pairdiff, cudaStream_t s) {
+    switch (r) {
+        case 1: return launch_vote_r<1, VEC>(X, ld, G, d, members, Z, ldz, pairdiff, s);
+        case 3: return launch_vote_r<3, VEC>(X, ld, G, d, members, Z, ldz, pairdiff, s);
+        case 5: return launch_vote_r<5, VEC>(X, ld, G, d, members, Z, ldz, pairdiff, s);
+        case 7: return launch_vote_r<7, VEC>(X, ld, G, d, members, Z, ldz, pairdiff, s);
+        case 9: return launch_vote_r<9, VEC>(X, ld, G, d, members, Z, ldz, pairdiff, s);
+        case 11: return launch_vote_r<11, VEC>(X, ld, G, d, members, Z, ldz, pairdiff, s);
+        case 13: return launch_vote_r<13, VEC>(X, ld, G, d, members, Z, ldz, pairdiff, s);
+        case 15: return launch_vote_r<15, VEC>(X, ld, G, d, members, Z, ldz, pairdiff, s);
+        default: return DETOX_ERR_UNSUPPORTED;
+    }
+}
+
+}  // namespace
+
+size_t vote_ws_bytes(int n, int r) {
+    int G = r > 0 ? n / r : 0;
+    return align_up((size_t)G * kPairWords * sizeof(uint32_t));
+}
+
+detox_status launch_vote(const float* X, int64_t ld, int n, int r, int64_t d, const IdTable& members,
+                         float* Z, int64_t ldz, int32_t* winner, void* ws, cudaStream_t s) {
+    const int G = n / r;
+    uint32_t* pairdiff = static_cast<uint32_t*>(ws);
+    if (cudaMemsetAsync(pairdiff, 0, (size_t)G * kPairWords * sizeof(uint32_t), s) != cudaSuccess)
+        return DETOX_ERR_CUDA;
+    const bool vec = aligned16(X) && ld % 4 == 0 && (!Z || (aligned16(Z) && ldz % 4 == 0));
+    detox_status st = vec ? launch_vote_vec<4>(X, ld, G, r, d, members, Z, ldz, pairdiff, s)
+                          : launch_vote_vec<1>(X, ld, G, r, d, members, Z, ldz, pairdiff, s);
+    if (st != DETOX_OK) return st;
+    vote_finalize_kernel<<<(G + 127) / 128, 128, 0, s>>>(G, r, members, pairdiff, winner);
+    if ((st = launch_status()) != DETOX_OK) return st;
+    if (Z) {
+        unsigned bx = (unsigned)(ceil_div(d, 256 * 8) < 64 ? ceil_div(d, 256 * 8) : 64);
+        vote_clear_kernel<<<dim3(bx, (unsigned)G), 256, 0, s>>>(winner, Z, ldz, d);
+        st = launch_status();
+    }
+    return st;
+}
+
+}  // namespace detox

@@ -1,0 +1,42 @@
+"""Shared test helpers (host side only): error norms and the near-tie screen for Krum-type decisions."""
+import numpy as np
+
+import oracle
+
+
+def rel_l2(y, ref) -> float:
+    y = np.asarray(y, dtype=np.float64)
+    ref = np.asarray(ref, dtype=np.float64)
+    den = np.linalg.norm(ref)
+    num = np.linalg.norm(y - ref)
+    return float(num) if den == 0.0 else float(num / den)
+
+
+def _gap_after(sorted_scores: np.ndarray, k: int) -> float:
+    """Relative gap between the k-th and (k+1)-th smallest *distinct-valued* neighbours at the cut."""
+    a, b = sorted_scores[k - 1], sorted_scores[k]
+    if a == b:
+        return np.inf  # an exact tie is decided by index on both sides
+    return abs(b - a) / max(abs(a), abs(b), 1e-300)
+
+
+def multikrum_min_gap(scores: np.ndarray, m_sel: int) -> float:
+    s = np.sort(scores)
+    return np.inf if m_sel >= len(s) else _gap_after(s, m_sel)
+
+
+def bulyan_min_gap(D: np.ndarray, f: int) -> float:
+    """Smallest relative gap between the best and the next distinct score over all selection rounds."""
+    m = D.shape[0]
+    alive = np.ones(m, np.uint8)
+    worst = np.inf
+    for _ in range(m - 2 * f):
+        sc = oracle.krum_scores(D, f, alive)
+        live = np.sort(sc[alive.astype(bool)])
+        best = live[0]
+        others = live[live != best]
+        if len(others):
+            worst = min(worst, abs(others[0] - best) / max(abs(others[0]), abs(best), 1e-300))
+        pick = min((i for i in range(m) if alive[i]), key=lambda i: (sc[i], i))
+        alive[pick] = 0
+    return worst
