@@ -1,0 +1,329 @@
+#!/usr/bin/env python
+"""Benchmark of the DETOX aggregation step (vote -> hierarchical mean -> robust aggregator) on B200.
+
+Default workload: n = 45 workers, r = 3, d = 11,173,962 (ResNet-18-sized), q = 5 ALIE attackers placed
+worst-case; one step = detox_aggregate(vote -> mean over 3 sets of 5 -> Multi-Krum(f=1, m_sel=1)).
+The metric is aggregation input throughput n*d*4 bytes per second.  Prints ONE JSON line.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload cfg2|cfg1|cfg3|cfg4]
+
+With N > 1 (launched by torch.distributed.run) every rank aggregates its own independent copy of the
+workload (replicas; the path has no exchange step) and rank 0 reports the sum over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "aggregation_input_throughput"
+UNIT = "GB/s"
+CLOCK_QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+               "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+               "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+
+def pipeline_for(name, w, dx):
+    """The DETOX leg and the direct (non-DETOX) leg of each named configuration."""
+    s = w.spec
+    G = s.n // s.r
+    if name == "cfg1":
+        return (dict(a0=dx.AGG_NONE, a1=dx.AGG_COORD_MEDIAN, f=0, m_sel=1), ("coord_median", {}))
+    if name == "cfg2":
+        return (dict(a0=dx.AGG_MEAN, a1=dx.AGG_MULTIKRUM, f=1, m_sel=1), ("multikrum", dict(f=5, m_sel=s.n - 5)))
+    if name == "cfg3":
+        return (dict(a0=dx.AGG_NONE, a1=dx.AGG_BULYAN, f=3, m_sel=1), ("bulyan", dict(f=9)))
+    if name == "cfg4":
+        return (dict(a0=dx.AGG_MEAN, a1=dx.AGG_COORD_MEDIAN, f=0, m_sel=1), ("coord_median", {}))
+    raise ValueError(name)
+
+
+ORACLE_A1 = {1: "mean", 2: "coord_median", 3: "multikrum", 4: "bulyan"}
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+
+    def __init__(self, index: int):
+        self.rows, self.proc, self.index = [], None, index
+
+    def __enter__(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={CLOCK_QUERY}",
+                                          "--format=csv,noheader,nounits", "-lms", "50"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+        return self
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def __exit__(self, *exc):
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except subprocess.TimeoutExpired:
+                self.proc.kill()
+            self.thread.join(timeout=2)
+
+    def summary(self):
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            if len(r) < 9:
+                continue
+            try:
+                sm.append(float(r[1])); mx.append(float(r[2]))
+            except ValueError:
+                continue
+            for nm, v in zip(names, r[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(nm)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(mx)), "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as fh:
+            return json.load(fh), "measured"
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0}, "fallback"
+
+
+def time_calls(torch, fn, steps, warmup):
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    st = torch.cuda.current_stream()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(st)
+    for _ in range(steps):
+        fn()
+    e1.record(st)
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / steps
+
+
+def oracle_step(w, cfg, X_host):
+    import oracle
+    s = w.spec
+    return oracle.detox_aggregate(X_host, w.members, s.r, "mean" if cfg["a0"] == 1 else "none", w.set_offsets,
+                                  w.set_members, ORACLE_A1[cfg["a1"]], cfg["f"], cfg["m_sel"])
+
+
+def run_reference(args, rank, world):
+    """The reference arm: the CPU oracle, as it stands, on the host cores (rank 0 only)."""
+    if rank != 0:
+        return
+    import oracle
+    import paper_1907_12205_b200 as dx  # constants only; nothing is launched
+    import workloads as wl
+    spec = wl.CONFIGS[args.workload]
+    w = wl.make_workload(spec)
+    cfg, _ = pipeline_for(args.workload, w, dx)
+    X = w.data().numpy()
+    for _ in range(min(args.warmup, 1)):
+        oracle_step(w, cfg, X)
+    steps = max(1, min(args.steps, 5))
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        oracle_step(w, cfg, X)
+    ms = (time.perf_counter() - t0) * 1e3 / steps
+    val = spec.n * spec.d * 4 / (ms * 1e-3) / 1e9
+    line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
+            "warmup": min(args.warmup, 1), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": workload_label(args.workload, spec, cfg)},
+            "cpu_baseline": {"value": val, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+                             "sample": "full workload, every step"},
+            "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def workload_label(name, spec, cfg):
+    a0 = {0: "none", 1: "mean"}[cfg["a0"]]
+    return (f"{name}: n={spec.n} r={spec.r} d={spec.d} q={spec.q} {spec.attack}/{spec.placement}; "
+            f"vote -> A0={a0} -> A1={ORACLE_A1[cfg['a1']]}(f={cfg['f']}, m_sel={cfg['m_sel']})")
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="detox", choices=["detox", "reference"])
+    ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "detox" else args.warmup
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        run_reference(args, rank, world)
+        return
+
+    import torch
+    import torch.distributed as dist
+
+    import paper_1907_12205_b200 as dx
+    import workloads as wl
+
+    torch.cuda.set_device(local)
+    dev = f"cuda:{local}"
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+    dx.load()
+
+    spec = wl.CONFIGS[args.workload]
+    if world > 1:  # every replica draws its own inputs
+        import dataclasses
+        spec = dataclasses.replace(spec, seed=spec.seed + rank)
+    w = wl.make_workload(spec, device=dev)
+    cfg, (direct_name, direct_args) = pipeline_for(args.workload, w, dx)
+    X = w.X[:, : spec.d]
+    pipe = dx.Pipeline(spec.n, spec.r, spec.d, w.members, cfg["a0"], w.set_offsets, w.set_members, cfg["a1"],
+                       cfg["f"], cfg["m_sel"])
+    ws = torch.empty(pipe.workspace_bytes(), dtype=torch.uint8, device=dev)
+    out = torch.empty(spec.d, dtype=torch.float32, device=dev)
+    winner = torch.empty(pipe.G, dtype=torch.int32, device=dev)
+    sel = torch.empty(max(pipe.n_selected, 1), dtype=torch.int32, device=dev)
+
+    def step():
+        dx.detox_aggregate(pipe, X, out=out, winner=winner, sel=sel, ws=ws)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- device-resident timing: K steps, barrier + synchronize on both sides, max over ranks ----
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    st = torch.cuda.current_stream()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(local) as clocks:
+        e0.record(st)
+        for _ in range(args.steps):
+            step()
+        e1.record(st)
+        barrier()
+        # the dominant kernel alone (vote: reads n*d*4, writes G*d*4), same inputs, same stream
+        Zbuf = torch.empty((pipe.G, w.ld), dtype=torch.float32, device=dev)[:, : spec.d]
+        vws = torch.empty(dx.detox_vote_workspace_bytes(spec.n, spec.r), dtype=torch.uint8, device=dev)
+        vote_ms = time_calls(torch, lambda: dx.detox_vote(X, spec.r, w.members, Z=Zbuf, winner=winner, ws=vws),
+                             max(args.steps, 10), 3)
+    total_ms = e0.elapsed_time(e1)
+    t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_per_step = float(t.item()) / args.steps
+    in_bytes = spec.n * spec.d * 4
+    value = world * in_bytes / (ms_per_step * 1e-3) / 1e9
+
+    # ---- end to end: pinned host input -> device, aggregate, result -> pinned host ----
+    Xh = torch.empty((spec.n, w.ld), dtype=torch.float32, pin_memory=True)
+    Xh.copy_(w.X)
+    Xd = torch.empty_like(w.X)
+    outh = torch.empty(spec.d, dtype=torch.float32, pin_memory=True)
+
+    def e2e_step():
+        Xd.copy_(Xh, non_blocking=True)
+        dx.detox_aggregate(pipe, Xd[:, : spec.d], out=out, winner=winner, sel=sel, ws=ws)
+        outh.copy_(out, non_blocking=True)
+
+    e2e_steps = max(2, min(args.steps, 5))
+    barrier()
+    e2e_ms = time_calls(torch, e2e_step, e2e_steps, 1)
+    t = torch.tensor([e2e_ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    e2e_ms = float(t.item())
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---- other legs on the same inputs (rank 0, N = 1 reporting only) ----
+    legs = {"detox_pipeline": {"ms": ms_per_step, "GBps": in_bytes / ms_per_step / 1e6}}
+    if direct_name == "multikrum":
+        dws = torch.empty(dx.agg_multikrum_workspace_bytes(spec.n, spec.d), dtype=torch.uint8, device=dev)
+        dsel = torch.empty(direct_args["m_sel"], dtype=torch.int32, device=dev)
+        dsc = torch.empty(spec.n, dtype=torch.float64, device=dev)
+        fn = lambda: dx.agg_multikrum(X, direct_args["f"], direct_args["m_sel"], out=out, sel=dsel, scores=dsc, ws=dws)
+    elif direct_name == "bulyan":
+        dws = torch.empty(dx.agg_bulyan_workspace_bytes(spec.n, spec.d), dtype=torch.uint8, device=dev)
+        dsel = torch.empty(spec.n - 2 * direct_args["f"], dtype=torch.int32, device=dev)
+        fn = lambda: dx.agg_bulyan(X, direct_args["f"], out=out, sel=dsel, ws=dws)
+    else:
+        fn = lambda: dx.agg_coord_median(X, out=out)
+    dms = time_calls(torch, fn, max(3, min(args.steps, 10)), 3)
+    legs[f"direct_{direct_name}"] = {"ms": dms, "GBps": in_bytes / dms / 1e6, "args": direct_args}
+    legs["detox_speedup_vs_direct"] = dms / ms_per_step
+
+    peaks, peak_kind = measured_peaks()
+    vote_bytes = (spec.n + pipe.G) * spec.d * 4
+    achieved = vote_bytes / (vote_ms * 1e-3) / 1e9
+    roofline = {"kernel": "vote_kernel", "bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"],
+                "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
+                "frac_of_8TBps": achieved / 8000.0, "ms_per_launch": vote_ms, "algorithmic_bytes": vote_bytes,
+                "traffic": None}
+
+    cpu_baseline = None
+    parity = None
+    if not args.no_cpu_baseline:
+        import oracle
+        Xn = w.X.cpu().numpy()[:, : spec.d]
+        t0 = time.perf_counter()
+        ref = oracle_step(w, cfg, Xn)
+        cpu_s = time.perf_counter() - t0
+        cpu_baseline = {"value": in_bytes / cpu_s / 1e9, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+                        "sample": "full workload, 1 repetition", "ms": cpu_s * 1e3}
+        step()
+        torch.cuda.synchronize()
+        o = out.cpu().numpy().astype(np.float64)
+        den = np.linalg.norm(ref["out"].astype(np.float64))
+        parity = {"winner_exact": winner.cpu().numpy().tolist() == ref["winner"].tolist(),
+                  "out_rel_l2": float(np.linalg.norm(o - ref["out"]) / (den if den else 1.0))}
+        if ref["sel"] is not None:
+            parity["sel_exact"] = sel.cpu().numpy()[: len(ref["sel"])].tolist() == ref["sel"].tolist()
+
+    kernels_per_step = {"cfg1": 4, "cfg2": 9, "cfg3": 8, "cfg4": 5}[args.workload]
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": workload_label(args.workload, spec, cfg), "l2": "inputs larger than L2"
+                       if in_bytes > 2 * 126e6 else "inputs fit in L2 (warm)", "replicas": world},
+            "clocks": clocks.summary(),
+            "e2e": {"value": world * in_bytes / (e2e_ms * 1e-3) / 1e9, "unit": UNIT, "ms_per_step": e2e_ms,
+                    "h2d_bytes_per_step": int(Xh.numel() * 4), "d2h_bytes_per_step": int(outh.numel() * 4)},
+            "gpu_launches": kernels_per_step * args.steps,
+            "roofline": roofline, "cpu_baseline": cpu_baseline, "legs": legs, "parity": parity}
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
