@@ -71,6 +71,30 @@ detox_status detox_vote(const float* X, int64_t ld, int n, int r, int64_t d, con
                         float* Z, int64_t ldz, int32_t* winner, void* ws, size_t ws_bytes, void* stream);
 
 /* ---------------------------------------------------------------------------------------------
+ * detox_vote without a workspace, for callers that must not allocate device memory.  (The paper has
+ * no counterpart; this is a packaging variant of detox_vote and computes exactly the same votes.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits - inside a framework's allocator
+ * callback, in a latency-critical serving loop with a frozen memory plan, or in a process whose
+ * memory budget is fixed at start-up - and that has nowhere to keep a workspace buffer.
+ *
+ * The scratch words of the vote live in a fixed array inside the library (4 KiB of global memory on
+ * every GPU that loads the library, held until the process exits), so at most
+ * DETOX_NOALLOC_MAX_GROUPS node groups (n / r) are accepted; more returns DETOX_ERR_UNSUPPORTED.
+ * The call itself performs no cudaMalloc / cudaFree and calls no allocating routine.
+ *
+ *   - Arguments as in detox_vote, minus ws / ws_bytes.  Inputs and outputs are still the caller's.
+ *   - The first call on each device looks up the device address of the built-in array (a one-time
+ *     set-up step, done with that device current).  Make that first call before any stream capture.
+ *   - All calls on a device share the one array.  Each call clears the words it uses before using
+ *     them, so results never depend on an earlier call; but two calls whose kernels overlap on the
+ *     GPU (different streams, no dependency between them) race on it.  Serialise them.
+ * ------------------------------------------------------------------------------------------- */
+#define DETOX_NOALLOC_MAX_GROUPS 256
+detox_status detox_vote_noalloc(const float* X, int64_t ld, int n, int r, int64_t d, const int32_t* members,
+                                float* Z, int64_t ldz, int32_t* winner, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
  * A_0 = mean over each vote group (Algorithm 2, step 3, with A_0 the mean as analysed in Section 4):
  * M[s] = (1/|Z_s|) sum_{j in Z_s} z_j.  A zero vote (no majority) counts as an ordinary member.
  *

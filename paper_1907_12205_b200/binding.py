@@ -21,7 +21,7 @@ AGG_NONE, AGG_MEAN, AGG_COORD_MEDIAN, AGG_MULTIKRUM, AGG_BULYAN = 0, 1, 2, 3, 4
 MAX_ROWS, MAX_R = 1024, 15
 
 EXPORTS = (
-    "detox_status_string", "detox_vote_workspace_bytes", "detox_vote", "detox_hier_mean",
+    "detox_status_string", "detox_vote_workspace_bytes", "detox_vote", "detox_vote_noalloc", "detox_hier_mean",
     "agg_coord_median_workspace_bytes", "agg_coord_median", "agg_multikrum_workspace_bytes", "agg_multikrum",
     "agg_bulyan_workspace_bytes", "agg_bulyan", "detox_aggregate_workspace_bytes", "detox_aggregate",
 )
@@ -62,6 +62,7 @@ def load() -> ctypes.CDLL:
     lib.detox_vote_workspace_bytes.restype = _sz
     lib.detox_vote_workspace_bytes.argtypes = [_int, _int]
     lib.detox_vote.argtypes = [_vp, _i64, _int, _int, _i64, _ip, _vp, _i64, _vp, _vp, _sz, _vp]
+    lib.detox_vote_noalloc.argtypes = [_vp, _i64, _int, _int, _i64, _ip, _vp, _i64, _vp, _vp]
     lib.detox_hier_mean.argtypes = [_vp, _i64, _int, _i64, _ip, _ip, _int, _vp, _i64, _vp]
     for name in ("agg_coord_median", "agg_multikrum", "agg_bulyan"):
         fn = getattr(lib, name + "_workspace_bytes")
@@ -134,6 +135,23 @@ def detox_vote(X, r: int, members, Z: Optional[torch.Tensor] = None, winner: Opt
     ws, wp, wb = _ws(lib.detox_vote_workspace_bytes(n, r), ws, X.device)
     _check(lib.detox_vote(xp, ld, n, r, d, mem.ctypes.data_as(_ip), zp, ldz, winner.data_ptr(), wp, wb,
                           _stream(stream)), "detox_vote")
+    return Z, winner
+
+
+NOALLOC_MAX_GROUPS = 256
+
+
+def detox_vote_noalloc(X, r: int, members, Z: torch.Tensor, winner: torch.Tensor, stream=None):
+    """detox_vote for callers that cannot allocate: the scratch is a fixed array inside the library,
+    and Z (or None) and winner must be passed in, so neither the library nor this wrapper allocates
+    device memory.  At most NOALLOC_MAX_GROUPS node groups.  Calls that overlap on the GPU race on
+    the shared scratch; the first call on a device should come before any stream capture."""
+    lib = load()
+    xp, ld, n, d = _mat(X)
+    mem = _host_i32(members)
+    zp, ldz = (None, 0) if Z is None else (Z.data_ptr(), Z.stride(0) if Z.shape[0] > 1 else max(Z.stride(0), d))
+    _check(lib.detox_vote_noalloc(xp, ld, n, r, d, mem.ctypes.data_as(_ip), zp, ldz, winner.data_ptr(),
+                                  _stream(stream)), "detox_vote_noalloc")
     return Z, winner
 
 
