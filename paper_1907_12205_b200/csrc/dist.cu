@@ -87,18 +87,25 @@ sqdist_direct_kernel(const float* __restrict__ X, int64_t ld, int64_t d, bool ve
     }
 }
 
-// D from the per-CTA pair partials of the direct kernel
+// D from the per-CTA pair partials of the direct kernel: one warp per pair, lanes take the partials
+// round-robin (independent loads), then a fixed shuffle tree.
 __global__ void sqdist_direct_reduce_kernel(const double* __restrict__ partial, int nblocks, int m,
                                             double* __restrict__ D) {
     const int np = m * (m - 1) / 2;
-    for (int p = blockIdx.x * blockDim.x + threadIdx.x; p < np; p += gridDim.x * blockDim.x) {
+    const int lane = threadIdx.x & 31;
+    const int warps = (gridDim.x * blockDim.x) >> 5;
+    for (int p = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; p < np; p += warps) {
         double v = 0.0;
-        for (int b = 0; b < nblocks; ++b) v += partial[(int64_t)b * np + p];
-        int i = 0, rem = p;
-        while (rem >= m - 1 - i) { rem -= m - 1 - i; ++i; }
-        const int j = i + 1 + rem;
-        D[i * m + j] = v;
-        D[j * m + i] = v;
+        for (int b = lane; b < nblocks; b += 32) v += partial[(int64_t)b * np + p];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) v += __shfl_down_sync(0xffffffffu, v, o);
+        if (lane == 0) {
+            int i = 0, rem = p;
+            while (rem >= m - 1 - i) { rem -= m - 1 - i; ++i; }
+            const int j = i + 1 + rem;
+            D[i * m + j] = v;
+            D[j * m + i] = v;
+        }
     }
     if (blockIdx.x == 0)
         for (int i = threadIdx.x; i < m; i += blockDim.x) D[i * m + i] = 0.0;
@@ -187,6 +194,7 @@ __global__ void gram_reduce_kernel(const double* __restrict__ partial, int m, in
         const int pair = bi * ntile - bi * (bi - 1) / 2 + (bj - bi);
         const double* p = partial + (int64_t)pair * nslab * (kGT * kGT) + (i % kGT) * kGT + (j % kGT);
         double v = 0.0;
+#pragma unroll 8
         for (int s = 0; s < nslab; ++s) v += p[(int64_t)s * (kGT * kGT)];
         gram[e] = v;
     }
@@ -235,7 +243,7 @@ detox_status launch_direct(const float* X, int64_t ld, int64_t d, double* D, dou
     sqdist_direct_kernel<M><<<nb, kDirThreads, 0, s>>>(X, ld, d, vec2, partial);
     detox_status st = launch_status();
     if (st != DETOX_OK) return st;
-    sqdist_direct_reduce_kernel<<<1, 128, 0, s>>>(partial, nb, M, D);
+    sqdist_direct_reduce_kernel<<<(M * (M - 1) / 2 + 3) / 4, 128, 0, s>>>(partial, nb, M, D);
     return launch_status();
 }
 
