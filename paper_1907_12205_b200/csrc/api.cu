@@ -54,6 +54,7 @@ detox_status check_matrix(const float* X, int64_t ld, int m, int64_t d) {
 
 // workspace of the Krum-type aggregators: D | distance scratch | selection scratch | index list
 struct KrumWs {
+    int* status;
     double* D;
     void* dist;
     void* select;
@@ -65,6 +66,8 @@ KrumWs krum_ws(void* ws, int m, int64_t d) {
     KrumWs k;
     char* p = static_cast<char*>(ws);
     size_t off = 0;
+    k.status = reinterpret_cast<int*>(p + off);   // first word of the workspace: device-side status
+    off += 256;
     k.D = reinterpret_cast<double*>(p + off);
     off += align_up((size_t)m * m * sizeof(double));
     k.dist = p + off;
@@ -81,7 +84,8 @@ detox_status run_multikrum(const float* X, int64_t ld, int m, int64_t d, int f, 
                            double* scores, void* ws, cudaStream_t s) {
     KrumWs k = krum_ws(ws, m, d);
     int32_t* sel_buf = sel ? sel : k.sel;
-    detox_status st = launch_sqdist(X, ld, m, d, k.D, k.dist, s);
+    if (cudaMemsetAsync(k.status, 0, sizeof(int), s) != cudaSuccess) return DETOX_ERR_CUDA;
+    detox_status st = launch_sqdist(X, ld, m, d, k.D, k.dist, k.status, s);
     if (st != DETOX_OK) return st;
     st = launch_multikrum_select(k.D, m, f, m_sel, sel_buf, scores, k.select, s);
     if (st != DETOX_OK) return st;
@@ -93,7 +97,8 @@ detox_status run_bulyan(const float* X, int64_t ld, int m, int64_t d, int f, flo
     KrumWs k = krum_ws(ws, m, d);
     int32_t* sel_buf = sel ? sel : k.sel;
     const int theta = m - 2 * f, beta = theta - 2 * f;
-    detox_status st = launch_sqdist(X, ld, m, d, k.D, k.dist, s);
+    if (cudaMemsetAsync(k.status, 0, sizeof(int), s) != cudaSuccess) return DETOX_ERR_CUDA;
+    detox_status st = launch_sqdist(X, ld, m, d, k.D, k.dist, k.status, s);
     if (st != DETOX_OK) return st;
     st = launch_bulyan_select(k.D, m, f, sel_buf, k.select, s);
     if (st != DETOX_OK) return st;

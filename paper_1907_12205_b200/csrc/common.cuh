@@ -77,9 +77,17 @@ detox_status launch_coord_select(const float* X, int64_t ld, int m, int64_t d, c
                                  int beta, float* out, cudaStream_t s);
 
 // dist.cu: squared distances D (m x m, fp64, symmetric, zero diagonal)
+//   status: device int32, must be 0 on entry; set to DETOX_ERR_TIMEOUT (and D to NaN) if a bounded
+//   device-side wait of the tensor-core path runs out
 size_t dist_ws_bytes(int m, int64_t d);
-detox_status launch_sqdist(const float* X, int64_t ld, int m, int64_t d, double* D, void* ws,
+detox_status launch_sqdist(const float* X, int64_t ld, int m, int64_t d, double* D, void* ws, int* status,
                            cudaStream_t s);
+
+// gram_tc.cu: the tcgen05 path for 16 < m <= 256 (needs 16-byte aligned rows)
+bool tc_supported(const float* X, int64_t ld, int m, int64_t d);
+size_t tc_ws_bytes(int m, int64_t d);
+detox_status launch_sqdist_tc(const float* X, int64_t ld, int m, int64_t d, double* D, void* ws, int* status,
+                              cudaStream_t s);
 
 // select.cu
 size_t select_ws_bytes(int m);

@@ -3,7 +3,8 @@
 //
 //   m <= 16 : differences are formed directly, (x_i - x_j)^2, with one fp32 accumulator per pair in
 //             registers; HBM-bound (m*d*4 bytes read once).
-//   m  > 16 : CUDA-core Gram tiles G = X X^T over K-slabs, D_ij = G_ii + G_jj - 2 G_ij.
+//   16 < m <= 256 with 16-byte aligned rows: the tensor-core Gram of gram_tc.cu.
+//   otherwise : CUDA-core Gram tiles G = X X^T over K-slabs, D_ij = G_ii + G_jj - 2 G_ij.
 // Both write per-CTA partial sums that a second kernel adds in a fixed order in fp64, so results
 // are deterministic and bitwise-equal rows get bitwise-equal distances.
 #include "common.cuh"
@@ -252,10 +253,13 @@ detox_status launch_direct(const float* X, int64_t ld, int64_t d, double* D, dou
 size_t dist_ws_bytes(int m, int64_t d) {
     if (m <= 16) return align_up((size_t)direct_blocks(d) * (size_t)(m * (m - 1) / 2 + 1) * sizeof(double));
     GramPlan g = gram_plan(m, d);
-    return align_up((size_t)g.npair * g.nslab * kGT * kGT * sizeof(double)) + align_up((size_t)m * m * sizeof(double));
+    size_t simt = align_up((size_t)g.npair * g.nslab * kGT * kGT * sizeof(double)) + align_up((size_t)m * m * sizeof(double));
+    size_t tc = m <= 256 ? tc_ws_bytes(m, d) : 0;
+    return simt > tc ? simt : tc;
 }
 
-detox_status launch_sqdist(const float* X, int64_t ld, int m, int64_t d, double* D, void* ws, cudaStream_t s) {
+detox_status launch_sqdist(const float* X, int64_t ld, int m, int64_t d, double* D, void* ws, int* status,
+                           cudaStream_t s) {
     double* partial = static_cast<double*>(ws);
     switch (m) {
         case 1:
@@ -268,6 +272,7 @@ detox_status launch_sqdist(const float* X, int64_t ld, int m, int64_t d, double*
 #undef DETOX_CASE
         default: break;
     }
+    if (tc_supported(X, ld, m, d)) return launch_sqdist_tc(X, ld, m, d, D, ws, status, s);
     GramPlan g = gram_plan(m, d);
     double* gram = reinterpret_cast<double*>(static_cast<char*>(ws) +
                                              align_up((size_t)g.npair * g.nslab * kGT * kGT * sizeof(double)));

@@ -1,0 +1,513 @@
+// Pairwise squared distances for 16 < m <= 256 on the 5th-generation tensor cores (tcgen05 + TMEM).
+//
+// G = X X^T is computed with error-compensated TF32: every fp32 x is split into hi = tf32(x) and
+// lo = x - hi (exact), and  x_i . x_j  ~=  hi_i.hi_j + hi_i.lo_j + lo_i.hi_j.  The last two terms are
+// folded by symmetry: with T = hi (hi + 2 lo)^T, accumulated as two MMAs per K-step into ONE fp32
+// accumulator in tensor memory, G_ij = (T_ij + T_ji) / 2.  Both MMA operands come from the same
+// shared-memory tiles (rows of X), so every row of X is read from HBM exactly once.
+//
+// One persistent CTA per SM.  One thread streams K-blocks of 32 columns (all m rows) into shared
+// memory with TMA (128-byte swizzle, which is the K-major layout the MMA expects; rows and columns
+// outside the matrix arrive as zeros).  The raw fp32 tile itself serves as the `hi` operand: a TF32
+// MMA reads only the upper 19 bits of each word.  Warps 0-7 read the tile back, form
+// 2 lo = 2 (x - (x with its low 13 bits cleared)) and write the second tile; lane 0 of warp 8
+// issues the MMAs; mbarriers form a ring of stages between the three roles.
+// Work is cut into K-slabs; at the end of a slab the accumulator is drained to a per-slab fp32
+// partial in global memory and the slabs are added in fp64 in a fixed order afterwards, so the long
+// sum never lives in one fp32 accumulator and the result is deterministic.
+//
+// The tensor cores add into their fp32 accumulator by truncation, so a long same-sign sum (a row with
+// itself, or with a copy of itself) comes out low by a few 1e-5 relative per slab.  The producers
+// therefore also accumulate each row's exact squared norm per slab on the CUDA cores; the final
+// reduction rescales every slab's T_ij by the mean of (exact norm / tensor-core norm) of rows i and
+// j.  The diagonal becomes exact, a pair of identical rows keeps distance zero, and entries
+// between unrelated rows (which hover around zero and lose nothing to truncation) are unchanged.
+//
+// Every wait on an mbarrier is bounded; if one runs out the kernel records DETOX_ERR_TIMEOUT in the
+// status word, stops waiting everywhere, frees its tensor memory and returns.
+#include <cuda.h>
+
+#include "common.cuh"
+
+namespace detox {
+
+namespace {
+
+constexpr int kKB = 32;                      // fp32 columns per K-block: one 128-byte swizzle row
+constexpr int kProdWarps = 8;
+constexpr int kProdThreads = kProdWarps * 32;
+constexpr int kTcThreads = kProdThreads + 64;  // + the MMA warp + the TMA warp
+constexpr int kMaxStages = 6;
+constexpr uint32_t kSpinLimit = 1u << 22;
+constexpr int64_t kSlabCols = 4096;          // columns accumulated in tensor memory before a drain
+constexpr int kReduceChunks = 32;
+
+struct TcPlan {
+    int rows_pad;    // rows of each shared-memory tile (128 or 256)
+    int box_rows;    // rows the TMA box brings in: m rounded up to 8
+    int nhalf;       // accumulator halves of 128 rows
+    int ncol;        // N of the MMA: m rounded up to 16
+    int tmem_cols;   // power of two >= nhalf * ncol, >= 32
+    int stages;
+    int nitems;      // K-slabs
+    int grid;
+    size_t smem_bytes;
+};
+
+TcPlan tc_plan(int m, int64_t d) {
+    TcPlan p;
+    p.nhalf = m > 128 ? 2 : 1;
+    p.rows_pad = 128 * p.nhalf;
+    p.box_rows = (m + 7) / 8 * 8;
+    p.ncol = (m + 15) / 16 * 16;
+    int need = p.nhalf * p.ncol;
+    p.tmem_cols = 32;
+    while (p.tmem_cols < need) p.tmem_cols <<= 1;
+    size_t stage = (size_t)2 * p.rows_pad * 128;
+    p.stages = (int)((192 * 1024) / stage);
+    if (p.stages > kMaxStages) p.stages = kMaxStages;
+    p.nitems = (int)ceil_div(d, kSlabCols);
+    p.grid = p.nitems < kSMs ? p.nitems : kSMs;
+    p.smem_bytes = stage * p.stages + 1024 /*barriers*/ + 1024 /*alignment slack*/;
+    return p;
+}
+
+// ------------------------------------------------------------------------------------ PTX wrappers
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_test(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait.  Returns false (and raises the CTA-wide abort flag) when the limit is hit.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status) {
+    for (uint32_t spin = 0; spin < kSpinLimit; ++spin) {
+        if (mbar_test(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (spin > 64) __nanosleep(64);
+    }
+    *abort_flag = 1;
+    atomicExch(status, (int)DETOX_ERR_TIMEOUT);
+    return false;
+}
+
+__device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_alloc(uint32_t* slot, uint32_t ncols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(slot)), "r"(ncols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+
+// Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, rows packed 128 bytes apart,
+// 8-row groups 1024 bytes apart.  `addr` must lie in a 1024-byte aligned tile.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
+    uint64_t desc = (uint64_t)((addr & 0x3FFFFu) >> 4);   // start address, 16-byte units
+    desc |= (uint64_t)1 << 16;                              // leading byte offset (unused for swizzled K-major)
+    desc |= (uint64_t)(1024 >> 4) << 32;                    // stride byte offset: next 8-row group
+    desc |= (uint64_t)1 << 46;                              // descriptor version of this architecture
+    desc |= (uint64_t)2 << 61;                              // 128-byte swizzle
+    return desc;
+}
+
+// D[tmem] (+)= A[smem] * B[smem]^T, TF32 inputs, fp32 accumulate, M = 128.
+__device__ __forceinline__ void mma_tf32(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// Arrive on `bar` once every MMA issued so far by this thread has finished.
+__device__ __forceinline__ void mma_commit(uint64_t* bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+                 : "memory");
+}
+
+__device__ __forceinline__ void tmem_load32(uint32_t taddr, uint32_t (&v)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+          "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+          "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+        : "r"(taddr)
+        : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+// 2-D tiled TMA load (no multicast): box at (x = column, y = row) -> shared memory, completion on `bar`.
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(smem_u32(bar))
+        : "memory");
+}
+
+__device__ __forceinline__ uint32_t to_tf32(float x) {
+    uint32_t r;
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
+    return r;
+}
+
+// What a TF32 MMA sees of x is hi = x with the low 13 mantissa bits cleared; x - hi is exact in fp32.
+// Returns 2 (x - hi) rounded to TF32.
+__device__ __forceinline__ uint32_t lo2_of(float x) {
+    const float hi = __uint_as_float(__float_as_uint(x) & 0xFFFFE000u);
+    return to_tf32(2.0f * (x - hi));
+}
+
+struct TcSmem {
+    uint64_t landed[kMaxStages];   // TMA bytes of the raw tile have arrived
+    uint64_t full[kMaxStages];     // the 2lo tile is written: both tiles ready for the MMA
+    uint64_t empty[kMaxStages];
+    uint64_t accum_full;
+    uint64_t accum_empty;
+    uint32_t tmem_base;
+    int abort_flag;
+};
+
+// J = 16-byte chunks per transform thread and K-block (m * 8 / 256 rounded up to a power of two)
+template <int J>
+__global__ void __launch_bounds__(kTcThreads, 1)
+gram_tc_kernel(const __grid_constant__ CUtensorMap xmap, int m, int64_t d, int rows_pad, int box_rows, int nhalf,
+               int ncol, int tmem_cols, int stages, int nitems, float* __restrict__ partial,
+               float* __restrict__ norms, int* __restrict__ status) {
+    extern __shared__ uint8_t smem_raw[];
+    // tiles need 1024-byte alignment for the 128-byte swizzle pattern
+    const uint32_t raw = smem_u32(smem_raw);
+    uint8_t* base = smem_raw + ((1024u - (raw & 1023u)) & 1023u);
+    const uint32_t tile_bytes = (uint32_t)rows_pad * 128u;
+    const uint32_t stage_bytes = 2u * tile_bytes;
+    TcSmem* sm = reinterpret_cast<TcSmem*>(base + (size_t)stage_bytes * stages);
+    volatile int* abort_flag = &sm->abort_flag;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+    if (tid == 0) {
+        for (int s = 0; s < stages; ++s) {
+            mbar_init(&sm->landed[s], 1);
+            mbar_init(&sm->full[s], kProdWarps);
+            mbar_init(&sm->empty[s], 1);
+        }
+        mbar_init(&sm->accum_full, 1);
+        mbar_init(&sm->accum_empty, kProdWarps);
+        sm->abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    // rows beyond the TMA box are never written: clear all tiles once so the padded rows are zeros
+    for (uint32_t off = (uint32_t)tid * 16u; off < stage_bytes * (uint32_t)stages; off += kTcThreads * 16u)
+        *reinterpret_cast<uint4*>(base + off) = make_uint4(0u, 0u, 0u, 0u);
+    fence_proxy_async_smem();
+    if (warp == 0) tmem_alloc(&sm->tmem_base, (uint32_t)tmem_cols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = sm->tmem_base;
+
+    // K-blocks of this CTA, over all its slabs, as one sequence t = 0 .. total-1.
+    // Every slab has kSlabCols / kKB blocks except the globally last one, which may be shorter.
+    constexpr int kBlocksPerSlab = (int)(kSlabCols / kKB);
+    const int my_items = (nitems - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
+    const int last_item = (int)blockIdx.x + (my_items - 1) * (int)gridDim.x;
+    const int last_nkb = (int)(((last_item == nitems - 1 ? d : (int64_t)(last_item + 1) * kSlabCols) -
+                                (int64_t)last_item * kSlabCols + kKB - 1) / kKB);
+    const int total = (my_items - 1) * kBlocksPerSlab + last_nkb;
+
+    if (warp < kProdWarps) {
+        // ------------------------------------------------ transform warps, then epilogue of each slab
+        const int nchunks = m * 8;
+        // this thread's chunks are (row, c) = ((tid >> 3) + 32 j, tid & 7) in every K-block
+        uint32_t off[J];
+#pragma unroll
+        for (int j = 0; j < J; ++j) {
+            const int row = (tid >> 3) + 32 * j, c = tid & 7;
+            off[j] = (uint32_t)(row >> 3) * 1024u + (uint32_t)(row & 7) * 128u + (uint32_t)((c ^ (row & 7)) << 4);
+        }
+        float sq[J];
+#pragma unroll
+        for (int j = 0; j < J; ++j) sq[j] = 0.f;
+
+        for (int t = 0; t < total; ++t) {
+            const int s = (int)((uint32_t)t % (uint32_t)stages);
+            const uint32_t ph = ((uint32_t)t / (uint32_t)stages) & 1u;
+            mbar_wait(&sm->landed[s], ph, abort_flag, status);
+            const uint8_t* hi_tile = base + (size_t)s * stage_bytes;
+            uint8_t* lo_tile = base + (size_t)s * stage_bytes + tile_bytes;
+#pragma unroll
+            for (int j = 0; j < J; ++j) {
+                if (tid + j * kProdThreads < nchunks) {
+                    const float4 x = *reinterpret_cast<const float4*>(hi_tile + off[j]);
+                    sq[j] = fmaf(x.x, x.x, fmaf(x.y, x.y, fmaf(x.z, x.z, fmaf(x.w, x.w, sq[j]))));
+                    *reinterpret_cast<uint4*>(lo_tile + off[j]) =
+                        make_uint4(lo2_of(x.x), lo2_of(x.y), lo2_of(x.z), lo2_of(x.w));
+                }
+            }
+            fence_proxy_async_smem();   // make the generic-proxy stores visible to the MMA's reads
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sm->full[s]);   // one arrival per transform warp
+
+            const int li = t / kBlocksPerSlab, kb = t - li * kBlocksPerSlab;
+            const int nkb = li == my_items - 1 ? last_nkb : kBlocksPerSlab;
+            if (kb != nkb - 1) continue;
+            const int item = (int)blockIdx.x + li * (int)gridDim.x;
+
+            // ---- end of a slab: exact squared norms (the 8 lanes that share a row add up) ...
+#pragma unroll
+            for (int j = 0; j < J; ++j) {
+                float v = sq[j];
+                v += __shfl_xor_sync(0xffffffffu, v, 1);
+                v += __shfl_xor_sync(0xffffffffu, v, 2);
+                v += __shfl_xor_sync(0xffffffffu, v, 4);
+                const int row = (tid >> 3) + 32 * j;
+                if ((tid & 7) == 0 && row < m) norms[(int64_t)item * m + row] = v;
+                sq[j] = 0.f;
+            }
+            // ... and the accumulator drain: warp w reads TMEM lanes 32*(w%4)..+31; the two warps that
+            // share a lane quarter take alternate 32-column chunks
+            mbar_wait(&sm->accum_full, (uint32_t)(li & 1), abort_flag, status);
+            tc_fence_after();
+            const int quarter = warp & 3;
+            float* out_item = partial + (int64_t)item * m * ncol;
+            for (int h = 0; h < nhalf; ++h) {
+                const int row = h * 128 + quarter * 32 + lane;
+                for (int cc = warp >> 2; cc * 32 < ncol; cc += 2) {
+                    uint32_t v[32];
+                    tmem_load32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(h * ncol + cc * 32), v);
+                    if (row < m) {
+                        float* dst = out_item + (int64_t)row * ncol + cc * 32;
+                        const int nvalid = ncol - cc * 32 < 32 ? ncol - cc * 32 : 32;
+#pragma unroll
+                        for (int j = 0; j < 32; j += 4) {
+                            if (j < nvalid)
+                                *reinterpret_cast<uint4*>(dst + j) = make_uint4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+                        }
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sm->accum_empty);
+        }
+    } else if (warp == kProdWarps + 1) {
+        // ------------------------------------------------ the TMA thread
+        if (lane == 0) {
+            const uint32_t tx_bytes = (uint32_t)box_rows * 128u;
+            int issued = 0;
+            for (int t = 0; t < total; ++t) {
+                const int s = (int)((uint32_t)t % (uint32_t)stages);
+                const uint32_t ph = ((uint32_t)t / (uint32_t)stages) & 1u;
+                mbar_wait(&sm->empty[s], ph ^ 1u, abort_flag, status);   // MMAs that read this stage are done
+                if (*abort_flag) break;
+                const int li = t / kBlocksPerSlab, kb = t - li * kBlocksPerSlab;
+                const int64_t c0 = ((int64_t)blockIdx.x + (int64_t)li * gridDim.x) * kSlabCols + (int64_t)kb * kKB;
+                mbar_expect_tx(&sm->landed[s], tx_bytes);
+                tma_load_2d(base + (size_t)s * stage_bytes, &xmap, (int)c0, 0, &sm->landed[s]);
+                issued = t + 1;
+            }
+            if (*abort_flag) {
+                // give the copies still in flight a bounded time to land before the CTA goes away
+                for (int t = issued > stages ? issued - stages : 0; t < issued; ++t) {
+                    const int s = (int)((uint32_t)t % (uint32_t)stages);
+                    const uint32_t ph = ((uint32_t)t / (uint32_t)stages) & 1u;
+                    for (uint32_t spin = 0; spin < (1u << 16) && !mbar_test(&sm->landed[s], ph); ++spin) __nanosleep(64);
+                }
+            }
+        }
+    } else if (lane == 0) {
+        // ------------------------------------------------ the MMA thread
+        const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(ncol >> 3) << 17) | ((128u >> 4) << 24);
+        uint32_t it = 0;
+        for (int local_item = 0; local_item < my_items; ++local_item) {
+            const int nkb = local_item == my_items - 1 ? last_nkb : kBlocksPerSlab;
+            if (local_item > 0) mbar_wait(&sm->accum_empty, (uint32_t)((local_item - 1) & 1), abort_flag, status);
+            tc_fence_after();
+            for (int kb = 0; kb < nkb; ++kb, ++it) {
+                const int s = (int)(it % (uint32_t)stages);
+                const uint32_t ph = (it / (uint32_t)stages) & 1u;
+                mbar_wait(&sm->full[s], ph, abort_flag, status);
+                tc_fence_after();
+                const uint32_t hi_addr = smem_u32(base + (size_t)s * stage_bytes);
+                const uint64_t hi_desc = smem_desc(hi_addr);
+                const uint64_t lo_desc = smem_desc(hi_addr + tile_bytes);
+#pragma unroll
+                for (int kk = 0; kk < kKB / 8; ++kk) {           // one MMA covers 8 columns = 32 bytes
+                    for (int h = 0; h < nhalf; ++h) {
+                        const uint64_t a = hi_desc + (uint64_t)(kk * 2 + h * (128 * 128 / 16));
+                        const uint32_t dcol = tmem_base + (uint32_t)(h * ncol);
+                        mma_tf32(dcol, a, hi_desc + (uint64_t)(kk * 2), idesc, (kb > 0 || kk > 0) ? 1u : 0u);
+                        mma_tf32(dcol, a, lo_desc + (uint64_t)(kk * 2), idesc, 1u);
+                    }
+                }
+                mma_commit(&sm->empty[s]);   // the stage may be refilled once these MMAs have read it
+            }
+            mma_commit(&sm->accum_full);
+        }
+    }
+
+    __syncwarp();
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    if (warp == 0) tmem_dealloc(tmem_base, (uint32_t)tmem_cols);
+}
+
+// For one chunk of slabs: gpart[chunk][i*m+j] (i < j) = sum_s sym(T(s))_ij * (r_i(s) + r_j(s)) / 2 with
+// r_i(s) = exact norm / tensor-core norm of row i in slab s; gpart[chunk][i*m+i] = sum_s exact norm.
+__global__ void tc_reduce_kernel(const float* __restrict__ partial, const float* __restrict__ norms, int nitems,
+                                 int m, int ncol, double* __restrict__ gpart) {
+    const int chunk = blockIdx.y;
+    const int per = (nitems + kReduceChunks - 1) / kReduceChunks;
+    const int s0 = chunk * per, s1 = (s0 + per) < nitems ? (s0 + per) : nitems;
+    const int64_t elems = (int64_t)m * ncol;
+    const int64_t total = (int64_t)m * m;
+    for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
+        const int i = (int)(e / m), j = (int)(e - (int64_t)i * m);
+        if (i > j) continue;
+        double acc = 0.0;
+        if (i == j) {
+            for (int s = s0; s < s1; ++s) acc += (double)norms[(int64_t)s * m + i];
+        } else {
+#pragma unroll 4
+            for (int s = s0; s < s1; ++s) {
+                const float* T = partial + (int64_t)s * elems;
+                const double tii = (double)T[(int64_t)i * ncol + i], tjj = (double)T[(int64_t)j * ncol + j];
+                const double ni = (double)norms[(int64_t)s * m + i], nj = (double)norms[(int64_t)s * m + j];
+                const double ri = tii > 0.0 ? ni / tii : 1.0;
+                const double rj = tjj > 0.0 ? nj / tjj : 1.0;
+                const double tij = 0.5 * ((double)T[(int64_t)i * ncol + j] + (double)T[(int64_t)j * ncol + i]);
+                acc += tij * (0.5 * (ri + rj));
+            }
+        }
+        gpart[(int64_t)chunk * total + e] = acc;
+    }
+}
+
+// D_ij = n_i + n_j - 2 G_ij (never negative, zero diagonal); status != 0 -> NaN
+__global__ void tc_dist_kernel(const double* __restrict__ gpart, int m, const int* __restrict__ status,
+                               double* __restrict__ D) {
+    const bool bad = *status != 0;
+    const int64_t total = (int64_t)m * m;
+    auto G = [&](int i, int j) {
+        double v = 0.0;
+#pragma unroll
+        for (int c = 0; c < kReduceChunks; ++c) v += gpart[(int64_t)c * total + (int64_t)i * m + j];
+        return v;
+    };
+    for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
+        const int i = (int)(e / m), j = (int)(e - (int64_t)i * m);
+        if (bad) { D[e] = __longlong_as_double(0x7ff8000000000000LL); continue; }
+        if (i == j) { D[e] = 0.0; continue; }
+        const int a = i < j ? i : j, b = i < j ? j : i;
+        const double v = G(a, a) + G(b, b) - 2.0 * G(a, b);
+        D[e] = v > 0.0 ? v : 0.0;
+    }
+}
+
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// The driver's tensor-map encoder, looked up through the runtime (no link against libcuda).
+EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = [] {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess)
+            p = nullptr;
+        return reinterpret_cast<EncodeTiledFn>(p);
+    }();
+    return fn;
+}
+
+// X as a 2-D fp32 tensor (d columns innermost, m rows, row pitch ld); box = 32 columns x box_rows rows,
+// 128-byte swizzle, zero fill outside.
+detox_status make_xmap(CUtensorMap* map, const float* X, int64_t ld, int m, int64_t d, int box_rows) {
+    EncodeTiledFn enc = encode_tiled_fn();
+    if (!enc) return DETOX_ERR_CUDA;
+    const cuuint64_t gdim[2] = {(cuuint64_t)d, (cuuint64_t)m};
+    const cuuint64_t gstride[1] = {(cuuint64_t)ld * sizeof(float)};
+    const cuuint32_t box[2] = {(cuuint32_t)kKB, (cuuint32_t)box_rows};
+    const cuuint32_t estride[2] = {1, 1};
+    CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(X), gdim, gstride, box, estride,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? DETOX_OK : DETOX_ERR_CUDA;
+}
+
+template <int J>
+detox_status launch_tc(const TcPlan& p, const CUtensorMap& xmap, int m, int64_t d, float* partial, float* norms,
+                       int* status, cudaStream_t s) {
+    if (cudaFuncSetAttribute(gram_tc_kernel<J>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem_bytes) !=
+        cudaSuccess)
+        return DETOX_ERR_CUDA;
+    gram_tc_kernel<J><<<p.grid, kTcThreads, p.smem_bytes, s>>>(xmap, m, d, p.rows_pad, p.box_rows, p.nhalf, p.ncol,
+                                                               p.tmem_cols, p.stages, p.nitems, partial, norms, status);
+    return launch_status();
+}
+
+}  // namespace
+
+bool tc_supported(const float* X, int64_t ld, int m, int64_t d) {
+    // TMA needs a 16-byte aligned base and row pitch; coordinates are 32-bit
+    return m > 16 && m <= 256 && aligned16(X) && ld % 4 == 0 && d < (int64_t)1 << 31 && encode_tiled_fn() != nullptr;
+}
+
+size_t tc_ws_bytes(int m, int64_t d) {
+    TcPlan p = tc_plan(m, d);
+    const size_t elems = (size_t)m * p.ncol;
+    return align_up((size_t)p.nitems * elems * sizeof(float)) + align_up((size_t)p.nitems * m * sizeof(float)) +
+           align_up((size_t)kReduceChunks * m * m * sizeof(double));
+}
+
+detox_status launch_sqdist_tc(const float* X, int64_t ld, int m, int64_t d, double* D, void* ws, int* status,
+                              cudaStream_t s) {
+    TcPlan p = tc_plan(m, d);
+    const int64_t elems = (int64_t)m * p.ncol;
+    char* base = static_cast<char*>(ws);
+    float* partial = reinterpret_cast<float*>(base);
+    float* norms = reinterpret_cast<float*>(base + align_up((size_t)p.nitems * elems * sizeof(float)));
+    double* gpart = reinterpret_cast<double*>(base + align_up((size_t)p.nitems * elems * sizeof(float)) +
+                                              align_up((size_t)p.nitems * m * sizeof(float)));
+    CUtensorMap xmap;
+    detox_status st = make_xmap(&xmap, X, ld, m, d, p.box_rows);
+    if (st != DETOX_OK) return st;
+    if (m <= 32) st = launch_tc<1>(p, xmap, m, d, partial, norms, status, s);
+    else if (m <= 64) st = launch_tc<2>(p, xmap, m, d, partial, norms, status, s);
+    else if (m <= 128) st = launch_tc<4>(p, xmap, m, d, partial, norms, status, s);
+    else st = launch_tc<8>(p, xmap, m, d, partial, norms, status, s);
+    if (st != DETOX_OK) return st;
+    tc_reduce_kernel<<<dim3((unsigned)ceil_div((int64_t)m * m, 256), kReduceChunks), 256, 0, s>>>(
+        partial, norms, p.nitems, m, p.ncol, gpart);
+    if ((st = launch_status()) != DETOX_OK) return st;
+    tc_dist_kernel<<<(unsigned)ceil_div((int64_t)m * m, 256), 256, 0, s>>>(gpart, m, status, D);
+    return launch_status();
+}
+
+}  // namespace detox
