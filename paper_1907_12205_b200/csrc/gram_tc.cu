@@ -36,9 +36,10 @@ namespace {
 constexpr int kKB = 32;                      // fp32 columns per K-block: one 128-byte swizzle row
 constexpr int kProdWarps = 8;
 constexpr int kProdThreads = kProdWarps * 32;
-constexpr int kTcThreads = kProdThreads + 64;  // + the MMA warp + the TMA warp
+constexpr int kMmaWarps = 2;                   // two issuing threads, so one's bookkeeping overlaps the other's MMAs
+constexpr int kTcThreads = kProdThreads + 32 * (kMmaWarps + 1);  // + the MMA warps + the TMA warp
 constexpr int kMaxStages = 6;
-constexpr uint32_t kSpinLimit = 1u << 22;
+constexpr long long kWaitLimitCycles = 2000000000LL;  // ~1 s at the SM clock
 constexpr int64_t kSlabCols = 4096;          // columns accumulated in tensor memory before a drain
 constexpr int kReduceChunks = 32;
 
@@ -47,7 +48,8 @@ struct TcPlan {
     int box_rows;    // rows the TMA box brings in: m rounded up to 8
     int nhalf;       // accumulator halves of 128 rows
     int ncol;        // N of the MMA: m rounded up to 16
-    int tmem_cols;   // power of two >= nhalf * ncol, >= 32
+    int chains;      // m <= 128: accumulators, one per MMA-issuing thread
+    int tmem_cols;   // power of two >= the accumulator columns, >= 32
     int stages;
     int nitems;      // K-slabs
     int grid;
@@ -60,7 +62,11 @@ TcPlan tc_plan(int m, int64_t d) {
     p.rows_pad = 128 * p.nhalf;
     p.box_rows = (m + 7) / 8 * 8;
     p.ncol = (m + 15) / 16 * 16;
-    int need = p.nhalf * p.ncol;
+    // m <= 128: one MMA per K-step with B = [hi ; 2lo] stacked (N = 2 ncol); the two issuing threads take
+    //           alternate K-blocks and own one accumulator each;
+    // m  > 128: two 128-row halves, one per issuing thread, B = hi and B = 2lo as separate MMAs
+    p.chains = p.nhalf == 1 ? kMmaWarps : 1;
+    int need = p.nhalf == 1 ? p.chains * 2 * p.ncol : 2 * p.ncol;
     p.tmem_cols = 32;
     while (p.tmem_cols < need) p.tmem_cols <<= 1;
     size_t stage = (size_t)2 * p.rows_pad * 128;
@@ -93,12 +99,28 @@ __device__ __forceinline__ bool mbar_test(uint64_t* bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
-// Bounded wait.  Returns false (and raises the CTA-wide abort flag) when the limit is hit.
+// Hardware-assisted wait: the thread is suspended until the phase completes or a short
+// implementation-defined time passes, whichever is first.
+__device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait (about a second of SM clocks).  Returns false, and raises the CTA-wide abort flag,
+// when the limit is hit; returns false at once when another thread has already given up.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status) {
-    for (uint32_t spin = 0; spin < kSpinLimit; ++spin) {
-        if (mbar_test(bar, parity)) return true;
+    if (mbar_try(bar, parity)) return true;
+    const long long start = clock64();
+    for (;;) {
+        if (mbar_try(bar, parity)) return true;
         if (*abort_flag) return false;
-        if (spin > 64) __nanosleep(64);
+        if (clock64() - start > kWaitLimitCycles) break;
     }
     *abort_flag = 1;
     atomicExch(status, (int)DETOX_ERR_TIMEOUT);
@@ -196,7 +218,7 @@ struct TcSmem {
 template <int J>
 __global__ void __launch_bounds__(kTcThreads, 1)
 gram_tc_kernel(const __grid_constant__ CUtensorMap xmap, int m, int64_t d, int rows_pad, int box_rows, int nhalf,
-               int ncol, int tmem_cols, int stages, int nitems, float* __restrict__ partial,
+               int ncol, int chains, int tmem_cols, int stages, int nitems, float* __restrict__ partial,
                float* __restrict__ norms, int* __restrict__ status) {
     extern __shared__ uint8_t smem_raw[];
     // tiles need 1024-byte alignment for the 128-byte swizzle pattern
@@ -213,9 +235,9 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap xmap, int m, int64_t d, int r
         for (int s = 0; s < stages; ++s) {
             mbar_init(&sm->landed[s], 1);
             mbar_init(&sm->full[s], kProdWarps);
-            mbar_init(&sm->empty[s], 1);
+            mbar_init(&sm->empty[s], nhalf == 1 ? 1 : kMmaWarps);
         }
-        mbar_init(&sm->accum_full, 1);
+        mbar_init(&sm->accum_full, kMmaWarps);
         mbar_init(&sm->accum_empty, kProdWarps);
         sm->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -258,7 +280,9 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap xmap, int m, int64_t d, int r
             const uint32_t ph = ((uint32_t)t / (uint32_t)stages) & 1u;
             mbar_wait(&sm->landed[s], ph, abort_flag, status);
             const uint8_t* hi_tile = base + (size_t)s * stage_bytes;
-            uint8_t* lo_tile = base + (size_t)s * stage_bytes + tile_bytes;
+            // m <= 128: the 2lo rows follow the hi rows at row `ncol` of the same tile (ncol % 8 == 0);
+            // m  > 128: they form a tile of their own
+            uint8_t* lo_tile = base + (size_t)s * stage_bytes + (nhalf == 1 ? (uint32_t)ncol * 128u : tile_bytes);
 #pragma unroll
             for (int j = 0; j < J; ++j) {
                 if (tid + j * kProdThreads < nchunks) {
@@ -297,15 +321,26 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap xmap, int m, int64_t d, int r
             for (int h = 0; h < nhalf; ++h) {
                 const int row = h * 128 + quarter * 32 + lane;
                 for (int cc = warp >> 2; cc * 32 < ncol; cc += 2) {
-                    uint32_t v[32];
-                    tmem_load32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(h * ncol + cc * 32), v);
+                    float acc[32];
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) acc[j] = 0.f;
+                    // m <= 128: add the hi.hi and hi.2lo parts of every chain; m > 128: one accumulator per half
+                    // (a slab of a single K-block leaves the second issuing thread's accumulator untouched: skip it)
+                    const int nparts = nhalf == 1 ? 2 * (nkb < chains ? nkb : chains) : 1;
+                    for (int part = 0; part < nparts; ++part) {
+                        uint32_t v[32];
+                        const int col = (nhalf == 1 ? part * ncol : h * ncol) + cc * 32;
+                        tmem_load32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)col, v);
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) acc[j] += __uint_as_float(v[j]);
+                    }
                     if (row < m) {
                         float* dst = out_item + (int64_t)row * ncol + cc * 32;
                         const int nvalid = ncol - cc * 32 < 32 ? ncol - cc * 32 : 32;
 #pragma unroll
                         for (int j = 0; j < 32; j += 4) {
                             if (j < nvalid)
-                                *reinterpret_cast<uint4*>(dst + j) = make_uint4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+                                *reinterpret_cast<float4*>(dst + j) = make_float4(acc[j], acc[j + 1], acc[j + 2], acc[j + 3]);
                         }
                     }
                 }
@@ -314,7 +349,7 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap xmap, int m, int64_t d, int r
             __syncwarp();
             if (lane == 0) mbar_arrive(&sm->accum_empty);
         }
-    } else if (warp == kProdWarps + 1) {
+    } else if (warp == kProdWarps + kMmaWarps) {
         // ------------------------------------------------ the TMA thread
         if (lane == 0) {
             const uint32_t tx_bytes = (uint32_t)box_rows * 128u;
@@ -340,28 +375,42 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap xmap, int m, int64_t d, int r
             }
         }
     } else if (lane == 0) {
-        // ------------------------------------------------ the MMA thread
-        const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(ncol >> 3) << 17) | ((128u >> 4) << 24);
+        // ------------------------------------------------ the MMA threads
+        // ------------------------------------------------ (two of them: warps 8 and 9, lane 0)
+        const int g = warp - kProdWarps;
+        const int n_mma = nhalf == 1 ? 2 * ncol : ncol;
+        const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(n_mma >> 3) << 17) | ((128u >> 4) << 24);
         uint32_t it = 0;
         for (int local_item = 0; local_item < my_items; ++local_item) {
             const int nkb = local_item == my_items - 1 ? last_nkb : kBlocksPerSlab;
             if (local_item > 0) mbar_wait(&sm->accum_empty, (uint32_t)((local_item - 1) & 1), abort_flag, status);
             tc_fence_after();
+            bool first = true;   // this thread's first MMA of the slab overwrites its accumulator
             for (int kb = 0; kb < nkb; ++kb, ++it) {
+                if (nhalf == 1 && (int)(it % kMmaWarps) != g) continue;   // m <= 128: alternate K-blocks
                 const int s = (int)(it % (uint32_t)stages);
                 const uint32_t ph = (it / (uint32_t)stages) & 1u;
                 mbar_wait(&sm->full[s], ph, abort_flag, status);
                 tc_fence_after();
                 const uint32_t hi_addr = smem_u32(base + (size_t)s * stage_bytes);
                 const uint64_t hi_desc = smem_desc(hi_addr);
-                const uint64_t lo_desc = smem_desc(hi_addr + tile_bytes);
+                if (nhalf == 1) {
+                    const uint32_t dcol = tmem_base + (uint32_t)(g * 2 * ncol);
 #pragma unroll
-                for (int kk = 0; kk < kKB / 8; ++kk) {           // one MMA covers 8 columns = 32 bytes
-                    for (int h = 0; h < nhalf; ++h) {
-                        const uint64_t a = hi_desc + (uint64_t)(kk * 2 + h * (128 * 128 / 16));
-                        const uint32_t dcol = tmem_base + (uint32_t)(h * ncol);
-                        mma_tf32(dcol, a, hi_desc + (uint64_t)(kk * 2), idesc, (kb > 0 || kk > 0) ? 1u : 0u);
+                    for (int kk = 0; kk < kKB / 8; ++kk) {       // one MMA covers 8 columns = 32 bytes
+                        const uint64_t ab = hi_desc + (uint64_t)(kk * 2);
+                        mma_tf32(dcol, ab, ab, idesc, first ? 0u : 1u);
+                        first = false;
+                    }
+                } else {
+                    const uint64_t lo_desc = smem_desc(hi_addr + tile_bytes);
+                    const uint32_t dcol = tmem_base + (uint32_t)(g * ncol);
+#pragma unroll
+                    for (int kk = 0; kk < kKB / 8; ++kk) {
+                        const uint64_t a = hi_desc + (uint64_t)(kk * 2 + g * (128 * 128 / 16));
+                        mma_tf32(dcol, a, hi_desc + (uint64_t)(kk * 2), idesc, first ? 0u : 1u);
                         mma_tf32(dcol, a, lo_desc + (uint64_t)(kk * 2), idesc, 1u);
+                        first = false;
                     }
                 }
                 mma_commit(&sm->empty[s]);   // the stage may be refilled once these MMAs have read it
@@ -468,7 +517,7 @@ detox_status launch_tc(const TcPlan& p, const CUtensorMap& xmap, int m, int64_t 
         cudaSuccess)
         return DETOX_ERR_CUDA;
     gram_tc_kernel<J><<<p.grid, kTcThreads, p.smem_bytes, s>>>(xmap, m, d, p.rows_pad, p.box_rows, p.nhalf, p.ncol,
-                                                               p.tmem_cols, p.stages, p.nitems, partial, norms, status);
+                                                               p.chains, p.tmem_cols, p.stages, p.nitems, partial, norms, status);
     return launch_status();
 }
 
