@@ -9,9 +9,9 @@
 // One persistent CTA per SM.  One thread streams K-blocks of 32 columns (all m rows) into shared
 // memory with TMA (128-byte swizzle, which is the K-major layout the MMA expects; rows and columns
 // outside the matrix arrive as zeros).  The raw fp32 tile itself serves as the `hi` operand: a TF32
-// MMA reads only the upper 19 bits of each word.  Warps 0-7 read the tile back, form
-// 2 lo = 2 (x - (x with its low 13 bits cleared)) and write the second tile; lane 0 of warp 8
-// issues the MMAs; mbarriers form a ring of stages between the three roles.
+// MMA reads only the upper 19 bits of each word.  Warps 0-15 read the tile back, form
+// 2 lo = 2 (x - (x with its low 13 bits cleared)) and write the second tile; lane 0 of warps 16, 17
+// issue the MMAs; mbarriers form a ring of stages between the three roles.
 // Work is cut into K-slabs; at the end of a slab the accumulator is drained to a per-slab fp32
 // partial in global memory and the slabs are added in fp64 in a fixed order afterwards, so the long
 // sum never lives in one fp32 accumulator and the result is deterministic.
@@ -34,7 +34,7 @@ namespace detox {
 namespace {
 
 constexpr int kKB = 32;                      // fp32 columns per K-block: one 128-byte swizzle row
-constexpr int kProdWarps = 8;
+constexpr int kProdWarps = 16;
 constexpr int kProdThreads = kProdWarps * 32;
 constexpr int kMmaWarps = 2;                   // two issuing threads, so one's bookkeeping overlaps the other's MMAs
 constexpr int kTcThreads = kProdThreads + 32 * (kMmaWarps + 1);  // + the MMA warps + the TMA warp
@@ -191,17 +191,27 @@ __device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, i
         : "memory");
 }
 
-__device__ __forceinline__ uint32_t to_tf32(float x) {
-    uint32_t r;
-    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
+// Packed pairs of fp32 (one instruction for two lanes).
+__device__ __forceinline__ uint64_t sub2(uint64_t a, uint64_t b) {
+    uint64_t r;
+    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
     return r;
 }
-
-// What a TF32 MMA sees of x is hi = x with the low 13 mantissa bits cleared; x - hi is exact in fp32.
-// Returns 2 (x - hi) rounded to TF32.
-__device__ __forceinline__ uint32_t lo2_of(float x) {
-    const float hi = __uint_as_float(__float_as_uint(x) & 0xFFFFE000u);
-    return to_tf32(2.0f * (x - hi));
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+    uint64_t r;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+// What a TF32 MMA sees of x is hi = x with the low 13 mantissa bits cleared; x - hi is exact in fp32
+// and so is its double.  (The MMA again reads only the upper 19 bits of 2 lo.)
+__device__ __forceinline__ uint64_t lo2_of(uint64_t x2) {
+    const uint64_t t = sub2(x2, x2 & 0xFFFFE000FFFFE000ull);
+    return add2(t, t);
 }
 
 struct TcSmem {
@@ -214,7 +224,7 @@ struct TcSmem {
     int abort_flag;
 };
 
-// J = 16-byte chunks per transform thread and K-block (m * 8 / 256 rounded up to a power of two)
+// J = 16-byte chunks per transform thread and K-block (m * 8 / 512 rounded up to a power of two)
 template <int J>
 __global__ void __launch_bounds__(kTcThreads, 1)
 gram_tc_kernel(const __grid_constant__ CUtensorMap xmap, int m, int64_t d, int rows_pad, int box_rows, int nhalf,
@@ -264,16 +274,16 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap xmap, int m, int64_t d, int r
     if (warp < kProdWarps) {
         // ------------------------------------------------ transform warps, then epilogue of each slab
         const int nchunks = m * 8;
-        // this thread's chunks are (row, c) = ((tid >> 3) + 32 j, tid & 7) in every K-block
+        // this thread's chunks are (row, c) = ((tid >> 3) + 64 j, tid & 7) in every K-block
         uint32_t off[J];
 #pragma unroll
         for (int j = 0; j < J; ++j) {
-            const int row = (tid >> 3) + 32 * j, c = tid & 7;
+            const int row = (tid >> 3) + (kProdThreads / 8) * j, c = tid & 7;
             off[j] = (uint32_t)(row >> 3) * 1024u + (uint32_t)(row & 7) * 128u + (uint32_t)((c ^ (row & 7)) << 4);
         }
-        float sq[J];
+        uint64_t sq[J];   // packed pair of partial sums of squares per chunk
 #pragma unroll
-        for (int j = 0; j < J; ++j) sq[j] = 0.f;
+        for (int j = 0; j < J; ++j) sq[j] = 0ull;
 
         for (int t = 0; t < total; ++t) {
             const int s = (int)((uint32_t)t % (uint32_t)stages);
@@ -286,10 +296,9 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap xmap, int m, int64_t d, int r
 #pragma unroll
             for (int j = 0; j < J; ++j) {
                 if (tid + j * kProdThreads < nchunks) {
-                    const float4 x = *reinterpret_cast<const float4*>(hi_tile + off[j]);
-                    sq[j] = fmaf(x.x, x.x, fmaf(x.y, x.y, fmaf(x.z, x.z, fmaf(x.w, x.w, sq[j]))));
-                    *reinterpret_cast<uint4*>(lo_tile + off[j]) =
-                        make_uint4(lo2_of(x.x), lo2_of(x.y), lo2_of(x.z), lo2_of(x.w));
+                    const ulonglong2 x = *reinterpret_cast<const ulonglong2*>(hi_tile + off[j]);
+                    sq[j] = fma2(x.x, x.x, fma2(x.y, x.y, sq[j]));
+                    *reinterpret_cast<ulonglong2*>(lo_tile + off[j]) = make_ulonglong2(lo2_of(x.x), lo2_of(x.y));
                 }
             }
             fence_proxy_async_smem();   // make the generic-proxy stores visible to the MMA's reads
@@ -304,23 +313,23 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap xmap, int m, int64_t d, int r
             // ---- end of a slab: exact squared norms (the 8 lanes that share a row add up) ...
 #pragma unroll
             for (int j = 0; j < J; ++j) {
-                float v = sq[j];
+                float v = __uint_as_float((uint32_t)sq[j]) + __uint_as_float((uint32_t)(sq[j] >> 32));
                 v += __shfl_xor_sync(0xffffffffu, v, 1);
                 v += __shfl_xor_sync(0xffffffffu, v, 2);
                 v += __shfl_xor_sync(0xffffffffu, v, 4);
-                const int row = (tid >> 3) + 32 * j;
+                const int row = (tid >> 3) + (kProdThreads / 8) * j;
                 if ((tid & 7) == 0 && row < m) norms[(int64_t)item * m + row] = v;
-                sq[j] = 0.f;
+                sq[j] = 0ull;
             }
-            // ... and the accumulator drain: warp w reads TMEM lanes 32*(w%4)..+31; the two warps that
-            // share a lane quarter take alternate 32-column chunks
+            // ... and the accumulator drain: warp w reads TMEM lanes 32*(w%4)..+31; the warps that share a
+            // lane quarter take 32-column chunks round-robin
             mbar_wait(&sm->accum_full, (uint32_t)(li & 1), abort_flag, status);
             tc_fence_after();
             const int quarter = warp & 3;
             float* out_item = partial + (int64_t)item * m * ncol;
             for (int h = 0; h < nhalf; ++h) {
                 const int row = h * 128 + quarter * 32 + lane;
-                for (int cc = warp >> 2; cc * 32 < ncol; cc += 2) {
+                for (int cc = warp >> 2; cc * 32 < ncol; cc += kProdWarps / 4) {
                     float acc[32];
 #pragma unroll
                     for (int j = 0; j < 32; ++j) acc[j] = 0.f;
@@ -376,7 +385,7 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap xmap, int m, int64_t d, int r
         }
     } else if (lane == 0) {
         // ------------------------------------------------ the MMA threads
-        // ------------------------------------------------ (two of them: warps 8 and 9, lane 0)
+        // ------------------------------------------------ (lane 0 of the two warps after the transform warps)
         const int g = warp - kProdWarps;
         const int n_mma = nhalf == 1 ? 2 * ncol : ncol;
         const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(n_mma >> 3) << 17) | ((128u >> 4) << 24);
@@ -547,10 +556,9 @@ detox_status launch_sqdist_tc(const float* X, int64_t ld, int m, int64_t d, doub
     CUtensorMap xmap;
     detox_status st = make_xmap(&xmap, X, ld, m, d, p.box_rows);
     if (st != DETOX_OK) return st;
-    if (m <= 32) st = launch_tc<1>(p, xmap, m, d, partial, norms, status, s);
-    else if (m <= 64) st = launch_tc<2>(p, xmap, m, d, partial, norms, status, s);
-    else if (m <= 128) st = launch_tc<4>(p, xmap, m, d, partial, norms, status, s);
-    else st = launch_tc<8>(p, xmap, m, d, partial, norms, status, s);
+    if (m <= 64) st = launch_tc<1>(p, xmap, m, d, partial, norms, status, s);
+    else if (m <= 128) st = launch_tc<2>(p, xmap, m, d, partial, norms, status, s);
+    else st = launch_tc<4>(p, xmap, m, d, partial, norms, status, s);
     if (st != DETOX_OK) return st;
     tc_reduce_kernel<<<dim3((unsigned)ceil_div((int64_t)m * m, 256), kReduceChunks), 256, 0, s>>>(
         partial, norms, p.nitems, m, p.ncol, gpart);
