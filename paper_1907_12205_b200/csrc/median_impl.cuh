@@ -1,0 +1,155 @@
+// Register-resident per-coordinate order statistics (shared by the translation units that
+// instantiate the network sizes; see median.cu for the overview).
+#pragma once
+
+#include "common.cuh"
+#include "sortnet.cuh"
+
+namespace detox {
+namespace regselect {
+
+constexpr int kRegThreads = 128;
+
+// Start of the window of `beta` consecutive sorted values that are closest to the median `med`.
+// dist(i) = |v_i - med| in fp32 falls, then rises, along the sorted order.  The window [L, L+beta) is
+// right when the value just above it is not strictly closer than its lowest value; on equal distance
+// the lower value stays.  The predicate below is true exactly for the starts that are too far left.
+template <typename KeyAt>
+__device__ __forceinline__ int window_start(int theta, int beta, float med, KeyAt key_at) {
+    const int h_lo = (theta - 1) >> 1;
+    int L = 0;
+    for (int s = 0; s < theta - beta; ++s) {
+        bool move_right;
+        if (s + beta <= h_lo) {
+            move_right = true;  // the window must reach the middle element
+        } else {
+            const float lo = float_of_key(key_at(s));
+            const float up = float_of_key(key_at(s + beta));
+            move_right = fabsf(up - med) < fabsf(lo - med);
+        }
+        L += move_right ? 1 : 0;
+    }
+    return L;
+}
+
+__host__ __device__ constexpr int reg_threads(int M, int C, bool trim) {
+    // the TRIM variant keeps M * C keys per thread in (static) shared memory
+    return (trim && M * C * kRegThreads * 4 > 48 * 1024) ? kRegThreads / 2 : kRegThreads;
+}
+
+// M = network size, m = rows actually present (M - m even; the gap is filled with lowest / highest keys)
+template <int M, int C, bool TRIM>
+__global__ void __launch_bounds__(reg_threads(M, C, TRIM))
+colselect_reg_kernel(const float* __restrict__ X, int64_t ld, int m, int64_t d, const int32_t* __restrict__ rows,
+                     int beta, float* __restrict__ out) {
+    constexpr int kThreads = reg_threads(M, C, TRIM);
+    const int64_t col0 = ((int64_t)blockIdx.x * kThreads + threadIdx.x) * C;
+    if (col0 >= d) return;
+    const int64_t left = d - col0;
+    const int valid = left >= C ? C : (int)left;
+
+    // Network sizes up to 32 are used with m == M; larger ones may carry padding.
+    constexpr bool kPadded = M > 32;
+    const int pad = kPadded ? (M - m) >> 1 : 0;   // lowest keys added (and as many highest)
+    int32_t key[C][M];
+    // All loads first, with no branch in between, so that they are in flight together; slots beyond m
+    // re-read the last row and are replaced by padding keys afterwards.
+#pragma unroll
+    for (int i = 0; i < M; ++i) {
+        const int ri = kPadded ? (i < m ? i : m - 1) : i;
+        const float* p = X + (int64_t)(rows ? rows[ri] : ri) * ld + col0;
+        if (C == 4 && valid == 4) {
+            uint4 v = ld_stream_u4(p);
+            key[0][i] = (int32_t)v.x;
+            key[1 % C][i] = (int32_t)v.y;
+            key[2 % C][i] = (int32_t)v.z;
+            key[3 % C][i] = (int32_t)v.w;
+        } else if (C == 2 && valid == 2) {
+            uint2 v = __ldcs(reinterpret_cast<const uint2*>(p));
+            key[0][i] = (int32_t)v.x;
+            key[1 % C][i] = (int32_t)v.y;
+        } else {
+#pragma unroll
+            for (int c = 0; c < C; ++c) key[c][i] = c < valid ? (int32_t)ld_stream_u1(p + c) : 0;
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < M; ++i) {
+#pragma unroll
+        for (int c = 0; c < C; ++c) {
+            int32_t k = key_of_bits((uint32_t)key[c][i]);
+            if (kPadded && i >= m) k = (i - m < pad) ? (int32_t)0x80000000 : 0x7fffffff;
+            key[c][i] = k;
+        }
+    }
+
+    __shared__ int32_t sorted[TRIM ? M * C * kThreads : 1];
+    float res[C];
+#pragma unroll
+    for (int c = 0; c < C; ++c) {
+        sort_registers<M>(key[c]);
+        float med;
+        if (M & 1) med = float_of_key(key[c][M / 2]);
+        else med = (float_of_key(key[c][M / 2 > 0 ? M / 2 - 1 : 0]) + float_of_key(key[c][M / 2])) * 0.5f;
+        if (!TRIM) {
+            res[c] = med;
+        } else {
+            // the m real values sit at sorted positions pad .. pad+m-1
+            int32_t* mine = sorted + (size_t)c * M * kThreads + threadIdx.x;
+#pragma unroll
+            for (int i = 0; i < M; ++i) mine[i * kThreads] = key[c][i];
+            const int L = pad + window_start(m, beta, med, [&](int i) { return mine[(i + pad) * kThreads]; });
+            float acc = 0.f;
+#pragma unroll
+            for (int i = 0; i < M; ++i)
+                if (i >= L && i < L + beta) acc += float_of_key(key[c][i]);
+            res[c] = acc / (float)beta;
+        }
+    }
+    if (C == 4 && valid == 4) {
+        st_stream_f4(out + col0, make_float4(res[0], res[1 % C], res[2 % C], res[3 % C]));
+    } else if (C == 2 && valid == 2) {
+        __stcs(reinterpret_cast<float2*>(out + col0), make_float2(res[0], res[1 % C]));
+    } else {
+#pragma unroll
+        for (int c = 0; c < C; ++c)
+            if (c < valid) out[col0 + c] = res[c];
+    }
+}
+
+template <int M, int C>
+detox_status launch_reg(const float* X, int64_t ld, int m, int64_t d, const int32_t* rows, int beta, float* out,
+                        cudaStream_t s) {
+    if (beta == 0) {
+        constexpr int T = reg_threads(M, C, false);
+        int64_t bx = ceil_div(d, (int64_t)T * C);
+        if (bx > 0x7fffffffLL) return DETOX_ERR_UNSUPPORTED;
+        colselect_reg_kernel<M, C, false><<<(unsigned)bx, T, 0, s>>>(X, ld, m, d, rows, beta, out);
+    } else {
+        constexpr int T = reg_threads(M, C, true);
+        int64_t bx = ceil_div(d, (int64_t)T * C);
+        if (bx > 0x7fffffffLL) return DETOX_ERR_UNSUPPORTED;
+        colselect_reg_kernel<M, C, true><<<(unsigned)bx, T, 0, s>>>(X, ld, m, d, rows, beta, out);
+    }
+    return launch_status();
+}
+
+template <int M>
+detox_status launch_reg_m(const float* X, int64_t ld, int m, int64_t d, const int32_t* rows, int beta, float* out,
+                          bool vec, cudaStream_t s) {
+    constexpr int C = M <= 8 ? 4 : (M <= 16 ? 2 : 1);
+    if (vec && C > 1) return launch_reg<M, C>(X, ld, m, d, rows, beta, out, s);
+    return launch_reg<M, 1>(X, ld, m, d, rows, beta, out, s);
+}
+
+}  // namespace regselect
+
+// Instantiated in median_m64.cu / median_m96.cu / median_m128.cu: network sizes 39..64, 79..96, 111..128.
+detox_status launch_reg_upto64(int M, const float* X, int64_t ld, int m, int64_t d, const int32_t* rows, int beta,
+                               float* out, bool vec, cudaStream_t s);
+detox_status launch_reg_upto96(int M, const float* X, int64_t ld, int m, int64_t d, const int32_t* rows, int beta,
+                               float* out, bool vec, cudaStream_t s);
+detox_status launch_reg_upto128(int M, const float* X, int64_t ld, int m, int64_t d, const int32_t* rows, int beta,
+                                float* out, bool vec, cudaStream_t s);
+
+}  // namespace detox

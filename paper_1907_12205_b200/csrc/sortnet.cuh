@@ -1,4 +1,4 @@
-// Compile-time sorting networks for small fixed sizes (Batcher's merge exchange, valid for any length),
+// Compile-time sorting networks for fixed sizes (Batcher's merge exchange, valid for any length),
 // applied to register arrays.  Comparators are emitted one by one with constant indices, so the array
 // never leaves registers and the compiler drops every comparator that cannot reach an output that
 // is actually used (a median needs far fewer than a full sort).
@@ -10,45 +10,50 @@
 
 namespace detox {
 
-struct Comparator {
-    int a, b;
-};
-
+// Number of comparators of the merge-exchange network on M inputs.
 template <int M>
-struct MergeExchange {
-    // Visit the comparators in network order; stop and return the idx-th one (or count them all).
-    __host__ __device__ static constexpr Comparator nth(int idx, int* total) {
+__host__ __device__ constexpr int merge_exchange_count() {
+    int c = 0;
+    for (int p = 1; p < M; p <<= 1)
+        for (int k = p; k >= 1; k >>= 1)
+            for (int j = k % p; j <= M - 1 - k; j += 2 * k) {
+                const int imax = k - 1 < M - j - k - 1 ? k - 1 : M - j - k - 1;
+                for (int i = 0; i <= imax; ++i)
+                    if ((i + j) / (2 * p) == (i + j + k) / (2 * p)) ++c;
+            }
+    return c;
+}
+
+// The comparators (a < b, minimum goes to a) in network order, built once per M at compile time.
+template <int M>
+struct MergeExchangeNet {
+    static constexpr int kCount = merge_exchange_count<M>();
+    int16_t a[kCount > 0 ? kCount : 1];
+    int16_t b[kCount > 0 ? kCount : 1];
+    __host__ __device__ constexpr MergeExchangeNet() : a{}, b{} {
         int c = 0;
-        for (int p = 1; p < M; p <<= 1) {
-            for (int k = p; k >= 1; k >>= 1) {
+        for (int p = 1; p < M; p <<= 1)
+            for (int k = p; k >= 1; k >>= 1)
                 for (int j = k % p; j <= M - 1 - k; j += 2 * k) {
-                    int imax = k - 1 < M - j - k - 1 ? k - 1 : M - j - k - 1;
-                    for (int i = 0; i <= imax; ++i) {
+                    const int imax = k - 1 < M - j - k - 1 ? k - 1 : M - j - k - 1;
+                    for (int i = 0; i <= imax; ++i)
                         if ((i + j) / (2 * p) == (i + j + k) / (2 * p)) {
-                            if (c == idx) return Comparator{i + j, i + j + k};
+                            a[c] = (int16_t)(i + j);
+                            b[c] = (int16_t)(i + j + k);
                             ++c;
                         }
-                    }
                 }
-            }
-        }
-        if (total) *total = c;
-        return Comparator{0, 0};
-    }
-    __host__ __device__ static constexpr int count() {
-        int t = 0;
-        nth(-1, &t);
-        return t;
     }
 };
 
 template <int M, int I>
 __device__ __forceinline__ void compare_exchange(int32_t (&k)[M]) {
-    constexpr Comparator c = MergeExchange<M>::nth(I, nullptr);
-    const int32_t lo = min(k[c.a], k[c.b]);
-    const int32_t hi = max(k[c.a], k[c.b]);
-    k[c.a] = lo;
-    k[c.b] = hi;
+    constexpr MergeExchangeNet<M> net{};
+    constexpr int a = net.a[I], b = net.b[I];
+    const int32_t lo = min(k[a], k[b]);
+    const int32_t hi = max(k[a], k[b]);
+    k[a] = lo;
+    k[b] = hi;
 }
 
 template <int M, int... Is>
@@ -59,7 +64,7 @@ __device__ __forceinline__ void run_network(int32_t (&k)[M], std::integer_sequen
 // Ascending sort of k[0..M-1] (signed compare).
 template <int M>
 __device__ __forceinline__ void sort_registers(int32_t (&k)[M]) {
-    if constexpr (M > 1) run_network<M>(k, std::make_integer_sequence<int, MergeExchange<M>::count()>{});
+    if constexpr (M > 1) run_network<M>(k, std::make_integer_sequence<int, MergeExchangeNet<M>::kCount>{});
 }
 
 }  // namespace detox

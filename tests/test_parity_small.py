@@ -102,7 +102,7 @@ def test_hier_mean_matches_oracle(G, d, offs):
 
 # ---------------------------------------------------------------------------------------- median
 
-@pytest.mark.parametrize("m", list(range(1, 34)) + [45, 64, 75, 105, 128, 225])
+@pytest.mark.parametrize("m", list(range(1, 42)) + [45, 47, 48, 64, 65, 75, 100, 105, 127, 128, 129, 225])
 def test_coord_median_bit_exact(m):
     rng = np.random.default_rng(m)
     d = 3000 + m if m <= 33 else 1000 + m
