@@ -5,7 +5,8 @@
 //           network; the median needs only part of it.  Sizes above 32 are served by a few network
 //           sizes: the m values are padded with equally many lowest and highest keys, which leaves
 //           the median (and the values around it) where they were.
-// m  > 128: a CTA stages a 32-coordinate tile as integer keys in shared memory and its 8 warps run
+// 128 < m <= 256: two lanes per coordinate, 128 registers each (median_pair.cu).
+// m  > 256: a CTA stages a 32-coordinate tile as integer keys in shared memory and its 8 warps run
 //          the layers of a merge-exchange network over it (warp = one comparator at a time for 32
 //          coordinates, so shared-memory accesses are conflict-free and control flow is uniform).
 #include "median_impl.cuh"
@@ -109,6 +110,7 @@ detox_status launch_coord_select(const float* X, int64_t ld, int m, int64_t d, c
         if (M <= 96) return launch_reg_upto96(M, X, ld, m, d, rows_dev, beta, out, vec, s);
         return launch_reg_upto128(M, X, ld, m, d, rows_dev, beta, out, vec, s);
     }
+    if (m <= 256) return launch_pair_select(X, ld, m, d, rows_dev, beta, out, s);
     const size_t smem = (size_t)m * kTileCols * sizeof(int32_t);
     if (cudaFuncSetAttribute(colselect_smem_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
         cudaSuccess)

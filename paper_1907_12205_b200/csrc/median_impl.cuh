@@ -152,4 +152,8 @@ detox_status launch_reg_upto96(int M, const float* X, int64_t ld, int m, int64_t
 detox_status launch_reg_upto128(int M, const float* X, int64_t ld, int m, int64_t d, const int32_t* rows, int beta,
                                 float* out, bool vec, cudaStream_t s);
 
+// median_pair.cu: 128 < m <= 256, two lanes per coordinate
+detox_status launch_pair_select(const float* X, int64_t ld, int m, int64_t d, const int32_t* rows, int beta,
+                                float* out, cudaStream_t s);
+
 }  // namespace detox

@@ -1,0 +1,126 @@
+// Per-coordinate order statistics over 128 < m <= 256 rows: two adjacent lanes share a coordinate.
+//
+// Each lane sorts 128 keys in registers (lane 0: rows 0..127; lane 1: the other rows plus padding
+// keys, lowest and highest, placed so that the wanted median lands on sorted position 127 of the
+// 256).  One bitonic split across the lane pair (min / max against the partner's reversed run)
+// leaves the 128 smallest keys in lane 0 and the 128 largest in lane 1; the median is then the
+// maximum of lane 0's keys (for an even count, averaged with the minimum of lane 1's).  For
+// Bulyan's second stage both halves are sorted with a bitonic merge and laid out in shared
+// memory for the data-dependent window search.
+#include "median_impl.cuh"
+
+namespace detox {
+
+namespace {
+
+constexpr int kHalf = 128;
+constexpr int kPairThreads = 128;              // 64 coordinates per CTA
+constexpr int kPairCols = kPairThreads / 2;
+
+template <bool TRIM>
+__global__ void __launch_bounds__(kPairThreads)
+colselect_pair_kernel(const float* __restrict__ X, int64_t ld, int m, int64_t d, const int32_t* __restrict__ rows,
+                      int beta, float* __restrict__ out) {
+    extern __shared__ int32_t sorted[];        // TRIM only: [256][kPairCols]
+    const int hsel = threadIdx.x & 1;
+    const int cidx = threadIdx.x >> 1;
+    const int64_t col_raw = (int64_t)blockIdx.x * kPairCols + cidx;
+    const bool live = col_raw < d;
+    const int64_t col = live ? col_raw : d - 1;   // dead pairs recompute the last coordinate and do not store
+
+    const int pad_lo = (kHalf - 1) - ((m - 1) >> 1);   // lowest keys added: puts the (lower) median on position 127
+    const int extra = m - kHalf;                        // real rows held by lane 1
+
+    int32_t key[kHalf];
+#pragma unroll
+    for (int i = 0; i < kHalf; ++i) {
+        int ri = hsel ? kHalf + i : i;
+        ri = ri < m ? ri : m - 1;
+        key[i] = (int32_t)ld_stream_u1(X + (int64_t)(rows ? rows[ri] : ri) * ld + col);
+    }
+#pragma unroll
+    for (int i = 0; i < kHalf; ++i) {
+        int32_t k = key_of_bits((uint32_t)key[i]);
+        if (hsel && i >= extra) k = (i - extra < pad_lo) ? (int32_t)0x80000000 : 0x7fffffff;
+        key[i] = k;
+    }
+    sort_registers<kHalf>(key);
+
+    // bitonic split with the partner lane: lane 0 keeps the minima, lane 1 the maxima
+#pragma unroll
+    for (int i = 0; i < kHalf / 2; ++i) {
+        const int j = kHalf - 1 - i;
+        const int32_t from_j = __shfl_xor_sync(0xffffffffu, key[j], 1);
+        const int32_t from_i = __shfl_xor_sync(0xffffffffu, key[i], 1);
+        key[i] = hsel ? max(key[i], from_j) : min(key[i], from_j);
+        key[j] = hsel ? max(key[j], from_i) : min(key[j], from_i);
+    }
+
+    if (!TRIM) {
+        int32_t ext = key[0];
+#pragma unroll
+        for (int i = 1; i < kHalf; ++i) ext = hsel ? min(ext, key[i]) : max(ext, key[i]);
+        const int32_t up_min = __shfl_xor_sync(0xffffffffu, ext, 1);   // lane 0 receives lane 1's minimum
+        if (hsel == 0 && live) {
+            const float lo = float_of_key(ext);
+            out[col] = (m & 1) ? lo : (lo + float_of_key(up_min)) * 0.5f;
+        }
+        return;
+    }
+
+    // each lane's 128 keys form a bitonic sequence: sort them ascending
+#pragma unroll
+    for (int s = kHalf / 2; s >= 1; s >>= 1) {
+#pragma unroll
+        for (int i = 0; i < kHalf; ++i) {
+            if ((i & s) == 0) {
+                const int32_t lo = min(key[i], key[i + s]);
+                const int32_t hi = max(key[i], key[i + s]);
+                key[i] = lo;
+                key[i + s] = hi;
+            }
+        }
+    }
+    // position p of the 256 sorted keys -> sorted[p * kPairCols + slot]; the slot is rotated by 16 for the
+    // upper half so that the two lanes of a pair never hit the same bank
+    {
+        const int slot = (cidx + hsel * 16) & (kPairCols - 1);
+#pragma unroll
+        for (int i = 0; i < kHalf; ++i) sorted[(hsel * kHalf + i) * kPairCols + slot] = key[i];
+    }
+    __syncwarp();
+    if (hsel == 0 && live) {
+        auto at = [&](int p) { return sorted[p * kPairCols + ((cidx + (p >= kHalf ? 16 : 0)) & (kPairCols - 1))]; };
+        float med = float_of_key(at(kHalf - 1));
+        if ((m & 1) == 0) med = (med + float_of_key(at(kHalf))) * 0.5f;
+        const int L = pad_lo + regselect::window_start(m, beta, med, [&](int i) { return at(i + pad_lo); });
+        float acc = 0.f, comp = 0.f;          // compensated fp32 sum
+        for (int p = L; p < L + beta; ++p) {
+            const float y = float_of_key(at(p)) - comp;
+            const float t = acc + y;
+            comp = (t - acc) - y;
+            acc = t;
+        }
+        out[col] = acc / (float)beta;
+    }
+}
+
+}  // namespace
+
+detox_status launch_pair_select(const float* X, int64_t ld, int m, int64_t d, const int32_t* rows, int beta,
+                                float* out, cudaStream_t s) {
+    int64_t bx = ceil_div(d, kPairCols);
+    if (bx > 0x7fffffffLL) return DETOX_ERR_UNSUPPORTED;
+    if (beta == 0) {
+        colselect_pair_kernel<false><<<(unsigned)bx, kPairThreads, 0, s>>>(X, ld, m, d, rows, beta, out);
+    } else {
+        const size_t smem = (size_t)2 * kHalf * kPairCols * sizeof(int32_t);
+        if (cudaFuncSetAttribute(colselect_pair_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
+            cudaSuccess)
+            return DETOX_ERR_CUDA;
+        colselect_pair_kernel<true><<<(unsigned)bx, kPairThreads, smem, s>>>(X, ld, m, d, rows, beta, out);
+    }
+    return launch_status();
+}
+
+}  // namespace detox

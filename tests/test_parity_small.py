@@ -102,7 +102,7 @@ def test_hier_mean_matches_oracle(G, d, offs):
 
 # ---------------------------------------------------------------------------------------- median
 
-@pytest.mark.parametrize("m", list(range(1, 42)) + [45, 47, 48, 64, 65, 75, 100, 105, 127, 128, 129, 225])
+@pytest.mark.parametrize("m", list(range(1, 42)) + [45, 47, 48, 64, 65, 75, 100, 105, 127, 128, 129, 130, 200, 225, 255, 256, 257, 300])
 def test_coord_median_bit_exact(m):
     rng = np.random.default_rng(m)
     d = 3000 + m if m <= 33 else 1000 + m
@@ -174,12 +174,15 @@ def test_multikrum_unaligned_rows():
 
 @pytest.mark.parametrize("m,d,f,copies", [(7, 10_001, 1, 1), (15, 20_000, 3, 1), (15, 4099, 1, 3), (11, 2048, 2, 1),
                                           (27, 3000, 6, 1), (45, 8000, 9, 3), (45, 5000, 4, 1), (64, 2000, 5, 1),
-                                          (105, 1500, 10, 3), (5, 1000, 0, 1), (36, 1200, 1, 1)])
+                                          (105, 1500, 10, 3), (5, 1000, 0, 1), (36, 1200, 1, 1), (150, 1100, 10, 1), (225, 1000, 22, 3),
+                                          (256, 700, 30, 1)])
 def test_bulyan_matches_oracle(m, d, f, copies):
     for attempt in range(16):                        # seeds with a near-tie in some selection round are skipped
         X = krum_inputs(m, d, seed=m * 11 + d + 1000 * attempt, copies=copies, outliers=f)
         out_o, sel_o, D_o = oracle.bulyan(X, f)
-        if bulyan_min_gap(D_o, f) > 1e-4:
+        # many rows mean many successive decisions among closely spaced scores: the screen is relaxed to a
+        # few times the tested score accuracy (2e-6) there
+        if bulyan_min_gap(D_o, f) > (1e-4 if m <= 64 else 5e-6):
             break
     else:
         pytest.fail("no seed without a near-tie")
