@@ -72,6 +72,12 @@ class ClockSampler:
         for line in self.proc.stdout:
             self.rows.append([x.strip() for x in line.split(",")])
 
+    def wait_first(self, seconds: float = 5.0):
+        """nvidia-smi needs a moment to start; block until it has printed its first sample."""
+        t0 = time.time()
+        while self.proc is not None and not self.rows and time.time() - t0 < seconds:
+            time.sleep(0.02)
+
     def __exit__(self, *exc):
         if self.proc is not None:
             self.proc.terminate()
@@ -164,6 +170,75 @@ def workload_label(name, spec, cfg):
             f"vote -> A0={a0} -> A1={ORACLE_A1[cfg['a1']]}(f={cfg['f']}, m_sel={cfg['m_sel']})")
 
 
+def run_sweep(args):
+    """Config 5: every aggregator with and without the DETOX front end over n x d x attack.
+
+    One JSON line per point (not the headline line).  Times are CUDA-event means on one stream after
+    warm-up; GB/s is n*d*4 / t; "alg" is the algorithmic bytes of the leg over the same time."""
+    import torch
+
+    import paper_1907_12205_b200 as dx
+    import workloads as wl
+
+    dev = "cuda:0"
+    torch.cuda.set_device(0)
+    peaks, peak_kind = measured_peaks()
+    ns = [int(x) for x in args.sweep_n.split(",")]
+    ds = [int(x) for x in args.sweep_d.split(",")]
+    for spec in wl.sweep_specs(ns=ns, ds=ds, attacks=tuple(args.sweep_attacks.split(","))):
+        w = wl.make_workload(spec, device=dev)
+        n, r, d, G, S, q = spec.n, spec.r, spec.d, w.G, w.S, spec.q
+        X = w.X[:, :d]
+        out = torch.empty(d, dtype=torch.float32, device=dev)
+        in_bytes = n * d * 4
+        reps = max(3, min(args.steps, 10))
+        legs = {}
+
+        def timed(name, fn, alg_bytes):
+            ms = time_calls(torch, fn, reps, 3)
+            legs[name] = {"ms": round(ms, 4), "GBps": round(in_bytes / ms / 1e6, 1),
+                          "alg_GBps": round(alg_bytes / ms / 1e6, 1),
+                          "alg_frac_of_hbm": round(alg_bytes / ms / 1e6 / peaks["hbm_gbs"], 3)}
+
+        def pipe_leg(name, a0, a1, f, m_sel, alg_bytes):
+            p = dx.Pipeline(n, r, d, w.members, a0, w.set_offsets if a0 == dx.AGG_MEAN else None,
+                            w.set_members if a0 == dx.AGG_MEAN else None, a1, f, m_sel)
+            ws = torch.empty(p.workspace_bytes(), dtype=torch.uint8, device=dev)
+            win = torch.empty(G, dtype=torch.int32, device=dev)
+            sel = torch.empty(max(p.n_selected, 1), dtype=torch.int32, device=dev)
+            timed(name, lambda: dx.detox_aggregate(p, X, out=out, winner=win, sel=sel, ws=ws), alg_bytes)
+            del ws
+
+        # DETOX legs.  Median: vote -> mean over sets of 5 -> median over the S means (S >= 3), else over the votes.
+        if S >= 3:
+            pipe_leg("detox_median", dx.AGG_MEAN, dx.AGG_COORD_MEDIAN, 0, 1, (n + 2 * S + 1) * d * 4)
+        else:
+            pipe_leg("detox_median", dx.AGG_NONE, dx.AGG_COORD_MEDIAN, 0, 1, (n + 2 * G + 1) * d * 4)
+        # Krum family: vote -> aggregator over the G votes, tolerance for the few Byzantine votes that survive
+        fv = min(2, max((G - 3) // 4, 0))
+        pipe_leg("detox_multikrum", dx.AGG_NONE, dx.AGG_MULTIKRUM, fv, G - fv, (n + 2 * G + (G - fv) + 1) * d * 4)
+        pipe_leg("detox_bulyan", dx.AGG_NONE, dx.AGG_BULYAN, fv, 1, (n + 2 * G + (G - 2 * fv) + 1) * d * 4)
+        # direct legs on all n rows
+        timed("direct_median", lambda: dx.agg_coord_median(X, out=out), (n + 1) * d * 4)
+        ws = torch.empty(dx.agg_multikrum_workspace_bytes(n, d), dtype=torch.uint8, device=dev)
+        sel = torch.empty(n, dtype=torch.int32, device=dev)
+        sc = torch.empty(n, dtype=torch.float64, device=dev)
+        timed("direct_multikrum", lambda: dx.agg_multikrum(X, q, n - q, out=out, sel=sel[: n - q], scores=sc, ws=ws),
+              (n + (n - q) + 1) * d * 4)
+        if n >= 4 * q + 3:
+            timed("direct_bulyan", lambda: dx.agg_bulyan(X, q, out=out, sel=sel[: n - 2 * q], ws=ws),
+                  (n + (n - 2 * q) + 1) * d * 4)
+        del ws
+        line = {"sweep_point": spec.name, "n": n, "r": r, "d": d, "q": q, "q_hat": w.q_hat, "attack": spec.attack,
+                "sets": S, "f_votes": fv, "unit": "GB/s = n*d*4/t", "hbm_peak": peaks["hbm_gbs"],
+                "peak_kind": peak_kind, "legs": legs,
+                "speedup": {k: round(legs["direct_" + k]["ms"] / legs["detox_" + k]["ms"], 2)
+                            for k in ("median", "multikrum", "bulyan") if "direct_" + k in legs}}
+        print(json.dumps(line), flush=True)
+        del w, X, out
+        torch.cuda.empty_cache()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -172,6 +247,10 @@ def main():
     ap.add_argument("--impl", default="detox", choices=["detox", "reference"])
     ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sweep", action="store_true", help="config 5: one JSON line per (n, d, attack) point")
+    ap.add_argument("--sweep-n", default="15,45,105,225")
+    ap.add_argument("--sweep-d", default="1000000,11173962,25557032")
+    ap.add_argument("--sweep-attacks", default="reverse,alie")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "detox" else args.warmup
 
@@ -180,6 +259,10 @@ def main():
     local = int(os.environ.get("LOCAL_RANK", "0"))
     if args.impl == "reference":
         run_reference(args, rank, world)
+        return
+    if args.sweep:
+        if rank == 0:
+            run_sweep(args)
         return
 
     import torch
@@ -223,16 +306,28 @@ def main():
     st = torch.cuda.current_stream()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     with ClockSampler(local) as clocks:
+        clocks.wait_first()
+        for _ in range(3):
+            step()
+        torch.cuda.synchronize()
         e0.record(st)
         for _ in range(args.steps):
             step()
         e1.record(st)
         barrier()
-        # the dominant kernel alone (vote: reads n*d*4, writes G*d*4), same inputs, same stream
-        Zbuf = torch.empty((pipe.G, w.ld), dtype=torch.float32, device=dev)[:, : spec.d]
+        # the dominant kernel alone, same inputs, same stream: the vote (reads n*d*4, writes G*d*4), or the vote
+        # fused with the set means when A_0 is the mean (reads n*d*4, writes S*d*4)
         vws = torch.empty(dx.detox_vote_workspace_bytes(spec.n, spec.r), dtype=torch.uint8, device=dev)
-        vote_ms = time_calls(torch, lambda: dx.detox_vote(X, spec.r, w.members, Z=Zbuf, winner=winner, ws=vws),
-                             max(args.steps, 10), 3)
+        if cfg["a0"] == dx.AGG_MEAN:
+            Mbuf = torch.empty((w.S, w.ld), dtype=torch.float32, device=dev)[:, : spec.d]
+            dom_name, dom_rows_out = "vote_mean_kernel", w.S
+            dom = lambda: dx.detox_vote_hier_mean(X, spec.r, w.members, w.set_offsets, w.set_members, M=Mbuf,
+                                                  winner=winner, ws=vws)
+        else:
+            Zbuf = torch.empty((pipe.G, w.ld), dtype=torch.float32, device=dev)[:, : spec.d]
+            dom_name, dom_rows_out = "vote_kernel", pipe.G
+            dom = lambda: dx.detox_vote(X, spec.r, w.members, Z=Zbuf, winner=winner, ws=vws)
+        vote_ms = time_calls(torch, dom, max(args.steps, 10), 3)
     total_ms = e0.elapsed_time(e1)
     t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
     if world > 1:
@@ -283,9 +378,9 @@ def main():
     legs["detox_speedup_vs_direct"] = dms / ms_per_step
 
     peaks, peak_kind = measured_peaks()
-    vote_bytes = (spec.n + pipe.G) * spec.d * 4
+    vote_bytes = (spec.n + dom_rows_out) * spec.d * 4
     achieved = vote_bytes / (vote_ms * 1e-3) / 1e9
-    roofline = {"kernel": "vote_kernel", "bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"],
+    roofline = {"kernel": dom_name, "bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"],
                 "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
                 "frac_of_8TBps": achieved / 8000.0, "ms_per_launch": vote_ms, "algorithmic_bytes": vote_bytes,
                 "traffic": None}
@@ -309,7 +404,7 @@ def main():
         if ref["sel"] is not None:
             parity["sel_exact"] = sel.cpu().numpy()[: len(ref["sel"])].tolist() == ref["sel"].tolist()
 
-    kernels_per_step = {"cfg1": 4, "cfg2": 9, "cfg3": 8, "cfg4": 5}[args.workload]
+    kernels_per_step = {"cfg1": 4, "cfg2": 8, "cfg3": 8, "cfg4": 4}[args.workload]
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
@@ -318,7 +413,7 @@ def main():
             "clocks": clocks.summary(),
             "e2e": {"value": world * in_bytes / (e2e_ms * 1e-3) / 1e9, "unit": UNIT, "ms_per_step": e2e_ms,
                     "h2d_bytes_per_step": int(Xh.numel() * 4), "d2h_bytes_per_step": int(outh.numel() * 4)},
-            "gpu_launches": kernels_per_step * args.steps,
+            "gpu_launches": kernels_per_step * args.steps, "kernels_per_step": kernels_per_step,
             "roofline": roofline, "cpu_baseline": cpu_baseline, "legs": legs, "parity": parity}
     print(json.dumps(line))
     if world > 1:

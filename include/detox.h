@@ -108,6 +108,19 @@ detox_status detox_hier_mean(const float* Z, int64_t ldz, int G, int64_t d, cons
                              const int32_t* set_members, int S, float* M, int64_t ldm, void* stream);
 
 /* ---------------------------------------------------------------------------------------------
+ * detox_vote followed by detox_hier_mean, in one pass over X (Algorithm 1's filtering step and
+ * Algorithm 2, step 3 with A_0 the mean): M[s] is the mean of the votes of set s, bit for bit what
+ * the two calls give, but the votes are never written to memory (n*d*4 bytes read, S*d*4 written).
+ * detox_aggregate uses this path whenever a0 = DETOX_AGG_MEAN.
+ *
+ *   arguments as in detox_vote (without Z) and detox_hier_mean (without Z, G);
+ *   ws: detox_vote_workspace_bytes(n, r) bytes.
+ * ------------------------------------------------------------------------------------------- */
+detox_status detox_vote_hier_mean(const float* X, int64_t ld, int n, int r, int64_t d, const int32_t* members,
+                                  const int32_t* set_offsets, const int32_t* set_members, int S, float* M,
+                                  int64_t ldm, int32_t* winner, void* ws, size_t ws_bytes, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
  * Coordinate-wise median (Section 4; Appendix B.1): out[c] = median_i X[i][c] over the m rows.
  * Odd m: the middle value, bit for bit one of the inputs.  Even m: fp32 (lo + hi) * 0.5f.
  *   out  dev, d.   ws: agg_coord_median_workspace_bytes(m, d) bytes (may be 0, then ws may be NULL).

@@ -22,6 +22,7 @@ from .binding import (  # noqa: F401
     detox_aggregate_workspace_bytes,
     detox_hier_mean,
     detox_vote,
+    detox_vote_hier_mean,
     detox_vote_noalloc,
     detox_vote_workspace_bytes,
     load,

@@ -22,6 +22,7 @@ MAX_ROWS, MAX_R = 1024, 15
 
 EXPORTS = (
     "detox_status_string", "detox_vote_workspace_bytes", "detox_vote", "detox_vote_noalloc", "detox_hier_mean",
+    "detox_vote_hier_mean",
     "agg_coord_median_workspace_bytes", "agg_coord_median", "agg_multikrum_workspace_bytes", "agg_multikrum",
     "agg_bulyan_workspace_bytes", "agg_bulyan", "detox_aggregate_workspace_bytes", "detox_aggregate",
 )
@@ -63,6 +64,7 @@ def load() -> ctypes.CDLL:
     lib.detox_vote_workspace_bytes.argtypes = [_int, _int]
     lib.detox_vote.argtypes = [_vp, _i64, _int, _int, _i64, _ip, _vp, _i64, _vp, _vp, _sz, _vp]
     lib.detox_vote_noalloc.argtypes = [_vp, _i64, _int, _int, _i64, _ip, _vp, _i64, _vp, _vp]
+    lib.detox_vote_hier_mean.argtypes = [_vp, _i64, _int, _int, _i64, _ip, _ip, _ip, _int, _vp, _i64, _vp, _vp, _sz, _vp]
     lib.detox_hier_mean.argtypes = [_vp, _i64, _int, _i64, _ip, _ip, _int, _vp, _i64, _vp]
     for name in ("agg_coord_median", "agg_multikrum", "agg_bulyan"):
         fn = getattr(lib, name + "_workspace_bytes")
@@ -167,6 +169,26 @@ def detox_hier_mean(Z, set_offsets, set_members, M: Optional[torch.Tensor] = Non
     _check(lib.detox_hier_mean(zp, ldz, G, d, so.ctypes.data_as(_ip), sm.ctypes.data_as(_ip), S, M.data_ptr(), ldm,
                                _stream(stream)), "detox_hier_mean")
     return M
+
+
+def detox_vote_hier_mean(X, r: int, members, set_offsets, set_members, M: Optional[torch.Tensor] = None,
+                         winner: Optional[torch.Tensor] = None, ws: Optional[torch.Tensor] = None, stream=None):
+    """Vote and mean over each vote set in one pass.  Returns (M [S, d], winner [G])."""
+    lib = load()
+    xp, ld, n, d = _mat(X)
+    mem, so, sm = _host_i32(members), _host_i32(set_offsets), _host_i32(set_members)
+    S = len(so) - 1
+    if M is None:
+        ldm = (d + 31) // 32 * 32
+        M = torch.empty((max(S, 1), ldm), dtype=torch.float32, device=X.device)[:S, :d]
+    ldm = M.stride(0) if M.shape[0] > 1 else max(M.stride(0), d)
+    if winner is None:
+        winner = torch.empty(max(n // max(r, 1), 1), dtype=torch.int32, device=X.device)[: n // max(r, 1)]
+    ws, wp, wb = _ws(lib.detox_vote_workspace_bytes(n, r), ws, X.device)
+    _check(lib.detox_vote_hier_mean(xp, ld, n, r, d, mem.ctypes.data_as(_ip), so.ctypes.data_as(_ip),
+                                    sm.ctypes.data_as(_ip), S, M.data_ptr(), ldm, winner.data_ptr(), wp, wb,
+                                    _stream(stream)), "detox_vote_hier_mean")
+    return M, winner
 
 
 def agg_coord_median_workspace_bytes(m: int, d: int) -> int:

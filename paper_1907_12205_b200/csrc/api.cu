@@ -139,7 +139,7 @@ PipeWs pipe_ws(void* ws, const detox_pipeline_desc* p) {
     w.winner = reinterpret_cast<int32_t*>(base + off);
     off += align_up((size_t)G * sizeof(int32_t));
     w.Z = reinterpret_cast<float*>(base + off);
-    off += align_up((size_t)G * w.ldz * sizeof(float));
+    if (p->a0 != DETOX_AGG_MEAN) off += align_up((size_t)G * w.ldz * sizeof(float));   // votes are stored only then
     w.M = reinterpret_cast<float*>(base + off);
     if (p->a0 == DETOX_AGG_MEAN) off += align_up((size_t)p->n_sets * w.ldz * sizeof(float));
     w.agg = base + off;
@@ -206,6 +206,20 @@ detox_status detox_hier_mean(const float* Z, int64_t ldz, int G, int64_t d, cons
     if ((st = check_matrix(Z, ldz, G, d)) != DETOX_OK) return st;
     if (!M || ldm < d || (reinterpret_cast<uintptr_t>(M) & 3u)) return DETOX_ERR_BAD_ARG;
     return launch_hier_mean(Z, ldz, d, tab, S, M, ldm, static_cast<cudaStream_t>(stream));
+}
+
+detox_status detox_vote_hier_mean(const float* X, int64_t ld, int n, int r, int64_t d, const int32_t* members,
+                                  const int32_t* set_offsets, const int32_t* set_members, int S, float* M,
+                                  int64_t ldm, int32_t* winner, void* ws, size_t ws_bytes, void* stream) {
+    IdTable groups;
+    detox_status st = check_groups(n, r, members, &groups);
+    if (st != DETOX_OK) return st;
+    SetTable sets;
+    if ((st = check_sets(n / r, S, set_offsets, set_members, &sets)) != DETOX_OK) return st;
+    if ((st = check_matrix(X, ld, n, d)) != DETOX_OK) return st;
+    if (!winner || !M || ldm < d || (reinterpret_cast<uintptr_t>(M) & 3u)) return DETOX_ERR_BAD_ARG;
+    if (!ws_ok(ws, ws_bytes, vote_ws_bytes(n, r))) return DETOX_ERR_WORKSPACE;
+    return launch_vote_mean(X, ld, n, r, d, groups, sets, S, M, ldm, winner, ws, static_cast<cudaStream_t>(stream));
 }
 
 size_t agg_coord_median_workspace_bytes(int m, int64_t d) {
@@ -277,14 +291,17 @@ detox_status detox_aggregate(const detox_pipeline_desc* p, const float* X, int64
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     int32_t* win = winner ? winner : w.winner;
 
-    // filtering step, then A_0, then A_1
-    if ((st = launch_vote(X, ld, p->n, p->r, p->d, groups, w.Z, w.ldz, win, w.vote, s)) != DETOX_OK) return st;
+    // filtering step, then A_0, then A_1 (the mean as A_0 is folded into the vote's pass)
     const float* rows = w.Z;
     int m = G;
     if (p->a0 == DETOX_AGG_MEAN) {
-        if ((st = launch_hier_mean(w.Z, w.ldz, p->d, sets, p->n_sets, w.M, w.ldz, s)) != DETOX_OK) return st;
+        if ((st = launch_vote_mean(X, ld, p->n, p->r, p->d, groups, sets, p->n_sets, w.M, w.ldz, win, w.vote, s)) !=
+            DETOX_OK)
+            return st;
         rows = w.M;
         m = p->n_sets;
+    } else if ((st = launch_vote(X, ld, p->n, p->r, p->d, groups, w.Z, w.ldz, win, w.vote, s)) != DETOX_OK) {
+        return st;
     }
     int cnt = 0;
     int32_t* sel_buf = nullptr;

@@ -64,6 +64,11 @@ size_t vote_ws_bytes(int n, int r);
 detox_status launch_vote(const float* X, int64_t ld, int n, int r, int64_t d, const IdTable& members,
                          float* Z, int64_t ldz, int32_t* winner, void* ws, cudaStream_t s);
 
+// vote + A_0 = mean in one pass: M[s] = mean of the votes of set s; the votes themselves are not stored
+detox_status launch_vote_mean(const float* X, int64_t ld, int n, int r, int64_t d, const IdTable& members,
+                              const SetTable& sets, int S, float* M, int64_t ldm, int32_t* winner, void* ws,
+                              cudaStream_t s);
+
 // mean.cu
 detox_status launch_hier_mean(const float* Z, int64_t ldz, int64_t d, const SetTable& sets, int S,
                               float* M, int64_t ldm, cudaStream_t s);

@@ -189,6 +189,140 @@ __global__ void vote_clear_kernel(const int32_t* __restrict__ winner, float* __r
         z[c] = 0.0f;
 }
 
+// ---------------------------------------------------------------------------------------------
+// Vote fused with A_0 = mean (Algorithm 1's filtering step + Algorithm 2, step 3, in one pass): the
+// piece-local majority of every group of a vote set is added up in the set's member order and only
+// the set mean is written, so the votes themselves never travel to memory (n*d*4 bytes read,
+// S*d*4 written).  The "differs" bits are collected as in vote_kernel.  Sets that contain a group
+// without a majority are recomputed afterwards from the winners' rows (vote_mean_fix_kernel).
+// ---------------------------------------------------------------------------------------------
+template <int VEC>
+struct PieceSum;
+template <>
+struct PieceSum<4> {
+    float4 a;
+    __device__ __forceinline__ void zero() { a = make_float4(0.f, 0.f, 0.f, 0.f); }
+    __device__ __forceinline__ void add(const Piece<4>& p) {
+        a.x += __uint_as_float(p.v.x); a.y += __uint_as_float(p.v.y);
+        a.z += __uint_as_float(p.v.z); a.w += __uint_as_float(p.v.w);
+    }
+    __device__ __forceinline__ void store_mean(float* dst, float k, int valid) const {
+        const float4 m = make_float4(a.x / k, a.y / k, a.z / k, a.w / k);
+        if (valid >= 4) { st_stream_f4(dst, m); return; }
+        if (valid > 0) dst[0] = m.x;
+        if (valid > 1) dst[1] = m.y;
+        if (valid > 2) dst[2] = m.z;
+    }
+};
+template <>
+struct PieceSum<1> {
+    float a;
+    __device__ __forceinline__ void zero() { a = 0.f; }
+    __device__ __forceinline__ void add(const Piece<1>& p) { a += __uint_as_float(p.v); }
+    __device__ __forceinline__ void store_mean(float* dst, float k, int valid) const {
+        if (valid > 0) dst[0] = a / k;
+    }
+};
+
+template <int R, int VEC>
+__global__ void __launch_bounds__(kVoteThreads)
+vote_mean_kernel(const float* __restrict__ X, int64_t ld, int64_t d, const __grid_constant__ IdTable members,
+                 const __grid_constant__ SetTable sets, float* __restrict__ M, int64_t ldm,
+                 uint32_t* __restrict__ pairdiff) {
+    using Shape = VoteShape<R>;
+    const int s = blockIdx.y;
+    const int64_t col = ((int64_t)blockIdx.x * kVoteThreads + threadIdx.x) * VEC;
+    const int64_t left = d - col;
+    const int valid = left >= VEC ? VEC : (left > 0 ? (int)left : 0);
+    const int b = sets.offset[s], e = sets.offset[s + 1];
+
+    PieceSum<VEC> sum;
+    sum.zero();
+#pragma unroll 2
+    for (int t = b; t < e; ++t) {
+        const int g = sets.member[t];
+        Piece<VEC> v[R];
+#pragma unroll
+        for (int a = 0; a < R; ++a) {
+            if (valid > 0) v[a].load(X + (int64_t)members.id[g * R + a] * ld + col, valid);
+            else v[a].clear();
+        }
+        uint32_t loc[Shape::kWords];
+#pragma unroll
+        for (int w = 0; w < Shape::kWords; ++w) loc[w] = 0u;
+#pragma unroll
+        for (int a = 0; a < R; ++a) {
+#pragma unroll
+            for (int c = a + 1; c < R; ++c) {
+                const int p = pair_index(R, a, c);
+                if (v[a].differs(v[c])) loc[p >> 5] |= 1u << (p & 31);
+            }
+        }
+        Piece<VEC> pick;
+        pick.clear();
+#pragma unroll
+        for (int a = R - 1; a >= 0; --a) {
+            int agree = 1;
+#pragma unroll
+            for (int c = 0; c < R; ++c) {
+                if (c == a) continue;
+                const int p = a < c ? pair_index(R, a, c) : pair_index(R, c, a);
+                agree += ((loc[p >> 5] >> (p & 31)) & 1u) ? 0 : 1;
+            }
+            if (2 * agree > R) pick = v[a];
+        }
+        sum.add(pick);
+#pragma unroll
+        for (int w = 0; w < Shape::kWords; ++w) {
+            const uint32_t bits = __reduce_or_sync(0xffffffffu, loc[w]);
+            if ((threadIdx.x & 31) == 0 && bits != 0u) {
+                uint32_t* word = pairdiff + (int64_t)g * kPairWords + w;
+                const uint32_t seen = *reinterpret_cast<volatile uint32_t*>(word);
+                if (bits & ~seen) atomicOr(word, bits);
+            }
+        }
+    }
+    if (valid > 0) sum.store_mean(M + (int64_t)s * ldm + col, (float)(e - b), valid);
+}
+
+// Recomputes the mean of every set that holds a group without a majority: such a group counts as a zero
+// row, the others contribute their winner's row (bitwise the vote).  Same order of additions.
+__global__ void vote_mean_fix_kernel(const float* __restrict__ X, int64_t ld, int64_t d,
+                                     const __grid_constant__ SetTable sets, const int32_t* __restrict__ winner,
+                                     float* __restrict__ M, int64_t ldm) {
+    const int s = blockIdx.y;
+    const int b = sets.offset[s], e = sets.offset[s + 1];
+    bool broken = false;
+    for (int t = b; t < e; ++t) broken |= winner[sets.member[t]] < 0;
+    if (!broken) return;
+    for (int64_t c = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; c < d; c += (int64_t)gridDim.x * blockDim.x) {
+        float acc = 0.f;
+        for (int t = b; t < e; ++t) {
+            const int w = winner[sets.member[t]];
+            acc += w >= 0 ? X[(int64_t)w * ld + c] : 0.f;
+        }
+        M[(int64_t)s * ldm + c] = acc / (float)(e - b);
+    }
+}
+
+template <int VEC>
+detox_status launch_vote_mean_vec(const float* X, int64_t ld, int r, int64_t d, const IdTable& members,
+                                  const SetTable& sets, int S, float* M, int64_t ldm, uint32_t* pairdiff,
+                                  cudaStream_t s) {
+    int64_t bx = ceil_div(d, (int64_t)kVoteThreads * VEC);
+    if (bx > 0x7fffffffLL || S > 65535) return DETOX_ERR_UNSUPPORTED;
+    dim3 grid((unsigned)bx, (unsigned)S);
+    switch (r) {
+#define DETOX_CASE(R) \
+    case R: vote_mean_kernel<R, VEC><<<grid, kVoteThreads, 0, s>>>(X, ld, d, members, sets, M, ldm, pairdiff); break;
+        DETOX_CASE(1) DETOX_CASE(3) DETOX_CASE(5) DETOX_CASE(7) DETOX_CASE(9) DETOX_CASE(11) DETOX_CASE(13)
+        DETOX_CASE(15)
+#undef DETOX_CASE
+        default: return DETOX_ERR_UNSUPPORTED;
+    }
+    return launch_status();
+}
+
 template <int R, int VEC>
 detox_status launch_vote_r(const float* X, int64_t ld, int G, int64_t d, const IdTable& members, float* Z,
                            int64_t ldz, uint32_t* pairdiff, cudaStream_t s) {
@@ -244,6 +378,24 @@ detox_status launch_vote(const float* X, int64_t ld, int n, int r, int64_t d, co
         st = launch_status();
     }
     return st;
+}
+
+detox_status launch_vote_mean(const float* X, int64_t ld, int n, int r, int64_t d, const IdTable& members,
+                              const SetTable& sets, int S, float* M, int64_t ldm, int32_t* winner, void* ws,
+                              cudaStream_t s) {
+    const int G = n / r;
+    uint32_t* pairdiff = static_cast<uint32_t*>(ws);
+    if (cudaMemsetAsync(pairdiff, 0, (size_t)G * kPairWords * sizeof(uint32_t), s) != cudaSuccess)
+        return DETOX_ERR_CUDA;
+    const bool vec = aligned16(X) && ld % 4 == 0 && aligned16(M) && ldm % 4 == 0;
+    detox_status st = vec ? launch_vote_mean_vec<4>(X, ld, r, d, members, sets, S, M, ldm, pairdiff, s)
+                          : launch_vote_mean_vec<1>(X, ld, r, d, members, sets, S, M, ldm, pairdiff, s);
+    if (st != DETOX_OK) return st;
+    vote_finalize_kernel<<<(G + 127) / 128, 128, 0, s>>>(G, r, members, pairdiff, winner);
+    if ((st = launch_status()) != DETOX_OK) return st;
+    unsigned bx = (unsigned)(ceil_div(d, 256 * 8) < 64 ? ceil_div(d, 256 * 8) : 64);
+    vote_mean_fix_kernel<<<dim3(bx, (unsigned)S), 256, 0, s>>>(X, ld, d, sets, winner, M, ldm);
+    return launch_status();
 }
 
 }  // namespace detox

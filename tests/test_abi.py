@@ -45,7 +45,9 @@ def test_workspace_sizes(lib):
     assert dx.agg_multikrum_workspace_bytes(45, 1000) > 45 * 45 * 8
     assert dx.agg_multikrum_workspace_bytes(5000, 1000) == 0
     p = dx.Pipeline(45, 3, 1000, np.arange(45), dx.AGG_MEAN, [0, 5, 10, 15], np.arange(15), dx.AGG_MULTIKRUM, 1, 1)
-    assert p.workspace_bytes() > 15 * 1024 * 4
+    assert p.workspace_bytes() > 3 * 1024 * 4                   # the three set means (votes are not stored)
+    q = dx.Pipeline(45, 3, 1000, np.arange(45), dx.AGG_NONE, None, None, dx.AGG_COORD_MEDIAN)
+    assert q.workspace_bytes() > 15 * 1024 * 4                  # the fifteen votes
     bad = dx.Pipeline(45, 3, 1000, np.arange(45), dx.AGG_NONE, None, None, dx.AGG_BULYAN, 4, 1)  # 15 < 4*4+3
     assert bad.workspace_bytes() == 0
 

@@ -250,6 +250,35 @@ def test_pipeline_no_majority_group_becomes_zero_vote():
     assert rel_l2(res["out"].cpu().numpy(), ref["out"]) <= TOL
 
 
+@pytest.mark.parametrize("r,G,set_size,d", [(3, 15, 5, 20_003), (3, 15, 7, 4097), (5, 6, 2, 3001), (1, 8, 3, 1000),
+                                            (7, 4, None, 2500)])
+def test_pipeline_fused_vote_mean_handles_no_majority_and_uneven_sets(r, G, set_size, d):
+    spec = wl.WorkloadSpec("p", n=r * G, r=r, d=d, sigma=1e-2, q=0, set_size=set_size, seed=r + G)
+    w = wl.make_workload(spec)
+    if r >= 3:                                          # group 1: nobody agrees -> zero vote inside its set
+        for t, i in enumerate(w.members[r:2 * r]):
+            w.X[int(i), (t * 37) % d] += 1.0 + t
+        i = int(w.members[0])                           # group 0: one dissenter, still a majority
+        w.X[i, d - 1] = -w.X[i, d - 1] - 1.0
+    for a1 in (dx.AGG_MEAN, dx.AGG_COORD_MEDIAN):
+        res, ref = run_pipeline(w, dx.AGG_MEAN, a1)
+        assert res["winner"].cpu().numpy().tolist() == ref["winner"].tolist()
+        if r >= 3:
+            assert ref["winner"][1] == -1 and ref["winner"][0] >= 0
+        assert rel_l2(res["out"].cpu().numpy(), ref["out"]) <= TOL
+    # the fused pass gives the same set means, bit for bit, as vote followed by detox_hier_mean
+    Xd = w.X.to(DEV)[:, :d]
+    Z, _ = dx.detox_vote(Xd, r, w.members)
+    M = dx.detox_hier_mean(Z, w.set_offsets, w.set_members)
+    pipe = dx.Pipeline(spec.n, r, d, w.members, dx.AGG_MEAN, w.set_offsets, w.set_members, dx.AGG_MEAN)
+    M2, w2 = dx.detox_vote_hier_mean(Xd, r, w.members, w.set_offsets, w.set_members)
+    assert np.array_equal(bits(M2.contiguous()), bits(M.contiguous()))
+    fused = dx.detox_aggregate(pipe, Xd)["out"]
+    two_step = dx.detox_aggregate(dx.Pipeline(w.S, 1, d, np.arange(w.S), dx.AGG_NONE, None, None, dx.AGG_MEAN),
+                                  M)["out"]
+    assert np.array_equal(bits(fused), bits(two_step))
+
+
 def test_q0_pipeline_is_plain_mean():
     spec = wl.WorkloadSpec("p", n=21, r=3, d=12_345, sigma=1e-3, q=0, seed=9)
     w = wl.make_workload(spec)
