@@ -5,7 +5,7 @@
 //           network; the median needs only part of it.  Sizes above 32 are served by a few network
 //           sizes: the m values are padded with equally many lowest and highest keys, which leaves
 //           the median (and the values around it) where they were.
-// 128 < m <= 256: two lanes per coordinate, 128 registers each (median_pair.cu).
+// 128 < m <= 256: two lanes per coordinate, up to 128 registers of keys each (median_pair.cu).
 // m  > 256: a CTA stages a 32-coordinate tile as integer keys in shared memory and its 8 warps run
 //          the layers of a merge-exchange network over it (warp = one comparator at a time for 32
 //          coordinates, so shared-memory accesses are conflict-free and control flow is uniform).

@@ -1,27 +1,27 @@
-// Per-coordinate order statistics over 128 < m <= 256 rows: two adjacent lanes share a coordinate.
+// Per-coordinate order statistics with two adjacent lanes per coordinate (128 < m <= 256 rows).
 //
-// Each lane sorts 128 keys in registers (lane 0: rows 0..127; lane 1: the other rows plus padding
-// keys, lowest and highest, placed so that the wanted median lands on sorted position 127 of the
-// 256).  One bitonic split across the lane pair (min / max against the partner's reversed run)
-// leaves the 128 smallest keys in lane 0 and the 128 largest in lane 1; the median is then the
-// maximum of lane 0's keys (for an even count, averaged with the minimum of lane 1's).  For
-// Bulyan's second stage both halves are sorted with a bitonic merge and laid out in shared
-// memory for the data-dependent window search.
+// Each lane sorts H keys in registers (lane 0: rows 0..H-1; lane 1: the other rows plus padding
+// keys, lowest and highest, placed so that the wanted median lands on sorted position H-1 of the
+// 2H).  One bitonic split across the lane pair (min / max against the partner's reversed run)
+// leaves the H smallest keys in lane 0 and the H largest in lane 1; the median is then the
+// maximum of lane 0's keys (for an even count, averaged with the minimum of lane 1's).  Sorting
+// two halves and splitting costs about half the comparators of one network over all m values.
+// For Bulyan's second stage (H a power of two) both halves are sorted with a bitonic merge and
+// laid out in shared memory for the data-dependent window search.
 #include "median_impl.cuh"
 
 namespace detox {
 
 namespace {
 
-constexpr int kHalf = 128;
 constexpr int kPairThreads = 128;              // 64 coordinates per CTA
 constexpr int kPairCols = kPairThreads / 2;
 
-template <bool TRIM>
+template <int kHalf, bool TRIM>
 __global__ void __launch_bounds__(kPairThreads)
 colselect_pair_kernel(const float* __restrict__ X, int64_t ld, int m, int64_t d, const int32_t* __restrict__ rows,
                       int beta, float* __restrict__ out) {
-    extern __shared__ int32_t sorted[];        // TRIM only: [256][kPairCols]
+    extern __shared__ int32_t sorted[];        // TRIM only: [2 * kHalf][kPairCols]
     const int hsel = threadIdx.x & 1;
     const int cidx = threadIdx.x >> 1;
     const int64_t col_raw = (int64_t)blockIdx.x * kPairCols + cidx;
@@ -105,22 +105,40 @@ colselect_pair_kernel(const float* __restrict__ X, int64_t ld, int m, int64_t d,
     }
 }
 
-}  // namespace
 
-detox_status launch_pair_select(const float* X, int64_t ld, int m, int64_t d, const int32_t* rows, int beta,
-                                float* out, cudaStream_t s) {
+template <int H>
+detox_status launch_pair(const float* X, int64_t ld, int m, int64_t d, const int32_t* rows, int beta, float* out,
+                         cudaStream_t s) {
     int64_t bx = ceil_div(d, kPairCols);
     if (bx > 0x7fffffffLL) return DETOX_ERR_UNSUPPORTED;
     if (beta == 0) {
-        colselect_pair_kernel<false><<<(unsigned)bx, kPairThreads, 0, s>>>(X, ld, m, d, rows, beta, out);
-    } else {
-        const size_t smem = (size_t)2 * kHalf * kPairCols * sizeof(int32_t);
-        if (cudaFuncSetAttribute(colselect_pair_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
-            cudaSuccess)
+        colselect_pair_kernel<H, false><<<(unsigned)bx, kPairThreads, 0, s>>>(X, ld, m, d, rows, beta, out);
+    } else if constexpr ((H & (H - 1)) == 0) {
+        const size_t smem = (size_t)2 * H * kPairCols * sizeof(int32_t);
+        if (cudaFuncSetAttribute(colselect_pair_kernel<H, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)smem) != cudaSuccess)
             return DETOX_ERR_CUDA;
-        colselect_pair_kernel<true><<<(unsigned)bx, kPairThreads, smem, s>>>(X, ld, m, d, rows, beta, out);
+        colselect_pair_kernel<H, true><<<(unsigned)bx, kPairThreads, smem, s>>>(X, ld, m, d, rows, beta, out);
+    } else {
+        return DETOX_ERR_UNSUPPORTED;
     }
     return launch_status();
+}
+
+}  // namespace
+
+// 128 < m <= 256.  Median: H = half of m rounded up to 8; Bulyan stage 2: H = 128 (a power of two).
+detox_status launch_pair_select(const float* X, int64_t ld, int m, int64_t d, const int32_t* rows, int beta,
+                                float* out, cudaStream_t s) {
+    int H = ((m + 1) / 2 + 7) / 8 * 8;
+    if (beta > 0) H = 128;
+    switch (H) {
+#define DETOX_CASE(HH) \
+    case HH: return launch_pair<HH>(X, ld, m, d, rows, beta, out, s);
+        DETOX_CASE(72) DETOX_CASE(80) DETOX_CASE(88) DETOX_CASE(96) DETOX_CASE(104) DETOX_CASE(112) DETOX_CASE(120) DETOX_CASE(128)
+#undef DETOX_CASE
+        default: return DETOX_ERR_UNSUPPORTED;
+    }
 }
 
 }  // namespace detox

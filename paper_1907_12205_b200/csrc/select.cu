@@ -5,8 +5,13 @@
 //   stored in ascending order together with their column indices.
 // Multi-Krum: score_i = sum of the first nb entries of row i's ascending list, added in that order;
 //   the m_sel smallest scores win (ties: lower index).
-// Bulyan: theta rounds in one CTA; each round sums, per remaining row, the first nb entries of its list
-//   that are still remaining, takes the argmin (ties: lower index) and removes it.
+// Bulyan: theta rounds in one CTA, one thread per row.  A row's score is the sum of its nb closest
+//   remaining rows, i.e. of the remaining entries of its ascending list up to a pointer.  Removing the
+//   round's winner changes every other row's sum by one entry at most (the winner's distance leaves
+//   if it was counted; the farthest counted entry leaves when nb shrinks), so each round costs O(1)
+//   per row instead of a walk over the list (the last few rounds, with at most 8 neighbours, re-add
+//   them from scratch so that exact ties stay exact).  Bitwise-equal rows see the same values in the same
+//   order, so their scores stay bitwise equal and ties keep going to the lower index.
 #include <math_constants.h>
 
 #include "common.cuh"
@@ -15,9 +20,12 @@ namespace detox {
 
 namespace {
 
+constexpr int kFreshSumBelow = 8;   // Bulyan rounds with at most this many neighbours re-add them from scratch
+
 struct SelectWs {
     double* sorted_d;    // m x m, row i ascending, self at the end (+inf)
     int32_t* sorted_j;   // m x m, matching column indices
+    int32_t* pos_t;      // m x m, pos_t[j][i] = position of column j in row i's list
     double* score;       // m
 };
 
@@ -28,12 +36,15 @@ SelectWs carve(void* ws, int m) {
     p += align_up((size_t)m * m * sizeof(double));
     w.sorted_j = reinterpret_cast<int32_t*>(p);
     p += align_up((size_t)m * m * sizeof(int32_t));
+    w.pos_t = reinterpret_cast<int32_t*>(p);
+    p += align_up((size_t)m * m * sizeof(int32_t));
     w.score = reinterpret_cast<double*>(p);
     return w;
 }
 
 __global__ void __launch_bounds__(256)
-rank_rows_kernel(const double* __restrict__ D, int m, double* __restrict__ sorted_d, int32_t* __restrict__ sorted_j) {
+rank_rows_kernel(const double* __restrict__ D, int m, double* __restrict__ sorted_d, int32_t* __restrict__ sorted_j,
+                 int32_t* __restrict__ pos_t) {
     extern __shared__ double rowv[];  // m
     const int i = blockIdx.x;
     for (int j = threadIdx.x; j < m; j += blockDim.x) rowv[j] = (j == i) ? CUDART_INF : D[(int64_t)i * m + j];
@@ -53,6 +64,7 @@ rank_rows_kernel(const double* __restrict__ D, int m, double* __restrict__ sorte
         }
         sorted_d[(int64_t)i * m + rank] = rowv[j];
         sorted_j[(int64_t)i * m + rank] = j;
+        pos_t[(int64_t)j * m + i] = rank;
     }
 }
 
@@ -93,35 +105,33 @@ multikrum_select_kernel(const double* __restrict__ sorted_d, int m, int f, int m
 }
 
 __global__ void __launch_bounds__(1024)
-bulyan_select_kernel(const double* __restrict__ sorted_d, const int32_t* __restrict__ sorted_j, int m, int f,
-                     int32_t* __restrict__ sel) {
+bulyan_select_kernel(const double* __restrict__ sorted_d, const int32_t* __restrict__ sorted_j,
+                     const int32_t* __restrict__ pos_t, int m, int f, int32_t* __restrict__ sel) {
     __shared__ unsigned char alive[kMaxRows];
     __shared__ double best_s[32];
     __shared__ int best_i[32];
     __shared__ int picked;
     const int i = threadIdx.x;
     const int lane = i & 31, warp = i >> 5;
-    if (i < kMaxRows) alive[i] = i < m ? 1 : 0;
+    const bool mine = i < m;
+    if (i < kMaxRows) alive[i] = mine ? 1 : 0;
+    const double* dist = sorted_d + (int64_t)i * m;   // row i's other rows, closest first (self last)
+    const int32_t* col = sorted_j + (int64_t)i * m;
+
+    // round 0: the nb closest rows, added in ascending order
+    int nb = krum_neighbours(m, f);
+    int last = nb - 1;        // position of the farthest counted entry; every remaining entry up to it is counted
+    int counted = nb;
+    double sum = 0.0;
+    if (mine)
+        for (int k = 0; k < nb; ++k) sum += dist[k];
     __syncthreads();
+
     const int theta = m - 2 * f;
     for (int round = 0; round < theta; ++round) {
-        const int remaining = m - round;
-        const int nb = krum_neighbours(remaining, f);
-        double s = CUDART_INF;
-        int idx = 0x7fffffff;
-        if (i < m && alive[i]) {
-            s = 0.0;
-            int taken = 0;
-            for (int k = 0; k < m - 1 && taken < nb; ++k) {
-                const int j = sorted_j[(int64_t)i * m + k];
-                if (alive[j]) {
-                    s += sorted_d[(int64_t)i * m + k];
-                    ++taken;
-                }
-            }
-            idx = i;
-        }
-        // argmin over (score, index)
+        // argmin over (score, index) among the remaining rows
+        double s = (mine && alive[i]) ? sum : CUDART_INF;
+        int idx = (mine && alive[i]) ? i : 0x7fffffff;
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) {
             const double s2 = __shfl_down_sync(0xffffffffu, s, o);
@@ -146,8 +156,49 @@ bulyan_select_kernel(const double* __restrict__ sorted_d, const int32_t* __restr
             }
         }
         __syncthreads();
+        const int gone = picked;
+        const int remaining = m - round - 1;
+        const int nb_next = remaining >= 1 ? krum_neighbours(remaining, f) : 0;
+        if (mine && alive[i] && remaining >= 1) {
+            // the removed row leaves the sum if it was counted
+            const int q = pos_t[(int64_t)gone * m + i];
+            if (q <= last) {
+                sum -= dist[q];
+                --counted;
+                if (q == last) {
+                    do { --last; } while (last >= 0 && !alive[col[last]]);
+                }
+            }
+            // then the count follows nb: drop the farthest counted entry, or take the next remaining one
+            while (counted > nb_next) {
+                sum -= dist[last];
+                --counted;
+                do { --last; } while (last >= 0 && !alive[col[last]]);
+            }
+            while (counted < nb_next) {
+                do { ++last; } while (last < m - 1 && !alive[col[last]]);
+                sum += dist[last];
+                ++counted;
+            }
+            if (counted == 0) sum = 0.0;
+            // Few neighbours left: add them afresh in ascending order.  With one neighbour two mutually
+            // closest rows must tie exactly (their score is the same distance), which running
+            // subtractions would blur in the last bit.
+            if (nb_next <= kFreshSumBelow) {
+                sum = 0.0;
+                int seen = 0;
+                for (int k = 0; seen < nb_next && k < m - 1; ++k) {
+                    if (alive[col[k]]) {
+                        sum += dist[k];
+                        ++seen;
+                    }
+                }
+            }
+        }
+        nb = nb_next;
+        __syncthreads();
     }
-    (void)picked;
+    (void)nb;
 }
 
 __global__ void map_indices_kernel(const int32_t* __restrict__ idx, const int32_t* __restrict__ map, int cnt,
@@ -161,14 +212,14 @@ int round_up_warp(int m) { return (m + 31) / 32 * 32; }
 }  // namespace
 
 size_t select_ws_bytes(int m) {
-    return align_up((size_t)m * m * sizeof(double)) + align_up((size_t)m * m * sizeof(int32_t)) +
+    return align_up((size_t)m * m * sizeof(double)) + 2 * align_up((size_t)m * m * sizeof(int32_t)) +
            align_up((size_t)m * sizeof(double));
 }
 
 detox_status launch_multikrum_select(const double* D, int m, int f, int m_sel, int32_t* sel_dev, double* scores_dev,
                                      void* ws, cudaStream_t s) {
     SelectWs w = carve(ws, m);
-    rank_rows_kernel<<<m, 256, (size_t)m * sizeof(double), s>>>(D, m, w.sorted_d, w.sorted_j);
+    rank_rows_kernel<<<m, 256, (size_t)m * sizeof(double), s>>>(D, m, w.sorted_d, w.sorted_j, w.pos_t);
     detox_status st = launch_status();
     if (st != DETOX_OK) return st;
     multikrum_select_kernel<<<1, round_up_warp(m), 0, s>>>(w.sorted_d, m, f, m_sel, sel_dev, scores_dev);
@@ -177,10 +228,10 @@ detox_status launch_multikrum_select(const double* D, int m, int f, int m_sel, i
 
 detox_status launch_bulyan_select(const double* D, int m, int f, int32_t* sel_dev, void* ws, cudaStream_t s) {
     SelectWs w = carve(ws, m);
-    rank_rows_kernel<<<m, 256, (size_t)m * sizeof(double), s>>>(D, m, w.sorted_d, w.sorted_j);
+    rank_rows_kernel<<<m, 256, (size_t)m * sizeof(double), s>>>(D, m, w.sorted_d, w.sorted_j, w.pos_t);
     detox_status st = launch_status();
     if (st != DETOX_OK) return st;
-    bulyan_select_kernel<<<1, round_up_warp(m), 0, s>>>(w.sorted_d, w.sorted_j, m, f, sel_dev);
+    bulyan_select_kernel<<<1, round_up_warp(m), 0, s>>>(w.sorted_d, w.sorted_j, w.pos_t, m, f, sel_dev);
     return launch_status();
 }
 
