@@ -128,6 +128,22 @@ def time_calls(torch, fn, steps, warmup):
     return e0.elapsed_time(e1) / steps
 
 
+def max_over_ranks(ms: float, device=None) -> float:
+    """The step time of a multi-rank run is the slowest rank's (all ranks start and stop at a barrier)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(ms)
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(bytes_per_rank: int, world: int, ms_per_step: float) -> float:
+    """Replicas: every rank aggregates its own workload, so the job's throughput is the sum over ranks (GB/s)."""
+    return world * bytes_per_rank / (ms_per_step * 1e-3) / 1e9
+
+
 def oracle_step(w, cfg, X_host):
     import oracle
     s = w.spec
@@ -328,13 +344,9 @@ def main():
             dom_name, dom_rows_out = "vote_kernel", pipe.G
             dom = lambda: dx.detox_vote(X, spec.r, w.members, Z=Zbuf, winner=winner, ws=vws)
         vote_ms = time_calls(torch, dom, max(args.steps, 10), 3)
-    total_ms = e0.elapsed_time(e1)
-    t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_per_step = float(t.item()) / args.steps
+    ms_per_step = max_over_ranks(e0.elapsed_time(e1), dev) / args.steps
     in_bytes = spec.n * spec.d * 4
-    value = world * in_bytes / (ms_per_step * 1e-3) / 1e9
+    value = whole_job_value(in_bytes, world, ms_per_step)
 
     # ---- end to end: pinned host input -> device, aggregate, result -> pinned host ----
     Xh = torch.empty((spec.n, w.ld), dtype=torch.float32, pin_memory=True)
@@ -349,11 +361,7 @@ def main():
 
     e2e_steps = max(2, min(args.steps, 5))
     barrier()
-    e2e_ms = time_calls(torch, e2e_step, e2e_steps, 1)
-    t = torch.tensor([e2e_ms], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    e2e_ms = float(t.item())
+    e2e_ms = max_over_ranks(time_calls(torch, e2e_step, e2e_steps, 1), dev)
 
     if rank != 0:
         if world > 1:
@@ -411,7 +419,7 @@ def main():
             "config": {"workload": workload_label(args.workload, spec, cfg), "l2": "inputs larger than L2"
                        if in_bytes > 2 * 126e6 else "inputs fit in L2 (warm)", "replicas": world},
             "clocks": clocks.summary(),
-            "e2e": {"value": world * in_bytes / (e2e_ms * 1e-3) / 1e9, "unit": UNIT, "ms_per_step": e2e_ms,
+            "e2e": {"value": whole_job_value(in_bytes, world, e2e_ms), "unit": UNIT, "ms_per_step": e2e_ms,
                     "h2d_bytes_per_step": int(Xh.numel() * 4), "d2h_bytes_per_step": int(outh.numel() * 4)},
             "gpu_launches": kernels_per_step * args.steps, "kernels_per_step": kernels_per_step,
             "roofline": roofline, "cpu_baseline": cpu_baseline, "legs": legs, "parity": parity}

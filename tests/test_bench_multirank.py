@@ -1,0 +1,50 @@
+"""The N > 1 path of bench.py on CPU: two gloo ranks, max-over-ranks timing and whole-job throughput.
+(The aggregation path has no exchange step, so ranks are independent replicas; only the reporting is shared.)"""
+import os
+import socket
+import sys
+
+import torch.multiprocessing as mp
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _free_port():
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def _worker(rank, world, port, q):
+    sys.path.insert(0, ROOT)
+    import torch.distributed as dist
+
+    import bench
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    ms = bench.max_over_ranks(10.0 + 5.0 * rank)          # rank 1 is the slower one
+    dist.barrier()
+    q.put((rank, ms, bench.whole_job_value(2_000_000_000, world, ms)))
+    dist.destroy_process_group()
+
+
+def test_two_ranks_report_the_slowest_time_and_the_summed_throughput():
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    port = _free_port()
+    procs = [ctx.Process(target=_worker, args=(r, 2, port, q)) for r in range(2)]
+    for p in procs:
+        p.start()
+    got = sorted(q.get(timeout=120) for _ in procs)
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    assert [g[1] for g in got] == [15.0, 15.0]
+    assert abs(got[0][2] - 2 * 2e9 / 15e-3 / 1e9) < 1e-9
+
+
+def test_single_process_is_passthrough():
+    sys.path.insert(0, ROOT)
+    import bench
+    assert bench.max_over_ranks(3.5) == 3.5
+    assert abs(bench.whole_job_value(10**9, 1, 1.0) - 1000.0) < 1e-9
