@@ -285,14 +285,16 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap xmap, int m, int64_t d, int r
 #pragma unroll
         for (int j = 0; j < J; ++j) sq[j] = 0ull;
 
+        // m <= 128: the 2lo rows follow the hi rows at row `ncol` of the same tile (ncol % 8 == 0);
+        // m  > 128: they form a tile of their own
+        const uint32_t lo_off = nhalf == 1 ? (uint32_t)ncol * 128u : tile_bytes;
+        // stage / phase / slab position are carried along instead of divided out every K-block
+        int s = 0, li = 0, kb = 0;
+        uint32_t ph = 0;
         for (int t = 0; t < total; ++t) {
-            const int s = (int)((uint32_t)t % (uint32_t)stages);
-            const uint32_t ph = ((uint32_t)t / (uint32_t)stages) & 1u;
             mbar_wait(&sm->landed[s], ph, abort_flag, status);
             const uint8_t* hi_tile = base + (size_t)s * stage_bytes;
-            // m <= 128: the 2lo rows follow the hi rows at row `ncol` of the same tile (ncol % 8 == 0);
-            // m  > 128: they form a tile of their own
-            uint8_t* lo_tile = base + (size_t)s * stage_bytes + (nhalf == 1 ? (uint32_t)ncol * 128u : tile_bytes);
+            uint8_t* lo_tile = base + (size_t)s * stage_bytes + lo_off;
 #pragma unroll
             for (int j = 0; j < J; ++j) {
                 if (tid + j * kProdThreads < nchunks) {
@@ -304,10 +306,10 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap xmap, int m, int64_t d, int r
             fence_proxy_async_smem();   // make the generic-proxy stores visible to the MMA's reads
             __syncwarp();
             if (lane == 0) mbar_arrive(&sm->full[s]);   // one arrival per transform warp
+            if (++s == stages) { s = 0; ph ^= 1u; }
 
-            const int li = t / kBlocksPerSlab, kb = t - li * kBlocksPerSlab;
             const int nkb = li == my_items - 1 ? last_nkb : kBlocksPerSlab;
-            if (kb != nkb - 1) continue;
+            if (++kb != nkb) continue;
             const int item = (int)blockIdx.x + li * (int)gridDim.x;
 
             // ---- end of a slab: exact squared norms (the 8 lanes that share a row add up) ...
@@ -357,22 +359,26 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap xmap, int m, int64_t d, int r
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&sm->accum_empty);
+            kb = 0;
+            ++li;
         }
     } else if (warp == kProdWarps + kMmaWarps) {
         // ------------------------------------------------ the TMA thread
         if (lane == 0) {
             const uint32_t tx_bytes = (uint32_t)box_rows * 128u;
             int issued = 0;
+            int s = 0, kb = 0;
+            uint32_t ph = 0;
+            int64_t c0 = (int64_t)blockIdx.x * kSlabCols;            // first column of the current K-block
             for (int t = 0; t < total; ++t) {
-                const int s = (int)((uint32_t)t % (uint32_t)stages);
-                const uint32_t ph = ((uint32_t)t / (uint32_t)stages) & 1u;
                 mbar_wait(&sm->empty[s], ph ^ 1u, abort_flag, status);   // MMAs that read this stage are done
                 if (*abort_flag) break;
-                const int li = t / kBlocksPerSlab, kb = t - li * kBlocksPerSlab;
-                const int64_t c0 = ((int64_t)blockIdx.x + (int64_t)li * gridDim.x) * kSlabCols + (int64_t)kb * kKB;
                 mbar_expect_tx(&sm->landed[s], tx_bytes);
                 tma_load_2d(base + (size_t)s * stage_bytes, &xmap, (int)c0, 0, &sm->landed[s]);
                 issued = t + 1;
+                if (++s == stages) { s = 0; ph ^= 1u; }
+                c0 += kKB;
+                if (++kb == kBlocksPerSlab) { kb = 0; c0 += (int64_t)(gridDim.x - 1) * kSlabCols; }   // next slab of this CTA
             }
             if (*abort_flag) {
                 // give the copies still in flight a bounded time to land before the CTA goes away
@@ -389,19 +395,23 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap xmap, int m, int64_t d, int r
         const int g = warp - kProdWarps;
         const int n_mma = nhalf == 1 ? 2 * ncol : ncol;
         const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(n_mma >> 3) << 17) | ((128u >> 4) << 24);
-        uint32_t it = 0;
+        int s = 0, turn = 0;
+        uint32_t ph = 0;
         for (int local_item = 0; local_item < my_items; ++local_item) {
             const int nkb = local_item == my_items - 1 ? last_nkb : kBlocksPerSlab;
             if (local_item > 0) mbar_wait(&sm->accum_empty, (uint32_t)((local_item - 1) & 1), abort_flag, status);
             tc_fence_after();
             bool first = true;   // this thread's first MMA of the slab overwrites its accumulator
-            for (int kb = 0; kb < nkb; ++kb, ++it) {
-                if (nhalf == 1 && (int)(it % kMmaWarps) != g) continue;   // m <= 128: alternate K-blocks
-                const int s = (int)(it % (uint32_t)stages);
-                const uint32_t ph = (it / (uint32_t)stages) & 1u;
-                mbar_wait(&sm->full[s], ph, abort_flag, status);
+            for (int kb = 0; kb < nkb; ++kb) {
+                const int my_s = s;
+                const uint32_t my_ph = ph;
+                const bool skip = nhalf == 1 && turn != g;   // m <= 128: the two threads alternate K-blocks
+                if (++s == stages) { s = 0; ph ^= 1u; }
+                turn ^= 1;
+                if (skip) continue;
+                mbar_wait(&sm->full[my_s], my_ph, abort_flag, status);
                 tc_fence_after();
-                const uint32_t hi_addr = smem_u32(base + (size_t)s * stage_bytes);
+                const uint32_t hi_addr = smem_u32(base + (size_t)my_s * stage_bytes);
                 const uint64_t hi_desc = smem_desc(hi_addr);
                 if (nhalf == 1) {
                     const uint32_t dcol = tmem_base + (uint32_t)(g * 2 * ncol);
@@ -422,7 +432,7 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap xmap, int m, int64_t d, int r
                         first = false;
                     }
                 }
-                mma_commit(&sm->empty[s]);   // the stage may be refilled once these MMAs have read it
+                mma_commit(&sm->empty[my_s]);   // the stage may be refilled once these MMAs have read it
             }
             mma_commit(&sm->accum_full);
         }
