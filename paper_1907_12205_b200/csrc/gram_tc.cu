@@ -566,8 +566,10 @@ detox_status launch_sqdist_tc(const float* X, int64_t ld, int m, int64_t d, doub
     CUtensorMap xmap;
     detox_status st = make_xmap(&xmap, X, ld, m, d, p.box_rows);
     if (st != DETOX_OK) return st;
-    if (m <= 64) st = launch_tc<1>(p, xmap, m, d, partial, norms, status, s);
-    else if (m <= 128) st = launch_tc<2>(p, xmap, m, d, partial, norms, status, s);
+    // chunks per transform thread: m * 8 / kProdThreads, rounded up to a power of two
+    const int per_thread = (m * 8 + kProdThreads - 1) / kProdThreads;
+    if (per_thread <= 1) st = launch_tc<1>(p, xmap, m, d, partial, norms, status, s);
+    else if (per_thread <= 2) st = launch_tc<2>(p, xmap, m, d, partial, norms, status, s);
     else st = launch_tc<4>(p, xmap, m, d, partial, norms, status, s);
     if (st != DETOX_OK) return st;
     tc_reduce_kernel<<<dim3((unsigned)ceil_div((int64_t)m * m, 256), kReduceChunks), 256, 0, s>>>(

@@ -1,0 +1,98 @@
+"""GPU parity at the edges of the supported ranges: the largest row counts and group sizes, the
+fallback paths (rows that are not 16-byte aligned, row counts beyond the tensor-core and register
+kernels), one-column inputs, and the device status word."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_1907_12205_b200 as dx
+from helpers import bulyan_min_gap, multikrum_min_gap, rel_l2
+from test_parity_small import bits, krum_inputs, padded
+
+pytestmark = pytest.mark.gpu
+TOL = 1e-5
+
+
+@pytest.mark.parametrize("r,G,d", [(3, 341, 257), (15, 68, 130), (1, 1024, 33), (5, 204, 64)])
+def test_vote_largest_group_counts(r, G, d):
+    rng = np.random.default_rng(G)
+    n = r * G
+    members = rng.permutation(n).astype(np.int32)
+    X = np.empty((n, d), np.float32)
+    for j in range(G):
+        grp = members[j * r:(j + 1) * r]
+        X[grp] = rng.standard_normal(d).astype(np.float32)
+        if r >= 3 and j % 3 == 0:
+            X[grp[0]] *= -100
+        if r >= 3 and j % 7 == 0:
+            for t, i in enumerate(grp):
+                X[i, t % d] += t + 1
+    Z, w = dx.detox_vote(padded(X), r, members)
+    Zo, wo = oracle.vote(X, members, r)
+    assert w.cpu().numpy().tolist() == wo.tolist()
+    assert np.array_equal(bits(Z), Zo.view(np.uint32))
+
+
+def test_hier_mean_largest_set_counts():
+    rng = np.random.default_rng(1)
+    G, d = 1024, 40
+    Z = rng.standard_normal((G, d)).astype(np.float32)
+    perm = rng.permutation(G).astype(np.int32)
+    for offs in (np.arange(G + 1), np.array([0, G]), np.array([0, 1, 1000, G])):
+        M = dx.detox_hier_mean(padded(Z), offs.astype(np.int32), perm)
+        assert rel_l2(M.cpu().numpy(), oracle.hier_mean(Z, offs, perm)) <= TOL
+
+
+@pytest.mark.parametrize("m,d", [(300, 200), (513, 70), (1024, 40), (1024, 1), (1, 1), (2, 1), (105, 1), (225, 1)])
+def test_coord_median_beyond_the_register_kernels_and_single_column(m, d):
+    X = np.random.default_rng(m + d).standard_normal((m, d)).astype(np.float32)
+    assert np.array_equal(bits(dx.agg_coord_median(padded(X))), oracle.coord_median(X).view(np.uint32))
+
+
+@pytest.mark.parametrize("m,d,f,m_sel,odd", [(300, 700, 30, 270, False), (1024, 48, 100, 900, False),
+                                              (45, 3001, 5, 40, True), (105, 1001, 10, 95, True), (3, 1, 0, 2, False)])
+def test_multikrum_fallback_paths(m, d, f, m_sel, odd):
+    for attempt in range(16):
+        X = krum_inputs(m, d, seed=m + d + 1000 * attempt, copies=1, outliers=min(f, 4))
+        out_o, sel_o, sc_o, _ = oracle.multikrum(X, f, m_sel)
+        if multikrum_min_gap(sc_o, m_sel) > 1e-5:
+            break
+    Xd = padded(X, ld=d + (1 if d % 2 == 0 else 2), offset=1) if odd else padded(X)
+    out, sel, sc = dx.agg_multikrum(Xd, f, m_sel)
+    assert sel.cpu().numpy().tolist() == sel_o.tolist()
+    np.testing.assert_allclose(sc.cpu().numpy(), sc_o, rtol=2e-6, atol=1e-30)
+    assert rel_l2(out.cpu().numpy(), out_o) <= TOL
+
+
+def test_bulyan_many_rows_through_the_shared_memory_stage_two():
+    m, d, f = 400, 96, 20                      # theta = 360 rows enter stage 2: beyond the register kernels
+    for attempt in range(8):
+        X = krum_inputs(m, d, seed=77 + 1000 * attempt, copies=1, outliers=f)
+        out_o, sel_o, D_o = oracle.bulyan(X, f)
+        if bulyan_min_gap(D_o, f) > 5e-6:
+            break
+    out, sel = dx.agg_bulyan(padded(X), f)
+    assert sel.cpu().numpy().tolist() == sel_o.tolist()
+    assert rel_l2(out.cpu().numpy(), out_o) <= TOL
+
+
+def test_status_word_is_clear_after_the_tensor_core_path():
+    m, d = 64, 5000
+    X = padded(krum_inputs(m, d, seed=5))
+    ws = torch.full((dx.agg_multikrum_workspace_bytes(m, d),), 0xFF, dtype=torch.uint8, device="cuda:0")
+    dx.agg_multikrum(X, 5, 50, ws=ws)
+    torch.cuda.synchronize()
+    assert int(ws[:4].view(torch.int32).item()) == 0       # first word of the workspace: device-side status
+
+
+def test_pipeline_with_the_largest_worker_count():
+    import workloads as wl
+    spec = wl.WorkloadSpec("p", n=1023, r=3, d=300, sigma=1e-3, q=100, attack="reverse", placement="random",
+                           set_size=11, group_jitter=0.05, seed=3)
+    w = wl.make_workload(spec)
+    pipe = dx.Pipeline(spec.n, 3, spec.d, w.members, dx.AGG_MEAN, w.set_offsets, w.set_members, dx.AGG_COORD_MEDIAN)
+    res = dx.detox_aggregate(pipe, w.X.to("cuda:0")[:, :spec.d])
+    ref = oracle.detox_aggregate(w.data().numpy(), w.members, 3, "mean", w.set_offsets, w.set_members, "coord_median")
+    assert res["winner"].cpu().numpy().tolist() == ref["winner"].tolist()
+    assert rel_l2(res["out"].cpu().numpy(), ref["out"]) <= TOL
