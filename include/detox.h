@@ -165,14 +165,20 @@ detox_status agg_bulyan(const float* X, int64_t ld, int m, int64_t d, int f, flo
  *
  *   a0 = DETOX_AGG_NONE : the G votes go to A_1 directly (sets are ignored)
  *   a0 = DETOX_AGG_MEAN : the S set means go to A_1
+ *   a0 = DETOX_AGG_MULTIKRUM | DETOX_AGG_BULYAN : the aggregator runs inside every vote set (the pairings the
+ *        paper found most resilient, Section 5.1 setups 2 and 3; set shapes as in Appendix B.1, e.g. 7 + 8 or
+ *        one set of 15) and its S results go to A_1, which must then be MEAN or COORD_MEDIAN.  f and m_sel
+ *        belong to A_0: every set of k votes averages its m_sel best (m_sel = 0: its k - f best), or, for
+ *        Bulyan, needs k >= 4f+3.
  *   a1 = MEAN | COORD_MEDIAN | MULTIKRUM (f, m_sel) | BULYAN (f)
  *
  *   out          dev, d
  *   winner       dev, G        out, as in detox_vote; may be NULL
  *   sel          dev           out, rows chosen by Multi-Krum (m_sel, ascending) or Bulyan (theta, in
- *                              selection order) among the rows that entered A_1; may be NULL
- *   sel_workers  dev           out, the same rows as worker ids (winner[sel[k]]), only meaningful
- *                              when a0 = DETOX_AGG_NONE; may be NULL
+ *                              selection order): indices among the rows that entered A_1 when A_1 is the
+ *                              Krum-type stage; vote (group) indices, set after set, when A_0 is; may be NULL
+ *   sel_workers  dev           out, the same rows as worker ids (winner[vote]), meaningful whenever sel
+ *                              indexes votes (a0 = NONE, MULTIKRUM or BULYAN); may be NULL
  *   ws           detox_aggregate_workspace_bytes(desc) bytes (holds the votes and set means too)
  * ------------------------------------------------------------------------------------------- */
 typedef struct {
@@ -180,8 +186,8 @@ typedef struct {
     int32_t r;                   /* redundancy ratio (odd, divides n) */
     int64_t d;                   /* gradient dimension */
     const int32_t* members;      /* host, G*r */
-    int32_t a0;                  /* detox_agg: NONE or MEAN */
-    int32_t n_sets;              /* S, used when a0 = MEAN */
+    int32_t a0;                  /* detox_agg: NONE, MEAN, MULTIKRUM or BULYAN */
+    int32_t n_sets;              /* S, used unless a0 = NONE */
     const int32_t* set_offsets;  /* host, S+1 */
     const int32_t* set_members;  /* host, G */
     int32_t a1;                  /* detox_agg: MEAN, COORD_MEDIAN, MULTIKRUM or BULYAN */

@@ -201,15 +201,33 @@ A0_NONE, A0_MEAN = "none", "mean"
 
 def detox_aggregate(X, members, r: int, a0: str, set_offsets, set_members, a1: str, f: int = 0,
                     m_sel: int = 1):
-    """Algorithm 1 (filtering step + hierarchical aggregation) with A_0 in {none, mean} and
-    A_1 in {mean, coord_median, multikrum, bulyan}.
+    """Algorithm 1 (filtering step + hierarchical aggregation) with A_0 in {none, mean, multikrum, bulyan}
+    and A_1 in {mean, coord_median, multikrum, bulyan}.
 
     Returns dict(out, winner, sel) where sel indexes the rows that entered A_1 (votes when a0 is
     "none", sets when a0 is "mean"), and sel_workers maps them through winner[] when a0 is "none".
     """
     Z, winner = vote(X, members, r)
-    rows = Z if a0 == A0_NONE else hier_mean(Z, set_offsets, set_members)
     sel = None
+    sel_votes = None
+    if a0 in ("multikrum", "bulyan"):
+        # Section 5.1, setups 2 and 3: the robust aggregator inside every vote group, then A_1 over the results.
+        # f and m_sel belong to A_0; m_sel = 0 means "all but f" of each group.
+        so, sm = np.asarray(set_offsets), np.asarray(set_members)
+        outs, sel_votes = [], []
+        for s in range(len(so) - 1):
+            idx = sm[so[s]:so[s + 1]]
+            if a0 == "multikrum":
+                keep = m_sel if m_sel > 0 else max(len(idx) - f, 1)
+                o, loc, _, _ = multikrum(Z[idx], f, keep)
+            else:
+                o, loc, _ = bulyan(Z[idx], f)
+            outs.append(o)
+            sel_votes.extend(int(v) for v in idx[loc])
+        rows = np.stack(outs)
+        sel_votes = np.asarray(sel_votes, dtype=np.int32)
+    else:
+        rows = Z if a0 == A0_NONE else hier_mean(Z, set_offsets, set_members)
     if a1 == "mean":
         out = mean_rows(rows)
     elif a1 == "coord_median":
@@ -221,6 +239,8 @@ def detox_aggregate(X, members, r: int, a0: str, set_offsets, set_members, a1: s
     else:
         raise ValueError(a1)
     sel_workers = None
-    if sel is not None and a0 == A0_NONE:
+    if sel_votes is not None:
+        sel, sel_workers = sel_votes, winner[sel_votes]
+    elif sel is not None and a0 == A0_NONE:
         sel_workers = winner[sel]
     return dict(out=out, winner=winner, sel=sel, sel_workers=sel_workers, rows=rows, Z=Z)

@@ -268,10 +268,15 @@ class Pipeline:
 
     @property
     def rows_into_a1(self) -> int:
-        return self.desc.n_sets if self.a0 == AGG_MEAN else self.G
+        return self.desc.n_sets if self.a0 != AGG_NONE else self.G
 
     @property
     def n_selected(self) -> int:
+        if self.a0 in (AGG_MULTIKRUM, AGG_BULYAN):      # chosen inside every vote set, concatenated in set order
+            sizes = np.diff(self.set_offsets)
+            if self.a0 == AGG_BULYAN:
+                return int(sum(k - 2 * self.f for k in sizes))
+            return int(sum(self.m_sel if self.m_sel > 0 else max(k - self.f, 1) for k in sizes))
         if self.a1 == AGG_MULTIKRUM:
             return self.m_sel
         if self.a1 == AGG_BULYAN:
@@ -289,7 +294,11 @@ def detox_aggregate_workspace_bytes(pipe: Pipeline) -> int:
 def detox_aggregate(pipe: Pipeline, X, out: Optional[torch.Tensor] = None, winner: Optional[torch.Tensor] = None,
                     sel: Optional[torch.Tensor] = None, sel_workers: Optional[torch.Tensor] = None,
                     ws: Optional[torch.Tensor] = None, stream=None):
-    """Vote -> A_0 -> A_1.  Returns dict(out, winner, sel, sel_workers)."""
+    """Vote -> A_0 -> A_1.  Returns dict(out, winner, sel, sel_workers).
+
+    sel lists the rows chosen by the Krum-type stage: rows that entered A_1 when A_1 is Multi-Krum / Bulyan;
+    vote (group) indices, set after set, when A_0 is Multi-Krum / Bulyan.  sel_workers gives the same rows
+    as worker ids whenever sel indexes votes."""
     lib = load()
     xp, ld, n, d = _mat(X)
     if n != pipe.n or d != pipe.d:
@@ -302,7 +311,7 @@ def detox_aggregate(pipe: Pipeline, X, out: Optional[torch.Tensor] = None, winne
     k = pipe.n_selected
     if k > 0 and sel is None:
         sel = torch.empty(k, dtype=torch.int32, device=dev)
-    if k > 0 and sel_workers is None and pipe.a0 == AGG_NONE:
+    if k > 0 and sel_workers is None and pipe.a0 != AGG_MEAN:
         sel_workers = torch.empty(k, dtype=torch.int32, device=dev)
     need = pipe.workspace_bytes()
     if need == 0:

@@ -117,7 +117,17 @@ detox_status check_bulyan(int m, int f) {
 
 int64_t pad_ld(int64_t d) { return (d + 31) / 32 * 32; }
 
+bool krum_type(int a) { return a == DETOX_AGG_MULTIKRUM || a == DETOX_AGG_BULYAN; }
+
+// rows a Krum-type A_0 keeps from a vote set of k rows
+int a0_selected(const detox_pipeline_desc* p, int k) {
+    if (p->a0 == DETOX_AGG_BULYAN) return k - 2 * p->f;
+    return p->m_sel > 0 ? p->m_sel : (k - p->f > 1 ? k - p->f : 1);
+}
+
 struct PipeWs {
+    int32_t* winner_set_order;   // Krum-type A_0: winners in set order
+    int32_t* sel_local;          // Krum-type A_0: rows chosen inside the current set
     void* vote;
     float* Z;
     float* M;
@@ -131,7 +141,7 @@ PipeWs pipe_ws(void* ws, const detox_pipeline_desc* p) {
     PipeWs w;
     char* base = static_cast<char*>(ws);
     const int G = p->n / p->r;
-    const int rows1 = p->a0 == DETOX_AGG_MEAN ? p->n_sets : G;
+    const int rows1 = p->a0 != DETOX_AGG_NONE ? p->n_sets : G;
     size_t off = 0;
     w.ldz = pad_ld(p->d);
     w.vote = base + off;
@@ -141,9 +151,21 @@ PipeWs pipe_ws(void* ws, const detox_pipeline_desc* p) {
     w.Z = reinterpret_cast<float*>(base + off);
     if (p->a0 != DETOX_AGG_MEAN) off += align_up((size_t)G * w.ldz * sizeof(float));   // votes are stored only then
     w.M = reinterpret_cast<float*>(base + off);
-    if (p->a0 == DETOX_AGG_MEAN) off += align_up((size_t)p->n_sets * w.ldz * sizeof(float));
+    if (p->a0 != DETOX_AGG_NONE) off += align_up((size_t)p->n_sets * w.ldz * sizeof(float));
+    w.winner_set_order = reinterpret_cast<int32_t*>(base + off);
+    off += align_up((size_t)G * sizeof(int32_t));
+    w.sel_local = reinterpret_cast<int32_t*>(base + off);
+    off += align_up((size_t)G * sizeof(int32_t));
     w.agg = base + off;
-    if (p->a1 == DETOX_AGG_MULTIKRUM || p->a1 == DETOX_AGG_BULYAN) off += krum_ws(nullptr, rows1, p->d).total;
+    if (krum_type(p->a1)) off += krum_ws(nullptr, rows1, p->d).total;
+    if (krum_type(p->a0)) {
+        int kmax = 1;
+        for (int s = 0; s < p->n_sets; ++s) {
+            const int k = p->set_offsets[s + 1] - p->set_offsets[s];
+            kmax = k > kmax ? k : kmax;
+        }
+        off += krum_ws(nullptr, kmax, p->d).total;
+    }
     w.total = off;
     return w;
 }
@@ -152,9 +174,22 @@ detox_status check_desc(const detox_pipeline_desc* p) {
     if (!p || p->d < 1) return DETOX_ERR_BAD_ARG;
     if (p->n < 1 || p->r < 1 || (p->r & 1) == 0 || p->n % p->r != 0) return DETOX_ERR_BAD_ARG;
     if (p->n > kMaxRows || p->r > kMaxR) return DETOX_ERR_UNSUPPORTED;
-    if (p->a0 != DETOX_AGG_NONE && p->a0 != DETOX_AGG_MEAN) return DETOX_ERR_UNSUPPORTED;
+    if (p->a0 != DETOX_AGG_NONE && p->a0 != DETOX_AGG_MEAN && !krum_type(p->a0)) return DETOX_ERR_BAD_ARG;
     const int G = p->n / p->r;
-    if (p->a0 == DETOX_AGG_MEAN && (p->n_sets < 1 || p->n_sets > G)) return DETOX_ERR_BAD_ARG;
+    if (p->a0 != DETOX_AGG_NONE && (p->n_sets < 1 || p->n_sets > G)) return DETOX_ERR_BAD_ARG;
+    if (krum_type(p->a0)) {
+        // Multi-Krum / Bulyan inside every vote set (f, m_sel belong to A_0), then a plain A_1 over the set results
+        if (p->a1 != DETOX_AGG_MEAN && p->a1 != DETOX_AGG_COORD_MEDIAN) return DETOX_ERR_UNSUPPORTED;
+        if (!p->set_offsets || p->f < 0 || p->m_sel < 0) return DETOX_ERR_BAD_ARG;
+        if (p->set_offsets[0] != 0 || p->set_offsets[p->n_sets] != G) return DETOX_ERR_BAD_ARG;
+        for (int s = 0; s < p->n_sets; ++s) {
+            const int k = p->set_offsets[s + 1] - p->set_offsets[s];
+            if (k < 1) return DETOX_ERR_BAD_ARG;
+            if (p->a0 == DETOX_AGG_BULYAN && check_bulyan(k, p->f) != DETOX_OK) return DETOX_ERR_BAD_ARG;
+            if (p->a0 == DETOX_AGG_MULTIKRUM && p->m_sel > k) return DETOX_ERR_BAD_ARG;
+        }
+        return DETOX_OK;
+    }
     const int rows1 = p->a0 == DETOX_AGG_MEAN ? p->n_sets : G;
     switch (p->a1) {
         case DETOX_AGG_MEAN:
@@ -283,7 +318,7 @@ detox_status detox_aggregate(const detox_pipeline_desc* p, const float* X, int64
     if (!out || (reinterpret_cast<uintptr_t>(out) & 3u)) return DETOX_ERR_BAD_ARG;
     const int G = p->n / p->r;
     SetTable sets;
-    if (p->a0 == DETOX_AGG_MEAN &&
+    if (p->a0 != DETOX_AGG_NONE &&
         (st = check_sets(G, p->n_sets, p->set_offsets, p->set_members, &sets)) != DETOX_OK)
         return st;
     PipeWs w = pipe_ws(ws, p);
@@ -298,6 +333,34 @@ detox_status detox_aggregate(const detox_pipeline_desc* p, const float* X, int64
         if ((st = launch_vote_mean(X, ld, p->n, p->r, p->d, groups, sets, p->n_sets, w.M, w.ldz, win, w.vote, s)) !=
             DETOX_OK)
             return st;
+        rows = w.M;
+        m = p->n_sets;
+    } else if (krum_type(p->a0)) {
+        // The paper's preferred pairings (Section 5.1, setups 2 and 3): Multi-Krum or Bulyan inside every
+        // vote set, then A_1.  The vote runs over the groups in set order, so each set's votes are
+        // consecutive rows of Z and the aggregators take them as ordinary matrices.
+        IdTable in_set_order;
+        for (int k = 0; k < G; ++k)
+            for (int a = 0; a < p->r; ++a) in_set_order.id[k * p->r + a] = groups.id[sets.member[k] * p->r + a];
+        if ((st = launch_vote(X, ld, p->n, p->r, p->d, in_set_order, w.Z, w.ldz, w.winner_set_order, w.vote, s)) !=
+            DETOX_OK)
+            return st;
+        if ((st = launch_scatter_by_set_order(w.winner_set_order, sets, G, win, s)) != DETOX_OK) return st;
+        int emitted = 0;
+        for (int t = 0; t < p->n_sets; ++t) {
+            const int b = sets.offset[t], k = sets.offset[t + 1] - b;
+            const int keep = a0_selected(p, k);
+            const float* rows_t = w.Z + (int64_t)b * w.ldz;
+            float* out_t = w.M + (int64_t)t * w.ldz;
+            st = p->a0 == DETOX_AGG_MULTIKRUM
+                     ? run_multikrum(rows_t, w.ldz, k, p->d, p->f, keep, out_t, w.sel_local, nullptr, w.agg, s)
+                     : run_bulyan(rows_t, w.ldz, k, p->d, p->f, out_t, w.sel_local, w.agg, s);
+            if (st != DETOX_OK) return st;
+            st = launch_map_set_selection(w.sel_local, keep, sets, b, w.winner_set_order, sel ? sel + emitted : nullptr,
+                                          sel_workers ? sel_workers + emitted : nullptr, s);
+            if (st != DETOX_OK) return st;
+            emitted += keep;
+        }
         rows = w.M;
         m = p->n_sets;
     } else if ((st = launch_vote(X, ld, p->n, p->r, p->d, groups, w.Z, w.ldz, win, w.vote, s)) != DETOX_OK) {

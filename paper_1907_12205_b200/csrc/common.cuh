@@ -106,4 +106,11 @@ detox_status launch_bulyan_select(const double* D, int m, int f, int32_t* sel_de
 detox_status launch_map_indices(const int32_t* idx, const int32_t* map, int cnt, int32_t* out,
                                 cudaStream_t s);
 
+// votes computed in set order: winner back to group order; selections inside a set to vote / worker ids
+detox_status launch_scatter_by_set_order(const int32_t* src, const SetTable& sets, int G, int32_t* dst,
+                                         cudaStream_t s);
+detox_status launch_map_set_selection(const int32_t* local, int cnt, const SetTable& sets, int set_begin,
+                                      const int32_t* winner_in_set_order, int32_t* sel_votes, int32_t* sel_workers,
+                                      cudaStream_t s);
+
 }  // namespace detox

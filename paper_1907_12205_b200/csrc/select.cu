@@ -207,6 +207,25 @@ __global__ void map_indices_kernel(const int32_t* __restrict__ idx, const int32_
     if (k < cnt) out[k] = map[idx[k]];
 }
 
+// dst[member[k]] = src[k] for the G votes (votes were produced in set order; give them back in group order)
+__global__ void scatter_by_set_order_kernel(const int32_t* __restrict__ src, const __grid_constant__ SetTable sets,
+                                            int G, int32_t* __restrict__ dst) {
+    int k = blockIdx.x * blockDim.x + threadIdx.x;
+    if (k < G) dst[sets.member[k]] = src[k];
+}
+
+// Rows chosen inside one vote set (local indices) -> vote indices and worker ids
+__global__ void map_set_selection_kernel(const int32_t* __restrict__ local, int cnt,
+                                         const __grid_constant__ SetTable sets, int set_begin,
+                                         const int32_t* __restrict__ winner_in_set_order,
+                                         int32_t* __restrict__ sel_votes, int32_t* __restrict__ sel_workers) {
+    int k = blockIdx.x * blockDim.x + threadIdx.x;
+    if (k >= cnt) return;
+    const int pos = set_begin + local[k];
+    if (sel_votes) sel_votes[k] = sets.member[pos];
+    if (sel_workers) sel_workers[k] = winner_in_set_order[pos];
+}
+
 int round_up_warp(int m) { return (m + 31) / 32 * 32; }
 
 }  // namespace
@@ -238,6 +257,21 @@ detox_status launch_bulyan_select(const double* D, int m, int f, int32_t* sel_de
 detox_status launch_map_indices(const int32_t* idx, const int32_t* map, int cnt, int32_t* out, cudaStream_t s) {
     if (cnt <= 0) return DETOX_OK;
     map_indices_kernel<<<(cnt + 127) / 128, 128, 0, s>>>(idx, map, cnt, out);
+    return launch_status();
+}
+
+detox_status launch_scatter_by_set_order(const int32_t* src, const SetTable& sets, int G, int32_t* dst,
+                                         cudaStream_t s) {
+    scatter_by_set_order_kernel<<<(G + 127) / 128, 128, 0, s>>>(src, sets, G, dst);
+    return launch_status();
+}
+
+detox_status launch_map_set_selection(const int32_t* local, int cnt, const SetTable& sets, int set_begin,
+                                      const int32_t* winner_in_set_order, int32_t* sel_votes, int32_t* sel_workers,
+                                      cudaStream_t s) {
+    if (cnt <= 0 || (!sel_votes && !sel_workers)) return DETOX_OK;
+    map_set_selection_kernel<<<(cnt + 127) / 128, 128, 0, s>>>(local, cnt, sets, set_begin, winner_in_set_order,
+                                                               sel_votes, sel_workers);
     return launch_status();
 }
 

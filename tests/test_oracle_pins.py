@@ -356,3 +356,31 @@ def test_pipeline_honest_majority_equals_aggregator_on_true_gradients():
     res = oracle.detox_aggregate(X, members, r, "none", None, None, "coord_median")
     assert np.array_equal(res["out"], np.median(honest, axis=0))
     assert np.array_equal(res["Z"], honest)
+
+
+def test_pipeline_krum_family_inside_vote_sets():
+    # Section 5.1, setups 2 and 3: the aggregator inside every vote group, then the mean.
+    G, r, d = 15, 3, 128
+    honest = rng(30).standard_normal((G, d)).astype(np.float32)
+    members = rng(31).permutation(G * r).astype(np.int32)
+    X = np.empty((G * r, d), np.float32)
+    for j in range(G):
+        X[members[j * r:(j + 1) * r]] = honest[j]
+    sm = rng(32).permutation(G).astype(np.int32)
+    # no Byzantine node, f = 0: Multi-Krum keeps everything -> mean of the two set means (7 and 8 votes)
+    res = oracle.detox_aggregate(X, members, r, "multikrum", [0, 7, 15], sm, "mean", f=0, m_sel=0)
+    exp = (honest[sm[:7]].astype(np.float64).mean(0).astype(np.float32).astype(np.float64) +
+           honest[sm[7:]].astype(np.float64).mean(0).astype(np.float32)) / 2
+    np.testing.assert_allclose(res["out"], exp, rtol=0, atol=1e-6)
+    assert sorted(res["sel"].tolist()) == list(range(G))
+    # one Byzantine vote (a colluding pair wins group sm[3]): Multi-Krum(f=1) drops it from its set
+    bad = int(sm[3])
+    X[members[bad * r:bad * r + 2]] = 50.0 * honest[bad]
+    res = oracle.detox_aggregate(X, members, r, "multikrum", [0, 7, 15], sm, "mean", f=1, m_sel=0)
+    assert bad not in res["sel"].tolist() and len(res["sel"]) == 6 + 7
+    assert res["sel_workers"].tolist() == res["winner"][res["sel"]].tolist()
+    # Bulyan over one set of 15 with f = 2, then the mean of a single result = Bulyan on the votes
+    res = oracle.detox_aggregate(X, members, r, "bulyan", [0, 15], sm, "mean", f=2)
+    direct, sel, _ = oracle.bulyan(res["Z"][sm], 2)
+    assert np.array_equal(res["out"], direct) and res["sel"].tolist() == sm[sel].tolist()
+    assert bad not in res["sel"].tolist()

@@ -279,6 +279,38 @@ def test_pipeline_fused_vote_mean_handles_no_majority_and_uneven_sets(r, G, set_
     assert np.array_equal(bits(fused), bits(two_step))
 
 
+@pytest.mark.parametrize("a0,f,m_sel,offs,a1", [("multikrum", 1, 0, [0, 7, 15], "mean"), ("bulyan", 2, 0, [0, 15], "mean"),
+                                                 ("multikrum", 1, 3, [0, 5, 10, 15], "coord_median")])
+def test_pipeline_krum_family_inside_vote_sets(a0, f, m_sel, offs, a1):
+    # the paper's preferred pairings (Section 5.1, setups 2 and 3; set shapes of Appendix B.1)
+    code = {"multikrum": dx.AGG_MULTIKRUM, "bulyan": dx.AGG_BULYAN, "mean": dx.AGG_MEAN,
+            "coord_median": dx.AGG_COORD_MEDIAN}
+    for attempt in range(16):
+        spec = wl.WorkloadSpec("p", n=45, r=3, d=20_011, sigma=1e-3, q=5, attack="alie", placement="worst",
+                               group_jitter=0.1, seed=40 + attempt)
+        w = wl.make_workload(spec)
+        sm = np.random.default_rng(spec.seed).permutation(15).astype(np.int32)
+        ref = oracle.detox_aggregate(w.data().numpy(), w.members, 3, a0, offs, sm, a1, f, m_sel)
+        gaps = []
+        for s in range(len(offs) - 1):
+            Zs = ref["Z"][sm[offs[s]:offs[s + 1]]]
+            if a0 == "multikrum":
+                keep = m_sel if m_sel > 0 else len(Zs) - f
+                gaps.append(multikrum_min_gap(oracle.multikrum(Zs, f, keep, want_out=False)[2], keep))
+            else:
+                gaps.append(bulyan_min_gap(oracle.sqdist(Zs), f))
+        if min(gaps) > 1e-4:
+            break
+    else:
+        pytest.fail("no seed without a near-tie")
+    pipe = dx.Pipeline(45, 3, spec.d, w.members, code[a0], offs, sm, code[a1], f, m_sel)
+    res = dx.detox_aggregate(pipe, w.X.to(DEV)[:, :spec.d])
+    assert res["winner"].cpu().numpy().tolist() == ref["winner"].tolist()
+    assert res["sel"].cpu().numpy().tolist() == ref["sel"].tolist()
+    assert res["sel_workers"].cpu().numpy().tolist() == ref["sel_workers"].tolist()
+    assert rel_l2(res["out"].cpu().numpy(), ref["out"]) <= TOL
+
+
 def test_q0_pipeline_is_plain_mean():
     spec = wl.WorkloadSpec("p", n=21, r=3, d=12_345, sigma=1e-3, q=0, seed=9)
     w = wl.make_workload(spec)
