@@ -130,6 +130,14 @@ detox_status agg_coord_median(const float* X, int64_t ld, int m, int64_t d, floa
                               size_t ws_bytes, void* stream);
 
 /* ---------------------------------------------------------------------------------------------
+ * Coordinate-wise alpha-trimmed mean (one of the A_1 choices analysed in Section 4, Theorem 4 with
+ * alpha = 1/4): per coordinate, drop the `trim` smallest and the `trim` largest of the m values and
+ * average the other m - 2*trim.  0 <= trim, m - 2*trim >= 1.  trim = 0 is the plain mean.
+ *   out  dev, d.   No workspace.
+ * ------------------------------------------------------------------------------------------- */
+detox_status agg_trimmed_mean(const float* X, int64_t ld, int m, int64_t d, int trim, float* out, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
  * Multi-Krum (cited in Section 4 "Improved speed" as the O(p^2 d) aggregator; requirement
  * m >= 2f+3 in Appendix B.1).  score_i = sum of the nb smallest squared distances from row i to the
  * other rows, nb = m - f - 2 clamped to [1, m-1]; the m_sel rows of smallest score (equal scores:

@@ -4,7 +4,7 @@ TEST INFRASTRUCTURE ONLY.  Imported by tests/, by the smoke check and by the ben
 leg; never by the CUDA library or its Python binding.  Every array is a host numpy array; fp32 in,
 fp64 accumulation inside, fp32 (values) / int32 (indices) out.
 
-Pin status: vote, hier_mean, coord_median, sqdist are pinned by tests/test_oracle_pins.py.
+Pin status: vote, hier_mean, coord_median, trimmed_mean, sqdist are pinned by tests/test_oracle_pins.py.
 Krum scores, Multi-Krum and Bulyan are pinned to brute-force subset definitions on tiny inputs and
 to their reductions; beyond those cases: parity unpinned (the paper cites them without a definition).
 """
@@ -55,6 +55,7 @@ def _load():
         lib.oracle_multikrum.argtypes = [_F, _i64, _int, _i64, _int, _int, _F, _I, _D, _D]
         lib.oracle_bulyan_select.argtypes = [_D, _int, _int, _I]
         lib.oracle_trimmed_around_median.argtypes = [_F, _i64, _i64, _I, _int, _int, _F]
+        lib.oracle_trimmed_mean.argtypes = [_F, _i64, _int, _i64, _int, _F]
         lib.oracle_bulyan.argtypes = [_F, _i64, _int, _i64, _int, _F, _I, _D]
         _lib = lib
     return _lib
@@ -132,6 +133,14 @@ def coord_median(X, rows=None):
     r = None if rows is None else _idx(rows)
     out = np.empty(d, dtype=np.float32)
     _check(_load().oracle_coord_median(_fp(X), ld, m if r is None else len(r), d, _ip(r), _fp(out)), "coord_median")
+    return out
+
+
+def trimmed_mean(X, trim: int):
+    X, ld = _mat(X)
+    m, d = X.shape
+    out = np.empty(d, dtype=np.float32)
+    _check(_load().oracle_trimmed_mean(_fp(X), ld, m, d, trim, _fp(out)), "trimmed_mean")
     return out
 
 

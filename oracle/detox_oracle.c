@@ -309,6 +309,28 @@ int oracle_trimmed_around_median(const float* X, int64_t ld, int64_t d, const in
     return 0;
 }
 
+/* ---------------------------------------------------------------------------------------------
+ * Coordinate-wise alpha-trimmed mean (Section 4, Theorem 4): drop the `trim` smallest and `trim`
+ * largest of the m values of a coordinate, average the rest.
+ * ------------------------------------------------------------------------------------------- */
+int oracle_trimmed_mean(const float* X, int64_t ld, int m, int64_t d, int trim, float* out) {
+    if (trim < 0 || m - 2 * trim < 1) return 1;
+#pragma omp parallel
+    {
+        uint32_t* k = (uint32_t*)malloc((size_t)m * sizeof(uint32_t));
+#pragma omp for schedule(static)
+        for (int64_t c = 0; c < d; ++c) {
+            for (int i = 0; i < m; ++i) k[i] = order_key(X[(int64_t)i * ld + c]);
+            qsort(k, (size_t)m, sizeof(uint32_t), cmp_u32);
+            double acc = 0.0;
+            for (int i = trim; i < m - trim; ++i) acc += (double)key_to_float(k[i]);
+            out[c] = (float)(acc / (double)(m - 2 * trim));
+        }
+        free(k);
+    }
+    return 0;
+}
+
 /* Bulyan = first stage on all m rows with tolerance f, then the second stage with beta = theta - 2f. */
 int oracle_bulyan(const float* X, int64_t ld, int m, int64_t d, int f, float* out, int32_t* sel,
                   double* D_out) {

@@ -23,7 +23,7 @@ MAX_ROWS, MAX_R = 1024, 15
 EXPORTS = (
     "detox_status_string", "detox_vote_workspace_bytes", "detox_vote", "detox_vote_noalloc", "detox_hier_mean",
     "detox_vote_hier_mean",
-    "agg_coord_median_workspace_bytes", "agg_coord_median", "agg_multikrum_workspace_bytes", "agg_multikrum",
+    "agg_coord_median_workspace_bytes", "agg_coord_median", "agg_trimmed_mean", "agg_multikrum_workspace_bytes", "agg_multikrum",
     "agg_bulyan_workspace_bytes", "agg_bulyan", "detox_aggregate_workspace_bytes", "detox_aggregate",
 )
 
@@ -71,6 +71,7 @@ def load() -> ctypes.CDLL:
         fn.restype = _sz
         fn.argtypes = [_int, _i64]
     lib.agg_coord_median.argtypes = [_vp, _i64, _int, _i64, _vp, _vp, _sz, _vp]
+    lib.agg_trimmed_mean.argtypes = [_vp, _i64, _int, _i64, _int, _vp, _vp]
     lib.agg_multikrum.argtypes = [_vp, _i64, _int, _i64, _int, _int, _vp, _vp, _vp, _vp, _sz, _vp]
     lib.agg_bulyan.argtypes = [_vp, _i64, _int, _i64, _int, _vp, _vp, _vp, _sz, _vp]
     lib.detox_aggregate_workspace_bytes.restype = _sz
@@ -202,6 +203,16 @@ def agg_coord_median(X, out: Optional[torch.Tensor] = None, ws: Optional[torch.T
         out = torch.empty(d, dtype=torch.float32, device=X.device)
     _check(lib.agg_coord_median(xp, ld, m, d, out.data_ptr(), _ptr(ws), 0 if ws is None else ws.numel(),
                                 _stream(stream)), "agg_coord_median")
+    return out
+
+
+def agg_trimmed_mean(X, trim: int, out: Optional[torch.Tensor] = None, stream=None):
+    """Coordinate-wise mean after dropping the `trim` smallest and `trim` largest values."""
+    lib = load()
+    xp, ld, m, d = _mat(X)
+    if out is None:
+        out = torch.empty(d, dtype=torch.float32, device=X.device)
+    _check(lib.agg_trimmed_mean(xp, ld, m, d, trim, out.data_ptr(), _stream(stream)), "agg_trimmed_mean")
     return out
 
 

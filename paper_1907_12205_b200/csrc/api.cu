@@ -273,6 +273,13 @@ detox_status agg_coord_median(const float* X, int64_t ld, int m, int64_t d, floa
     return launch_coord_select(X, ld, m, d, nullptr, 0, out, static_cast<cudaStream_t>(stream));
 }
 
+detox_status agg_trimmed_mean(const float* X, int64_t ld, int m, int64_t d, int trim, float* out, void* stream) {
+    detox_status st = check_matrix(X, ld, m, d);
+    if (st != DETOX_OK) return st;
+    if (!out || (reinterpret_cast<uintptr_t>(out) & 3u) || trim < 0 || m - 2 * trim < 1) return DETOX_ERR_BAD_ARG;
+    return launch_coord_select(X, ld, m, d, nullptr, -(m - 2 * trim), out, static_cast<cudaStream_t>(stream));
+}
+
 size_t agg_multikrum_workspace_bytes(int m, int64_t d) {
     if (m < 1 || m > kMaxRows || d < 1) return 0;
     return krum_ws(nullptr, m, d).total;

@@ -77,7 +77,8 @@ detox_status launch_mean_rows(const float* X, int64_t ld, int64_t d, const int32
                               float* out, cudaStream_t s);
 
 // median.cu: per-coordinate order statistics over m rows (rows_dev: device int32 list or NULL)
-//   beta == 0 : coordinate median;  beta >= 1 : mean of the beta values closest to the median
+//   beta == 0 : coordinate median;  beta >= 1 : mean of the beta values closest to the median;
+//   beta <= -1 : mean of the middle -beta values of the sorted column (m + beta even): the trimmed mean
 detox_status launch_coord_select(const float* X, int64_t ld, int m, int64_t d, const int32_t* rows_dev,
                                  int beta, float* out, cudaStream_t s);
 

@@ -70,16 +70,18 @@ colselect_smem_kernel(const float* __restrict__ X, int64_t ld, int m, int64_t d,
         if (beta == 0) {
             out[col] = med;
         } else {
-            const int L = window_start(m, beta, med, [&](int i) { return keys[i * kTileCols + c]; });
+            const int cnt = beta < 0 ? -beta : beta;   // beta < 0: the middle -beta values (trimmed mean)
+            const int L = beta < 0 ? (m - cnt) >> 1
+                                   : window_start(m, beta, med, [&](int i) { return keys[i * kTileCols + c]; });
             // compensated fp32 sum over up to 1024 values
             float acc = 0.f, comp = 0.f;
-            for (int i = L; i < L + beta; ++i) {
+            for (int i = L; i < L + cnt; ++i) {
                 const float y = float_of_key(keys[i * kTileCols + c]) - comp;
                 const float t = acc + y;
                 comp = (t - acc) - y;
                 acc = t;
             }
-            out[col] = acc / (float)beta;
+            out[col] = acc / (float)cnt;
         }
     }
 }

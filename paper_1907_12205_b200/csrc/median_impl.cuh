@@ -98,12 +98,15 @@ colselect_reg_kernel(const float* __restrict__ X, int64_t ld, int m, int64_t d, 
             int32_t* mine = sorted + (size_t)c * M * kThreads + threadIdx.x;
 #pragma unroll
             for (int i = 0; i < M; ++i) mine[i * kThreads] = key[c][i];
-            const int L = pad + window_start(m, beta, med, [&](int i) { return mine[(i + pad) * kThreads]; });
+            // beta > 0: the beta values closest to the median; beta < 0: the middle -beta values (trimmed mean)
+            const int cnt = beta < 0 ? -beta : beta;
+            const int L = pad + (beta < 0 ? (m - cnt) >> 1
+                                          : window_start(m, beta, med, [&](int i) { return mine[(i + pad) * kThreads]; }));
             float acc = 0.f;
 #pragma unroll
             for (int i = 0; i < M; ++i)
-                if (i >= L && i < L + beta) acc += float_of_key(key[c][i]);
-            res[c] = acc / (float)beta;
+                if (i >= L && i < L + cnt) acc += float_of_key(key[c][i]);
+            res[c] = acc / (float)cnt;
         }
     }
     if (C == 4 && valid == 4) {

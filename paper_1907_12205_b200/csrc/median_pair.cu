@@ -93,15 +93,17 @@ colselect_pair_kernel(const float* __restrict__ X, int64_t ld, int m, int64_t d,
         auto at = [&](int p) { return sorted[p * kPairCols + ((cidx + (p >= kHalf ? 16 : 0)) & (kPairCols - 1))]; };
         float med = float_of_key(at(kHalf - 1));
         if ((m & 1) == 0) med = (med + float_of_key(at(kHalf))) * 0.5f;
-        const int L = pad_lo + regselect::window_start(m, beta, med, [&](int i) { return at(i + pad_lo); });
+        const int cnt = beta < 0 ? -beta : beta;   // beta < 0: the middle -beta values (trimmed mean)
+        const int L = pad_lo + (beta < 0 ? (m - cnt) >> 1
+                                         : regselect::window_start(m, beta, med, [&](int i) { return at(i + pad_lo); }));
         float acc = 0.f, comp = 0.f;          // compensated fp32 sum
-        for (int p = L; p < L + beta; ++p) {
+        for (int p = L; p < L + cnt; ++p) {
             const float y = float_of_key(at(p)) - comp;
             const float t = acc + y;
             comp = (t - acc) - y;
             acc = t;
         }
-        out[col] = acc / (float)beta;
+        out[col] = acc / (float)cnt;
     }
 }
 
@@ -131,7 +133,7 @@ detox_status launch_pair(const float* X, int64_t ld, int m, int64_t d, const int
 detox_status launch_pair_select(const float* X, int64_t ld, int m, int64_t d, const int32_t* rows, int beta,
                                 float* out, cudaStream_t s) {
     int H = ((m + 1) / 2 + 7) / 8 * 8;
-    if (beta > 0) H = 128;
+    if (beta != 0) H = 128;
     switch (H) {
 #define DETOX_CASE(HH) \
     case HH: return launch_pair<HH>(X, ld, m, d, rows, beta, out, s);

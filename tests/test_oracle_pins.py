@@ -384,3 +384,15 @@ def test_pipeline_krum_family_inside_vote_sets():
     direct, sel, _ = oracle.bulyan(res["Z"][sm], 2)
     assert np.array_equal(res["out"], direct) and res["sel"].tolist() == sm[sel].tolist()
     assert bad not in res["sel"].tolist()
+
+
+def test_trimmed_mean_against_library_and_reductions():
+    from scipy import stats
+    X = rng(40).standard_normal((12, 300)).astype(np.float32)
+    np.testing.assert_allclose(oracle.trimmed_mean(X, 3), stats.trim_mean(X.astype(np.float64), 0.25, axis=0),
+                               rtol=1e-6)
+    assert np.array_equal(oracle.trimmed_mean(X, 0), (X.astype(np.float64).sum(0) / 12).astype(np.float32))
+    Y = rng(41).standard_normal((9, 50)).astype(np.float32)
+    assert np.array_equal(oracle.trimmed_mean(Y, 4), np.median(Y, axis=0))      # one value left: the median
+    Z = np.array([[5.0], [1.0], [100.0], [3.0], [-7.0]], np.float32)            # sorted -7 1 3 5 100
+    assert oracle.trimmed_mean(Z, 1).tolist() == [3.0]

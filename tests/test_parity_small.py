@@ -127,6 +127,15 @@ def test_coord_median_special_values(m):
     assert np.array_equal(bits(got), oracle.coord_median(X).view(np.uint32))
 
 
+@pytest.mark.parametrize("m,trim", [(5, 1), (7, 0), (12, 3), (15, 7), (27, 6), (35, 8), (64, 16), (105, 26), (225, 56),
+                                    (300, 75)])
+def test_trimmed_mean_matches_oracle(m, trim):
+    X = (np.random.default_rng(m).standard_normal((m, 2000 + m)) * 1e-3).astype(np.float32)
+    X[0] *= -100
+    got = dx.agg_trimmed_mean(padded(X), trim)
+    assert rel_l2(got.cpu().numpy(), oracle.trimmed_mean(X, trim)) <= TOL
+
+
 # ------------------------------------------------------------------------------------ Multi-Krum
 
 def krum_inputs(m, d, seed, copies=1, outliers=0):
