@@ -241,6 +241,8 @@ def detox_aggregate(X, members, r: int, a0: str, set_offsets, set_members, a1: s
         out = mean_rows(rows)
     elif a1 == "coord_median":
         out = coord_median(rows)
+    elif a1 == "trimmed_mean":
+        out = trimmed_mean(rows, f)
     elif a1 == "multikrum":
         out, sel, _, _ = multikrum(rows, f, m_sel)
     elif a1 == "bulyan":

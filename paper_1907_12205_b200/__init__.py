@@ -8,6 +8,7 @@ from .binding import (  # noqa: F401
     AGG_MEAN,
     AGG_MULTIKRUM,
     AGG_NONE,
+    AGG_TRIMMED_MEAN,
     EXPORTS,
     LIB_PATH,
     DetoxError,

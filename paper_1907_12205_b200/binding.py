@@ -17,7 +17,7 @@ import torch
 _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "libdetox.so")
 
-AGG_NONE, AGG_MEAN, AGG_COORD_MEDIAN, AGG_MULTIKRUM, AGG_BULYAN = 0, 1, 2, 3, 4
+AGG_NONE, AGG_MEAN, AGG_COORD_MEDIAN, AGG_MULTIKRUM, AGG_BULYAN, AGG_TRIMMED_MEAN = 0, 1, 2, 3, 4, 5
 MAX_ROWS, MAX_R = 1024, 15
 
 EXPORTS = (

@@ -179,7 +179,7 @@ detox_status check_desc(const detox_pipeline_desc* p) {
     if (p->a0 != DETOX_AGG_NONE && (p->n_sets < 1 || p->n_sets > G)) return DETOX_ERR_BAD_ARG;
     if (krum_type(p->a0)) {
         // Multi-Krum / Bulyan inside every vote set (f, m_sel belong to A_0), then a plain A_1 over the set results
-        if (p->a1 != DETOX_AGG_MEAN && p->a1 != DETOX_AGG_COORD_MEDIAN) return DETOX_ERR_UNSUPPORTED;
+        if (p->a1 != DETOX_AGG_MEAN && p->a1 != DETOX_AGG_COORD_MEDIAN) return DETOX_ERR_UNSUPPORTED;  // f is A_0's
         if (!p->set_offsets || p->f < 0 || p->m_sel < 0) return DETOX_ERR_BAD_ARG;
         if (p->set_offsets[0] != 0 || p->set_offsets[p->n_sets] != G) return DETOX_ERR_BAD_ARG;
         for (int s = 0; s < p->n_sets; ++s) {
@@ -194,6 +194,7 @@ detox_status check_desc(const detox_pipeline_desc* p) {
     switch (p->a1) {
         case DETOX_AGG_MEAN:
         case DETOX_AGG_COORD_MEDIAN: return DETOX_OK;
+        case DETOX_AGG_TRIMMED_MEAN: return (p->f >= 0 && rows1 - 2 * p->f >= 1) ? DETOX_OK : DETOX_ERR_BAD_ARG;
         case DETOX_AGG_MULTIKRUM: return check_multikrum(rows1, p->f, p->m_sel);
         case DETOX_AGG_BULYAN: return check_bulyan(rows1, p->f);
         default: return DETOX_ERR_BAD_ARG;
@@ -378,6 +379,9 @@ detox_status detox_aggregate(const detox_pipeline_desc* p, const float* X, int64
     switch (p->a1) {
         case DETOX_AGG_MEAN: st = launch_mean_rows(rows, w.ldz, p->d, nullptr, m, out, s); break;
         case DETOX_AGG_COORD_MEDIAN: st = launch_coord_select(rows, w.ldz, m, p->d, nullptr, 0, out, s); break;
+        case DETOX_AGG_TRIMMED_MEAN:
+            st = launch_coord_select(rows, w.ldz, m, p->d, nullptr, -(m - 2 * p->f), out, s);
+            break;
         case DETOX_AGG_MULTIKRUM:
             cnt = p->m_sel;
             sel_buf = sel ? sel : krum_ws(w.agg, m, p->d).sel;
