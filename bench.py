@@ -50,6 +50,13 @@ def pipeline_for(name, w, dx):
 
 ORACLE_A1 = {1: "mean", 2: "coord_median", 3: "multikrum", 4: "bulyan"}
 
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu captures summarised in
+# profiles/vote_kernels_cfg2.md (same kernel code; reset an entry to None when its kernel changes).
+NCU_TRAFFIC_BYTES = {
+    ("cfg2", "vote_mean_kernel"): 2_011_333_000 + 117_863_424,
+    ("cfg3", "vote_kernel"): 2_011_359_000 + 639_171_584,      # same shape as config 2's vote
+}
+
 
 class ClockSampler:
     """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
@@ -391,7 +398,7 @@ def main():
     roofline = {"kernel": dom_name, "bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"],
                 "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
                 "frac_of_8TBps": achieved / 8000.0, "ms_per_launch": vote_ms, "algorithmic_bytes": vote_bytes,
-                "traffic": None}
+                "traffic": NCU_TRAFFIC_BYTES.get((args.workload, dom_name))}
 
     cpu_baseline = None
     parity = None
