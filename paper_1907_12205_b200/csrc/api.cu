@@ -59,6 +59,7 @@ struct KrumWs {
     void* dist;
     void* select;
     int32_t* sel;
+    int32_t* mapped;   // the selection as rows of X when the m rows are given by a row list
     size_t total;
 };
 
@@ -76,33 +77,47 @@ KrumWs krum_ws(void* ws, int m, int64_t d) {
     off += select_ws_bytes(m);
     k.sel = reinterpret_cast<int32_t*>(p + off);
     off += align_up((size_t)m * sizeof(int32_t));
+    k.mapped = reinterpret_cast<int32_t*>(p + off);
+    off += align_up((size_t)m * sizeof(int32_t));
     k.total = off;
     return k;
 }
 
-detox_status run_multikrum(const float* X, int64_t ld, int m, int64_t d, int f, int m_sel, float* out, int32_t* sel,
-                           double* scores, void* ws, cudaStream_t s) {
+// `rows` (optional, device, m <= 16): the m rows are X[rows[i]], a negative entry standing for a zero row
+// (this is how the votes are consumed straight from the workers' rows through winner[], without a copy).
+detox_status run_multikrum(const float* X, int64_t ld, int m, int64_t d, const int32_t* rows, int f, int m_sel,
+                           float* out, int32_t* sel, double* scores, void* ws, cudaStream_t s) {
     KrumWs k = krum_ws(ws, m, d);
     int32_t* sel_buf = sel ? sel : k.sel;
     if (cudaMemsetAsync(k.status, 0, sizeof(int), s) != cudaSuccess) return DETOX_ERR_CUDA;
-    detox_status st = launch_sqdist(X, ld, m, d, k.D, k.dist, k.status, s);
+    detox_status st = launch_sqdist(X, ld, m, d, rows, k.D, k.dist, k.status, s);
     if (st != DETOX_OK) return st;
     st = launch_multikrum_select(k.D, m, f, m_sel, sel_buf, scores, k.select, s);
     if (st != DETOX_OK) return st;
-    return launch_mean_rows(X, ld, d, sel_buf, m_sel, out, s);
+    const int32_t* take = sel_buf;
+    if (rows) {
+        if ((st = launch_map_indices(sel_buf, rows, m_sel, k.mapped, s)) != DETOX_OK) return st;
+        take = k.mapped;
+    }
+    return launch_mean_rows(X, ld, d, take, m_sel, out, s);
 }
 
-detox_status run_bulyan(const float* X, int64_t ld, int m, int64_t d, int f, float* out, int32_t* sel, void* ws,
-                        cudaStream_t s) {
+detox_status run_bulyan(const float* X, int64_t ld, int m, int64_t d, const int32_t* rows, int f, float* out,
+                        int32_t* sel, void* ws, cudaStream_t s) {
     KrumWs k = krum_ws(ws, m, d);
     int32_t* sel_buf = sel ? sel : k.sel;
     const int theta = m - 2 * f, beta = theta - 2 * f;
     if (cudaMemsetAsync(k.status, 0, sizeof(int), s) != cudaSuccess) return DETOX_ERR_CUDA;
-    detox_status st = launch_sqdist(X, ld, m, d, k.D, k.dist, k.status, s);
+    detox_status st = launch_sqdist(X, ld, m, d, rows, k.D, k.dist, k.status, s);
     if (st != DETOX_OK) return st;
     st = launch_bulyan_select(k.D, m, f, sel_buf, k.select, s);
     if (st != DETOX_OK) return st;
-    return launch_coord_select(X, ld, theta, d, sel_buf, beta, out, s);
+    const int32_t* take = sel_buf;
+    if (rows) {
+        if ((st = launch_map_indices(sel_buf, rows, theta, k.mapped, s)) != DETOX_OK) return st;
+        take = k.mapped;
+    }
+    return launch_coord_select(X, ld, theta, d, take, beta, out, s);
 }
 
 detox_status check_multikrum(int m, int f, int m_sel) {
@@ -123,6 +138,14 @@ bool krum_type(int a) { return a == DETOX_AGG_MULTIKRUM || a == DETOX_AGG_BULYAN
 int a0_selected(const detox_pipeline_desc* p, int k) {
     if (p->a0 == DETOX_AGG_BULYAN) return k - 2 * p->f;
     return p->m_sel > 0 ? p->m_sel : (k - p->f > 1 ? k - p->f : 1);
+}
+
+// With A_0 = none the votes are rows of X, so A_1 can read them through winner[] and the votes need not be
+// written: always for the per-coordinate aggregators, and for the Krum type up to 16 votes (the
+// direct-difference distance kernel takes a row list; the tensor-core Gram wants consecutive rows).
+bool votes_by_index(const detox_pipeline_desc* p) {
+    if (p->a0 != DETOX_AGG_NONE) return false;
+    return !krum_type(p->a1) || p->n / p->r <= 16;
 }
 
 struct PipeWs {
@@ -149,7 +172,8 @@ PipeWs pipe_ws(void* ws, const detox_pipeline_desc* p) {
     w.winner = reinterpret_cast<int32_t*>(base + off);
     off += align_up((size_t)G * sizeof(int32_t));
     w.Z = reinterpret_cast<float*>(base + off);
-    if (p->a0 != DETOX_AGG_MEAN) off += align_up((size_t)G * w.ldz * sizeof(float));   // votes are stored only then
+    if (p->a0 != DETOX_AGG_MEAN && !votes_by_index(p))
+        off += align_up((size_t)G * w.ldz * sizeof(float));   // the votes are stored only when a stage needs them as a matrix
     w.M = reinterpret_cast<float*>(base + off);
     if (p->a0 != DETOX_AGG_NONE) off += align_up((size_t)p->n_sets * w.ldz * sizeof(float));
     w.winner_set_order = reinterpret_cast<int32_t*>(base + off);
@@ -293,7 +317,7 @@ detox_status agg_multikrum(const float* X, int64_t ld, int m, int64_t d, int f, 
     if ((st = check_multikrum(m, f, m_sel)) != DETOX_OK) return st;
     if (!out || (reinterpret_cast<uintptr_t>(out) & 3u)) return DETOX_ERR_BAD_ARG;
     if (!ws_ok(ws, ws_bytes, krum_ws(nullptr, m, d).total)) return DETOX_ERR_WORKSPACE;
-    return run_multikrum(X, ld, m, d, f, m_sel, out, sel, scores, ws, static_cast<cudaStream_t>(stream));
+    return run_multikrum(X, ld, m, d, nullptr, f, m_sel, out, sel, scores, ws, static_cast<cudaStream_t>(stream));
 }
 
 size_t agg_bulyan_workspace_bytes(int m, int64_t d) {
@@ -308,7 +332,7 @@ detox_status agg_bulyan(const float* X, int64_t ld, int m, int64_t d, int f, flo
     if ((st = check_bulyan(m, f)) != DETOX_OK) return st;
     if (!out || (reinterpret_cast<uintptr_t>(out) & 3u)) return DETOX_ERR_BAD_ARG;
     if (!ws_ok(ws, ws_bytes, krum_ws(nullptr, m, d).total)) return DETOX_ERR_WORKSPACE;
-    return run_bulyan(X, ld, m, d, f, out, sel, ws, static_cast<cudaStream_t>(stream));
+    return run_bulyan(X, ld, m, d, nullptr, f, out, sel, ws, static_cast<cudaStream_t>(stream));
 }
 
 size_t detox_aggregate_workspace_bytes(const detox_pipeline_desc* desc) {
@@ -336,6 +360,8 @@ detox_status detox_aggregate(const detox_pipeline_desc* p, const float* X, int64
 
     // filtering step, then A_0, then A_1 (the mean as A_0 is folded into the vote's pass)
     const float* rows = w.Z;
+    int64_t row_ld = w.ldz;
+    const int32_t* row_list = nullptr;
     int m = G;
     if (p->a0 == DETOX_AGG_MEAN) {
         if ((st = launch_vote_mean(X, ld, p->n, p->r, p->d, groups, sets, p->n_sets, w.M, w.ldz, win, w.vote, s)) !=
@@ -361,8 +387,8 @@ detox_status detox_aggregate(const detox_pipeline_desc* p, const float* X, int64
             const float* rows_t = w.Z + (int64_t)b * w.ldz;
             float* out_t = w.M + (int64_t)t * w.ldz;
             st = p->a0 == DETOX_AGG_MULTIKRUM
-                     ? run_multikrum(rows_t, w.ldz, k, p->d, p->f, keep, out_t, w.sel_local, nullptr, w.agg, s)
-                     : run_bulyan(rows_t, w.ldz, k, p->d, p->f, out_t, w.sel_local, w.agg, s);
+                     ? run_multikrum(rows_t, w.ldz, k, p->d, nullptr, p->f, keep, out_t, w.sel_local, nullptr, w.agg, s)
+                     : run_bulyan(rows_t, w.ldz, k, p->d, nullptr, p->f, out_t, w.sel_local, w.agg, s);
             if (st != DETOX_OK) return st;
             st = launch_map_set_selection(w.sel_local, keep, sets, b, w.winner_set_order, sel ? sel + emitted : nullptr,
                                           sel_workers ? sel_workers + emitted : nullptr, s);
@@ -371,26 +397,33 @@ detox_status detox_aggregate(const detox_pipeline_desc* p, const float* X, int64
         }
         rows = w.M;
         m = p->n_sets;
+    } else if (votes_by_index(p)) {
+        // The votes are rows of X: only winner[] is produced and A_1 reads the winners' rows through it
+        // (a group without a majority has winner -1, which the consumers take as a zero row).
+        if ((st = launch_vote(X, ld, p->n, p->r, p->d, groups, nullptr, 0, win, w.vote, s)) != DETOX_OK) return st;
+        rows = X;
+        row_ld = ld;
+        row_list = win;
     } else if ((st = launch_vote(X, ld, p->n, p->r, p->d, groups, w.Z, w.ldz, win, w.vote, s)) != DETOX_OK) {
         return st;
     }
     int cnt = 0;
     int32_t* sel_buf = nullptr;
     switch (p->a1) {
-        case DETOX_AGG_MEAN: st = launch_mean_rows(rows, w.ldz, p->d, nullptr, m, out, s); break;
-        case DETOX_AGG_COORD_MEDIAN: st = launch_coord_select(rows, w.ldz, m, p->d, nullptr, 0, out, s); break;
+        case DETOX_AGG_MEAN: st = launch_mean_rows(rows, row_ld, p->d, row_list, m, out, s); break;
+        case DETOX_AGG_COORD_MEDIAN: st = launch_coord_select(rows, row_ld, m, p->d, row_list, 0, out, s); break;
         case DETOX_AGG_TRIMMED_MEAN:
-            st = launch_coord_select(rows, w.ldz, m, p->d, nullptr, -(m - 2 * p->f), out, s);
+            st = launch_coord_select(rows, row_ld, m, p->d, row_list, -(m - 2 * p->f), out, s);
             break;
         case DETOX_AGG_MULTIKRUM:
             cnt = p->m_sel;
             sel_buf = sel ? sel : krum_ws(w.agg, m, p->d).sel;
-            st = run_multikrum(rows, w.ldz, m, p->d, p->f, p->m_sel, out, sel_buf, nullptr, w.agg, s);
+            st = run_multikrum(rows, row_ld, m, p->d, row_list, p->f, p->m_sel, out, sel_buf, nullptr, w.agg, s);
             break;
         case DETOX_AGG_BULYAN:
             cnt = m - 2 * p->f;
             sel_buf = sel ? sel : krum_ws(w.agg, m, p->d).sel;
-            st = run_bulyan(rows, w.ldz, m, p->d, p->f, out, sel_buf, w.agg, s);
+            st = run_bulyan(rows, row_ld, m, p->d, row_list, p->f, out, sel_buf, w.agg, s);
             break;
         default: st = DETOX_ERR_BAD_ARG;
     }

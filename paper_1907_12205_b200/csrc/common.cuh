@@ -72,11 +72,12 @@ detox_status launch_vote_mean(const float* X, int64_t ld, int n, int r, int64_t 
 // mean.cu
 detox_status launch_hier_mean(const float* Z, int64_t ldz, int64_t d, const SetTable& sets, int S,
                               float* M, int64_t ldm, cudaStream_t s);
-// mean of k rows of X listed in rows_dev (device int32; NULL = rows 0..k-1)
+// mean of k rows of X listed in rows_dev (device int32; NULL = rows 0..k-1; a negative entry = a zero row)
 detox_status launch_mean_rows(const float* X, int64_t ld, int64_t d, const int32_t* rows_dev, int k,
                               float* out, cudaStream_t s);
 
-// median.cu: per-coordinate order statistics over m rows (rows_dev: device int32 list or NULL)
+// median.cu: per-coordinate order statistics over m rows (rows_dev: device int32 list or NULL; a negative
+// entry = a zero row)
 //   beta == 0 : coordinate median;  beta >= 1 : mean of the beta values closest to the median;
 //   beta <= -1 : mean of the middle -beta values of the sorted column (m + beta even): the trimmed mean
 detox_status launch_coord_select(const float* X, int64_t ld, int m, int64_t d, const int32_t* rows_dev,
@@ -86,8 +87,9 @@ detox_status launch_coord_select(const float* X, int64_t ld, int m, int64_t d, c
 //   status: device int32, must be 0 on entry; set to DETOX_ERR_TIMEOUT (and D to NaN) if a bounded
 //   device-side wait of the tensor-core path runs out
 size_t dist_ws_bytes(int m, int64_t d);
-detox_status launch_sqdist(const float* X, int64_t ld, int m, int64_t d, double* D, void* ws, int* status,
-                           cudaStream_t s);
+//   rows: optional device list of the m rows of X to use (m <= 16 only); a negative entry stands for a zero row
+detox_status launch_sqdist(const float* X, int64_t ld, int m, int64_t d, const int32_t* rows, double* D, void* ws,
+                           int* status, cudaStream_t s);
 
 // gram_tc.cu: the tcgen05 path for 16 < m <= 256 (needs 16-byte aligned rows)
 bool tc_supported(const float* X, int64_t ld, int m, int64_t d);

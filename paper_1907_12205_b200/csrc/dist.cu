@@ -20,11 +20,21 @@ constexpr int kDirWarps = kDirThreads / 32;
 
 template <int M>
 __global__ void __launch_bounds__(kDirThreads)
-sqdist_direct_kernel(const float* __restrict__ X, int64_t ld, int64_t d, bool vec2, double* __restrict__ partial) {
+sqdist_direct_kernel(const float* __restrict__ X, int64_t ld, int64_t d, const int32_t* __restrict__ rows,
+                     bool vec2, double* __restrict__ partial) {
     constexpr int NP = M * (M - 1) / 2;
     float acc[NP];
 #pragma unroll
     for (int p = 0; p < NP; ++p) acc[p] = 0.f;
+    // rows (optional): the M rows are X[rows[i]]; a negative entry stands for a zero row
+    const float* rowp[M];
+    float keep[M];
+#pragma unroll
+    for (int i = 0; i < M; ++i) {
+        const int r = rows ? rows[i] : i;
+        rowp[i] = X + (int64_t)(r < 0 ? 0 : r) * ld;
+        keep[i] = r < 0 ? 0.f : 1.f;
+    }
 
     const int64_t stride = (int64_t)gridDim.x * kDirThreads;
     if (vec2) {
@@ -32,7 +42,10 @@ sqdist_direct_kernel(const float* __restrict__ X, int64_t ld, int64_t d, bool ve
         for (int64_t c = (int64_t)blockIdx.x * kDirThreads + threadIdx.x; c < n2; c += stride) {
             float2 v[M];
 #pragma unroll
-            for (int i = 0; i < M; ++i) v[i] = __ldcs(reinterpret_cast<const float2*>(X + (int64_t)i * ld) + c);
+            for (int i = 0; i < M; ++i) {
+                v[i] = __ldcs(reinterpret_cast<const float2*>(rowp[i]) + c);
+                if (keep[i] == 0.f) v[i] = make_float2(0.f, 0.f);
+            }
             int p = 0;
 #pragma unroll
             for (int i = 0; i < M; ++i)
@@ -49,7 +62,7 @@ sqdist_direct_kernel(const float* __restrict__ X, int64_t ld, int64_t d, bool ve
             for (int i = 0; i < M; ++i)
 #pragma unroll
                 for (int j = i + 1; j < M; ++j, ++p) {
-                    const float a = X[(int64_t)i * ld + d - 1] - X[(int64_t)j * ld + d - 1];
+                    const float a = (keep[i] == 0.f ? 0.f : rowp[i][d - 1]) - (keep[j] == 0.f ? 0.f : rowp[j][d - 1]);
                     acc[p] = fmaf(a, a, acc[p]);
                 }
         }
@@ -57,7 +70,10 @@ sqdist_direct_kernel(const float* __restrict__ X, int64_t ld, int64_t d, bool ve
         for (int64_t c = (int64_t)blockIdx.x * kDirThreads + threadIdx.x; c < d; c += stride) {
             float v[M];
 #pragma unroll
-            for (int i = 0; i < M; ++i) v[i] = __ldcs(X + (int64_t)i * ld + c);
+            for (int i = 0; i < M; ++i) {
+                v[i] = __ldcs(rowp[i] + c);
+                if (keep[i] == 0.f) v[i] = 0.f;
+            }
             int p = 0;
 #pragma unroll
             for (int i = 0; i < M; ++i)
@@ -238,10 +254,11 @@ int direct_blocks(int64_t d) {
 }
 
 template <int M>
-detox_status launch_direct(const float* X, int64_t ld, int64_t d, double* D, double* partial, cudaStream_t s) {
+detox_status launch_direct(const float* X, int64_t ld, int64_t d, const int32_t* rows, double* D, double* partial,
+                           cudaStream_t s) {
     const int nb = direct_blocks(d);
     const bool vec2 = (reinterpret_cast<uintptr_t>(X) & 7u) == 0 && ld % 2 == 0;
-    sqdist_direct_kernel<M><<<nb, kDirThreads, 0, s>>>(X, ld, d, vec2, partial);
+    sqdist_direct_kernel<M><<<nb, kDirThreads, 0, s>>>(X, ld, d, rows, vec2, partial);
     detox_status st = launch_status();
     if (st != DETOX_OK) return st;
     sqdist_direct_reduce_kernel<<<(M * (M - 1) / 2 + 3) / 4, 128, 0, s>>>(partial, nb, M, D);
@@ -258,14 +275,15 @@ size_t dist_ws_bytes(int m, int64_t d) {
     return simt > tc ? simt : tc;
 }
 
-detox_status launch_sqdist(const float* X, int64_t ld, int m, int64_t d, double* D, void* ws, int* status,
-                           cudaStream_t s) {
+detox_status launch_sqdist(const float* X, int64_t ld, int m, int64_t d, const int32_t* rows, double* D, void* ws,
+                           int* status, cudaStream_t s) {
     double* partial = static_cast<double*>(ws);
+    if (rows && m > 16) return DETOX_ERR_UNSUPPORTED;   // only the direct kernel takes a row list
     switch (m) {
         case 1:
             return cudaMemsetAsync(D, 0, sizeof(double), s) == cudaSuccess ? DETOX_OK : DETOX_ERR_CUDA;
 #define DETOX_CASE(M) \
-    case M: return launch_direct<M>(X, ld, d, D, partial, s);
+    case M: return launch_direct<M>(X, ld, d, rows, D, partial, s);
         DETOX_CASE(2) DETOX_CASE(3) DETOX_CASE(4) DETOX_CASE(5) DETOX_CASE(6) DETOX_CASE(7) DETOX_CASE(8)
         DETOX_CASE(9) DETOX_CASE(10) DETOX_CASE(11) DETOX_CASE(12) DETOX_CASE(13) DETOX_CASE(14) DETOX_CASE(15)
         DETOX_CASE(16)

@@ -18,6 +18,14 @@ struct Acc<4> {
     __device__ __forceinline__ void div(float k) { a.x /= k; a.y /= k; a.z /= k; a.w /= k; }
 };
 
+// Row r of X at column `col`; a negative r stands for a zero row.
+__device__ __forceinline__ const float* row_ptr(const float* X, int64_t ld, int r, int64_t col) {
+    return X + (int64_t)(r < 0 ? 0 : r) * ld + col;
+}
+__device__ __forceinline__ float4 mask_piece(float4 v, int r) {
+    return r < 0 ? make_float4(0.f, 0.f, 0.f, 0.f) : v;
+}
+
 __device__ __forceinline__ float4 load_piece(const float* p, int valid) {
     if (valid >= 4) return ld_stream_f4(p);
     float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -46,18 +54,26 @@ __device__ __forceinline__ void mean_columns(const float* __restrict__ X, int64_
         acc.zero();
         int t = 0;
         for (; t + 4 <= k; t += 4) {
-            float4 v0 = load_piece(X + (int64_t)row_of(t) * ld + col, valid);
-            float4 v1 = load_piece(X + (int64_t)row_of(t + 1) * ld + col, valid);
-            float4 v2 = load_piece(X + (int64_t)row_of(t + 2) * ld + col, valid);
-            float4 v3 = load_piece(X + (int64_t)row_of(t + 3) * ld + col, valid);
-            acc.add(v0); acc.add(v1); acc.add(v2); acc.add(v3);
+            const int r0 = row_of(t), r1 = row_of(t + 1), r2 = row_of(t + 2), r3 = row_of(t + 3);
+            float4 v0 = load_piece(row_ptr(X, ld, r0, col), valid);
+            float4 v1 = load_piece(row_ptr(X, ld, r1, col), valid);
+            float4 v2 = load_piece(row_ptr(X, ld, r2, col), valid);
+            float4 v3 = load_piece(row_ptr(X, ld, r3, col), valid);
+            acc.add(mask_piece(v0, r0)); acc.add(mask_piece(v1, r1)); acc.add(mask_piece(v2, r2)); acc.add(mask_piece(v3, r3));
         }
-        for (; t < k; ++t) acc.add(load_piece(X + (int64_t)row_of(t) * ld + col, valid));
+        for (; t < k; ++t) {
+            const int r = row_of(t);
+            acc.add(mask_piece(load_piece(row_ptr(X, ld, r, col), valid), r));
+        }
         acc.div((float)k);
         store_piece(out + col, acc.a, valid);
     } else {
         float acc = 0.f;
-        for (int t = 0; t < k; ++t) acc += __ldcs(X + (int64_t)row_of(t) * ld + col);
+        for (int t = 0; t < k; ++t) {
+            const int r = row_of(t);
+            const float v = __ldcs(row_ptr(X, ld, r, col));
+            acc += r < 0 ? 0.f : v;
+        }
         out[col] = acc / (float)k;
     }
 }

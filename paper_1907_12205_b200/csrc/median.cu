@@ -33,8 +33,8 @@ colselect_smem_kernel(const float* __restrict__ X, int64_t ld, int m, int64_t d,
     const bool live = col < d;
 
     for (int i = w; i < m; i += kBigWarps) {
-        const int64_t r = rows ? rows[i] : i;
-        keys[i * kTileCols + c] = live ? key_of_bits(ld_stream_u1(X + r * ld + col)) : 0;
+        const int64_t r = rows ? rows[i] : i;     // a negative entry of the row list stands for a zero row
+        keys[i * kTileCols + c] = (live && r >= 0) ? key_of_bits(ld_stream_u1(X + r * ld + col)) : key_of_bits(0u);
     }
     __syncthreads();
 

@@ -36,7 +36,9 @@ colselect_pair_kernel(const float* __restrict__ X, int64_t ld, int m, int64_t d,
     for (int i = 0; i < kHalf; ++i) {
         int ri = hsel ? kHalf + i : i;
         ri = ri < m ? ri : m - 1;
-        key[i] = (int32_t)ld_stream_u1(X + (int64_t)(rows ? rows[ri] : ri) * ld + col);
+        const int rr = rows ? rows[ri] : ri;      // a negative entry of the row list stands for a zero row
+        const uint32_t v = ld_stream_u1(X + (int64_t)(rr < 0 ? 0 : rr) * ld + col);
+        key[i] = (int32_t)(rr < 0 ? 0u : v);
     }
 #pragma unroll
     for (int i = 0; i < kHalf; ++i) {

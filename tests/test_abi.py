@@ -46,8 +46,10 @@ def test_workspace_sizes(lib):
     assert dx.agg_multikrum_workspace_bytes(5000, 1000) == 0
     p = dx.Pipeline(45, 3, 1000, np.arange(45), dx.AGG_MEAN, [0, 5, 10, 15], np.arange(15), dx.AGG_MULTIKRUM, 1, 1)
     assert p.workspace_bytes() > 3 * 1024 * 4                   # the three set means (votes are not stored)
+    q = dx.Pipeline(105, 3, 1000, np.arange(105), dx.AGG_NONE, None, None, dx.AGG_MULTIKRUM, 3, 30)
+    assert q.workspace_bytes() > 35 * 1024 * 4                  # the 35 votes, stored for the Gram kernel
     q = dx.Pipeline(45, 3, 1000, np.arange(45), dx.AGG_NONE, None, None, dx.AGG_COORD_MEDIAN)
-    assert q.workspace_bytes() > 15 * 1024 * 4                  # the fifteen votes
+    assert 0 < q.workspace_bytes() < 15 * 1000 * 4              # votes are read through winner[]: no copy
     bad = dx.Pipeline(45, 3, 1000, np.arange(45), dx.AGG_NONE, None, None, dx.AGG_BULYAN, 4, 1)  # 15 < 4*4+3
     assert bad.workspace_bytes() == 0
 
