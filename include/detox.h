@@ -139,6 +139,18 @@ detox_status agg_coord_median(const float* X, int64_t ld, int m, int64_t d, floa
 detox_status agg_trimmed_mean(const float* X, int64_t ld, int m, int64_t d, int trim, float* out, void* stream);
 
 /* ---------------------------------------------------------------------------------------------
+ * Geometric median (one of the A_1 choices analysed in Section 4, Theorem 4; the paper does not fix
+ * an algorithm).  Computed by Weiszfeld's iteration started at the mean:
+ *     y <- sum_j w_j x_j / sum_j w_j,   w_j = 1 / max(||x_j - y||_2, eps),   `iters` times.
+ * m <= 32 rows (it aggregates the few set results of the hierarchical step); more returns
+ * DETOX_ERR_UNSUPPORTED.  iters >= 0 (0 gives the mean), eps > 0.
+ *   out  dev, d.   ws: agg_geometric_median_workspace_bytes(m, d) bytes.
+ * ------------------------------------------------------------------------------------------- */
+size_t agg_geometric_median_workspace_bytes(int m, int64_t d);
+detox_status agg_geometric_median(const float* X, int64_t ld, int m, int64_t d, int iters, float eps, float* out,
+                                  void* ws, size_t ws_bytes, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
  * Multi-Krum (cited in Section 4 "Improved speed" as the O(p^2 d) aggregator; requirement
  * m >= 2f+3 in Appendix B.1).  score_i = sum of the nb smallest squared distances from row i to the
  * other rows, nb = m - f - 2 clamped to [1, m-1]; the m_sel rows of smallest score (equal scores:

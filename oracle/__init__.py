@@ -56,6 +56,7 @@ def _load():
         lib.oracle_bulyan_select.argtypes = [_D, _int, _int, _I]
         lib.oracle_trimmed_around_median.argtypes = [_F, _i64, _i64, _I, _int, _int, _F]
         lib.oracle_trimmed_mean.argtypes = [_F, _i64, _int, _i64, _int, _F]
+        lib.oracle_geometric_median.argtypes = [_F, _i64, _int, _i64, _int, ctypes.c_double, _F]
         lib.oracle_bulyan.argtypes = [_F, _i64, _int, _i64, _int, _F, _I, _D]
         _lib = lib
     return _lib
@@ -141,6 +142,14 @@ def trimmed_mean(X, trim: int):
     m, d = X.shape
     out = np.empty(d, dtype=np.float32)
     _check(_load().oracle_trimmed_mean(_fp(X), ld, m, d, trim, _fp(out)), "trimmed_mean")
+    return out
+
+
+def geometric_median(X, iters: int = 32, eps: float = 1e-12):
+    X, ld = _mat(X)
+    m, d = X.shape
+    out = np.empty(d, dtype=np.float32)
+    _check(_load().oracle_geometric_median(_fp(X), ld, m, d, iters, float(eps), _fp(out)), "geometric_median")
     return out
 
 

@@ -331,6 +331,43 @@ int oracle_trimmed_mean(const float* X, int64_t ld, int m, int64_t d, int trim, 
     return 0;
 }
 
+/* ---------------------------------------------------------------------------------------------
+ * Geometric median by Weiszfeld's iteration (Section 4, Theorem 4 names the aggregator; the
+ * iteration is the textbook one): y_0 = mean; y <- sum_j w_j x_j / sum_j w_j with
+ * w_j = 1 / max(||x_j - y||, eps), `iters` times.  Everything in fp64; rounded to fp32 at the end.
+ * ------------------------------------------------------------------------------------------- */
+int oracle_geometric_median(const float* X, int64_t ld, int m, int64_t d, int iters, double eps, float* out) {
+    if (m < 1 || iters < 0 || !(eps > 0.0)) return 1;
+    double* y = (double*)malloc((size_t)d * sizeof(double));
+    double* w = (double*)malloc((size_t)m * sizeof(double));
+    for (int j = 0; j < m; ++j) w[j] = 1.0;
+    for (int t = 0; t <= iters; ++t) {
+        double tot = 0.0;
+        for (int j = 0; j < m; ++j) tot += w[j];
+#pragma omp parallel for schedule(static)
+        for (int64_t c = 0; c < d; ++c) {
+            double acc = 0.0;
+            for (int j = 0; j < m; ++j) acc += w[j] * (double)X[(int64_t)j * ld + c];
+            y[c] = acc / tot;
+        }
+        if (t == iters) break;
+        for (int j = 0; j < m; ++j) {
+            double dist2 = 0.0;
+#pragma omp parallel for schedule(static) reduction(+ : dist2)
+            for (int64_t c = 0; c < d; ++c) {
+                const double diff = (double)X[(int64_t)j * ld + c] - y[c];
+                dist2 += diff * diff;
+            }
+            const double dist = sqrt(dist2);
+            w[j] = 1.0 / (dist > eps ? dist : eps);
+        }
+    }
+    for (int64_t c = 0; c < d; ++c) out[c] = (float)y[c];
+    free(w);
+    free(y);
+    return 0;
+}
+
 /* Bulyan = first stage on all m rows with tolerance f, then the second stage with beta = theta - 2f. */
 int oracle_bulyan(const float* X, int64_t ld, int m, int64_t d, int f, float* out, int32_t* sel,
                   double* D_out) {

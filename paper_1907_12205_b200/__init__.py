@@ -17,6 +17,7 @@ from .binding import (  # noqa: F401
     agg_bulyan_workspace_bytes,
     agg_coord_median,
     agg_coord_median_workspace_bytes,
+    agg_geometric_median,
     agg_multikrum,
     agg_trimmed_mean,
     agg_multikrum_workspace_bytes,

@@ -23,7 +23,7 @@ MAX_ROWS, MAX_R = 1024, 15
 EXPORTS = (
     "detox_status_string", "detox_vote_workspace_bytes", "detox_vote", "detox_vote_noalloc", "detox_hier_mean",
     "detox_vote_hier_mean",
-    "agg_coord_median_workspace_bytes", "agg_coord_median", "agg_trimmed_mean", "agg_multikrum_workspace_bytes", "agg_multikrum",
+    "agg_coord_median_workspace_bytes", "agg_coord_median", "agg_trimmed_mean", "agg_geometric_median_workspace_bytes", "agg_geometric_median", "agg_multikrum_workspace_bytes", "agg_multikrum",
     "agg_bulyan_workspace_bytes", "agg_bulyan", "detox_aggregate_workspace_bytes", "detox_aggregate",
 )
 
@@ -72,6 +72,9 @@ def load() -> ctypes.CDLL:
         fn.argtypes = [_int, _i64]
     lib.agg_coord_median.argtypes = [_vp, _i64, _int, _i64, _vp, _vp, _sz, _vp]
     lib.agg_trimmed_mean.argtypes = [_vp, _i64, _int, _i64, _int, _vp, _vp]
+    lib.agg_geometric_median_workspace_bytes.restype = _sz
+    lib.agg_geometric_median_workspace_bytes.argtypes = [_int, _i64]
+    lib.agg_geometric_median.argtypes = [_vp, _i64, _int, _i64, _int, ctypes.c_float, _vp, _vp, _sz, _vp]
     lib.agg_multikrum.argtypes = [_vp, _i64, _int, _i64, _int, _int, _vp, _vp, _vp, _vp, _sz, _vp]
     lib.agg_bulyan.argtypes = [_vp, _i64, _int, _i64, _int, _vp, _vp, _vp, _sz, _vp]
     lib.detox_aggregate_workspace_bytes.restype = _sz
@@ -213,6 +216,19 @@ def agg_trimmed_mean(X, trim: int, out: Optional[torch.Tensor] = None, stream=No
     if out is None:
         out = torch.empty(d, dtype=torch.float32, device=X.device)
     _check(lib.agg_trimmed_mean(xp, ld, m, d, trim, out.data_ptr(), _stream(stream)), "agg_trimmed_mean")
+    return out
+
+
+def agg_geometric_median(X, iters: int = 32, eps: float = 1e-12, out: Optional[torch.Tensor] = None,
+                         ws: Optional[torch.Tensor] = None, stream=None):
+    """Geometric median of at most 32 rows by `iters` Weiszfeld iterations started at the mean."""
+    lib = load()
+    xp, ld, m, d = _mat(X)
+    if out is None:
+        out = torch.empty(d, dtype=torch.float32, device=X.device)
+    ws, wp, wb = _ws(lib.agg_geometric_median_workspace_bytes(m, d), ws, X.device)
+    _check(lib.agg_geometric_median(xp, ld, m, d, iters, eps, out.data_ptr(), wp, wb, _stream(stream)),
+           "agg_geometric_median")
     return out
 
 

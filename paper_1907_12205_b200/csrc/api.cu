@@ -305,6 +305,21 @@ detox_status agg_trimmed_mean(const float* X, int64_t ld, int m, int64_t d, int 
     return launch_coord_select(X, ld, m, d, nullptr, -(m - 2 * trim), out, static_cast<cudaStream_t>(stream));
 }
 
+size_t agg_geometric_median_workspace_bytes(int m, int64_t d) {
+    if (m < 1 || m > 32 || d < 1) return 0;
+    return geomed_ws_bytes(d);
+}
+
+detox_status agg_geometric_median(const float* X, int64_t ld, int m, int64_t d, int iters, float eps, float* out,
+                                  void* ws, size_t ws_bytes, void* stream) {
+    detox_status st = check_matrix(X, ld, m, d);
+    if (st != DETOX_OK) return st;
+    if (!out || (reinterpret_cast<uintptr_t>(out) & 3u) || iters < 0 || !(eps > 0.f)) return DETOX_ERR_BAD_ARG;
+    if (m > 32) return DETOX_ERR_UNSUPPORTED;
+    if (!ws_ok(ws, ws_bytes, geomed_ws_bytes(d))) return DETOX_ERR_WORKSPACE;
+    return launch_geometric_median(X, ld, m, d, iters, eps, out, ws, static_cast<cudaStream_t>(stream));
+}
+
 size_t agg_multikrum_workspace_bytes(int m, int64_t d) {
     if (m < 1 || m > kMaxRows || d < 1) return 0;
     return krum_ws(nullptr, m, d).total;

@@ -97,6 +97,11 @@ size_t tc_ws_bytes(int m, int64_t d);
 detox_status launch_sqdist_tc(const float* X, int64_t ld, int m, int64_t d, double* D, void* ws, int* status,
                               cudaStream_t s);
 
+// geomed.cu: Weiszfeld iterations for the geometric median of m <= 32 rows
+size_t geomed_ws_bytes(int64_t d);
+detox_status launch_geometric_median(const float* X, int64_t ld, int m, int64_t d, int iters, float eps, float* out,
+                                     void* ws, cudaStream_t s);
+
 // select.cu
 size_t select_ws_bytes(int m);
 // Multi-Krum scoring + selection of the m_sel best rows (ascending indices in sel_dev)

@@ -396,3 +396,42 @@ def test_trimmed_mean_against_library_and_reductions():
     assert np.array_equal(oracle.trimmed_mean(Y, 4), np.median(Y, axis=0))      # one value left: the median
     Z = np.array([[5.0], [1.0], [100.0], [3.0], [-7.0]], np.float32)            # sorted -7 1 3 5 100
     assert oracle.trimmed_mean(Z, 1).tolist() == [3.0]
+
+
+# ----------------------------------------------------------------------------- geometric median
+
+def _objective(X, y):
+    return float(np.sqrt(((X.astype(np.float64) - y.astype(np.float64)) ** 2).sum(1)).sum())
+
+
+def test_geometric_median_zero_iterations_is_the_mean_and_symmetric_points_stay():
+    X = rng(50).standard_normal((7, 40)).astype(np.float32)
+    assert np.array_equal(oracle.geometric_median(X, iters=0), (X.astype(np.float64).sum(0) / 7).astype(np.float32))
+    ang = np.arange(6) * np.pi / 3
+    P = np.stack([np.cos(ang), np.sin(ang)], 1).astype(np.float32) * 4 + np.float32(2.5)   # regular hexagon
+    np.testing.assert_allclose(oracle.geometric_median(P, iters=50), [2.5, 2.5], atol=1e-6)
+
+
+def test_geometric_median_is_a_stationary_point_and_the_objective_never_rises():
+    # 3-4-5 triangle (all angles < 120 degrees): at the Fermat point the three unit vectors cancel
+    T = np.array([[0.0, 0.0], [3.0, 0.0], [0.0, 4.0]], np.float32)
+    y = oracle.geometric_median(T, iters=300).astype(np.float64)
+    u = (T - y) / np.linalg.norm(T - y, axis=1, keepdims=True)
+    assert np.abs(u.sum(0)).max() < 1e-5
+    X = rng(51).standard_normal((9, 25)).astype(np.float32)
+    obj = [_objective(X, oracle.geometric_median(X, iters=t)) for t in range(12)]
+    assert all(b <= a + 1e-9 for a, b in zip(obj, obj[1:])) and obj[-1] < obj[0]
+    g = oracle.geometric_median(X, iters=400).astype(np.float64)
+    u = (X - g) / np.linalg.norm(X - g, axis=1, keepdims=True)
+    assert np.abs(u.sum(0)).max() < 1e-4
+
+
+def test_geometric_median_resists_an_outlier_and_is_equivariant():
+    X = (rng(52).standard_normal((8, 30)) * 0.1).astype(np.float32)
+    X[3] = 1000.0
+    g = oracle.geometric_median(X, iters=100)
+    assert np.linalg.norm(g) < 1.0 < np.linalg.norm(X.mean(0))        # the mean is dragged away, the median is not
+    assert np.array_equal(oracle.geometric_median(X * np.float32(4), iters=20), oracle.geometric_median(X, iters=20) * 4)
+    shift = np.float32(3.0)
+    np.testing.assert_allclose(oracle.geometric_median(X + shift, iters=20), oracle.geometric_median(X, iters=20) + shift,
+                               atol=1e-4)

@@ -136,6 +136,17 @@ def test_trimmed_mean_matches_oracle(m, trim):
     assert rel_l2(got.cpu().numpy(), oracle.trimmed_mean(X, trim)) <= TOL
 
 
+@pytest.mark.parametrize("m,d,iters", [(3, 20_001, 10), (7, 4099, 25), (15, 10_000, 8), (32, 3000, 5), (1, 500, 3),
+                                       (5, 1, 4), (9, 1003, 0)])
+def test_geometric_median_matches_oracle(m, d, iters):
+    X = (np.random.default_rng(m + d).standard_normal((m, d)) * 1e-3).astype(np.float32)
+    if m > 2:
+        X[m - 1] *= -100                                   # a Byzantine row
+    ref = oracle.geometric_median(X, iters=iters)
+    assert rel_l2(dx.agg_geometric_median(padded(X), iters=iters).cpu().numpy(), ref) <= TOL
+    assert rel_l2(dx.agg_geometric_median(padded(X, ld=d + 3, offset=1), iters=iters).cpu().numpy(), ref) <= TOL
+
+
 # ------------------------------------------------------------------------------------ Multi-Krum
 
 def krum_inputs(m, d, seed, copies=1, outliers=0):
