@@ -51,7 +51,8 @@ typedef enum {
     DETOX_AGG_COORD_MEDIAN = 2,
     DETOX_AGG_MULTIKRUM = 3,
     DETOX_AGG_BULYAN = 4,
-    DETOX_AGG_TRIMMED_MEAN = 5  /* A_1 only: drops the f smallest and f largest values per coordinate */
+    DETOX_AGG_TRIMMED_MEAN = 5, /* A_1 only: drops the f smallest and f largest values per coordinate */
+    DETOX_AGG_GEOMETRIC_MEDIAN = 6  /* A_1 only: gm_iters Weiszfeld iterations over at most 32 rows */
 } detox_agg;
 
 const char* detox_status_string(detox_status s);
@@ -191,7 +192,8 @@ detox_status agg_bulyan(const float* X, int64_t ld, int m, int64_t d, int f, flo
  *        one set of 15) and its S results go to A_1, which must then be MEAN or COORD_MEDIAN.  f and m_sel
  *        belong to A_0: every set of k votes averages its m_sel best (m_sel = 0: its k - f best), or, for
  *        Bulyan, needs k >= 4f+3.
- *   a1 = MEAN | COORD_MEDIAN | TRIMMED_MEAN (f per side) | MULTIKRUM (f, m_sel) | BULYAN (f)
+ *   a1 = MEAN | COORD_MEDIAN | TRIMMED_MEAN (f per side) | GEOMETRIC_MEDIAN (gm_iters, gm_eps; at most 32 rows
+ *        enter it) | MULTIKRUM (f, m_sel) | BULYAN (f)
  *
  *   out          dev, d
  *   winner       dev, G        out, as in detox_vote; may be NULL
@@ -211,9 +213,11 @@ typedef struct {
     int32_t n_sets;              /* S, used unless a0 = NONE */
     const int32_t* set_offsets;  /* host, S+1 */
     const int32_t* set_members;  /* host, G */
-    int32_t a1;                  /* detox_agg: MEAN, COORD_MEDIAN, TRIMMED_MEAN, MULTIKRUM or BULYAN */
+    int32_t a1;                  /* detox_agg: MEAN, COORD_MEDIAN, TRIMMED_MEAN, GEOMETRIC_MEDIAN, MULTIKRUM or BULYAN */
     int32_t f;                   /* tolerance given to Multi-Krum / Bulyan */
     int32_t m_sel;               /* rows averaged by Multi-Krum */
+    int32_t gm_iters;            /* Weiszfeld iterations when a1 = GEOMETRIC_MEDIAN */
+    float gm_eps;                /* floor on the distances in its weights (> 0) */
 } detox_pipeline_desc;
 
 size_t detox_aggregate_workspace_bytes(const detox_pipeline_desc* desc);

@@ -218,7 +218,7 @@ A0_NONE, A0_MEAN = "none", "mean"
 
 
 def detox_aggregate(X, members, r: int, a0: str, set_offsets, set_members, a1: str, f: int = 0,
-                    m_sel: int = 1):
+                    m_sel: int = 1, gm_iters: int = 32, gm_eps: float = 1e-12):
     """Algorithm 1 (filtering step + hierarchical aggregation) with A_0 in {none, mean, multikrum, bulyan}
     and A_1 in {mean, coord_median, multikrum, bulyan}.
 
@@ -252,6 +252,8 @@ def detox_aggregate(X, members, r: int, a0: str, set_offsets, set_members, a1: s
         out = coord_median(rows)
     elif a1 == "trimmed_mean":
         out = trimmed_mean(rows, f)
+    elif a1 == "geometric_median":
+        out = geometric_median(rows, gm_iters, gm_eps)
     elif a1 == "multikrum":
         out, sel, _, _ = multikrum(rows, f, m_sel)
     elif a1 == "bulyan":

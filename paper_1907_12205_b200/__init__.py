@@ -5,6 +5,7 @@ The product is the C-ABI library built from csrc/ (include/detox.h); this packag
 from .binding import (  # noqa: F401
     AGG_BULYAN,
     AGG_COORD_MEDIAN,
+    AGG_GEOMETRIC_MEDIAN,
     AGG_MEAN,
     AGG_MULTIKRUM,
     AGG_NONE,

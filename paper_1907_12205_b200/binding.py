@@ -17,7 +17,7 @@ import torch
 _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "libdetox.so")
 
-AGG_NONE, AGG_MEAN, AGG_COORD_MEDIAN, AGG_MULTIKRUM, AGG_BULYAN, AGG_TRIMMED_MEAN = 0, 1, 2, 3, 4, 5
+AGG_NONE, AGG_MEAN, AGG_COORD_MEDIAN, AGG_MULTIKRUM, AGG_BULYAN, AGG_TRIMMED_MEAN, AGG_GEOMETRIC_MEDIAN = range(7)
 MAX_ROWS, MAX_R = 1024, 15
 
 EXPORTS = (
@@ -41,6 +41,7 @@ class PipelineDesc(ctypes.Structure):
         ("a0", ctypes.c_int32), ("n_sets", ctypes.c_int32),
         ("set_offsets", ctypes.POINTER(ctypes.c_int32)), ("set_members", ctypes.POINTER(ctypes.c_int32)),
         ("a1", ctypes.c_int32), ("f", ctypes.c_int32), ("m_sel", ctypes.c_int32),
+        ("gm_iters", ctypes.c_int32), ("gm_eps", ctypes.c_float),
     ]
 
 
@@ -275,7 +276,7 @@ class Pipeline:
     """Holds the host-side description of one DETOX configuration (Algorithm 1 + Algorithm 2)."""
 
     def __init__(self, n: int, r: int, d: int, members, a0: int = AGG_NONE, set_offsets=None, set_members=None,
-                 a1: int = AGG_COORD_MEDIAN, f: int = 0, m_sel: int = 1):
+                 a1: int = AGG_COORD_MEDIAN, f: int = 0, m_sel: int = 1, gm_iters: int = 32, gm_eps: float = 1e-12):
         self.members = _host_i32(members)
         self.set_offsets = None if set_offsets is None else _host_i32(set_offsets)
         self.set_members = None if set_members is None else _host_i32(set_members)
@@ -287,6 +288,7 @@ class Pipeline:
         self.desc.set_offsets = None if self.set_offsets is None else self.set_offsets.ctypes.data_as(_ip)
         self.desc.set_members = None if self.set_members is None else self.set_members.ctypes.data_as(_ip)
         self.desc.a1, self.desc.f, self.desc.m_sel = a1, f, m_sel
+        self.desc.gm_iters, self.desc.gm_eps = gm_iters, gm_eps
         self.n, self.r, self.d, self.a0, self.a1, self.f, self.m_sel = n, r, d, a0, a1, f, m_sel
 
     @property

@@ -144,7 +144,7 @@ int a0_selected(const detox_pipeline_desc* p, int k) {
 // written: always for the per-coordinate aggregators, and for the Krum type up to 16 votes (the
 // direct-difference distance kernel takes a row list; the tensor-core Gram wants consecutive rows).
 bool votes_by_index(const detox_pipeline_desc* p) {
-    if (p->a0 != DETOX_AGG_NONE) return false;
+    if (p->a0 != DETOX_AGG_NONE || p->a1 == DETOX_AGG_GEOMETRIC_MEDIAN) return false;
     return !krum_type(p->a1) || p->n / p->r <= 16;
 }
 
@@ -182,6 +182,7 @@ PipeWs pipe_ws(void* ws, const detox_pipeline_desc* p) {
     off += align_up((size_t)G * sizeof(int32_t));
     w.agg = base + off;
     if (krum_type(p->a1)) off += krum_ws(nullptr, rows1, p->d).total;
+    if (p->a1 == DETOX_AGG_GEOMETRIC_MEDIAN) off += geomed_ws_bytes(p->d);
     if (krum_type(p->a0)) {
         int kmax = 1;
         for (int s = 0; s < p->n_sets; ++s) {
@@ -203,7 +204,10 @@ detox_status check_desc(const detox_pipeline_desc* p) {
     if (p->a0 != DETOX_AGG_NONE && (p->n_sets < 1 || p->n_sets > G)) return DETOX_ERR_BAD_ARG;
     if (krum_type(p->a0)) {
         // Multi-Krum / Bulyan inside every vote set (f, m_sel belong to A_0), then a plain A_1 over the set results
-        if (p->a1 != DETOX_AGG_MEAN && p->a1 != DETOX_AGG_COORD_MEDIAN) return DETOX_ERR_UNSUPPORTED;  // f is A_0's
+        if (p->a1 != DETOX_AGG_MEAN && p->a1 != DETOX_AGG_COORD_MEDIAN && p->a1 != DETOX_AGG_GEOMETRIC_MEDIAN)
+            return DETOX_ERR_UNSUPPORTED;  // f and m_sel are A_0's
+        if (p->a1 == DETOX_AGG_GEOMETRIC_MEDIAN && (p->gm_iters < 0 || !(p->gm_eps > 0.f) || p->n_sets > 32))
+            return p->n_sets > 32 ? DETOX_ERR_UNSUPPORTED : DETOX_ERR_BAD_ARG;
         if (!p->set_offsets || p->f < 0 || p->m_sel < 0) return DETOX_ERR_BAD_ARG;
         if (p->set_offsets[0] != 0 || p->set_offsets[p->n_sets] != G) return DETOX_ERR_BAD_ARG;
         for (int s = 0; s < p->n_sets; ++s) {
@@ -219,6 +223,9 @@ detox_status check_desc(const detox_pipeline_desc* p) {
         case DETOX_AGG_MEAN:
         case DETOX_AGG_COORD_MEDIAN: return DETOX_OK;
         case DETOX_AGG_TRIMMED_MEAN: return (p->f >= 0 && rows1 - 2 * p->f >= 1) ? DETOX_OK : DETOX_ERR_BAD_ARG;
+        case DETOX_AGG_GEOMETRIC_MEDIAN:
+            if (p->gm_iters < 0 || !(p->gm_eps > 0.f)) return DETOX_ERR_BAD_ARG;
+            return rows1 <= 32 ? DETOX_OK : DETOX_ERR_UNSUPPORTED;
         case DETOX_AGG_MULTIKRUM: return check_multikrum(rows1, p->f, p->m_sel);
         case DETOX_AGG_BULYAN: return check_bulyan(rows1, p->f);
         default: return DETOX_ERR_BAD_ARG;
@@ -429,6 +436,9 @@ detox_status detox_aggregate(const detox_pipeline_desc* p, const float* X, int64
         case DETOX_AGG_COORD_MEDIAN: st = launch_coord_select(rows, row_ld, m, p->d, row_list, 0, out, s); break;
         case DETOX_AGG_TRIMMED_MEAN:
             st = launch_coord_select(rows, row_ld, m, p->d, row_list, -(m - 2 * p->f), out, s);
+            break;
+        case DETOX_AGG_GEOMETRIC_MEDIAN:
+            st = launch_geometric_median(rows, row_ld, m, p->d, p->gm_iters, p->gm_eps, out, w.agg, s);
             break;
         case DETOX_AGG_MULTIKRUM:
             cnt = p->m_sel;

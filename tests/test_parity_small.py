@@ -220,7 +220,8 @@ def run_pipeline(w, a0, a1, f=0, m_sel=1):
     Xd = w.X.to(DEV)[:, :spec.d]
     res = dx.detox_aggregate(pipe, Xd)
     names = {dx.AGG_MEAN: "mean", dx.AGG_COORD_MEDIAN: "coord_median", dx.AGG_MULTIKRUM: "multikrum",
-             dx.AGG_BULYAN: "bulyan", dx.AGG_TRIMMED_MEAN: "trimmed_mean"}
+             dx.AGG_BULYAN: "bulyan", dx.AGG_TRIMMED_MEAN: "trimmed_mean",
+             dx.AGG_GEOMETRIC_MEDIAN: "geometric_median"}
     ref = oracle.detox_aggregate(w.data().numpy(), w.members, spec.r, "mean" if a0 == dx.AGG_MEAN else "none",
                                  w.set_offsets, w.set_members, names[a1], f, m_sel)
     return res, ref
@@ -236,7 +237,7 @@ def test_pipeline_cfg1_vote_then_median_is_bit_exact():
 
 
 @pytest.mark.parametrize("a1,f,m_sel", [(dx.AGG_MULTIKRUM, 1, 1), (dx.AGG_COORD_MEDIAN, 0, 1), (dx.AGG_MEAN, 0, 1),
-                                        (dx.AGG_TRIMMED_MEAN, 1, 1)])
+                                        (dx.AGG_TRIMMED_MEAN, 1, 1), (dx.AGG_GEOMETRIC_MEDIAN, 0, 1)])
 def test_pipeline_vote_mean_then_a1(a1, f, m_sel):
     spec = wl.WorkloadSpec("p", n=45, r=3, d=50_003, sigma=1e-3, q=5, attack="alie", placement="worst", set_size=5,
                            group_jitter=0.05, seed=11)
