@@ -52,7 +52,8 @@ typedef enum {
     DETOX_AGG_MULTIKRUM = 3,
     DETOX_AGG_BULYAN = 4,
     DETOX_AGG_TRIMMED_MEAN = 5, /* A_1 only: drops the f smallest and f largest values per coordinate */
-    DETOX_AGG_GEOMETRIC_MEDIAN = 6  /* A_1 only: gm_iters Weiszfeld iterations over at most 32 rows */
+    DETOX_AGG_GEOMETRIC_MEDIAN = 6, /* A_1 only: gm_iters Weiszfeld iterations over at most 32 rows */
+    DETOX_AGG_SIGN_MAJORITY = 7 /* A_0 and A_1: coordinate-wise sign(sum of signs), the signSGD pairing */
 } detox_agg;
 
 const char* detox_status_string(detox_status s);
@@ -140,6 +141,14 @@ detox_status agg_coord_median(const float* X, int64_t ld, int m, int64_t d, floa
 detox_status agg_trimmed_mean(const float* X, int64_t ld, int m, int64_t d, int trim, float* out, void* stream);
 
 /* ---------------------------------------------------------------------------------------------
+ * Coordinate-wise sign majority, the aggregator of signSGD with majority vote (Section 5.1, setup 4:
+ * A_0 = A_1 = coordinate-wise majority): out[c] = sign(sum_i sign(X[i][c])), one of -1, 0, +1
+ * (sign(0) = sign(NaN) = 0; a tie gives 0).
+ *   out  dev, d.   No workspace.
+ * ------------------------------------------------------------------------------------------- */
+detox_status agg_sign_majority(const float* X, int64_t ld, int m, int64_t d, float* out, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
  * Geometric median (one of the A_1 choices analysed in Section 4, Theorem 4; the paper does not fix
  * an algorithm).  Computed by Weiszfeld's iteration started at the mean:
  *     y <- sum_j w_j x_j / sum_j w_j,   w_j = 1 / max(||x_j - y||_2, eps),   `iters` times.
@@ -187,12 +196,13 @@ detox_status agg_bulyan(const float* X, int64_t ld, int m, int64_t d, int f, flo
  *
  *   a0 = DETOX_AGG_NONE : the G votes go to A_1 directly (sets are ignored)
  *   a0 = DETOX_AGG_MEAN : the S set means go to A_1
+ *   a0 = DETOX_AGG_SIGN_MAJORITY : the S coordinate-wise sign majorities of the sets go to A_1
  *   a0 = DETOX_AGG_MULTIKRUM | DETOX_AGG_BULYAN : the aggregator runs inside every vote set (the pairings the
  *        paper found most resilient, Section 5.1 setups 2 and 3; set shapes as in Appendix B.1, e.g. 7 + 8 or
  *        one set of 15) and its S results go to A_1, which must then be MEAN or COORD_MEDIAN.  f and m_sel
  *        belong to A_0: every set of k votes averages its m_sel best (m_sel = 0: its k - f best), or, for
  *        Bulyan, needs k >= 4f+3.
- *   a1 = MEAN | COORD_MEDIAN | TRIMMED_MEAN (f per side) | GEOMETRIC_MEDIAN (gm_iters, gm_eps; at most 32 rows
+ *   a1 = MEAN | SIGN_MAJORITY | COORD_MEDIAN | TRIMMED_MEAN (f per side) | GEOMETRIC_MEDIAN (gm_iters, gm_eps; at most 32 rows
  *        enter it) | MULTIKRUM (f, m_sel) | BULYAN (f)
  *
  *   out          dev, d
@@ -209,7 +219,7 @@ typedef struct {
     int32_t r;                   /* redundancy ratio (odd, divides n) */
     int64_t d;                   /* gradient dimension */
     const int32_t* members;      /* host, G*r */
-    int32_t a0;                  /* detox_agg: NONE, MEAN, MULTIKRUM or BULYAN */
+    int32_t a0;                  /* detox_agg: NONE, MEAN, SIGN_MAJORITY, MULTIKRUM or BULYAN */
     int32_t n_sets;              /* S, used unless a0 = NONE */
     const int32_t* set_offsets;  /* host, S+1 */
     const int32_t* set_members;  /* host, G */

@@ -57,6 +57,7 @@ def _load():
         lib.oracle_trimmed_around_median.argtypes = [_F, _i64, _i64, _I, _int, _int, _F]
         lib.oracle_trimmed_mean.argtypes = [_F, _i64, _int, _i64, _int, _F]
         lib.oracle_geometric_median.argtypes = [_F, _i64, _int, _i64, _int, ctypes.c_double, _F]
+        lib.oracle_sign_majority.argtypes = [_F, _i64, _int, _i64, _I, _F]
         lib.oracle_bulyan.argtypes = [_F, _i64, _int, _i64, _int, _F, _I, _D]
         _lib = lib
     return _lib
@@ -142,6 +143,15 @@ def trimmed_mean(X, trim: int):
     m, d = X.shape
     out = np.empty(d, dtype=np.float32)
     _check(_load().oracle_trimmed_mean(_fp(X), ld, m, d, trim, _fp(out)), "trimmed_mean")
+    return out
+
+
+def sign_majority(X, rows=None):
+    X, ld = _mat(X)
+    m, d = X.shape
+    r = None if rows is None else _idx(rows)
+    out = np.empty(d, dtype=np.float32)
+    _check(_load().oracle_sign_majority(_fp(X), ld, m if r is None else len(r), d, _ip(r), _fp(out)), "sign_majority")
     return out
 
 
@@ -244,10 +254,15 @@ def detox_aggregate(X, members, r: int, a0: str, set_offsets, set_members, a1: s
             sel_votes.extend(int(v) for v in idx[loc])
         rows = np.stack(outs)
         sel_votes = np.asarray(sel_votes, dtype=np.int32)
+    elif a0 == "sign_majority":
+        so, sm = np.asarray(set_offsets), np.asarray(set_members)
+        rows = np.stack([sign_majority(Z, sm[so[s]:so[s + 1]]) for s in range(len(so) - 1)])
     else:
         rows = Z if a0 == A0_NONE else hier_mean(Z, set_offsets, set_members)
     if a1 == "mean":
         out = mean_rows(rows)
+    elif a1 == "sign_majority":
+        out = sign_majority(rows)
     elif a1 == "coord_median":
         out = coord_median(rows)
     elif a1 == "trimmed_mean":

@@ -368,6 +368,24 @@ int oracle_geometric_median(const float* X, int64_t ld, int m, int64_t d, int it
     return 0;
 }
 
+/* ---------------------------------------------------------------------------------------------
+ * Coordinate-wise sign majority (signSGD with majority vote; Section 5.1, setup 4):
+ * out[c] = sign(sum_i sign(x_ic)); sign(0) = sign(NaN) = 0.  rows == NULL means rows 0..m-1.
+ * ------------------------------------------------------------------------------------------- */
+int oracle_sign_majority(const float* X, int64_t ld, int m, int64_t d, const int32_t* rows, float* out) {
+    if (m < 1) return 1;
+#pragma omp parallel for schedule(static)
+    for (int64_t c = 0; c < d; ++c) {
+        long votes = 0;
+        for (int i = 0; i < m; ++i) {
+            const float v = X[(int64_t)(rows ? rows[i] : i) * ld + c];
+            votes += (v > 0.0f) - (v < 0.0f);
+        }
+        out[c] = (float)((votes > 0) - (votes < 0));
+    }
+    return 0;
+}
+
 /* Bulyan = first stage on all m rows with tolerance f, then the second stage with beta = theta - 2f. */
 int oracle_bulyan(const float* X, int64_t ld, int m, int64_t d, int f, float* out, int32_t* sel,
                   double* D_out) {

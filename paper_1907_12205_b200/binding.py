@@ -17,13 +17,13 @@ import torch
 _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "libdetox.so")
 
-AGG_NONE, AGG_MEAN, AGG_COORD_MEDIAN, AGG_MULTIKRUM, AGG_BULYAN, AGG_TRIMMED_MEAN, AGG_GEOMETRIC_MEDIAN = range(7)
+AGG_NONE, AGG_MEAN, AGG_COORD_MEDIAN, AGG_MULTIKRUM, AGG_BULYAN, AGG_TRIMMED_MEAN, AGG_GEOMETRIC_MEDIAN, AGG_SIGN_MAJORITY = range(8)
 MAX_ROWS, MAX_R = 1024, 15
 
 EXPORTS = (
     "detox_status_string", "detox_vote_workspace_bytes", "detox_vote", "detox_vote_noalloc", "detox_hier_mean",
     "detox_vote_hier_mean",
-    "agg_coord_median_workspace_bytes", "agg_coord_median", "agg_trimmed_mean", "agg_geometric_median_workspace_bytes", "agg_geometric_median", "agg_multikrum_workspace_bytes", "agg_multikrum",
+    "agg_coord_median_workspace_bytes", "agg_coord_median", "agg_trimmed_mean", "agg_sign_majority", "agg_geometric_median_workspace_bytes", "agg_geometric_median", "agg_multikrum_workspace_bytes", "agg_multikrum",
     "agg_bulyan_workspace_bytes", "agg_bulyan", "detox_aggregate_workspace_bytes", "detox_aggregate",
 )
 
@@ -76,6 +76,7 @@ def load() -> ctypes.CDLL:
     lib.agg_geometric_median_workspace_bytes.restype = _sz
     lib.agg_geometric_median_workspace_bytes.argtypes = [_int, _i64]
     lib.agg_geometric_median.argtypes = [_vp, _i64, _int, _i64, _int, ctypes.c_float, _vp, _vp, _sz, _vp]
+    lib.agg_sign_majority.argtypes = [_vp, _i64, _int, _i64, _vp, _vp]
     lib.agg_multikrum.argtypes = [_vp, _i64, _int, _i64, _int, _int, _vp, _vp, _vp, _vp, _sz, _vp]
     lib.agg_bulyan.argtypes = [_vp, _i64, _int, _i64, _int, _vp, _vp, _vp, _sz, _vp]
     lib.detox_aggregate_workspace_bytes.restype = _sz
@@ -217,6 +218,16 @@ def agg_trimmed_mean(X, trim: int, out: Optional[torch.Tensor] = None, stream=No
     if out is None:
         out = torch.empty(d, dtype=torch.float32, device=X.device)
     _check(lib.agg_trimmed_mean(xp, ld, m, d, trim, out.data_ptr(), _stream(stream)), "agg_trimmed_mean")
+    return out
+
+
+def agg_sign_majority(X, out: Optional[torch.Tensor] = None, stream=None):
+    """Coordinate-wise sign(sum of signs): -1, 0 or +1 per coordinate."""
+    lib = load()
+    xp, ld, m, d = _mat(X)
+    if out is None:
+        out = torch.empty(d, dtype=torch.float32, device=X.device)
+    _check(lib.agg_sign_majority(xp, ld, m, d, out.data_ptr(), _stream(stream)), "agg_sign_majority")
     return out
 
 

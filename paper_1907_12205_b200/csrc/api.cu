@@ -199,7 +199,8 @@ detox_status check_desc(const detox_pipeline_desc* p) {
     if (!p || p->d < 1) return DETOX_ERR_BAD_ARG;
     if (p->n < 1 || p->r < 1 || (p->r & 1) == 0 || p->n % p->r != 0) return DETOX_ERR_BAD_ARG;
     if (p->n > kMaxRows || p->r > kMaxR) return DETOX_ERR_UNSUPPORTED;
-    if (p->a0 != DETOX_AGG_NONE && p->a0 != DETOX_AGG_MEAN && !krum_type(p->a0)) return DETOX_ERR_BAD_ARG;
+    if (p->a0 != DETOX_AGG_NONE && p->a0 != DETOX_AGG_MEAN && p->a0 != DETOX_AGG_SIGN_MAJORITY && !krum_type(p->a0))
+        return DETOX_ERR_BAD_ARG;
     const int G = p->n / p->r;
     if (p->a0 != DETOX_AGG_NONE && (p->n_sets < 1 || p->n_sets > G)) return DETOX_ERR_BAD_ARG;
     if (krum_type(p->a0)) {
@@ -218,9 +219,10 @@ detox_status check_desc(const detox_pipeline_desc* p) {
         }
         return DETOX_OK;
     }
-    const int rows1 = p->a0 == DETOX_AGG_MEAN ? p->n_sets : G;
+    const int rows1 = p->a0 != DETOX_AGG_NONE ? p->n_sets : G;
     switch (p->a1) {
         case DETOX_AGG_MEAN:
+        case DETOX_AGG_SIGN_MAJORITY:
         case DETOX_AGG_COORD_MEDIAN: return DETOX_OK;
         case DETOX_AGG_TRIMMED_MEAN: return (p->f >= 0 && rows1 - 2 * p->f >= 1) ? DETOX_OK : DETOX_ERR_BAD_ARG;
         case DETOX_AGG_GEOMETRIC_MEDIAN:
@@ -312,6 +314,13 @@ detox_status agg_trimmed_mean(const float* X, int64_t ld, int m, int64_t d, int 
     return launch_coord_select(X, ld, m, d, nullptr, -(m - 2 * trim), out, static_cast<cudaStream_t>(stream));
 }
 
+detox_status agg_sign_majority(const float* X, int64_t ld, int m, int64_t d, float* out, void* stream) {
+    detox_status st = check_matrix(X, ld, m, d);
+    if (st != DETOX_OK) return st;
+    if (!out || (reinterpret_cast<uintptr_t>(out) & 3u)) return DETOX_ERR_BAD_ARG;
+    return launch_mean_rows(X, ld, d, nullptr, m, out, static_cast<cudaStream_t>(stream), true);
+}
+
 size_t agg_geometric_median_workspace_bytes(int m, int64_t d) {
     if (m < 1 || m > 32 || d < 1) return 0;
     return geomed_ws_bytes(d);
@@ -391,6 +400,12 @@ detox_status detox_aggregate(const detox_pipeline_desc* p, const float* X, int64
             return st;
         rows = w.M;
         m = p->n_sets;
+    } else if (p->a0 == DETOX_AGG_SIGN_MAJORITY) {
+        // signSGD pairing (Section 5.1, setup 4): coordinate-wise sign majority inside every vote set
+        if ((st = launch_vote(X, ld, p->n, p->r, p->d, groups, w.Z, w.ldz, win, w.vote, s)) != DETOX_OK) return st;
+        if ((st = launch_hier_mean(w.Z, w.ldz, p->d, sets, p->n_sets, w.M, w.ldz, s, true)) != DETOX_OK) return st;
+        rows = w.M;
+        m = p->n_sets;
     } else if (krum_type(p->a0)) {
         // The paper's preferred pairings (Section 5.1, setups 2 and 3): Multi-Krum or Bulyan inside every
         // vote set, then A_1.  The vote runs over the groups in set order, so each set's votes are
@@ -433,6 +448,7 @@ detox_status detox_aggregate(const detox_pipeline_desc* p, const float* X, int64
     int32_t* sel_buf = nullptr;
     switch (p->a1) {
         case DETOX_AGG_MEAN: st = launch_mean_rows(rows, row_ld, p->d, row_list, m, out, s); break;
+        case DETOX_AGG_SIGN_MAJORITY: st = launch_mean_rows(rows, row_ld, p->d, row_list, m, out, s, true); break;
         case DETOX_AGG_COORD_MEDIAN: st = launch_coord_select(rows, row_ld, m, p->d, row_list, 0, out, s); break;
         case DETOX_AGG_TRIMMED_MEAN:
             st = launch_coord_select(rows, row_ld, m, p->d, row_list, -(m - 2 * p->f), out, s);

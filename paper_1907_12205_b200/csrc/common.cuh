@@ -70,11 +70,12 @@ detox_status launch_vote_mean(const float* X, int64_t ld, int n, int r, int64_t 
                               cudaStream_t s);
 
 // mean.cu
+// (sign = true: coordinate-wise sign majority sign(sum sign(x)) instead of the mean, in both launchers)
 detox_status launch_hier_mean(const float* Z, int64_t ldz, int64_t d, const SetTable& sets, int S,
-                              float* M, int64_t ldm, cudaStream_t s);
+                              float* M, int64_t ldm, cudaStream_t s, bool sign = false);
 // mean of k rows of X listed in rows_dev (device int32; NULL = rows 0..k-1; a negative entry = a zero row)
 detox_status launch_mean_rows(const float* X, int64_t ld, int64_t d, const int32_t* rows_dev, int k,
-                              float* out, cudaStream_t s);
+                              float* out, cudaStream_t s, bool sign = false);
 
 // median.cu: per-coordinate order statistics over m rows (rows_dev: device int32 list or NULL; a negative
 // entry = a zero row)

@@ -435,3 +435,15 @@ def test_geometric_median_resists_an_outlier_and_is_equivariant():
     shift = np.float32(3.0)
     np.testing.assert_allclose(oracle.geometric_median(X + shift, iters=20), oracle.geometric_median(X, iters=20) + shift,
                                atol=1e-4)
+
+
+def test_sign_majority_against_numpy_and_hand_worked_column():
+    X = rng(60).standard_normal((9, 500)).astype(np.float32)
+    X[:, 3] = 0.0
+    X[0, 4] = np.nan
+    exp = np.sign(np.where(np.isnan(X), 0.0, np.sign(X)).sum(0)).astype(np.float32)
+    assert np.array_equal(oracle.sign_majority(X), exp)
+    col = np.array([[2.0], [-1.0], [-3.0], [0.0], [5.0], [-0.0]], np.float32)   # two up, two down, two zeros: a tie
+    assert oracle.sign_majority(col).tolist() == [0.0]
+    assert oracle.sign_majority(col[:3]).tolist() == [-1.0]
+    assert np.array_equal(oracle.sign_majority(X, [2, 5, 7]), np.sign(np.sign(X[[2, 5, 7]]).sum(0)).astype(np.float32))

@@ -147,6 +147,32 @@ def test_geometric_median_matches_oracle(m, d, iters):
     assert rel_l2(dx.agg_geometric_median(padded(X, ld=d + 3, offset=1), iters=iters).cpu().numpy(), ref) <= TOL
 
 
+@pytest.mark.parametrize("m,d", [(1, 100), (3, 4099), (4, 1001), (15, 20_000), (45, 3000), (200, 513)])
+def test_sign_majority_bit_exact(m, d):
+    X = np.random.default_rng(m * d).standard_normal((m, d)).astype(np.float32)
+    X[:, 1] = 0.0
+    X[0, 2] = np.nan
+    X[:, 5] = -1.0                                          # the constant attack of Section 5.2
+    assert np.array_equal(bits(dx.agg_sign_majority(padded(X))), oracle.sign_majority(X).view(np.uint32))
+    assert np.array_equal(bits(dx.agg_sign_majority(padded(X, ld=d + 1, offset=1))),
+                          oracle.sign_majority(X).view(np.uint32))
+
+
+def test_pipeline_signsgd_pairing():
+    # Section 5.1, setup 4: sign majority inside the vote sets and over their results; constant attack (-1)
+    spec = wl.WorkloadSpec("p", n=45, r=3, d=30_001, sigma=1.0, q=5, attack="constant", placement="worst", set_size=5,
+                           seed=8)
+    w = wl.make_workload(spec)
+    w.X[:, :spec.d] = torch.sign(w.X[:, :spec.d])           # workers send signs
+    pipe = dx.Pipeline(45, 3, spec.d, w.members, dx.AGG_SIGN_MAJORITY, w.set_offsets, w.set_members,
+                       dx.AGG_SIGN_MAJORITY)
+    res = dx.detox_aggregate(pipe, w.X.to(DEV)[:, :spec.d])
+    ref = oracle.detox_aggregate(w.data().numpy(), w.members, 3, "sign_majority", w.set_offsets, w.set_members,
+                                 "sign_majority")
+    assert res["winner"].cpu().numpy().tolist() == ref["winner"].tolist()
+    assert np.array_equal(bits(res["out"]), ref["out"].view(np.uint32))
+
+
 # ------------------------------------------------------------------------------------ Multi-Krum
 
 def krum_inputs(m, d, seed, copies=1, outliers=0):
