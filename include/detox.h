@@ -3,7 +3,8 @@
  *
  * C ABI.  Every entry point enqueues its kernels on the caller's CUDA stream and returns without
  * synchronising the host.  The library allocates nothing and keeps no state between calls: every
- * buffer, including scratch ("workspace"), belongs to the caller.
+ * buffer, including scratch ("workspace"), belongs to the caller (the one exception, a fixed
+ * scratch array inside the library, is detox_vote_noalloc below).
  *
  * Notation follows arXiv 1907.12205: n compute nodes (the paper's p) each send a gradient of
  * dimension d; node groups have size r (odd, r divides n), so there are G = n / r votes; f is the
@@ -19,7 +20,10 @@
  *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
  *   - Workspace pointers must be 256-byte aligned; sizes come from the *_workspace_bytes helpers.
  *   - Errors: argument problems are reported before anything is launched; a failed launch returns
- *     DETOX_ERR_CUDA.  Nothing aborts or throws.
+ *     DETOX_ERR_CUDA.  Nothing aborts or throws.  Multi-Krum and Bulyan on 17 to 256 rows run a
+ *     tensor-core kernel whose device-side waits are bounded: should one run out, the first int32 of
+ *     the workspace passed to agg_multikrum / agg_bulyan reads DETOX_ERR_TIMEOUT after the stream
+ *     has been synchronised (0 otherwise) and the outputs are not valid.
  *   - Ranking of values (medians, "closest to the median") uses the total order
  *     -NaN < -Inf < ... < -0 < +0 < ... < +Inf < +NaN on fp32 bit patterns.
  */
