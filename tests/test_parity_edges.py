@@ -96,3 +96,42 @@ def test_pipeline_with_the_largest_worker_count():
     ref = oracle.detox_aggregate(w.data().numpy(), w.members, 3, "mean", w.set_offsets, w.set_members, "coord_median")
     assert res["winner"].cpu().numpy().tolist() == ref["winner"].tolist()
     assert rel_l2(res["out"].cpu().numpy(), ref["out"]) <= TOL
+
+
+@pytest.mark.parametrize("a1,f,m_sel", [("median", 0, 1), ("multikrum", 4, 30)])
+def test_pipeline_replays_from_a_cuda_graph(a1, f, m_sel):
+    # Everything is enqueued on the caller's stream with host tables passed as kernel parameters, so a step
+    # can be captured once and replayed on new data in the same buffers.
+    import workloads as wl
+    code = {"median": dx.AGG_COORD_MEDIAN, "multikrum": dx.AGG_MULTIKRUM}[a1]
+    oname = {"median": "coord_median", "multikrum": "multikrum"}[a1]
+    specs = [wl.WorkloadSpec("g", n=105, r=3, d=6001, sigma=1e-3, q=10, attack="reverse", placement="random",
+                             set_size=5, group_jitter=0.2, seed=s) for s in (1, 2)]
+    w0 = wl.make_workload(specs[0])
+    a0 = dx.AGG_MEAN if a1 == "median" else dx.AGG_NONE
+    pipe = dx.Pipeline(105, 3, 6001, w0.members, a0, w0.set_offsets, w0.set_members, code, f, m_sel)
+    X = w0.X.to("cuda:0")
+    out = torch.empty(6001, dtype=torch.float32, device="cuda:0")
+    winner = torch.empty(35, dtype=torch.int32, device="cuda:0")
+    sel = torch.empty(max(pipe.n_selected, 1), dtype=torch.int32, device="cuda:0")
+    selw = torch.empty(max(pipe.n_selected, 1), dtype=torch.int32, device="cuda:0")
+    ws = torch.empty(pipe.workspace_bytes(), dtype=torch.uint8, device="cuda:0")
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        dx.detox_aggregate(pipe, X[:, :6001], out=out, winner=winner, sel=sel, sel_workers=selw, ws=ws)   # warm-up
+        stream.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            dx.detox_aggregate(pipe, X[:, :6001], out=out, winner=winner, sel=sel, sel_workers=selw, ws=ws)
+    for spec in specs:
+        w = wl.make_workload(spec)            # new gradients, moved onto the captured partition (the tables are
+        Xn = torch.empty_like(w.X)            # kernel parameters baked into the graph)
+        Xn[torch.as_tensor(w0.members, dtype=torch.long)] = w.X[torch.as_tensor(w.members, dtype=torch.long)]
+        X.copy_(Xn)
+        out.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        ref = oracle.detox_aggregate(Xn.numpy()[:, :6001], w0.members, 3, "mean" if a1 == "median" else "none",
+                                     w0.set_offsets, w0.set_members, oname, f, m_sel)
+        assert winner.cpu().numpy().tolist() == ref["winner"].tolist()
+        assert rel_l2(out.cpu().numpy(), ref["out"]) <= TOL
