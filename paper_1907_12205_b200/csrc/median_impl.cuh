@@ -53,28 +53,33 @@ colselect_reg_kernel(const float* __restrict__ X, int64_t ld, int m, int64_t d, 
     const int pad = kPadded ? (M - m) >> 1 : 0;   // lowest keys added (and as many highest)
     int32_t key[C][M];
     // All loads first, with no branch in between, so that they are in flight together; slots beyond m
-    // re-read the last row and are replaced by padding keys afterwards.
+    // re-read the last row and are replaced by padding keys afterwards.  The test for a row list is
+    // taken once, outside the loads: a per-load test would serialise them.
+    auto load_all = [&](auto row_of) {
 #pragma unroll
-    for (int i = 0; i < M; ++i) {
-        const int ri = kPadded ? (i < m ? i : m - 1) : i;
-        const int rr = rows ? rows[ri] : ri;          // a negative entry of the row list stands for a zero row
-        const uint32_t keep = rr < 0 ? 0u : 0xFFFFFFFFu;
-        const float* p = X + (int64_t)(rr < 0 ? 0 : rr) * ld + col0;
-        if (C == 4 && valid == 4) {
-            uint4 v = ld_stream_u4(p);
-            key[0][i] = (int32_t)(v.x & keep);
-            key[1 % C][i] = (int32_t)(v.y & keep);
-            key[2 % C][i] = (int32_t)(v.z & keep);
-            key[3 % C][i] = (int32_t)(v.w & keep);
-        } else if (C == 2 && valid == 2) {
-            uint2 v = __ldcs(reinterpret_cast<const uint2*>(p));
-            key[0][i] = (int32_t)(v.x & keep);
-            key[1 % C][i] = (int32_t)(v.y & keep);
-        } else {
+        for (int i = 0; i < M; ++i) {
+            const int ri = kPadded ? (i < m ? i : m - 1) : i;
+            const int rr = row_of(ri);                    // a negative entry of the row list stands for a zero row
+            const uint32_t keep = rr < 0 ? 0u : 0xFFFFFFFFu;
+            const float* p = X + (int64_t)(rr < 0 ? 0 : rr) * ld + col0;
+            if (C == 4 && valid == 4) {
+                uint4 v = ld_stream_u4(p);
+                key[0][i] = (int32_t)(v.x & keep);
+                key[1 % C][i] = (int32_t)(v.y & keep);
+                key[2 % C][i] = (int32_t)(v.z & keep);
+                key[3 % C][i] = (int32_t)(v.w & keep);
+            } else if (C == 2 && valid == 2) {
+                uint2 v = __ldcs(reinterpret_cast<const uint2*>(p));
+                key[0][i] = (int32_t)(v.x & keep);
+                key[1 % C][i] = (int32_t)(v.y & keep);
+            } else {
 #pragma unroll
-            for (int c = 0; c < C; ++c) key[c][i] = c < valid ? (int32_t)(ld_stream_u1(p + c) & keep) : 0;
+                for (int c = 0; c < C; ++c) key[c][i] = c < valid ? (int32_t)(ld_stream_u1(p + c) & keep) : 0;
+            }
         }
-    }
+    };
+    if (rows) load_all([&](int ri) { return rows[ri]; });
+    else load_all([](int ri) { return ri; });
 #pragma unroll
     for (int i = 0; i < M; ++i) {
 #pragma unroll

@@ -32,14 +32,19 @@ colselect_pair_kernel(const float* __restrict__ X, int64_t ld, int m, int64_t d,
     const int extra = m - kHalf;                        // real rows held by lane 1
 
     int32_t key[kHalf];
+    // the test for a row list is taken once, outside the loads: a per-load test would serialise them
+    auto load_all = [&](auto row_of) {
 #pragma unroll
-    for (int i = 0; i < kHalf; ++i) {
-        int ri = hsel ? kHalf + i : i;
-        ri = ri < m ? ri : m - 1;
-        const int rr = rows ? rows[ri] : ri;      // a negative entry of the row list stands for a zero row
-        const uint32_t v = ld_stream_u1(X + (int64_t)(rr < 0 ? 0 : rr) * ld + col);
-        key[i] = (int32_t)(rr < 0 ? 0u : v);
-    }
+        for (int i = 0; i < kHalf; ++i) {
+            int ri = hsel ? kHalf + i : i;
+            ri = ri < m ? ri : m - 1;
+            const int rr = row_of(ri);                // a negative entry of the row list stands for a zero row
+            const uint32_t v = ld_stream_u1(X + (int64_t)(rr < 0 ? 0 : rr) * ld + col);
+            key[i] = (int32_t)(rr < 0 ? 0u : v);
+        }
+    };
+    if (rows) load_all([&](int ri) { return rows[ri]; });
+    else load_all([](int ri) { return ri; });
 #pragma unroll
     for (int i = 0; i < kHalf; ++i) {
         int32_t k = key_of_bits((uint32_t)key[i]);
