@@ -38,13 +38,14 @@ constexpr int kProdWarps = 16;
 constexpr int kProdThreads = kProdWarps * 32;
 constexpr int kMmaWarps = 2;                   // two issuing threads, so one's bookkeeping overlaps the other's MMAs
 constexpr int kTcThreads = kProdThreads + 32 * (kMmaWarps + 1);  // + the MMA warps + the TMA warp
-constexpr int kMaxStages = 6;
+constexpr int kMaxStages = 12;
 constexpr long long kWaitLimitCycles = 2000000000LL;  // ~1 s at the SM clock
 constexpr int64_t kSlabCols = 4096;          // columns accumulated in tensor memory before a drain
 constexpr int kReduceChunks = 32;
 
 struct TcPlan {
-    int rows_pad;    // rows of each shared-memory tile (128 or 256)
+    int rows_pad;    // rows of each shared-memory tile (64, 128 or 256); a stage holds two tiles
+    int mrows;       // M of the MMA: 64 for m <= 64, else 128
     int box_rows;    // rows the TMA box brings in: m rounded up to 8
     int nhalf;       // accumulator halves of 128 rows
     int ncol;        // N of the MMA: m rounded up to 16
@@ -59,7 +60,8 @@ struct TcPlan {
 TcPlan tc_plan(int m, int64_t d) {
     TcPlan p;
     p.nhalf = m > 128 ? 2 : 1;
-    p.rows_pad = 128 * p.nhalf;
+    p.mrows = m <= 64 ? 64 : 128;
+    p.rows_pad = m <= 64 ? 64 : 128 * p.nhalf;
     p.box_rows = (m + 7) / 8 * 8;
     p.ncol = (m + 15) / 16 * 16;
     // m <= 128: one MMA per K-step with B = [hi ; 2lo] stacked (N = 2 ncol); the two issuing threads take
@@ -227,7 +229,7 @@ struct TcSmem {
 // J = 16-byte chunks per transform thread and K-block (m * 8 / 512 rounded up to a power of two)
 template <int J>
 __global__ void __launch_bounds__(kTcThreads, 1)
-gram_tc_kernel(const __grid_constant__ CUtensorMap xmap, int m, int64_t d, int rows_pad, int box_rows, int nhalf,
+gram_tc_kernel(const __grid_constant__ CUtensorMap xmap, int m, int64_t d, int rows_pad, int mrows, int box_rows, int nhalf,
                int ncol, int chains, int tmem_cols, int stages, int nitems, float* __restrict__ partial,
                float* __restrict__ norms, int* __restrict__ status) {
     extern __shared__ uint8_t smem_raw[];
@@ -330,7 +332,8 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap xmap, int m, int64_t d, int r
             const int quarter = warp & 3;
             float* out_item = partial + (int64_t)item * m * ncol;
             for (int h = 0; h < nhalf; ++h) {
-                const int row = h * 128 + quarter * 32 + lane;
+                // M = 128: accumulator row i sits in TMEM lane i; M = 64: in lane 32 (i / 16) + i % 16
+                const int row = mrows == 64 ? (lane < 16 ? quarter * 16 + lane : m) : h * 128 + quarter * 32 + lane;
                 for (int cc = warp >> 2; cc * 32 < ncol; cc += kProdWarps / 4) {
                     float acc[32];
 #pragma unroll
@@ -394,7 +397,7 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap xmap, int m, int64_t d, int r
         // ------------------------------------------------ (lane 0 of the two warps after the transform warps)
         const int g = warp - kProdWarps;
         const int n_mma = nhalf == 1 ? 2 * ncol : ncol;
-        const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(n_mma >> 3) << 17) | ((128u >> 4) << 24);
+        const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(n_mma >> 3) << 17) | ((uint32_t)(mrows >> 4) << 24);
         int s = 0, turn = 0;
         uint32_t ph = 0;
         for (int local_item = 0; local_item < my_items; ++local_item) {
@@ -535,7 +538,7 @@ detox_status launch_tc(const TcPlan& p, const CUtensorMap& xmap, int m, int64_t 
     if (cudaFuncSetAttribute(gram_tc_kernel<J>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem_bytes) !=
         cudaSuccess)
         return DETOX_ERR_CUDA;
-    gram_tc_kernel<J><<<p.grid, kTcThreads, p.smem_bytes, s>>>(xmap, m, d, p.rows_pad, p.box_rows, p.nhalf, p.ncol,
+    gram_tc_kernel<J><<<p.grid, kTcThreads, p.smem_bytes, s>>>(xmap, m, d, p.rows_pad, p.mrows, p.box_rows, p.nhalf, p.ncol,
                                                                p.chains, p.tmem_cols, p.stages, p.nitems, partial, norms, status);
     return launch_status();
 }
