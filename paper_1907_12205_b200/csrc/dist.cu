@@ -18,10 +18,12 @@ namespace {
 constexpr int kDirThreads = 256;
 constexpr int kDirWarps = kDirThreads / 32;
 
-template <int M>
+// VEC = columns per thread and step (4: 16-byte loads; 2: 8-byte; 1: scalar).  Columns past the last
+// multiple of VEC are added by one thread.
+template <int M, int VEC>
 __global__ void __launch_bounds__(kDirThreads)
 sqdist_direct_kernel(const float* __restrict__ X, int64_t ld, int64_t d, const int32_t* __restrict__ rows,
-                     bool vec2, double* __restrict__ partial) {
+                     double* __restrict__ partial) {
     constexpr int NP = M * (M - 1) / 2;
     float acc[NP];
 #pragma unroll
@@ -37,49 +39,43 @@ sqdist_direct_kernel(const float* __restrict__ X, int64_t ld, int64_t d, const i
     }
 
     const int64_t stride = (int64_t)gridDim.x * kDirThreads;
-    if (vec2) {
-        const int64_t n2 = d >> 1;
-        for (int64_t c = (int64_t)blockIdx.x * kDirThreads + threadIdx.x; c < n2; c += stride) {
-            float2 v[M];
+    const int64_t nv = d / VEC;
+    for (int64_t c = (int64_t)blockIdx.x * kDirThreads + threadIdx.x; c < nv; c += stride) {
+        float v[M][VEC];
 #pragma unroll
-            for (int i = 0; i < M; ++i) {
-                v[i] = __ldcs(reinterpret_cast<const float2*>(rowp[i]) + c);
-                if (keep[i] == 0.f) v[i] = make_float2(0.f, 0.f);
+        for (int i = 0; i < M; ++i) {
+            if (VEC == 4) {
+                const float4 t = ld_stream_f4(rowp[i] + c * 4);
+                v[i][0] = t.x; v[i][1 % VEC] = t.y; v[i][2 % VEC] = t.z; v[i][3 % VEC] = t.w;
+            } else if (VEC == 2) {
+                const float2 t = __ldcs(reinterpret_cast<const float2*>(rowp[i]) + c);
+                v[i][0] = t.x; v[i][1 % VEC] = t.y;
+            } else {
+                v[i][0] = __ldcs(rowp[i] + c);
             }
-            int p = 0;
 #pragma unroll
-            for (int i = 0; i < M; ++i)
-#pragma unroll
-                for (int j = i + 1; j < M; ++j, ++p) {
-                    const float a = v[i].x - v[j].x, b = v[i].y - v[j].y;
-                    acc[p] = fmaf(a, a, acc[p]);
-                    acc[p] = fmaf(b, b, acc[p]);
-                }
+            for (int e = 0; e < VEC; ++e) v[i][e] = keep[i] == 0.f ? 0.f : v[i][e];
         }
-        if ((d & 1) && blockIdx.x == 0 && threadIdx.x == 0) {
-            int p = 0;
+        int p = 0;
 #pragma unroll
-            for (int i = 0; i < M; ++i)
+        for (int i = 0; i < M; ++i)
 #pragma unroll
-                for (int j = i + 1; j < M; ++j, ++p) {
-                    const float a = (keep[i] == 0.f ? 0.f : rowp[i][d - 1]) - (keep[j] == 0.f ? 0.f : rowp[j][d - 1]);
+            for (int j = i + 1; j < M; ++j, ++p) {
+#pragma unroll
+                for (int e = 0; e < VEC; ++e) {
+                    const float a = v[i][e] - v[j][e];
                     acc[p] = fmaf(a, a, acc[p]);
                 }
-        }
-    } else {
-        for (int64_t c = (int64_t)blockIdx.x * kDirThreads + threadIdx.x; c < d; c += stride) {
-            float v[M];
-#pragma unroll
-            for (int i = 0; i < M; ++i) {
-                v[i] = __ldcs(rowp[i] + c);
-                if (keep[i] == 0.f) v[i] = 0.f;
             }
+    }
+    if (VEC > 1 && blockIdx.x == 0 && threadIdx.x == 0) {
+        for (int64_t c = nv * VEC; c < d; ++c) {
             int p = 0;
 #pragma unroll
             for (int i = 0; i < M; ++i)
 #pragma unroll
                 for (int j = i + 1; j < M; ++j, ++p) {
-                    const float a = v[i] - v[j];
+                    const float a = (keep[i] == 0.f ? 0.f : rowp[i][c]) - (keep[j] == 0.f ? 0.f : rowp[j][c]);
                     acc[p] = fmaf(a, a, acc[p]);
                 }
         }
@@ -257,8 +253,10 @@ template <int M>
 detox_status launch_direct(const float* X, int64_t ld, int64_t d, const int32_t* rows, double* D, double* partial,
                            cudaStream_t s) {
     const int nb = direct_blocks(d);
-    const bool vec2 = (reinterpret_cast<uintptr_t>(X) & 7u) == 0 && ld % 2 == 0;
-    sqdist_direct_kernel<M><<<nb, kDirThreads, 0, s>>>(X, ld, d, rows, vec2, partial);
+    const uintptr_t addr = reinterpret_cast<uintptr_t>(X);
+    if ((addr & 15u) == 0 && ld % 4 == 0) sqdist_direct_kernel<M, 4><<<nb, kDirThreads, 0, s>>>(X, ld, d, rows, partial);
+    else if ((addr & 7u) == 0 && ld % 2 == 0) sqdist_direct_kernel<M, 2><<<nb, kDirThreads, 0, s>>>(X, ld, d, rows, partial);
+    else sqdist_direct_kernel<M, 1><<<nb, kDirThreads, 0, s>>>(X, ld, d, rows, partial);
     detox_status st = launch_status();
     if (st != DETOX_OK) return st;
     sqdist_direct_reduce_kernel<<<(M * (M - 1) / 2 + 3) / 4, 128, 0, s>>>(partial, nb, M, D);

@@ -12,9 +12,10 @@
 // MMA reads only the upper 19 bits of each word.  Warps 0-15 read the tile back, form
 // 2 lo = 2 (x - (x with its low 13 bits cleared)) and write the second tile; lane 0 of warps 16, 17
 // issue the MMAs; mbarriers form a ring of stages between the three roles.
-// Work is cut into K-slabs; at the end of a slab the accumulator is drained to a per-slab fp32
-// partial in global memory and the slabs are added in fp64 in a fixed order afterwards, so the long
-// sum never lives in one fp32 accumulator and the result is deterministic.
+// K-blocks are dealt round-robin to the CTAs and every 128 of a CTA's K-blocks form a slab; at the end
+// of a slab the accumulator is drained to a per-slab fp32 partial in global memory and the slabs are
+// added in fp64 in a fixed order afterwards, so the long sum never lives in one fp32 accumulator and
+// the result is deterministic.
 //
 // The tensor cores add into their fp32 accumulator by truncation, so a long same-sign sum (a row with
 // itself, or with a copy of itself) comes out low by a few 1e-5 relative per slab.  The producers
@@ -40,7 +41,7 @@ constexpr int kMmaWarps = 2;                   // two issuing threads, so one's 
 constexpr int kTcThreads = kProdThreads + 32 * (kMmaWarps + 1);  // + the MMA warps + the TMA warp
 constexpr int kMaxStages = 12;
 constexpr long long kWaitLimitCycles = 2000000000LL;  // ~1 s at the SM clock
-constexpr int64_t kSlabCols = 4096;          // columns accumulated in tensor memory before a drain
+constexpr int64_t kSlabCols = 4096;          // columns (128 K-blocks) accumulated in tensor memory before a drain
 constexpr int kReduceChunks = 32;
 
 struct TcPlan {
@@ -52,7 +53,8 @@ struct TcPlan {
     int chains;      // m <= 128: accumulators, one per MMA-issuing thread
     int tmem_cols;   // power of two >= the accumulator columns, >= 32
     int stages;
-    int nitems;      // K-slabs
+    int nkb_total;   // K-blocks in all: d / 32 rounded up
+    int nitems;      // slab slots: grid x the largest number of slabs a CTA has
     int grid;
     size_t smem_bytes;
 };
@@ -74,8 +76,12 @@ TcPlan tc_plan(int m, int64_t d) {
     size_t stage = (size_t)2 * p.rows_pad * 128;
     p.stages = (int)((192 * 1024) / stage);
     if (p.stages > kMaxStages) p.stages = kMaxStages;
-    p.nitems = (int)ceil_div(d, kSlabCols);
-    p.grid = p.nitems < kSMs ? p.nitems : kSMs;
+    // K-blocks are dealt round-robin to the CTAs, so that every CTA has the same number of them (to within one)
+    // whatever d is, and neighbouring CTAs read neighbouring 128-byte pieces of a row
+    p.nkb_total = (int)ceil_div(d, (int64_t)kKB);
+    p.grid = p.nkb_total < kSMs ? p.nkb_total : kSMs;
+    const int per_cta = (p.nkb_total + p.grid - 1) / p.grid;
+    p.nitems = p.grid * (int)ceil_div((int64_t)per_cta, kSlabCols / kKB);
     p.smem_bytes = stage * p.stages + 1024 /*barriers*/ + 1024 /*alignment slack*/;
     return p;
 }
@@ -153,7 +159,7 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
     return desc;
 }
 
-// D[tmem] (+)= A[smem] * B[smem]^T, TF32 inputs, fp32 accumulate, M = 128.
+// D[tmem] (+)= A[smem] * B[smem]^T, TF32 inputs, fp32 accumulate; M and N come with the instruction descriptor.
 __device__ __forceinline__ void mma_tf32(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
@@ -230,7 +236,7 @@ struct TcSmem {
 template <int J>
 __global__ void __launch_bounds__(kTcThreads, 1)
 gram_tc_kernel(const __grid_constant__ CUtensorMap xmap, int m, int64_t d, int rows_pad, int mrows, int box_rows, int nhalf,
-               int ncol, int chains, int tmem_cols, int stages, int nitems, float* __restrict__ partial,
+               int ncol, int chains, int tmem_cols, int stages, int nkb_total, int nitems, float* __restrict__ partial,
                float* __restrict__ norms, int* __restrict__ status) {
     extern __shared__ uint8_t smem_raw[];
     // tiles need 1024-byte alignment for the 128-byte swizzle pattern
@@ -264,14 +270,13 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap xmap, int m, int64_t d, int r
     tc_fence_after();
     const uint32_t tmem_base = sm->tmem_base;
 
-    // K-blocks of this CTA, over all its slabs, as one sequence t = 0 .. total-1.
-    // Every slab has kSlabCols / kKB blocks except the globally last one, which may be shorter.
+    // This CTA owns the K-blocks b, b + G, b + 2G, ... (b = blockIdx.x, G = gridDim.x), t = 0 .. total-1 in its own
+    // count; a slab is kBlocksPerSlab consecutive ones of them (the last slab may be shorter) and goes to slot
+    // b + G * (slab number).
     constexpr int kBlocksPerSlab = (int)(kSlabCols / kKB);
-    const int my_items = (nitems - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
-    const int last_item = (int)blockIdx.x + (my_items - 1) * (int)gridDim.x;
-    const int last_nkb = (int)(((last_item == nitems - 1 ? d : (int64_t)(last_item + 1) * kSlabCols) -
-                                (int64_t)last_item * kSlabCols + kKB - 1) / kKB);
-    const int total = (my_items - 1) * kBlocksPerSlab + last_nkb;
+    const int total = (nkb_total - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
+    const int my_items = (total + kBlocksPerSlab - 1) / kBlocksPerSlab;
+    const int last_nkb = total - (my_items - 1) * kBlocksPerSlab;
 
     if (warp < kProdWarps) {
         // ------------------------------------------------ transform warps, then epilogue of each slab
@@ -365,14 +370,20 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap xmap, int m, int64_t d, int r
             kb = 0;
             ++li;
         }
+        // slots of slabs this CTA does not have (it owns one K-block fewer than others) read as zero
+        for (int l2 = my_items; l2 * (int)gridDim.x < nitems; ++l2) {
+            const int64_t item = (int64_t)blockIdx.x + (int64_t)l2 * gridDim.x;
+            for (int e = tid; e < m * ncol; e += kProdThreads) partial[item * m * ncol + e] = 0.f;
+            for (int e = tid; e < m; e += kProdThreads) norms[item * m + e] = 0.f;
+        }
     } else if (warp == kProdWarps + kMmaWarps) {
         // ------------------------------------------------ the TMA thread
         if (lane == 0) {
             const uint32_t tx_bytes = (uint32_t)box_rows * 128u;
             int issued = 0;
-            int s = 0, kb = 0;
+            int s = 0;
             uint32_t ph = 0;
-            int64_t c0 = (int64_t)blockIdx.x * kSlabCols;            // first column of the current K-block
+            int64_t c0 = (int64_t)blockIdx.x * kKB;                  // first column of the current K-block
             for (int t = 0; t < total; ++t) {
                 mbar_wait(&sm->empty[s], ph ^ 1u, abort_flag, status);   // MMAs that read this stage are done
                 if (*abort_flag) break;
@@ -380,8 +391,7 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap xmap, int m, int64_t d, int r
                 tma_load_2d(base + (size_t)s * stage_bytes, &xmap, (int)c0, 0, &sm->landed[s]);
                 issued = t + 1;
                 if (++s == stages) { s = 0; ph ^= 1u; }
-                c0 += kKB;
-                if (++kb == kBlocksPerSlab) { kb = 0; c0 += (int64_t)(gridDim.x - 1) * kSlabCols; }   // next slab of this CTA
+                c0 += (int64_t)gridDim.x * kKB;
             }
             if (*abort_flag) {
                 // give the copies still in flight a bounded time to land before the CTA goes away
@@ -539,7 +549,7 @@ detox_status launch_tc(const TcPlan& p, const CUtensorMap& xmap, int m, int64_t 
         cudaSuccess)
         return DETOX_ERR_CUDA;
     gram_tc_kernel<J><<<p.grid, kTcThreads, p.smem_bytes, s>>>(xmap, m, d, p.rows_pad, p.mrows, p.box_rows, p.nhalf, p.ncol,
-                                                               p.chains, p.tmem_cols, p.stages, p.nitems, partial, norms, status);
+                                                               p.chains, p.tmem_cols, p.stages, p.nkb_total, p.nitems, partial, norms, status);
     return launch_status();
 }
 
