@@ -13,28 +13,31 @@ constexpr int kRegThreads = 128;
 // Start of the window of `beta` consecutive sorted values that are closest to the median `med`.
 // dist(i) = |v_i - med| in fp32 falls, then rises, along the sorted order.  The window [L, L+beta) is
 // right when the value just above it is not strictly closer than its lowest value; on equal distance
-// the lower value stays.  The predicate below is true exactly for the starts that are too far left.
+// the lower value stays.  The predicate below is true exactly for the starts that are too far left
+// (true for s < L, false from L on), so L is found by bisection over s in [0, theta - beta].
 template <typename KeyAt>
 __device__ __forceinline__ int window_start(int theta, int beta, float med, KeyAt key_at) {
     const int h_lo = (theta - 1) >> 1;
-    int L = 0;
-    for (int s = 0; s < theta - beta; ++s) {
+    int lo = 0, hi = theta - beta;
+    while (lo < hi) {
+        const int s = (lo + hi) >> 1;
         bool move_right;
         if (s + beta <= h_lo) {
             move_right = true;  // the window must reach the middle element
         } else {
-            const float lo = float_of_key(key_at(s));
-            const float up = float_of_key(key_at(s + beta));
-            move_right = fabsf(up - med) < fabsf(lo - med);
+            const float below = float_of_key(key_at(s));
+            const float above = float_of_key(key_at(s + beta));
+            move_right = fabsf(above - med) < fabsf(below - med);
         }
-        L += move_right ? 1 : 0;
+        if (move_right) lo = s + 1;
+        else hi = s;
     }
-    return L;
+    return lo;
 }
 
 __host__ __device__ constexpr int reg_threads(int M, int C, bool trim) {
-    // the TRIM variant keeps M * C keys per thread in (static) shared memory
-    return (trim && M * C * kRegThreads * 4 > 48 * 1024) ? kRegThreads / 2 : kRegThreads;
+    // the TRIM variant keeps M * C keys per thread in (static) shared memory, next to a staged row list
+    return (trim && M * C * kRegThreads * 4 + M * 4 > 48 * 1024) ? kRegThreads / 2 : kRegThreads;
 }
 
 // M = network size, m = rows actually present (M - m even; the gap is filled with lowest / highest keys)
@@ -43,6 +46,13 @@ __global__ void __launch_bounds__(reg_threads(M, C, TRIM))
 colselect_reg_kernel(const float* __restrict__ X, int64_t ld, int m, int64_t d, const int32_t* __restrict__ rows,
                      int beta, float* __restrict__ out) {
     constexpr int kThreads = reg_threads(M, C, TRIM);
+    // a row list is staged in shared memory once per CTA: read from global memory it would put an index
+    // load in front of every data load
+    __shared__ int32_t srow[M];
+    if (rows) {
+        for (int i = threadIdx.x; i < m; i += kThreads) srow[i] = rows[i];
+        __syncthreads();
+    }
     const int64_t col0 = ((int64_t)blockIdx.x * kThreads + threadIdx.x) * C;
     if (col0 >= d) return;
     const int64_t left = d - col0;
@@ -78,7 +88,7 @@ colselect_reg_kernel(const float* __restrict__ X, int64_t ld, int m, int64_t d, 
             }
         }
     };
-    if (rows) load_all([&](int ri) { return rows[ri]; });
+    if (rows) load_all([&](int ri) { return srow[ri]; });
     else load_all([](int ri) { return ri; });
 #pragma unroll
     for (int i = 0; i < M; ++i) {
@@ -109,11 +119,11 @@ colselect_reg_kernel(const float* __restrict__ X, int64_t ld, int m, int64_t d, 
             const int cnt = beta < 0 ? -beta : beta;
             const int L = pad + (beta < 0 ? (m - cnt) >> 1
                                           : window_start(m, beta, med, [&](int i) { return mine[(i + pad) * kThreads]; }));
-            float acc = 0.f;
+            // four interleaved partial sums (shorter dependency chains, smaller rounding error)
+            float acc[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-            for (int i = 0; i < M; ++i)
-                if (i >= L && i < L + cnt) acc += float_of_key(key[c][i]);
-            res[c] = acc / (float)cnt;
+            for (int i = 0; i < M; ++i) acc[i & 3] += (i >= L && i < L + cnt) ? float_of_key(key[c][i]) : 0.f;
+            res[c] = ((acc[0] + acc[1]) + (acc[2] + acc[3])) / (float)cnt;
         }
     }
     if (C == 4 && valid == 4) {

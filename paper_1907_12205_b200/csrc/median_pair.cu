@@ -22,6 +22,13 @@ __global__ void __launch_bounds__(kPairThreads)
 colselect_pair_kernel(const float* __restrict__ X, int64_t ld, int m, int64_t d, const int32_t* __restrict__ rows,
                       int beta, float* __restrict__ out) {
     extern __shared__ int32_t sorted[];        // TRIM only: [2 * kHalf][kPairCols]
+    // a row list is staged in shared memory once per CTA: read from global memory it would put an index
+    // load in front of every data load
+    __shared__ int32_t srow[2 * kHalf];
+    if (rows) {
+        for (int i = threadIdx.x; i < m; i += kPairThreads) srow[i] = rows[i];
+        __syncthreads();
+    }
     const int hsel = threadIdx.x & 1;
     const int cidx = threadIdx.x >> 1;
     const int64_t col_raw = (int64_t)blockIdx.x * kPairCols + cidx;
@@ -43,7 +50,7 @@ colselect_pair_kernel(const float* __restrict__ X, int64_t ld, int m, int64_t d,
             key[i] = (int32_t)(rr < 0 ? 0u : v);
         }
     };
-    if (rows) load_all([&](int ri) { return rows[ri]; });
+    if (rows) load_all([&](int ri) { return srow[ri]; });
     else load_all([](int ri) { return ri; });
 #pragma unroll
     for (int i = 0; i < kHalf; ++i) {
@@ -96,22 +103,20 @@ colselect_pair_kernel(const float* __restrict__ X, int64_t ld, int m, int64_t d,
         for (int i = 0; i < kHalf; ++i) sorted[(hsel * kHalf + i) * kPairCols + slot] = key[i];
     }
     __syncwarp();
-    if (hsel == 0 && live) {
-        auto at = [&](int p) { return sorted[p * kPairCols + ((cidx + (p >= kHalf ? 16 : 0)) & (kPairCols - 1))]; };
-        float med = float_of_key(at(kHalf - 1));
-        if ((m & 1) == 0) med = (med + float_of_key(at(kHalf))) * 0.5f;
-        const int cnt = beta < 0 ? -beta : beta;   // beta < 0: the middle -beta values (trimmed mean)
-        const int L = pad_lo + (beta < 0 ? (m - cnt) >> 1
-                                         : regselect::window_start(m, beta, med, [&](int i) { return at(i + pad_lo); }));
-        float acc = 0.f, comp = 0.f;          // compensated fp32 sum
-        for (int p = L; p < L + cnt; ++p) {
-            const float y = float_of_key(at(p)) - comp;
-            const float t = acc + y;
-            comp = (t - acc) - y;
-            acc = t;
-        }
-        out[col] = acc / (float)cnt;
-    }
+    auto at = [&](int p) { return sorted[p * kPairCols + ((cidx + (p >= kHalf ? 16 : 0)) & (kPairCols - 1))]; };
+    float med = float_of_key(at(kHalf - 1));
+    if ((m & 1) == 0) med = (med + float_of_key(at(kHalf))) * 0.5f;
+    const int cnt = beta < 0 ? -beta : beta;   // beta < 0: the middle -beta values (trimmed mean)
+    // both lanes of the pair find the same window; each adds the part of it that sits in its own registers
+    const int L = pad_lo + (beta < 0 ? (m - cnt) >> 1
+                                     : regselect::window_start(m, beta, med, [&](int i) { return at(i + pad_lo); }));
+    const int first = L - hsel * kHalf, last = first + cnt;     // window in this lane's positions
+    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int i = 0; i < kHalf; ++i) acc[i & 3] += (i >= first && i < last) ? float_of_key(key[i]) : 0.f;
+    float sum = (acc[0] + acc[1]) + (acc[2] + acc[3]);
+    sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+    if (hsel == 0 && live) out[col] = sum / (float)cnt;
 }
 
 
