@@ -42,7 +42,7 @@ constexpr int kTcThreads = kProdThreads + 32 * (kMmaWarps + 1);  // + the MMA wa
 constexpr int kMaxStages = 12;
 constexpr long long kWaitLimitCycles = 2000000000LL;  // ~1 s at the SM clock
 constexpr int64_t kSlabCols = 4096;          // columns (128 K-blocks) accumulated in tensor memory before a drain
-constexpr int kReduceChunks = 32;
+constexpr int kMinReduceChunks = 32, kMaxReduceChunks = 256;
 
 struct TcPlan {
     int rows_pad;    // rows of each shared-memory tile (64, 128 or 256); a stage holds two tiles
@@ -84,6 +84,17 @@ TcPlan tc_plan(int m, int64_t d) {
     p.nitems = p.grid * (int)ceil_div((int64_t)per_cta, kSlabCols / kKB);
     p.smem_bytes = stage * p.stages + 1024 /*barriers*/ + 1024 /*alignment slack*/;
     return p;
+}
+
+// Slab slots are added up in `chunks` independent groups (one CTA per group and pair of 32-row blocks), enough
+// of them to fill the GPU when m is small.
+int reduce_chunks(int m, int nitems) {
+    const int nt = (m + 31) / 32, pairs = nt * (nt + 1) / 2;
+    int c = (8 * kSMs + pairs - 1) / pairs;
+    if (c < kMinReduceChunks) c = kMinReduceChunks;
+    if (c > kMaxReduceChunks) c = kMaxReduceChunks;
+    if (c > nitems) c = nitems;
+    return c;
 }
 
 // ------------------------------------------------------------------------------------ PTX wrappers
@@ -460,53 +471,103 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap xmap, int m, int64_t d, int r
 
 // For one chunk of slabs: gpart[chunk][i*m+j] (i < j) = sum_s sym(T(s))_ij * (r_i(s) + r_j(s)) / 2 with
 // r_i(s) = exact norm / tensor-core norm of row i in slab s; gpart[chunk][i*m+i] = sum_s exact norm.
-__global__ void tc_reduce_kernel(const float* __restrict__ partial, const float* __restrict__ norms, int nitems,
-                                 int m, int ncol, double* __restrict__ gpart) {
+// One CTA per pair of 32-row blocks (bi <= bj) and chunk: per slab it reads the tile T[bi][bj] and the
+// mirrored tile T[bj][bi] row by row (coalesced) and transposes the second through shared memory.
+constexpr int kRT = 32;
+__global__ void __launch_bounds__(kRT * 8)
+tc_reduce_kernel(const float* __restrict__ partial, const float* __restrict__ norms, int nitems, int m, int ncol,
+                 double* __restrict__ gpart) {
+    __shared__ float mirror[kRT][kRT + 1];
+    __shared__ double ratio_i[kRT], ratio_j[kRT];
+    const int nt = (m + kRT - 1) / kRT;
+    int bi = 0, rem = blockIdx.x;
+    while (rem >= nt - bi) { rem -= nt - bi; ++bi; }
+    const int bj = bi + rem;
     const int chunk = blockIdx.y;
-    const int per = (nitems + kReduceChunks - 1) / kReduceChunks;
+    const int per = (nitems + (int)gridDim.y - 1) / (int)gridDim.y;
     const int s0 = chunk * per, s1 = (s0 + per) < nitems ? (s0 + per) : nitems;
     const int64_t elems = (int64_t)m * ncol;
-    const int64_t total = (int64_t)m * m;
-    for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
-        const int i = (int)(e / m), j = (int)(e - (int64_t)i * m);
-        if (i > j) continue;
-        double acc = 0.0;
-        if (i == j) {
-            for (int s = s0; s < s1; ++s) acc += (double)norms[(int64_t)s * m + i];
-        } else {
-#pragma unroll 4
-            for (int s = s0; s < s1; ++s) {
-                const float* T = partial + (int64_t)s * elems;
-                const double tii = (double)T[(int64_t)i * ncol + i], tjj = (double)T[(int64_t)j * ncol + j];
-                const double ni = (double)norms[(int64_t)s * m + i], nj = (double)norms[(int64_t)s * m + j];
-                const double ri = tii > 0.0 ? ni / tii : 1.0;
-                const double rj = tjj > 0.0 ? nj / tjj : 1.0;
-                const double tij = 0.5 * ((double)T[(int64_t)i * ncol + j] + (double)T[(int64_t)j * ncol + i]);
-                acc += tij * (0.5 * (ri + rj));
+    const int tx = threadIdx.x & (kRT - 1), ty = threadIdx.x / kRT;   // ty = 0..7
+
+    double acc[kRT / 8];
+#pragma unroll
+    for (int k = 0; k < kRT / 8; ++k) acc[k] = 0.0;
+    double nsum = 0.0;                       // ty == 0 on a diagonal tile: exact norm of row bi*32 + tx
+    const int j = bj * kRT + tx;             // this thread's column of the tile
+
+    for (int s = s0; s < s1; ++s) {
+        const float* T = partial + (int64_t)s * elems;
+        const float* nrm = norms + (int64_t)s * m;
+        if (ty < 2) {
+            const int r = (ty == 0 ? bi : bj) * kRT + tx;
+            double ratio = 1.0;
+            if (r < m) {
+                const double t = (double)T[(int64_t)r * ncol + r], nv = (double)nrm[r];
+                if (t > 0.0) ratio = nv / t;
+                if (ty == 0 && bi == bj) nsum += nv;
             }
+            (ty == 0 ? ratio_i : ratio_j)[tx] = ratio;
         }
-        gpart[(int64_t)chunk * total + e] = acc;
+        float a[kRT / 8];
+#pragma unroll
+        for (int k = 0; k < kRT / 8; ++k) {
+            const int rl = ty + 8 * k;
+            const int ri = bi * kRT + rl, rj = bj * kRT + rl;
+            a[k] = (ri < m && j < m) ? T[(int64_t)ri * ncol + j] : 0.f;                                  // T[bi][bj]
+            mirror[rl][tx] = (rj < m && bi * kRT + tx < m) ? T[(int64_t)rj * ncol + bi * kRT + tx] : 0.f;   // T[bj][bi]
+        }
+        __syncthreads();
+#pragma unroll
+        for (int k = 0; k < kRT / 8; ++k) {
+            const int il = ty + 8 * k;
+            const double tij = 0.5 * ((double)a[k] + (double)mirror[tx][il]);
+            acc[k] += tij * (0.5 * (ratio_i[il] + ratio_j[tx]));
+        }
+        __syncthreads();
     }
+    const int64_t total = (int64_t)m * m;
+#pragma unroll
+    for (int k = 0; k < kRT / 8; ++k) {
+        const int i = bi * kRT + ty + 8 * k;
+        if (i < m && j < m && i < j) gpart[(int64_t)chunk * total + (int64_t)i * m + j] = acc[k];
+    }
+    if (ty == 0 && bi == bj && j < m) gpart[(int64_t)chunk * total + (int64_t)j * m + j] = nsum;
 }
 
-// D_ij = n_i + n_j - 2 G_ij (never negative, zero diagonal); status != 0 -> NaN
-__global__ void tc_dist_kernel(const double* __restrict__ gpart, int m, const int* __restrict__ status,
+// D_ij = n_i + n_j - 2 G_ij (never negative, zero diagonal); status != 0 -> NaN.
+// One warp per pair i < j: the lanes add the chunks round-robin, then a fixed butterfly.
+__global__ void tc_dist_kernel(const double* __restrict__ gpart, int nchunks, int m, const int* __restrict__ status,
                                double* __restrict__ D) {
     const bool bad = *status != 0;
     const int64_t total = (int64_t)m * m;
-    auto G = [&](int i, int j) {
-        double v = 0.0;
+    const int lane = threadIdx.x & 31;
+    const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    if (warp >= total) return;
+    const int i = (int)(warp / m), j = (int)(warp - (int64_t)i * m);
+    if (i > j) return;
+    if (i == j) {
+        if (lane == 0) D[warp] = bad ? __longlong_as_double(0x7ff8000000000000LL) : 0.0;
+        return;
+    }
+    double gii = 0.0, gjj = 0.0, gij = 0.0;
+    for (int c = lane; c < nchunks; c += 32) {
+        const double* g = gpart + (int64_t)c * total;
+        gii += g[(int64_t)i * m + i];
+        gjj += g[(int64_t)j * m + j];
+        gij += g[(int64_t)i * m + j];
+    }
 #pragma unroll
-        for (int c = 0; c < kReduceChunks; ++c) v += gpart[(int64_t)c * total + (int64_t)i * m + j];
-        return v;
-    };
-    for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
-        const int i = (int)(e / m), j = (int)(e - (int64_t)i * m);
-        if (bad) { D[e] = __longlong_as_double(0x7ff8000000000000LL); continue; }
-        if (i == j) { D[e] = 0.0; continue; }
-        const int a = i < j ? i : j, b = i < j ? j : i;
-        const double v = G(a, a) + G(b, b) - 2.0 * G(a, b);
-        D[e] = v > 0.0 ? v : 0.0;
+    for (int o = 16; o > 0; o >>= 1) {
+        gii += __shfl_xor_sync(0xffffffffu, gii, o);
+        gjj += __shfl_xor_sync(0xffffffffu, gjj, o);
+        gij += __shfl_xor_sync(0xffffffffu, gij, o);
+    }
+    if (lane == 0) {
+        double v = gii + gjj - 2.0 * gij;
+        v = v > 0.0 ? v : 0.0;
+        if (bad) v = __longlong_as_double(0x7ff8000000000000LL);
+        D[(int64_t)i * m + j] = v;
+        D[(int64_t)j * m + i] = v;
     }
 }
 
@@ -564,7 +625,7 @@ size_t tc_ws_bytes(int m, int64_t d) {
     TcPlan p = tc_plan(m, d);
     const size_t elems = (size_t)m * p.ncol;
     return align_up((size_t)p.nitems * elems * sizeof(float)) + align_up((size_t)p.nitems * m * sizeof(float)) +
-           align_up((size_t)kReduceChunks * m * m * sizeof(double));
+           align_up((size_t)reduce_chunks(m, p.nitems) * m * m * sizeof(double));
 }
 
 detox_status launch_sqdist_tc(const float* X, int64_t ld, int m, int64_t d, double* D, void* ws, int* status,
@@ -585,10 +646,12 @@ detox_status launch_sqdist_tc(const float* X, int64_t ld, int m, int64_t d, doub
     else if (per_thread <= 2) st = launch_tc<2>(p, xmap, m, d, partial, norms, status, s);
     else st = launch_tc<4>(p, xmap, m, d, partial, norms, status, s);
     if (st != DETOX_OK) return st;
-    tc_reduce_kernel<<<dim3((unsigned)ceil_div((int64_t)m * m, 256), kReduceChunks), 256, 0, s>>>(
-        partial, norms, p.nitems, m, p.ncol, gpart);
+    const int nt = (m + kRT - 1) / kRT;
+    const int nchunks = reduce_chunks(m, p.nitems);
+    tc_reduce_kernel<<<dim3((unsigned)(nt * (nt + 1) / 2), (unsigned)nchunks), kRT * 8, 0, s>>>(partial, norms, p.nitems, m,
+                                                                                           p.ncol, gpart);
     if ((st = launch_status()) != DETOX_OK) return st;
-    tc_dist_kernel<<<(unsigned)ceil_div((int64_t)m * m, 256), 256, 0, s>>>(gpart, m, status, D);
+    tc_dist_kernel<<<(unsigned)ceil_div((int64_t)m * m * 32, 256), 256, 0, s>>>(gpart, nchunks, m, status, D);
     return launch_status();
 }
 
