@@ -89,8 +89,17 @@ detox_status run_multikrum(const float* X, int64_t ld, int m, int64_t d, const i
                            float* out, int32_t* sel, double* scores, void* ws, cudaStream_t s) {
     KrumWs k = krum_ws(ws, m, d);
     int32_t* sel_buf = sel ? sel : k.sel;
+    detox_status st;
+    if (m >= 2 && m <= 16) {   // distance pass, then one small kernel for everything up to the chosen rows
+        int nblocks = 0;
+        if ((st = launch_sqdist_partials(X, ld, m, d, rows, k.dist, &nblocks, s)) != DETOX_OK) return st;
+        st = launch_krum_small(false, static_cast<const double*>(k.dist), nblocks, m, f, m_sel, rows, sel_buf, k.mapped,
+                               scores, k.status, s);
+        if (st != DETOX_OK) return st;
+        return launch_mean_rows(X, ld, d, rows ? k.mapped : sel_buf, m_sel, out, s);
+    }
     if (cudaMemsetAsync(k.status, 0, sizeof(int), s) != cudaSuccess) return DETOX_ERR_CUDA;
-    detox_status st = launch_sqdist(X, ld, m, d, rows, k.D, k.dist, k.status, s);
+    st = launch_sqdist(X, ld, m, d, rows, k.D, k.dist, k.status, s);
     if (st != DETOX_OK) return st;
     st = launch_multikrum_select(k.D, m, f, m_sel, sel_buf, scores, k.select, s);
     if (st != DETOX_OK) return st;
@@ -107,8 +116,17 @@ detox_status run_bulyan(const float* X, int64_t ld, int m, int64_t d, const int3
     KrumWs k = krum_ws(ws, m, d);
     int32_t* sel_buf = sel ? sel : k.sel;
     const int theta = m - 2 * f, beta = theta - 2 * f;
+    detox_status st;
+    if (m >= 2 && m <= 16) {   // distance pass, then one small kernel for everything up to the chosen rows
+        int nblocks = 0;
+        if ((st = launch_sqdist_partials(X, ld, m, d, rows, k.dist, &nblocks, s)) != DETOX_OK) return st;
+        st = launch_krum_small(true, static_cast<const double*>(k.dist), nblocks, m, f, 0, rows, sel_buf, k.mapped, nullptr,
+                               k.status, s);
+        if (st != DETOX_OK) return st;
+        return launch_coord_select(X, ld, theta, d, rows ? k.mapped : sel_buf, beta, out, s);
+    }
     if (cudaMemsetAsync(k.status, 0, sizeof(int), s) != cudaSuccess) return DETOX_ERR_CUDA;
-    detox_status st = launch_sqdist(X, ld, m, d, rows, k.D, k.dist, k.status, s);
+    st = launch_sqdist(X, ld, m, d, rows, k.D, k.dist, k.status, s);
     if (st != DETOX_OK) return st;
     st = launch_bulyan_select(k.D, m, f, sel_buf, k.select, s);
     if (st != DETOX_OK) return st;

@@ -95,6 +95,9 @@ detox_status launch_sqdist(const float* X, int64_t ld, int m, int64_t d, const i
 // gram_tc.cu: the tcgen05 path for 16 < m <= 256 (needs 16-byte aligned rows)
 bool tc_supported(const float* X, int64_t ld, int m, int64_t d);
 size_t tc_ws_bytes(int m, int64_t d);
+// 2 <= m <= 16: the direct kernel's per-CTA pair partials only (consumed by launch_krum_small)
+detox_status launch_sqdist_partials(const float* X, int64_t ld, int m, int64_t d, const int32_t* rows, void* ws,
+                                    int* nblocks, cudaStream_t s);
 detox_status launch_sqdist_tc(const float* X, int64_t ld, int m, int64_t d, double* D, void* ws, int* status,
                               cudaStream_t s);
 
@@ -109,6 +112,10 @@ size_t select_ws_bytes(int m);
 detox_status launch_multikrum_select(const double* D, int m, int f, int m_sel, int32_t* sel_dev,
                                      double* scores_dev, void* ws, cudaStream_t s);
 // Bulyan stage 1: theta = m - 2f rounds; sel_dev in selection order
+// 2 <= m <= 16: pair partials -> distances -> ranked lists -> selection (-> rows of X through the row list), one CTA
+detox_status launch_krum_small(bool bulyan, const double* partial, int nblocks, int m, int f, int m_sel,
+                               const int32_t* rows_dev, int32_t* sel_dev, int32_t* mapped_dev, double* scores_dev,
+                               int* status_dev, cudaStream_t s);
 detox_status launch_bulyan_select(const double* D, int m, int f, int32_t* sel_dev, void* ws,
                                   cudaStream_t s);
 // out[k] = map[idx[k]] (k < cnt), all device int32

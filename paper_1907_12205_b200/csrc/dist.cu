@@ -250,14 +250,21 @@ int direct_blocks(int64_t d) {
 }
 
 template <int M>
-detox_status launch_direct(const float* X, int64_t ld, int64_t d, const int32_t* rows, double* D, double* partial,
-                           cudaStream_t s) {
+detox_status launch_direct_partials(const float* X, int64_t ld, int64_t d, const int32_t* rows, double* partial,
+                                    cudaStream_t s) {
     const int nb = direct_blocks(d);
     const uintptr_t addr = reinterpret_cast<uintptr_t>(X);
     if ((addr & 15u) == 0 && ld % 4 == 0) sqdist_direct_kernel<M, 4><<<nb, kDirThreads, 0, s>>>(X, ld, d, rows, partial);
     else if ((addr & 7u) == 0 && ld % 2 == 0) sqdist_direct_kernel<M, 2><<<nb, kDirThreads, 0, s>>>(X, ld, d, rows, partial);
     else sqdist_direct_kernel<M, 1><<<nb, kDirThreads, 0, s>>>(X, ld, d, rows, partial);
-    detox_status st = launch_status();
+    return launch_status();
+}
+
+template <int M>
+detox_status launch_direct(const float* X, int64_t ld, int64_t d, const int32_t* rows, double* D, double* partial,
+                           cudaStream_t s) {
+    const int nb = direct_blocks(d);
+    detox_status st = launch_direct_partials<M>(X, ld, d, rows, partial, s);
     if (st != DETOX_OK) return st;
     sqdist_direct_reduce_kernel<<<(M * (M - 1) / 2 + 3) / 4, 128, 0, s>>>(partial, nb, M, D);
     return launch_status();
@@ -271,6 +278,23 @@ size_t dist_ws_bytes(int m, int64_t d) {
     size_t simt = align_up((size_t)g.npair * g.nslab * kGT * kGT * sizeof(double)) + align_up((size_t)m * m * sizeof(double));
     size_t tc = m <= 256 ? tc_ws_bytes(m, d) : 0;
     return simt > tc ? simt : tc;
+}
+
+// 2 <= m <= 16: only the per-CTA pair partials (ws: [nblocks][m (m-1) / 2] fp64, pairs in row-major order of
+// i < j); *nblocks says how many there are.
+detox_status launch_sqdist_partials(const float* X, int64_t ld, int m, int64_t d, const int32_t* rows, void* ws,
+                                    int* nblocks, cudaStream_t s) {
+    double* partial = static_cast<double*>(ws);
+    *nblocks = direct_blocks(d);
+    switch (m) {
+#define DETOX_CASE(M) \
+    case M: return launch_direct_partials<M>(X, ld, d, rows, partial, s);
+        DETOX_CASE(2) DETOX_CASE(3) DETOX_CASE(4) DETOX_CASE(5) DETOX_CASE(6) DETOX_CASE(7) DETOX_CASE(8)
+        DETOX_CASE(9) DETOX_CASE(10) DETOX_CASE(11) DETOX_CASE(12) DETOX_CASE(13) DETOX_CASE(14) DETOX_CASE(15)
+        DETOX_CASE(16)
+#undef DETOX_CASE
+        default: return DETOX_ERR_UNSUPPORTED;
+    }
 }
 
 detox_status launch_sqdist(const float* X, int64_t ld, int m, int64_t d, const int32_t* rows, double* D, void* ws,

@@ -75,10 +75,9 @@ __device__ __forceinline__ int krum_neighbours(int alive, int f) {
     return nb;
 }
 
-// One CTA, one thread per row (m <= 1024).
-__global__ void __launch_bounds__(1024)
-multikrum_select_kernel(const double* __restrict__ sorted_d, int m, int f, int m_sel, int32_t* __restrict__ sel,
-                        double* __restrict__ scores_out) {
+// One CTA, one thread per row (m <= blockDim.x); the lists may live in global or in shared memory.
+__device__ __forceinline__ void multikrum_select_body(const double* sorted_d, int m, int f, int m_sel, int32_t* sel,
+                                                      double* scores_out) {
     __shared__ double score[kMaxRows];
     __shared__ int chosen[kMaxRows];
     const int i = threadIdx.x;
@@ -104,9 +103,8 @@ multikrum_select_kernel(const double* __restrict__ sorted_d, int m, int f, int m
     }
 }
 
-__global__ void __launch_bounds__(1024)
-bulyan_select_kernel(const double* __restrict__ sorted_d, const int32_t* __restrict__ sorted_j,
-                     const int32_t* __restrict__ pos_t, int m, int f, int32_t* __restrict__ sel) {
+__device__ __forceinline__ void bulyan_select_body(const double* sorted_d, const int32_t* sorted_j, const int32_t* pos_t,
+                                                   int m, int f, int32_t* sel) {
     __shared__ unsigned char alive[kMaxRows];
     __shared__ double best_s[32];
     __shared__ int best_i[32];
@@ -201,6 +199,89 @@ bulyan_select_kernel(const double* __restrict__ sorted_d, const int32_t* __restr
     (void)nb;
 }
 
+__global__ void __launch_bounds__(1024)
+multikrum_select_kernel(const double* __restrict__ sorted_d, int m, int f, int m_sel, int32_t* __restrict__ sel,
+                        double* __restrict__ scores_out) {
+    multikrum_select_body(sorted_d, m, f, m_sel, sel, scores_out);
+}
+
+__global__ void __launch_bounds__(1024)
+bulyan_select_kernel(const double* __restrict__ sorted_d, const int32_t* __restrict__ sorted_j,
+                     const int32_t* __restrict__ pos_t, int m, int f, int32_t* __restrict__ sel) {
+    bulyan_select_body(sorted_d, sorted_j, pos_t, m, f, sel);
+}
+
+// m <= 16: everything between the distance pass and the final mean / order statistics in one CTA:
+// the per-CTA pair partials of the direct distance kernel are added up (one warp per pair, lanes
+// round-robin over the partials, then a fixed shuffle tree), every row's distances are ranked, the
+// selection runs on the lists in shared memory, and the chosen indices are mapped through the row
+// list when there is one.  The device status word is cleared on the way.
+constexpr int kSmallRows = 16;
+constexpr int kSmallThreads = 512;
+
+template <bool BULYAN>
+__global__ void __launch_bounds__(kSmallThreads)
+krum_small_kernel(const double* __restrict__ partial, int nblocks, int m, int f, int m_sel,
+                  const int32_t* __restrict__ rows, int32_t* __restrict__ sel, int32_t* __restrict__ mapped,
+                  double* __restrict__ scores_out, int* __restrict__ status) {
+    __shared__ double dmat[kSmallRows][kSmallRows];
+    __shared__ double s_sorted_d[kSmallRows * kSmallRows];
+    __shared__ int32_t s_sorted_j[kSmallRows * kSmallRows];
+    __shared__ int32_t s_pos_t[kSmallRows * kSmallRows];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (tid == 0) *status = 0;
+
+    const int np = m * (m - 1) / 2;
+    for (int p = warp; p < np; p += kSmallThreads / 32) {
+        double v = 0.0;
+        for (int b = lane; b < nblocks; b += 32) v += partial[(int64_t)b * np + p];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) v += __shfl_down_sync(0xffffffffu, v, o);
+        if (lane == 0) {
+            int i = 0, rem = p;
+            while (rem >= m - 1 - i) { rem -= m - 1 - i; ++i; }
+            const int j = i + 1 + rem;
+            dmat[i][j] = v;
+            dmat[j][i] = v;
+        }
+    }
+    if (tid < m) dmat[tid][tid] = CUDART_INF;   // a row never counts itself: it goes to the end of its own list
+    __syncthreads();
+
+    if (tid < m * m) {
+        const int i = tid / m, j = tid - i * m;
+        int rank;
+        if (j == i) {
+            rank = m - 1;
+        } else {
+            const double v = dmat[i][j];
+            rank = 0;
+            for (int k = 0; k < m; ++k) {
+                if (k == i) continue;
+                const double u = dmat[i][k];
+                rank += (u < v || (u == v && k < j)) ? 1 : 0;
+            }
+        }
+        s_sorted_d[i * m + rank] = dmat[i][j];
+        s_sorted_j[i * m + rank] = j;
+        s_pos_t[j * m + i] = rank;
+    }
+    __syncthreads();
+
+    int count;
+    if (BULYAN) {
+        bulyan_select_body(s_sorted_d, s_sorted_j, s_pos_t, m, f, sel);
+        count = m - 2 * f;
+    } else {
+        multikrum_select_body(s_sorted_d, m, f, m_sel, sel, scores_out);
+        count = m_sel;
+    }
+    if (rows && mapped) {
+        __syncthreads();
+        if (tid < count) mapped[tid] = rows[sel[tid]];
+    }
+}
+
 __global__ void map_indices_kernel(const int32_t* __restrict__ idx, const int32_t* __restrict__ map, int cnt,
                                    int32_t* __restrict__ out) {
     int k = blockIdx.x * blockDim.x + threadIdx.x;
@@ -251,6 +332,19 @@ detox_status launch_bulyan_select(const double* D, int m, int f, int32_t* sel_de
     detox_status st = launch_status();
     if (st != DETOX_OK) return st;
     bulyan_select_kernel<<<1, round_up_warp(m), 0, s>>>(w.sorted_d, w.sorted_j, w.pos_t, m, f, sel_dev);
+    return launch_status();
+}
+
+detox_status launch_krum_small(bool bulyan, const double* partial, int nblocks, int m, int f, int m_sel,
+                               const int32_t* rows_dev, int32_t* sel_dev, int32_t* mapped_dev, double* scores_dev,
+                               int* status_dev, cudaStream_t s) {
+    if (m < 2 || m > kSmallRows) return DETOX_ERR_UNSUPPORTED;
+    if (bulyan)
+        krum_small_kernel<true><<<1, kSmallThreads, 0, s>>>(partial, nblocks, m, f, m_sel, rows_dev, sel_dev, mapped_dev,
+                                                           scores_dev, status_dev);
+    else
+        krum_small_kernel<false><<<1, kSmallThreads, 0, s>>>(partial, nblocks, m, f, m_sel, rows_dev, sel_dev, mapped_dev,
+                                                            scores_dev, status_dev);
     return launch_status();
 }
 
