@@ -422,7 +422,7 @@ def main():
         if ref["sel"] is not None:
             parity["sel_exact"] = sel.cpu().numpy()[: len(ref["sel"])].tolist() == ref["sel"].tolist()
 
-    kernels_per_step = {"cfg1": 3, "cfg2": 8, "cfg3": 9, "cfg4": 4}[args.workload]
+    kernels_per_step = {"cfg1": 3, "cfg2": 6, "cfg3": 6, "cfg4": 4}[args.workload]
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",

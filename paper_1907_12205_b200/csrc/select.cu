@@ -75,7 +75,15 @@ __device__ __forceinline__ int krum_neighbours(int alive, int f) {
     return nb;
 }
 
-// One CTA, one thread per row (m <= blockDim.x); the lists may live in global or in shared memory.
+// One thread per row; the lists may live in global or in shared memory.  ONE_WARP: m <= 32 and only the first
+// warp of the CTA is inside (it synchronises by itself); otherwise the whole CTA is (m <= blockDim.x).
+template <bool ONE_WARP>
+__device__ __forceinline__ void group_sync() {
+    if (ONE_WARP) __syncwarp();
+    else __syncthreads();
+}
+
+template <bool ONE_WARP>
 __device__ __forceinline__ void multikrum_select_body(const double* sorted_d, int m, int f, int m_sel, int32_t* sel,
                                                       double* scores_out) {
     __shared__ double score[kMaxRows];
@@ -88,14 +96,14 @@ __device__ __forceinline__ void multikrum_select_body(const double* sorted_d, in
         score[i] = s;
         if (scores_out) scores_out[i] = s;
     }
-    __syncthreads();
+    group_sync<ONE_WARP>();
     if (i < m) {
         int rank = 0;
         const double s = score[i];
         for (int k = 0; k < m; ++k) rank += (score[k] < s || (score[k] == s && k < i)) ? 1 : 0;
         chosen[i] = rank < m_sel ? 1 : 0;
     }
-    __syncthreads();
+    group_sync<ONE_WARP>();
     if (i < m && chosen[i] && sel) {
         int pos = 0;
         for (int k = 0; k < i; ++k) pos += chosen[k];
@@ -103,6 +111,7 @@ __device__ __forceinline__ void multikrum_select_body(const double* sorted_d, in
     }
 }
 
+template <bool ONE_WARP>
 __device__ __forceinline__ void bulyan_select_body(const double* sorted_d, const int32_t* sorted_j, const int32_t* pos_t,
                                                    int m, int f, int32_t* sel) {
     __shared__ unsigned char alive[kMaxRows];
@@ -111,6 +120,7 @@ __device__ __forceinline__ void bulyan_select_body(const double* sorted_d, const
     __shared__ int picked;
     const int i = threadIdx.x;
     const int lane = i & 31, warp = i >> 5;
+    const int nwarps = ONE_WARP ? 1 : (int)(blockDim.x >> 5);
     const bool mine = i < m;
     if (i < kMaxRows) alive[i] = mine ? 1 : 0;
     const double* dist = sorted_d + (int64_t)i * m;   // row i's other rows, closest first (self last)
@@ -123,7 +133,7 @@ __device__ __forceinline__ void bulyan_select_body(const double* sorted_d, const
     double sum = 0.0;
     if (mine)
         for (int k = 0; k < nb; ++k) sum += dist[k];
-    __syncthreads();
+    group_sync<ONE_WARP>();
 
     const int theta = m - 2 * f;
     for (int round = 0; round < theta; ++round) {
@@ -137,10 +147,10 @@ __device__ __forceinline__ void bulyan_select_body(const double* sorted_d, const
             if (s2 < s || (s2 == s && i2 < idx)) { s = s2; idx = i2; }
         }
         if (lane == 0) { best_s[warp] = s; best_i[warp] = idx; }
-        __syncthreads();
+        group_sync<ONE_WARP>();
         if (warp == 0) {
-            s = lane < (int)(blockDim.x >> 5) ? best_s[lane] : CUDART_INF;
-            idx = lane < (int)(blockDim.x >> 5) ? best_i[lane] : 0x7fffffff;
+            s = lane < nwarps ? best_s[lane] : CUDART_INF;
+            idx = lane < nwarps ? best_i[lane] : 0x7fffffff;
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) {
                 const double s2 = __shfl_down_sync(0xffffffffu, s, o);
@@ -153,7 +163,7 @@ __device__ __forceinline__ void bulyan_select_body(const double* sorted_d, const
                 alive[idx] = 0;
             }
         }
-        __syncthreads();
+        group_sync<ONE_WARP>();
         const int gone = picked;
         const int remaining = m - round - 1;
         const int nb_next = remaining >= 1 ? krum_neighbours(remaining, f) : 0;
@@ -194,7 +204,7 @@ __device__ __forceinline__ void bulyan_select_body(const double* sorted_d, const
             }
         }
         nb = nb_next;
-        __syncthreads();
+        group_sync<ONE_WARP>();
     }
     (void)nb;
 }
@@ -202,13 +212,13 @@ __device__ __forceinline__ void bulyan_select_body(const double* sorted_d, const
 __global__ void __launch_bounds__(1024)
 multikrum_select_kernel(const double* __restrict__ sorted_d, int m, int f, int m_sel, int32_t* __restrict__ sel,
                         double* __restrict__ scores_out) {
-    multikrum_select_body(sorted_d, m, f, m_sel, sel, scores_out);
+    multikrum_select_body<false>(sorted_d, m, f, m_sel, sel, scores_out);
 }
 
 __global__ void __launch_bounds__(1024)
 bulyan_select_kernel(const double* __restrict__ sorted_d, const int32_t* __restrict__ sorted_j,
                      const int32_t* __restrict__ pos_t, int m, int f, int32_t* __restrict__ sel) {
-    bulyan_select_body(sorted_d, sorted_j, pos_t, m, f, sel);
+    bulyan_select_body<false>(sorted_d, sorted_j, pos_t, m, f, sel);
 }
 
 // m <= 16: everything between the distance pass and the final mean / order statistics in one CTA:
@@ -217,7 +227,8 @@ bulyan_select_kernel(const double* __restrict__ sorted_d, const int32_t* __restr
 // selection runs on the lists in shared memory, and the chosen indices are mapped through the row
 // list when there is one.  The device status word is cleared on the way.
 constexpr int kSmallRows = 16;
-constexpr int kSmallThreads = 512;
+constexpr int kSmallThreads = 1024;
+constexpr int kSmallPartialsPerLane = 19;   // covers the direct distance kernel's 4 CTAs per SM
 
 template <bool BULYAN>
 __global__ void __launch_bounds__(kSmallThreads)
@@ -233,8 +244,18 @@ krum_small_kernel(const double* __restrict__ partial, int nblocks, int m, int f,
 
     const int np = m * (m - 1) / 2;
     for (int p = warp; p < np; p += kSmallThreads / 32) {
+        // all of a lane's partials are requested before the first is added (the order of the additions stays)
+        double part[kSmallPartialsPerLane];
+#pragma unroll
+        for (int k = 0; k < kSmallPartialsPerLane; ++k) {
+            const int b = lane + 32 * k;
+            part[k] = b < nblocks ? partial[(int64_t)b * np + p] : 0.0;
+        }
         double v = 0.0;
-        for (int b = lane; b < nblocks; b += 32) v += partial[(int64_t)b * np + p];
+#pragma unroll
+        for (int k = 0; k < kSmallPartialsPerLane; ++k)
+            if (lane + 32 * k < nblocks) v += part[k];
+        for (int b = lane + 32 * kSmallPartialsPerLane; b < nblocks; b += 32) v += partial[(int64_t)b * np + p];
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) v += __shfl_down_sync(0xffffffffu, v, o);
         if (lane == 0) {
@@ -268,13 +289,11 @@ krum_small_kernel(const double* __restrict__ partial, int nblocks, int m, int f,
     }
     __syncthreads();
 
-    int count;
-    if (BULYAN) {
-        bulyan_select_body(s_sorted_d, s_sorted_j, s_pos_t, m, f, sel);
-        count = m - 2 * f;
-    } else {
-        multikrum_select_body(s_sorted_d, m, f, m_sel, sel, scores_out);
-        count = m_sel;
+    // m <= 16 rows: the selection runs in the first warp alone
+    const int count = BULYAN ? m - 2 * f : m_sel;
+    if (warp == 0) {
+        if (BULYAN) bulyan_select_body<true>(s_sorted_d, s_sorted_j, s_pos_t, m, f, sel);
+        else multikrum_select_body<true>(s_sorted_d, m, f, m_sel, sel, scores_out);
     }
     if (rows && mapped) {
         __syncthreads();
