@@ -54,6 +54,10 @@ ORACLE_A1 = {1: "mean", 2: "coord_median", 3: "multikrum", 4: "bulyan"}
 # profiles/vote_kernels_cfg2.md (same kernel code; reset an entry to None when its kernel changes).
 NCU_TRAFFIC_BYTES = {
     ("cfg2", "vote_mean_kernel"): 2_011_333_000 + 117_863_424,
+    ("cfg3", "vote_kernel (winners only)"): 2_011_344_896 + 3_232_768,
+    # config 4 holds 11.8 GB, too much for a multi-pass capture: config 2's traffic of the same streaming kernel,
+    # scaled by the algorithmic bytes (12,544,000,000 / 2,145,400,704)
+    ("cfg4", "vote_mean_kernel"): int((2_011_333_000 + 117_863_424) * 12_544_000_000 / 2_145_400_704),
 }
 
 
