@@ -6,13 +6,14 @@
 // accumulator in tensor memory, G_ij = (T_ij + T_ji) / 2.  Both MMA operands come from the same
 // shared-memory tiles (rows of X), so every row of X is read from HBM exactly once.
 //
-// One persistent CTA per SM.  One thread streams K-blocks of 32 columns (all m rows) into shared
-// memory with TMA (128-byte swizzle, which is the K-major layout the MMA expects; rows and columns
-// outside the matrix arrive as zeros).  The raw fp32 tile itself serves as the `hi` operand: a TF32
-// MMA reads only the upper 19 bits of each word.  Warps 0-15 read the tile back, form
-// 2 lo = 2 (x - (x with its low 13 bits cleared)) and write the second tile; lane 0 of warps 16, 17
-// issue the MMAs; mbarriers form a ring of stages between the three roles.
-// K-blocks are dealt round-robin to the CTAs and every 128 of a CTA's K-blocks form a slab; at the end
+// One persistent CTA per SM: copy-issuing threads stream column blocks of all m rows into shared memory with
+// TMA (rows and columns outside the matrix arrive as zeros), warps 0-15 form 2 lo = 2 (x - (x with its low 13
+// bits cleared)) -- the raw fp32 values themselves serve as `hi`, because a TF32 MMA reads only the upper 19
+// bits of each word -- and lane 0 of warps 16, 17 issues the MMAs; mbarriers form rings of stages between the
+// roles.  Two kernels share this scheme: up to 128 rows the copies are 64 columns wide, land in a staging ring
+// and the transform warps write both MMA operands (see the staged kernel); above, the copies land directly in
+// the swizzled hi tile (see the wide kernel).
+// Column blocks are dealt round-robin to the CTAs and every 4096 columns of a CTA form a slab; at the end
 // of a slab the accumulator is drained to a per-slab fp32 partial in global memory and the slabs are
 // added in fp64 in a fixed order afterwards, so the long sum never lives in one fp32 accumulator and
 // the result is deterministic.
@@ -38,53 +39,12 @@ constexpr int kKB = 32;                      // fp32 columns per K-block: one 12
 constexpr int kProdWarps = 16;
 constexpr int kProdThreads = kProdWarps * 32;
 constexpr int kMmaWarps = 2;                   // two issuing threads, so one's bookkeeping overlaps the other's MMAs
-constexpr int kTcThreads = kProdThreads + 32 * (kMmaWarps + 1);  // + the MMA warps + the TMA warp
-constexpr int kMaxStages = 12;
+constexpr int kTmaWarps = 2;                   // copy-issuing threads (the kernel for m > 128 uses the first only)
+constexpr int kTcThreads = kProdThreads + 32 * (kMmaWarps + kTmaWarps);
+constexpr size_t kSmemBudget = 227 * 1024;     // dynamic shared memory one CTA may have
 constexpr long long kWaitLimitCycles = 2000000000LL;  // ~1 s at the SM clock
-constexpr int64_t kSlabCols = 4096;          // columns (128 K-blocks) accumulated in tensor memory before a drain
+constexpr int64_t kSlabCols = 4096;          // columns accumulated in tensor memory before a drain
 constexpr int kMinReduceChunks = 32, kMaxReduceChunks = 256;
-
-struct TcPlan {
-    int rows_pad;    // rows of each shared-memory tile (64, 128 or 256); a stage holds two tiles
-    int mrows;       // M of the MMA: 64 for m <= 64, else 128
-    int box_rows;    // rows the TMA box brings in: m rounded up to 8
-    int nhalf;       // accumulator halves of 128 rows
-    int ncol;        // N of the MMA: m rounded up to 16
-    int chains;      // m <= 128: accumulators, one per MMA-issuing thread
-    int tmem_cols;   // power of two >= the accumulator columns, >= 32
-    int stages;
-    int nkb_total;   // K-blocks in all: d / 32 rounded up
-    int nitems;      // slab slots: grid x the largest number of slabs a CTA has
-    int grid;
-    size_t smem_bytes;
-};
-
-TcPlan tc_plan(int m, int64_t d) {
-    TcPlan p;
-    p.nhalf = m > 128 ? 2 : 1;
-    p.mrows = m <= 64 ? 64 : 128;
-    p.rows_pad = m <= 64 ? 64 : 128 * p.nhalf;
-    p.box_rows = (m + 7) / 8 * 8;
-    p.ncol = (m + 15) / 16 * 16;
-    // m <= 128: one MMA per K-step with B = [hi ; 2lo] stacked (N = 2 ncol); the two issuing threads take
-    //           alternate K-blocks and own one accumulator each;
-    // m  > 128: two 128-row halves, one per issuing thread, B = hi and B = 2lo as separate MMAs
-    p.chains = p.nhalf == 1 ? kMmaWarps : 1;
-    int need = p.nhalf == 1 ? p.chains * 2 * p.ncol : 2 * p.ncol;
-    p.tmem_cols = 32;
-    while (p.tmem_cols < need) p.tmem_cols <<= 1;
-    size_t stage = (size_t)2 * p.rows_pad * 128;
-    p.stages = (int)((192 * 1024) / stage);
-    if (p.stages > kMaxStages) p.stages = kMaxStages;
-    // K-blocks are dealt round-robin to the CTAs, so that every CTA has the same number of them (to within one)
-    // whatever d is, and neighbouring CTAs read neighbouring 128-byte pieces of a row
-    p.nkb_total = (int)ceil_div(d, (int64_t)kKB);
-    p.grid = p.nkb_total < kSMs ? p.nkb_total : kSMs;
-    const int per_cta = (p.nkb_total + p.grid - 1) / p.grid;
-    p.nitems = p.grid * (int)ceil_div((int64_t)per_cta, kSlabCols / kKB);
-    p.smem_bytes = stage * p.stages + 1024 /*barriers*/ + 1024 /*alignment slack*/;
-    return p;
-}
 
 // Slab slots are added up in `chunks` independent groups (one CTA per group and pair of 32-row blocks), enough
 // of them to fill the GPU when m is small.
@@ -185,15 +145,12 @@ __device__ __forceinline__ void mma_commit(uint64_t* bar) {
                  : "memory");
 }
 
-__device__ __forceinline__ void tmem_load32(uint32_t taddr, uint32_t (&v)[32]) {
+__device__ __forceinline__ void tmem_load16(uint32_t taddr, uint32_t (&v)[16]) {
     asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
         : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
-          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
-          "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
-          "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
         : "r"(taddr)
         : "memory");
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
@@ -233,29 +190,67 @@ __device__ __forceinline__ uint64_t lo2_of(uint64_t x2) {
     return add2(t, t);
 }
 
-struct TcSmem {
-    uint64_t landed[kMaxStages];   // TMA bytes of the raw tile have arrived
-    uint64_t full[kMaxStages];     // the 2lo tile is written: both tiles ready for the MMA
-    uint64_t empty[kMaxStages];
+// ------------------------------------------------------------------------------------ 128 < m <= 256: wide kernel
+//
+// The accumulator has two halves of 128 rows, one per MMA-issuing thread; per K-step each thread issues
+// A = hi rows of its half with B = hi and with B = 2lo.  Sixteen MMAs of N = ncol per K-block keep the tensor pipe
+// busier than the copies, so the copies stay 32 columns wide and land directly in the swizzled hi tile.
+constexpr int kMaxWideStages = 4;
+
+struct WidePlan {
+    int box_rows;     // rows the TMA box brings in: m rounded up to 8
+    int ncol;         // m rounded up to 16
+    int tmem_cols;    // power of two >= 2 ncol
+    int stages;
+    uint32_t lo_off;       // where the 2lo tile starts inside a stage: after 256 hi rows (the second half's A operand
+                           // reads rows 128..255)
+    uint32_t stage_bytes;
+    int nkb_total;    // K-blocks in all: d / 32 rounded up
+    int nitems;       // slab slots: grid x the largest number of slabs a CTA has
+    int grid;
+    size_t smem_bytes;
+};
+
+WidePlan wide_plan(int m, int64_t d) {
+    WidePlan p;
+    p.box_rows = (m + 7) / 8 * 8;
+    p.ncol = (m + 15) / 16 * 16;
+    p.tmem_cols = 512;
+    p.lo_off = 256u * 128u;
+    p.stage_bytes = p.lo_off + (uint32_t)p.ncol * 128u;
+    p.stages = (int)((kSmemBudget - 2048) / p.stage_bytes);
+    if (p.stages > kMaxWideStages) p.stages = kMaxWideStages;
+    // K-blocks are dealt round-robin to the CTAs, so that every CTA has the same number of them (to within one)
+    // whatever d is, and neighbouring CTAs read neighbouring 128-byte pieces of a row
+    p.nkb_total = (int)ceil_div(d, (int64_t)kKB);
+    p.grid = p.nkb_total < kSMs ? p.nkb_total : kSMs;
+    const int per_cta = (p.nkb_total + p.grid - 1) / p.grid;
+    p.nitems = p.grid * (int)ceil_div((int64_t)per_cta, kSlabCols / kKB);
+    p.smem_bytes = (size_t)p.stage_bytes * p.stages + 1024 /*barriers*/ + 1024 /*alignment slack*/;
+    return p;
+}
+
+struct WideSmem {
+    uint64_t landed[kMaxWideStages];   // TMA bytes of the raw tile have arrived
+    uint64_t full[kMaxWideStages];     // the 2lo tile is written: both tiles ready for the MMA
+    uint64_t empty[kMaxWideStages];
     uint64_t accum_full;
     uint64_t accum_empty;
     uint32_t tmem_base;
     int abort_flag;
 };
 
-// J = 16-byte chunks per transform thread and K-block (m * 8 / 512 rounded up to a power of two)
+// J = 16-byte pieces per transform thread and K-block (m * 8 / 512, rounded up)
 template <int J>
 __global__ void __launch_bounds__(kTcThreads, 1)
-gram_tc_kernel(const __grid_constant__ CUtensorMap xmap, int m, int64_t d, int rows_pad, int mrows, int box_rows, int nhalf,
-               int ncol, int chains, int tmem_cols, int stages, int nkb_total, int nitems, float* __restrict__ partial,
-               float* __restrict__ norms, int* __restrict__ status) {
+gram_wide_kernel(const __grid_constant__ CUtensorMap xmap, int m, uint32_t lo_off, uint32_t stage_bytes, int box_rows,
+                 int ncol, int tmem_cols, int stages, int nkb_total, int nitems, float* __restrict__ partial,
+                 float* __restrict__ norms, int* __restrict__ status) {
     extern __shared__ uint8_t smem_raw[];
     // tiles need 1024-byte alignment for the 128-byte swizzle pattern
     const uint32_t raw = smem_u32(smem_raw);
     uint8_t* base = smem_raw + ((1024u - (raw & 1023u)) & 1023u);
-    const uint32_t tile_bytes = (uint32_t)rows_pad * 128u;
-    const uint32_t stage_bytes = 2u * tile_bytes;
-    TcSmem* sm = reinterpret_cast<TcSmem*>(base + (size_t)stage_bytes * stages);
+    WideSmem* sm = reinterpret_cast<WideSmem*>(base + (size_t)stage_bytes * stages);
     volatile int* abort_flag = &sm->abort_flag;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -264,7 +259,7 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap xmap, int m, int64_t d, int r
         for (int s = 0; s < stages; ++s) {
             mbar_init(&sm->landed[s], 1);
             mbar_init(&sm->full[s], kProdWarps);
-            mbar_init(&sm->empty[s], nhalf == 1 ? 1 : kMmaWarps);
+            mbar_init(&sm->empty[s], kMmaWarps);
         }
         mbar_init(&sm->accum_full, kMmaWarps);
         mbar_init(&sm->accum_empty, kProdWarps);
@@ -282,8 +277,8 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap xmap, int m, int64_t d, int r
     const uint32_t tmem_base = sm->tmem_base;
 
     // This CTA owns the K-blocks b, b + G, b + 2G, ... (b = blockIdx.x, G = gridDim.x), t = 0 .. total-1 in its own
-    // count; a slab is kBlocksPerSlab consecutive ones of them (the last slab may be shorter) and goes to slot
-    // b + G * (slab number).
+    // count; K-block t goes through stage t % stages; a slab is kBlocksPerSlab consecutive ones of them (the last
+    // slab may be shorter) and goes to slot b + G * (slab number).
     constexpr int kBlocksPerSlab = (int)(kSlabCols / kKB);
     const int total = (nkb_total - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
     const int my_items = (total + kBlocksPerSlab - 1) / kBlocksPerSlab;
@@ -291,43 +286,38 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap xmap, int m, int64_t d, int r
 
     if (warp < kProdWarps) {
         // ------------------------------------------------ transform warps, then epilogue of each slab
-        const int nchunks = m * 8;
-        // this thread's chunks are (row, c) = ((tid >> 3) + 64 j, tid & 7) in every K-block
-        uint32_t off[J];
-#pragma unroll
-        for (int j = 0; j < J; ++j) {
-            const int row = (tid >> 3) + (kProdThreads / 8) * j, c = tid & 7;
-            off[j] = (uint32_t)(row >> 3) * 1024u + (uint32_t)(row & 7) * 128u + (uint32_t)((c ^ (row & 7)) << 4);
-        }
-        uint64_t sq[J];   // packed pair of partial sums of squares per chunk
+        const int npieces = m * 8;
+        // this thread's pieces are (row, c) = ((tid >> 3) + 64 j, tid & 7) in every K-block; 64 is a multiple of 8,
+        // so the swizzle term is the same for all j
+        const int row0 = tid >> 3, c = tid & 7;
+        const uint32_t off0 = (uint32_t)(row0 >> 3) * 1024u + (uint32_t)(row0 & 7) * 128u + (uint32_t)((c ^ (row0 & 7)) << 4);
+        constexpr uint32_t kOffStep = (uint32_t)(kProdThreads / 64) * 1024u;
+        uint64_t sq[J];   // packed pair of partial sums of squares per piece
 #pragma unroll
         for (int j = 0; j < J; ++j) sq[j] = 0ull;
 
-        // m <= 128: the 2lo rows follow the hi rows at row `ncol` of the same tile (ncol % 8 == 0);
-        // m  > 128: they form a tile of their own
-        const uint32_t lo_off = nhalf == 1 ? (uint32_t)ncol * 128u : tile_bytes;
-        // stage / phase / slab position are carried along instead of divided out every K-block
-        int s = 0, li = 0, kb = 0;
+        int s = 0, t = 0;
         uint32_t ph = 0;
-        for (int t = 0; t < total; ++t) {
-            mbar_wait(&sm->landed[s], ph, abort_flag, status);
-            const uint8_t* hi_tile = base + (size_t)s * stage_bytes;
-            uint8_t* lo_tile = base + (size_t)s * stage_bytes + lo_off;
-#pragma unroll
-            for (int j = 0; j < J; ++j) {
-                if (tid + j * kProdThreads < nchunks) {
-                    const ulonglong2 x = *reinterpret_cast<const ulonglong2*>(hi_tile + off[j]);
-                    sq[j] = fma2(x.x, x.x, fma2(x.y, x.y, sq[j]));
-                    *reinterpret_cast<ulonglong2*>(lo_tile + off[j]) = make_ulonglong2(lo2_of(x.x), lo2_of(x.y));
-                }
-            }
-            fence_proxy_async_smem();   // make the generic-proxy stores visible to the MMA's reads
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&sm->full[s]);   // one arrival per transform warp
-            if (++s == stages) { s = 0; ph ^= 1u; }
-
+        for (int li = 0; li < my_items; ++li) {
             const int nkb = li == my_items - 1 ? last_nkb : kBlocksPerSlab;
-            if (++kb != nkb) continue;
+            const int t_end = li * kBlocksPerSlab + nkb;
+            for (; t < t_end; ++t) {
+                mbar_wait(&sm->landed[s], ph, abort_flag, status);
+                const uint8_t* hi_tile = base + (size_t)s * stage_bytes + off0;
+                uint8_t* lo_tile = base + (size_t)s * stage_bytes + lo_off + off0;
+#pragma unroll
+                for (int j = 0; j < J; ++j) {
+                    if (tid + j * kProdThreads < npieces) {
+                        const ulonglong2 x = *reinterpret_cast<const ulonglong2*>(hi_tile + j * kOffStep);
+                        sq[j] = fma2(x.x, x.x, fma2(x.y, x.y, sq[j]));
+                        *reinterpret_cast<ulonglong2*>(lo_tile + j * kOffStep) = make_ulonglong2(lo2_of(x.x), lo2_of(x.y));
+                    }
+                }
+                fence_proxy_async_smem();   // make the generic-proxy stores visible to the MMA's reads
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sm->full[s]);   // one arrival per transform warp
+                if (++s == stages) { s = 0; ph ^= 1u; }
+            }
             const int item = (int)blockIdx.x + li * (int)gridDim.x;
 
             // ---- end of a slab: exact squared norms (the 8 lanes that share a row add up) ...
@@ -337,49 +327,34 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap xmap, int m, int64_t d, int r
                 v += __shfl_xor_sync(0xffffffffu, v, 1);
                 v += __shfl_xor_sync(0xffffffffu, v, 2);
                 v += __shfl_xor_sync(0xffffffffu, v, 4);
-                const int row = (tid >> 3) + (kProdThreads / 8) * j;
-                if ((tid & 7) == 0 && row < m) norms[(int64_t)item * m + row] = v;
+                const int row = row0 + (kProdThreads / 8) * j;
+                if (c == 0 && row < m) norms[(int64_t)item * m + row] = v;
                 sq[j] = 0ull;
             }
-            // ... and the accumulator drain: warp w reads TMEM lanes 32*(w%4)..+31; the warps that share a
-            // lane quarter take 32-column chunks round-robin
+            // ... and the accumulator drain: warp w reads TMEM lanes 32*(w%4)..+31 (accumulator row i of a half sits
+            // in lane i); the warps that share a lane quarter take 16-column chunks round-robin
             mbar_wait(&sm->accum_full, (uint32_t)(li & 1), abort_flag, status);
             tc_fence_after();
             const int quarter = warp & 3;
             float* out_item = partial + (int64_t)item * m * ncol;
-            for (int h = 0; h < nhalf; ++h) {
-                // M = 128: accumulator row i sits in TMEM lane i; M = 64: in lane 32 (i / 16) + i % 16
-                const int row = mrows == 64 ? (lane < 16 ? quarter * 16 + lane : m) : h * 128 + quarter * 32 + lane;
-                for (int cc = warp >> 2; cc * 32 < ncol; cc += kProdWarps / 4) {
-                    float acc[32];
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) acc[j] = 0.f;
-                    // m <= 128: add the hi.hi and hi.2lo parts of every chain; m > 128: one accumulator per half
-                    // (a slab of a single K-block leaves the second issuing thread's accumulator untouched: skip it)
-                    const int nparts = nhalf == 1 ? 2 * (nkb < chains ? nkb : chains) : 1;
-                    for (int part = 0; part < nparts; ++part) {
-                        uint32_t v[32];
-                        const int col = (nhalf == 1 ? part * ncol : h * ncol) + cc * 32;
-                        tmem_load32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)col, v);
-#pragma unroll
-                        for (int j = 0; j < 32; ++j) acc[j] += __uint_as_float(v[j]);
-                    }
+            for (int h = 0; h < 2; ++h) {
+                const int row = h * 128 + quarter * 32 + lane;
+                for (int cc = warp >> 2; cc * 16 < ncol; cc += kProdWarps / 4) {   // ncol is a multiple of 16
+                    uint32_t v[16];
+                    tmem_load16(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(h * ncol + cc * 16), v);
                     if (row < m) {
-                        float* dst = out_item + (int64_t)row * ncol + cc * 32;
-                        const int nvalid = ncol - cc * 32 < 32 ? ncol - cc * 32 : 32;
+                        float* dstp = out_item + (int64_t)row * ncol + cc * 16;
 #pragma unroll
-                        for (int j = 0; j < 32; j += 4) {
-                            if (j < nvalid)
-                                *reinterpret_cast<float4*>(dst + j) = make_float4(acc[j], acc[j + 1], acc[j + 2], acc[j + 3]);
-                        }
+                        for (int j = 0; j < 16; j += 4)
+                            *reinterpret_cast<float4*>(dstp + j) =
+                                make_float4(__uint_as_float(v[j]), __uint_as_float(v[j + 1]), __uint_as_float(v[j + 2]),
+                                            __uint_as_float(v[j + 3]));
                     }
                 }
             }
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&sm->accum_empty);
-            kb = 0;
-            ++li;
         }
         // slots of slabs this CTA does not have (it owns one K-block fewer than others) read as zero
         for (int l2 = my_items; l2 * (int)gridDim.x < nitems; ++l2) {
@@ -396,8 +371,8 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap xmap, int m, int64_t d, int r
             uint32_t ph = 0;
             int64_t c0 = (int64_t)blockIdx.x * kKB;                  // first column of the current K-block
             for (int t = 0; t < total; ++t) {
-                mbar_wait(&sm->empty[s], ph ^ 1u, abort_flag, status);   // MMAs that read this stage are done
-                if (*abort_flag) break;
+                // the MMAs that read this stage are done
+                if (!mbar_wait(&sm->empty[s], ph ^ 1u, abort_flag, status)) break;
                 mbar_expect_tx(&sm->landed[s], tx_bytes);
                 tma_load_2d(base + (size_t)s * stage_bytes, &xmap, (int)c0, 0, &sm->landed[s]);
                 issued = t + 1;
@@ -406,57 +381,327 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap xmap, int m, int64_t d, int r
             }
             if (*abort_flag) {
                 // give the copies still in flight a bounded time to land before the CTA goes away
-                for (int t = issued > stages ? issued - stages : 0; t < issued; ++t) {
-                    const int s = (int)((uint32_t)t % (uint32_t)stages);
-                    const uint32_t ph = ((uint32_t)t / (uint32_t)stages) & 1u;
-                    for (uint32_t spin = 0; spin < (1u << 16) && !mbar_test(&sm->landed[s], ph); ++spin) __nanosleep(64);
+                for (int tt = issued > stages ? issued - stages : 0; tt < issued; ++tt) {
+                    const int s2 = (int)((uint32_t)tt % (uint32_t)stages);
+                    const uint32_t ph2 = ((uint32_t)tt / (uint32_t)stages) & 1u;
+                    for (uint32_t spin = 0; spin < (1u << 16) && !mbar_test(&sm->landed[s2], ph2); ++spin) __nanosleep(64);
+                }
+            }
+        }
+    } else if (warp < kProdWarps + kMmaWarps && lane == 0) {
+        // ------------------------------------------------ the MMA threads (lane 0 of the two warps after the
+        // transform warps): thread g owns the accumulator half of rows 128 g .. 128 g + 127
+        const int g = warp - kProdWarps;
+        const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(ncol >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+        const uint32_t dcol = tmem_base + (uint32_t)(g * ncol);
+        int s = 0;
+        uint32_t ph = 0;
+        for (int li = 0; li < my_items; ++li) {
+            const int nkb = li == my_items - 1 ? last_nkb : kBlocksPerSlab;
+            if (li > 0) mbar_wait(&sm->accum_empty, (uint32_t)((li - 1) & 1), abort_flag, status);
+            tc_fence_after();
+            bool first = true;   // this thread's first MMA of the slab overwrites its accumulator
+            for (int kb = 0; kb < nkb; ++kb) {
+                mbar_wait(&sm->full[s], ph, abort_flag, status);
+                tc_fence_after();
+                const uint32_t hi_addr = smem_u32(base + (size_t)s * stage_bytes);
+                const uint64_t hi_desc = smem_desc(hi_addr);
+                const uint64_t lo_desc = smem_desc(hi_addr + lo_off);
+#pragma unroll
+                for (int kk = 0; kk < kKB / 8; ++kk) {       // one MMA covers 8 columns = 32 bytes
+                    const uint64_t a = hi_desc + (uint64_t)(kk * 2 + g * (128 * 128 / 16));
+                    mma_tf32(dcol, a, hi_desc + (uint64_t)(kk * 2), idesc, first ? 0u : 1u);
+                    mma_tf32(dcol, a, lo_desc + (uint64_t)(kk * 2), idesc, 1u);
+                    first = false;
+                }
+                mma_commit(&sm->empty[s]);   // the stage may be refilled once both threads' MMAs have read it
+                if (++s == stages) { s = 0; ph ^= 1u; }
+            }
+            mma_commit(&sm->accum_full);
+        }
+    }
+
+    __syncwarp();
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    if (warp == 0) tmem_dealloc(tmem_base, (uint32_t)tmem_cols);
+}
+
+// ------------------------------------------------------------------------------------ m <= 128: staged kernel
+//
+// A TMA box with the 128-byte swizzle is at most 32 fp32 columns wide, and the copy engine takes about 8 cycles
+// per row of a box whatever the row's width: boxes of 128-byte rows top out near 4.5 TB/s over all SMs, boxes of
+// 256-byte rows reach the HBM rate.  So for m <= 128 the copies are 64 columns wide and land, unswizzled, in a
+// staging ring; the transform warps read a staging stage (two K-blocks), and write both MMA operands of each
+// K-block, the raw values (= hi for the MMA) and 2 lo, into a ring of MMA stages in the swizzled K-major layout.
+constexpr int kStageCols = 64;                       // columns per staging stage: two K-blocks
+constexpr int kKbPerStage = kStageCols / kKB;
+constexpr int kMaxStg = 8, kMaxMst = 4;
+
+struct StagedPlan {
+    int mrows, box_rows, ncol, tmem_cols;
+    int groups;                  // groups of transform warps, each on a stage of its own
+    int nstg, nmst;              // staging stages, MMA stages
+    uint32_t stg_bytes;          // box_rows x 256 bytes
+    uint32_t tile_bytes;         // one K-block's [hi ; 2lo] tile: 2 ncol rows of 128 bytes
+    int nst_total;               // 64-column stages in all
+    int nitems, grid;
+    size_t smem_bytes;
+};
+
+StagedPlan staged_plan(int m, int64_t d) {
+    StagedPlan p;
+    p.mrows = m <= 64 ? 64 : 128;
+    p.box_rows = (m + 7) / 8 * 8;
+    p.ncol = (m + 15) / 16 * 16;
+    p.tmem_cols = 32;
+    while (p.tmem_cols < kMmaWarps * 2 * p.ncol) p.tmem_cols <<= 1;
+    p.stg_bytes = (uint32_t)p.box_rows * (uint32_t)kStageCols * 4u;
+    p.tile_bytes = 2u * (uint32_t)p.ncol * 128u;
+    const size_t mst_bytes = (size_t)kKbPerStage * p.tile_bytes;
+    // up to 64 rows there is room for four MMA stages: two groups of transform warps write two of them while the
+    // tensor cores read the others; above, two MMA stages and one group
+    p.nmst = m <= 64 ? 4 : 2;
+    p.groups = m <= 64 ? 2 : 1;
+    const size_t left = kSmemBudget - 2048 - p.nmst * mst_bytes;
+    p.nstg = (int)(left / p.stg_bytes);
+    if (p.nstg > kMaxStg) p.nstg = kMaxStg;
+    while (p.nstg > 2 && (size_t)p.nstg * p.stg_bytes > 112 * 1024) --p.nstg;   // ~100 KB in flight saturates HBM
+    p.nst_total = (int)ceil_div(d, (int64_t)kStageCols);
+    p.grid = p.nst_total < kSMs ? p.nst_total : kSMs;
+    const int per_cta = (p.nst_total + p.grid - 1) / p.grid;
+    p.nitems = p.grid * (int)ceil_div((int64_t)per_cta, kSlabCols / kStageCols);
+    p.smem_bytes = (size_t)p.nstg * p.stg_bytes + p.nmst * mst_bytes + 1024 /*barriers*/ + 1024 /*alignment slack*/;
+    return p;
+}
+
+struct StagedSmem {
+    uint64_t stg_full[kMaxStg];    // TMA bytes of a staging stage have arrived
+    uint64_t stg_empty[kMaxStg];   // the transform warps have read it
+    uint64_t mst_full[kMaxMst];    // both operands of both K-blocks are written
+    uint64_t mst_empty[kMaxMst];   // the MMAs that read them are done
+    uint64_t accum_full;
+    uint64_t accum_empty;
+    uint32_t tmem_base;
+    int abort_flag;
+};
+
+// LX = groups of transform warps; J = 16-byte pieces per transform thread and stage (m * 16 / (512 / LX), rounded up)
+template <int J, int LX>
+__global__ void __launch_bounds__(kTcThreads, 1)
+gram_staged_kernel(const __grid_constant__ CUtensorMap xmap, int m, uint32_t stg_bytes, uint32_t tile_bytes, int mrows,
+                   int ncol, int tmem_cols, int nstg, int nmst, int nst_total, int nitems, float* __restrict__ partial,
+                   float* __restrict__ norms, int* __restrict__ status) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    uint8_t* stg_base = smem_raw + ((1024u - (raw & 1023u)) & 1023u);       // MMA tiles need 1024-byte alignment
+    const uint32_t mst_bytes = (uint32_t)kKbPerStage * tile_bytes;
+    uint8_t* mst_base = stg_base + (size_t)nstg * stg_bytes;                // stg_bytes is a multiple of 2048
+    StagedSmem* sm = reinterpret_cast<StagedSmem*>(mst_base + (size_t)nmst * mst_bytes);
+    volatile int* abort_flag = &sm->abort_flag;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    constexpr int kGroupThreads = kProdThreads / LX, kGroupWarps = kProdWarps / LX;
+
+    if (tid == 0) {
+        for (int s = 0; s < nstg; ++s) {
+            mbar_init(&sm->stg_full[s], 1);
+            mbar_init(&sm->stg_empty[s], kGroupWarps);
+        }
+        for (int s = 0; s < nmst; ++s) {
+            mbar_init(&sm->mst_full[s], kGroupWarps);
+            mbar_init(&sm->mst_empty[s], 1);
+        }
+        mbar_init(&sm->accum_full, kMmaWarps);
+        mbar_init(&sm->accum_empty, kProdWarps);
+        sm->abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    // rows m .. 2 ncol of the MMA tiles are never written: clear the MMA stages once so that they read as zeros
+    for (uint32_t off = (uint32_t)tid * 16u; off < mst_bytes * (uint32_t)nmst; off += kTcThreads * 16u)
+        *reinterpret_cast<uint4*>(mst_base + off) = make_uint4(0u, 0u, 0u, 0u);
+    fence_proxy_async_smem();
+    if (warp == 0) tmem_alloc(&sm->tmem_base, (uint32_t)tmem_cols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = sm->tmem_base;
+
+    // This CTA owns the 64-column stages b, b + G, b + 2G, ... (b = blockIdx.x, G = gridDim.x), t = 0 .. total-1 in
+    // its own count; stage t lands in staging slot t % nstg and is transformed into MMA slot t % nmst; a slab is
+    // kStagesPerSlab consecutive ones (the last slab may be shorter) and goes to slot b + G * (slab number).
+    constexpr int kStagesPerSlab = (int)(kSlabCols / kStageCols);
+    static_assert(kStagesPerSlab % LX == 0 && kStagesPerSlab % kMmaWarps == 0, "slabs start at every role's own offset");
+    const int total = (nst_total - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
+    const int my_items = (total + kStagesPerSlab - 1) / kStagesPerSlab;
+    const int last_nst = total - (my_items - 1) * kStagesPerSlab;
+
+    if (warp < kProdWarps) {
+        // ------------------------------------------------ transform warps, then epilogue of each slab
+        const int group = warp / kGroupWarps, gtid = tid - group * kGroupThreads;
+        const int npieces = m * (kStageCols / 4);
+        // this thread's pieces are (row, q) = ((gtid >> 4) + (kGroupThreads / 16) j, gtid & 15): 16 bytes at column
+        // 4 q of the stage, i.e. piece q & 7 of K-block q >> 3.  kGroupThreads / 16 is a multiple of 8, so the
+        // swizzle term of the destination is the same for all j.
+        const int row0 = gtid >> 4, q = gtid & 15, cq = q & 7;
+        const uint32_t src0 = (uint32_t)row0 * (uint32_t)(kStageCols * 4) + (uint32_t)q * 16u;
+        constexpr uint32_t kSrcStep = (uint32_t)(kGroupThreads / 16) * (uint32_t)(kStageCols * 4);
+        const uint32_t dst0 = (uint32_t)(q >> 3) * tile_bytes + (uint32_t)(row0 >> 3) * 1024u + (uint32_t)(row0 & 7) * 128u +
+                              (uint32_t)((cq ^ (row0 & 7)) << 4);
+        constexpr uint32_t kDstStep = (uint32_t)(kGroupThreads / 128) * 1024u;
+        const uint32_t lo_off = (uint32_t)ncol * 128u;      // the 2lo rows follow the hi rows inside a tile
+        uint64_t sq[J];   // packed pair of partial sums of squares per piece
+#pragma unroll
+        for (int j = 0; j < J; ++j) sq[j] = 0ull;
+
+        // slots / phases are carried along instead of divided out every stage (LX <= nstg, nmst)
+        int ss = group, ms = group, t = group;
+        uint32_t sph = 0, mph = 0;
+        for (int li = 0; li < my_items; ++li) {
+            const int nst = li == my_items - 1 ? last_nst : kStagesPerSlab;
+            const int t_end = li * kStagesPerSlab + nst;
+            for (; t < t_end; t += LX) {
+                mbar_wait(&sm->stg_full[ss], sph, abort_flag, status);
+                const uint8_t* src = stg_base + (size_t)ss * stg_bytes + src0;
+                ulonglong2 x[J];
+#pragma unroll
+                for (int j = 0; j < J; ++j)
+                    if (gtid + j * kGroupThreads < npieces) x[j] = *reinterpret_cast<const ulonglong2*>(src + j * kSrcStep);
+                mbar_wait(&sm->mst_empty[ms], mph ^ 1u, abort_flag, status);   // the MMAs that read this slot are done
+                uint8_t* dst = mst_base + (size_t)ms * mst_bytes + dst0;
+#pragma unroll
+                for (int j = 0; j < J; ++j) {
+                    if (gtid + j * kGroupThreads < npieces) {
+                        sq[j] = fma2(x[j].x, x[j].x, fma2(x[j].y, x[j].y, sq[j]));
+                        *reinterpret_cast<ulonglong2*>(dst + j * kDstStep) = x[j];
+                        *reinterpret_cast<ulonglong2*>(dst + lo_off + j * kDstStep) = make_ulonglong2(lo2_of(x[j].x), lo2_of(x[j].y));
+                    }
+                }
+                fence_proxy_async_smem();   // make the generic-proxy stores visible to the MMA's reads
+                __syncwarp();
+                if (lane == 0) {
+                    mbar_arrive(&sm->stg_empty[ss]);   // the staging slot has been read: it may be refilled
+                    mbar_arrive(&sm->mst_full[ms]);    // one arrival per transform warp of the group
+                }
+                ss += LX;
+                if (ss >= nstg) { ss -= nstg; sph ^= 1u; }
+                ms += LX;
+                if (ms >= nmst) { ms -= nmst; mph ^= 1u; }
+            }
+            const int item = (int)blockIdx.x + li * (int)gridDim.x;
+
+            // ---- end of a slab: this group's share of the exact squared norms (the 16 lanes that share a row
+            // add up; the reduction kernel adds the groups) ...
+#pragma unroll
+            for (int j = 0; j < J; ++j) {
+                float v = __uint_as_float((uint32_t)sq[j]) + __uint_as_float((uint32_t)(sq[j] >> 32));
+                v += __shfl_xor_sync(0xffffffffu, v, 1);
+                v += __shfl_xor_sync(0xffffffffu, v, 2);
+                v += __shfl_xor_sync(0xffffffffu, v, 4);
+                v += __shfl_xor_sync(0xffffffffu, v, 8);
+                const int row = row0 + (kGroupThreads / 16) * j;
+                if (q == 0 && row < m) norms[((int64_t)item * LX + group) * m + row] = v;
+                sq[j] = 0ull;
+            }
+            // ... and the accumulator drain: warp w reads TMEM lanes 32*(w%4)..+31; the warps that share a
+            // lane quarter take 16-column chunks round-robin
+            mbar_wait(&sm->accum_full, (uint32_t)(li & 1), abort_flag, status);
+            tc_fence_after();
+            const int quarter = warp & 3;
+            float* out_item = partial + (int64_t)item * m * ncol;
+            // M = 128: accumulator row i sits in TMEM lane i; M = 64: in lane 32 (i / 16) + i % 16
+            const int row = mrows == 64 ? (lane < 16 ? quarter * 16 + lane : m) : quarter * 32 + lane;
+            // the hi.hi and hi.2lo parts of every issuing thread's accumulator (a slab of a single stage leaves the
+            // second thread's accumulator untouched: skip it)
+            const int nparts = 2 * (nst < kMmaWarps ? nst : kMmaWarps);
+            for (int cc = warp >> 2; cc * 16 < ncol; cc += kProdWarps / 4) {   // ncol is a multiple of 16
+                float acc[16];
+#pragma unroll
+                for (int j = 0; j < 16; ++j) acc[j] = 0.f;
+                for (int part = 0; part < nparts; ++part) {
+                    uint32_t v[16];
+                    tmem_load16(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(part * ncol + cc * 16), v);
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) acc[j] += __uint_as_float(v[j]);
+                }
+                if (row < m) {
+                    float* dstp = out_item + (int64_t)row * ncol + cc * 16;
+#pragma unroll
+                    for (int j = 0; j < 16; j += 4)
+                        *reinterpret_cast<float4*>(dstp + j) = make_float4(acc[j], acc[j + 1], acc[j + 2], acc[j + 3]);
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sm->accum_empty);
+        }
+        // slots of slabs this CTA does not have (it owns one stage fewer than others) read as zero
+        for (int l2 = my_items; l2 * (int)gridDim.x < nitems; ++l2) {
+            const int64_t item = (int64_t)blockIdx.x + (int64_t)l2 * gridDim.x;
+            for (int e = tid; e < m * ncol; e += kProdThreads) partial[item * m * ncol + e] = 0.f;
+            for (int e = tid; e < m * LX; e += kProdThreads) norms[item * LX * m + e] = 0.f;
+        }
+    } else if (warp >= kProdWarps + kMmaWarps) {
+        // ------------------------------------------------ the TMA threads: thread l issues the stages l, l + kTmaWarps, ...
+        if (lane == 0) {
+            const int l = warp - (kProdWarps + kMmaWarps);
+            int last = -1;
+            int s = l % nstg;
+            uint32_t ph = (uint32_t)(l / nstg) & 1u;
+            int64_t c0 = ((int64_t)blockIdx.x + (int64_t)l * gridDim.x) * kStageCols;   // first column of the stage
+            for (int t = l; t < total; t += kTmaWarps) {
+                if (!mbar_wait(&sm->stg_empty[s], ph ^ 1u, abort_flag, status)) break;   // the slot has been read
+                mbar_expect_tx(&sm->stg_full[s], stg_bytes);
+                tma_load_2d(stg_base + (size_t)s * stg_bytes, &xmap, (int)c0, 0, &sm->stg_full[s]);
+                last = t;
+                s += kTmaWarps;
+                while (s >= nstg) { s -= nstg; ph ^= 1u; }
+                c0 += (int64_t)kTmaWarps * gridDim.x * kStageCols;
+            }
+            if (*abort_flag) {
+                // give this thread's copies still in flight a bounded time to land before the CTA goes away
+                for (int tt = last; tt >= 0 && tt > last - nstg; tt -= kTmaWarps) {
+                    const int s2 = (int)((uint32_t)tt % (uint32_t)nstg);
+                    const uint32_t ph2 = ((uint32_t)tt / (uint32_t)nstg) & 1u;
+                    for (uint32_t spin = 0; spin < (1u << 16) && !mbar_test(&sm->stg_full[s2], ph2); ++spin) __nanosleep(64);
                 }
             }
         }
     } else if (lane == 0) {
-        // ------------------------------------------------ the MMA threads
-        // ------------------------------------------------ (lane 0 of the two warps after the transform warps)
+        // ------------------------------------------------ the MMA threads (lane 0 of the two warps after the
+        // transform warps): they alternate stages and own one accumulator of 2 ncol columns each
         const int g = warp - kProdWarps;
-        const int n_mma = nhalf == 1 ? 2 * ncol : ncol;
-        const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(n_mma >> 3) << 17) | ((uint32_t)(mrows >> 4) << 24);
+        const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)((2 * ncol) >> 3) << 17) | ((uint32_t)(mrows >> 4) << 24);
+        const uint32_t dcol = tmem_base + (uint32_t)(g * 2 * ncol);
         int s = 0, turn = 0;
         uint32_t ph = 0;
-        for (int local_item = 0; local_item < my_items; ++local_item) {
-            const int nkb = local_item == my_items - 1 ? last_nkb : kBlocksPerSlab;
-            if (local_item > 0) mbar_wait(&sm->accum_empty, (uint32_t)((local_item - 1) & 1), abort_flag, status);
+        for (int li = 0; li < my_items; ++li) {
+            const int nst = li == my_items - 1 ? last_nst : kStagesPerSlab;
+            if (li > 0) mbar_wait(&sm->accum_empty, (uint32_t)((li - 1) & 1), abort_flag, status);
             tc_fence_after();
             bool first = true;   // this thread's first MMA of the slab overwrites its accumulator
-            for (int kb = 0; kb < nkb; ++kb) {
+            for (int k = 0; k < nst; ++k) {
                 const int my_s = s;
                 const uint32_t my_ph = ph;
-                const bool skip = nhalf == 1 && turn != g;   // m <= 128: the two threads alternate K-blocks
-                if (++s == stages) { s = 0; ph ^= 1u; }
+                const bool skip = turn != g;
+                if (++s == nmst) { s = 0; ph ^= 1u; }
                 turn ^= 1;
                 if (skip) continue;
-                mbar_wait(&sm->full[my_s], my_ph, abort_flag, status);
+                mbar_wait(&sm->mst_full[my_s], my_ph, abort_flag, status);
                 tc_fence_after();
-                const uint32_t hi_addr = smem_u32(base + (size_t)my_s * stage_bytes);
-                const uint64_t hi_desc = smem_desc(hi_addr);
-                if (nhalf == 1) {
-                    const uint32_t dcol = tmem_base + (uint32_t)(g * 2 * ncol);
+                const uint32_t addr = smem_u32(mst_base + (size_t)my_s * mst_bytes);
+#pragma unroll
+                for (int kb = 0; kb < kKbPerStage; ++kb) {
+                    const uint64_t desc = smem_desc(addr + (uint32_t)kb * tile_bytes);
 #pragma unroll
                     for (int kk = 0; kk < kKB / 8; ++kk) {       // one MMA covers 8 columns = 32 bytes
-                        const uint64_t ab = hi_desc + (uint64_t)(kk * 2);
-                        mma_tf32(dcol, ab, ab, idesc, first ? 0u : 1u);
-                        first = false;
-                    }
-                } else {
-                    const uint64_t lo_desc = smem_desc(hi_addr + tile_bytes);
-                    const uint32_t dcol = tmem_base + (uint32_t)(g * ncol);
-#pragma unroll
-                    for (int kk = 0; kk < kKB / 8; ++kk) {
-                        const uint64_t a = hi_desc + (uint64_t)(kk * 2 + g * (128 * 128 / 16));
-                        mma_tf32(dcol, a, hi_desc + (uint64_t)(kk * 2), idesc, first ? 0u : 1u);
-                        mma_tf32(dcol, a, lo_desc + (uint64_t)(kk * 2), idesc, 1u);
+                        const uint64_t ab = desc + (uint64_t)(kk * 2);
+                        mma_tf32(dcol, ab, ab, idesc, first ? 0u : 1u);   // A = hi rows, B = [hi ; 2lo]
                         first = false;
                     }
                 }
-                mma_commit(&sm->empty[my_s]);   // the stage may be refilled once these MMAs have read it
+                mma_commit(&sm->mst_empty[my_s]);   // the slot may be rewritten once these MMAs have read it
             }
             mma_commit(&sm->accum_full);
         }
@@ -470,13 +715,14 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap xmap, int m, int64_t d, int r
 }
 
 // For one chunk of slabs: gpart[chunk][i*m+j] (i < j) = sum_s sym(T(s))_ij * (r_i(s) + r_j(s)) / 2 with
-// r_i(s) = exact norm / tensor-core norm of row i in slab s; gpart[chunk][i*m+i] = sum_s exact norm.
+// r_i(s) = exact norm / tensor-core norm of row i in slab s; gpart[chunk][i*m+i] = sum_s exact norm
+// (the exact norm of a slab comes in `ngroups` shares, added here in a fixed order).
 // One CTA per pair of 32-row blocks (bi <= bj) and chunk: per slab it reads the tile T[bi][bj] and the
 // mirrored tile T[bj][bi] row by row (coalesced) and transposes the second through shared memory.
 constexpr int kRT = 32;
 __global__ void __launch_bounds__(kRT * 8)
-tc_reduce_kernel(const float* __restrict__ partial, const float* __restrict__ norms, int nitems, int m, int ncol,
-                 double* __restrict__ gpart) {
+tc_reduce_kernel(const float* __restrict__ partial, const float* __restrict__ norms, int ngroups, int nitems, int m,
+                 int ncol, double* __restrict__ gpart) {
     __shared__ float mirror[kRT][kRT + 1];
     __shared__ double ratio_i[kRT], ratio_j[kRT];
     const int nt = (m + kRT - 1) / kRT;
@@ -497,12 +743,14 @@ tc_reduce_kernel(const float* __restrict__ partial, const float* __restrict__ no
 
     for (int s = s0; s < s1; ++s) {
         const float* T = partial + (int64_t)s * elems;
-        const float* nrm = norms + (int64_t)s * m;
+        const float* nrm = norms + (int64_t)s * ngroups * m;   // one share per group of transform warps
         if (ty < 2) {
             const int r = (ty == 0 ? bi : bj) * kRT + tx;
             double ratio = 1.0;
             if (r < m) {
-                const double t = (double)T[(int64_t)r * ncol + r], nv = (double)nrm[r];
+                const double t = (double)T[(int64_t)r * ncol + r];
+                double nv = 0.0;
+                for (int g = 0; g < ngroups; ++g) nv += (double)nrm[g * m + r];
                 if (t > 0.0) ratio = nv / t;
                 if (ty == 0 && bi == bj) nsum += nv;
             }
@@ -590,28 +838,60 @@ EncodeTiledFn encode_tiled_fn() {
 
 // X as a 2-D fp32 tensor (d columns innermost, m rows, row pitch ld); box = 32 columns x box_rows rows,
 // 128-byte swizzle, zero fill outside.
-detox_status make_xmap(CUtensorMap* map, const float* X, int64_t ld, int m, int64_t d, int box_rows) {
+detox_status make_xmap(CUtensorMap* map, const float* X, int64_t ld, int m, int64_t d, int box_cols, int box_rows,
+                       CUtensorMapSwizzle swizzle) {
     EncodeTiledFn enc = encode_tiled_fn();
     if (!enc) return DETOX_ERR_CUDA;
     const cuuint64_t gdim[2] = {(cuuint64_t)d, (cuuint64_t)m};
     const cuuint64_t gstride[1] = {(cuuint64_t)ld * sizeof(float)};
-    const cuuint32_t box[2] = {(cuuint32_t)kKB, (cuuint32_t)box_rows};
+    const cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows};
     const cuuint32_t estride[2] = {1, 1};
     CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(X), gdim, gstride, box, estride,
-                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? DETOX_OK : DETOX_ERR_CUDA;
 }
 
 template <int J>
-detox_status launch_tc(const TcPlan& p, const CUtensorMap& xmap, int m, int64_t d, float* partial, float* norms,
-                       int* status, cudaStream_t s) {
-    if (cudaFuncSetAttribute(gram_tc_kernel<J>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem_bytes) !=
+detox_status launch_wide(const WidePlan& p, const CUtensorMap& xmap, int m, float* partial, float* norms, int* status,
+                         cudaStream_t s) {
+    if (cudaFuncSetAttribute(gram_wide_kernel<J>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem_bytes) !=
         cudaSuccess)
         return DETOX_ERR_CUDA;
-    gram_tc_kernel<J><<<p.grid, kTcThreads, p.smem_bytes, s>>>(xmap, m, d, p.rows_pad, p.mrows, p.box_rows, p.nhalf, p.ncol,
-                                                               p.chains, p.tmem_cols, p.stages, p.nkb_total, p.nitems, partial, norms, status);
+    gram_wide_kernel<J><<<p.grid, kTcThreads, p.smem_bytes, s>>>(xmap, m, p.lo_off, p.stage_bytes, p.box_rows, p.ncol,
+                                                                 p.tmem_cols, p.stages, p.nkb_total, p.nitems, partial,
+                                                                 norms, status);
     return launch_status();
+}
+
+template <int J, int LX>
+detox_status launch_staged(const StagedPlan& p, const CUtensorMap& xmap, int m, float* partial, float* norms, int* status,
+                           cudaStream_t s) {
+    if (cudaFuncSetAttribute(gram_staged_kernel<J, LX>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem_bytes) !=
+        cudaSuccess)
+        return DETOX_ERR_CUDA;
+    gram_staged_kernel<J, LX><<<p.grid, kTcThreads, p.smem_bytes, s>>>(xmap, m, p.stg_bytes, p.tile_bytes, p.mrows, p.ncol,
+                                                                       p.tmem_cols, p.nstg, p.nmst, p.nst_total, p.nitems,
+                                                                       partial, norms, status);
+    return launch_status();
+}
+
+// What the two kernels' outputs look like to the reduction: slab slots, shares of the norms per slot, row pitch.
+struct TcShape {
+    bool staged;
+    int nitems, groups, ncol;
+};
+TcShape tc_shape(int m, int64_t d) {
+    TcShape o;
+    o.staged = m <= 128;
+    if (o.staged) {
+        const StagedPlan p = staged_plan(m, d);
+        o.nitems = p.nitems, o.groups = p.groups, o.ncol = p.ncol;
+    } else {
+        const WidePlan p = wide_plan(m, d);
+        o.nitems = p.nitems, o.groups = 1, o.ncol = p.ncol;
+    }
+    return o;
 }
 
 }  // namespace
@@ -622,34 +902,50 @@ bool tc_supported(const float* X, int64_t ld, int m, int64_t d) {
 }
 
 size_t tc_ws_bytes(int m, int64_t d) {
-    TcPlan p = tc_plan(m, d);
-    const size_t elems = (size_t)m * p.ncol;
-    return align_up((size_t)p.nitems * elems * sizeof(float)) + align_up((size_t)p.nitems * m * sizeof(float)) +
-           align_up((size_t)reduce_chunks(m, p.nitems) * m * m * sizeof(double));
+    const TcShape o = tc_shape(m, d);
+    const size_t elems = (size_t)m * o.ncol;
+    return align_up((size_t)o.nitems * elems * sizeof(float)) + align_up((size_t)o.nitems * o.groups * m * sizeof(float)) +
+           align_up((size_t)reduce_chunks(m, o.nitems) * m * m * sizeof(double));
 }
 
 detox_status launch_sqdist_tc(const float* X, int64_t ld, int m, int64_t d, double* D, void* ws, int* status,
                               cudaStream_t s) {
-    TcPlan p = tc_plan(m, d);
-    const int64_t elems = (int64_t)m * p.ncol;
+    const TcShape o = tc_shape(m, d);
+    const int64_t elems = (int64_t)m * o.ncol;
     char* base = static_cast<char*>(ws);
     float* partial = reinterpret_cast<float*>(base);
-    float* norms = reinterpret_cast<float*>(base + align_up((size_t)p.nitems * elems * sizeof(float)));
-    double* gpart = reinterpret_cast<double*>(base + align_up((size_t)p.nitems * elems * sizeof(float)) +
-                                              align_up((size_t)p.nitems * m * sizeof(float)));
+    float* norms = reinterpret_cast<float*>(base + align_up((size_t)o.nitems * elems * sizeof(float)));
+    double* gpart = reinterpret_cast<double*>(base + align_up((size_t)o.nitems * elems * sizeof(float)) +
+                                              align_up((size_t)o.nitems * o.groups * m * sizeof(float)));
     CUtensorMap xmap;
-    detox_status st = make_xmap(&xmap, X, ld, m, d, p.box_rows);
-    if (st != DETOX_OK) return st;
-    // chunks per transform thread: m * 8 / kProdThreads, rounded up to a power of two
-    const int per_thread = (m * 8 + kProdThreads - 1) / kProdThreads;
-    if (per_thread <= 1) st = launch_tc<1>(p, xmap, m, d, partial, norms, status, s);
-    else if (per_thread <= 2) st = launch_tc<2>(p, xmap, m, d, partial, norms, status, s);
-    else st = launch_tc<4>(p, xmap, m, d, partial, norms, status, s);
+    detox_status st;
+    if (o.staged) {
+        const StagedPlan p = staged_plan(m, d);
+        if ((st = make_xmap(&xmap, X, ld, m, d, kStageCols, p.box_rows, CU_TENSOR_MAP_SWIZZLE_NONE)) != DETOX_OK) return st;
+        // 16-byte pieces per transform thread and stage: m * 16 / (threads of a group), rounded up
+        const int gt = kProdThreads / p.groups;
+        const int per_thread = (m * (kStageCols / 4) + gt - 1) / gt;
+        if (p.groups == 2) {
+            if (per_thread <= 2) st = launch_staged<2, 2>(p, xmap, m, partial, norms, status, s);
+            else if (per_thread <= 3) st = launch_staged<3, 2>(p, xmap, m, partial, norms, status, s);
+            else st = launch_staged<4, 2>(p, xmap, m, partial, norms, status, s);
+        } else {
+            if (per_thread <= 2) st = launch_staged<2, 1>(p, xmap, m, partial, norms, status, s);
+            else if (per_thread <= 3) st = launch_staged<3, 1>(p, xmap, m, partial, norms, status, s);
+            else st = launch_staged<4, 1>(p, xmap, m, partial, norms, status, s);
+        }
+    } else {
+        const WidePlan p = wide_plan(m, d);
+        if ((st = make_xmap(&xmap, X, ld, m, d, kKB, p.box_rows, CU_TENSOR_MAP_SWIZZLE_128B)) != DETOX_OK) return st;
+        // 16-byte pieces per transform thread and K-block: m * 8 / 512, rounded up
+        if (m * 8 <= 3 * kProdThreads) st = launch_wide<3>(p, xmap, m, partial, norms, status, s);
+        else st = launch_wide<4>(p, xmap, m, partial, norms, status, s);
+    }
     if (st != DETOX_OK) return st;
     const int nt = (m + kRT - 1) / kRT;
-    const int nchunks = reduce_chunks(m, p.nitems);
-    tc_reduce_kernel<<<dim3((unsigned)(nt * (nt + 1) / 2), (unsigned)nchunks), kRT * 8, 0, s>>>(partial, norms, p.nitems, m,
-                                                                                           p.ncol, gpart);
+    const int nchunks = reduce_chunks(m, o.nitems);
+    tc_reduce_kernel<<<dim3((unsigned)(nt * (nt + 1) / 2), (unsigned)nchunks), kRT * 8, 0, s>>>(partial, norms, o.groups,
+                                                                                           o.nitems, m, o.ncol, gpart);
     if ((st = launch_status()) != DETOX_OK) return st;
     tc_dist_kernel<<<(unsigned)ceil_div((int64_t)m * m * 32, 256), 256, 0, s>>>(gpart, nchunks, m, status, D);
     return launch_status();
