@@ -58,44 +58,52 @@ colselect_reg_kernel(const float* __restrict__ X, int64_t ld, int m, int64_t d, 
     const int64_t left = d - col0;
     const int valid = left >= C ? C : (int)left;
 
-    // Network sizes up to 32 are used with m == M; larger ones may carry padding.
+    // Network sizes up to 32 are used with m == M; larger ones may carry padding: at most kMaxGap slots, the top ones
+    // (the dispatcher rounds m up to the next network size, 8 apart up to 64 and 16 apart above).  Only those slots
+    // pay for the clamped row index and the padding test; the others have a compile-time row.
     constexpr bool kPadded = M > 32;
+    constexpr int kMaxGap = !kPadded ? 0 : (M <= 64 ? 7 : 15);
+    constexpr int kSure = M - kMaxGap;            // slots below this always hold a row
     const int pad = kPadded ? (M - m) >> 1 : 0;   // lowest keys added (and as many highest)
     int32_t key[C][M];
+    const uint32_t col32 = (uint32_t)col0;        // the launcher keeps d below 2^31 per launch
+    auto load_piece = [&](const float* rowp, uint32_t keep, int i) {
+        // row pointer (the same for the whole warp) + 4 * column: one 32 x 32 + 64 bit multiply-add
+        const float* p = reinterpret_cast<const float*>(reinterpret_cast<const char*>(rowp) + (uint64_t)col32 * 4u);
+        if (C == 4 && valid == 4) {
+            uint4 v = ld_stream_u4(p);
+            key[0][i] = (int32_t)(v.x & keep);
+            key[1 % C][i] = (int32_t)(v.y & keep);
+            key[2 % C][i] = (int32_t)(v.z & keep);
+            key[3 % C][i] = (int32_t)(v.w & keep);
+        } else if (C == 2 && valid == 2) {
+            uint2 v = __ldcs(reinterpret_cast<const uint2*>(p));
+            key[0][i] = (int32_t)(v.x & keep);
+            key[1 % C][i] = (int32_t)(v.y & keep);
+        } else {
+#pragma unroll
+            for (int c = 0; c < C; ++c) key[c][i] = c < valid ? (int32_t)(ld_stream_u1(p + c) & keep) : 0;
+        }
+    };
     // All loads first, with no branch in between, so that they are in flight together; slots beyond m
     // re-read the last row and are replaced by padding keys afterwards.  The test for a row list is
     // taken once, outside the loads: a per-load test would serialise them.
-    auto load_all = [&](auto row_of) {
+    if (rows) {
 #pragma unroll
         for (int i = 0; i < M; ++i) {
-            const int ri = kPadded ? (i < m ? i : m - 1) : i;
-            const int rr = row_of(ri);                    // a negative entry of the row list stands for a zero row
-            const uint32_t keep = rr < 0 ? 0u : 0xFFFFFFFFu;
-            const float* p = X + (int64_t)(rr < 0 ? 0 : rr) * ld + col0;
-            if (C == 4 && valid == 4) {
-                uint4 v = ld_stream_u4(p);
-                key[0][i] = (int32_t)(v.x & keep);
-                key[1 % C][i] = (int32_t)(v.y & keep);
-                key[2 % C][i] = (int32_t)(v.z & keep);
-                key[3 % C][i] = (int32_t)(v.w & keep);
-            } else if (C == 2 && valid == 2) {
-                uint2 v = __ldcs(reinterpret_cast<const uint2*>(p));
-                key[0][i] = (int32_t)(v.x & keep);
-                key[1 % C][i] = (int32_t)(v.y & keep);
-            } else {
-#pragma unroll
-                for (int c = 0; c < C; ++c) key[c][i] = c < valid ? (int32_t)(ld_stream_u1(p + c) & keep) : 0;
-            }
+            const int rr = srow[i < kSure ? i : (i < m ? i : m - 1)];   // a negative entry stands for a zero row
+            load_piece(X + (int64_t)(rr < 0 ? 0 : rr) * ld, rr < 0 ? 0u : 0xFFFFFFFFu, i);
         }
-    };
-    if (rows) load_all([&](int ri) { return srow[ri]; });
-    else load_all([](int ri) { return ri; });
+    } else {
+#pragma unroll
+        for (int i = 0; i < M; ++i) load_piece(X + (int64_t)(i < kSure ? i : (i < m ? i : m - 1)) * ld, 0xFFFFFFFFu, i);
+    }
 #pragma unroll
     for (int i = 0; i < M; ++i) {
 #pragma unroll
         for (int c = 0; c < C; ++c) {
             int32_t k = key_of_bits((uint32_t)key[c][i]);
-            if (kPadded && i >= m) k = (i - m < pad) ? (int32_t)0x80000000 : 0x7fffffff;
+            if (i >= kSure && i >= m) k = (i - m < pad) ? (int32_t)0x80000000 : 0x7fffffff;
             key[c][i] = k;
         }
     }
@@ -140,18 +148,23 @@ colselect_reg_kernel(const float* __restrict__ X, int64_t ld, int m, int64_t d, 
 template <int M, int C>
 detox_status launch_reg(const float* X, int64_t ld, int m, int64_t d, const int32_t* rows, int beta, float* out,
                         cudaStream_t s) {
-    if (beta == 0) {
-        constexpr int T = reg_threads(M, C, false);
-        int64_t bx = ceil_div(d, (int64_t)T * C);
-        if (bx > 0x7fffffffLL) return DETOX_ERR_UNSUPPORTED;
-        colselect_reg_kernel<M, C, false><<<(unsigned)bx, T, 0, s>>>(X, ld, m, d, rows, beta, out);
-    } else {
-        constexpr int T = reg_threads(M, C, true);
-        int64_t bx = ceil_div(d, (int64_t)T * C);
-        if (bx > 0x7fffffffLL) return DETOX_ERR_UNSUPPORTED;
-        colselect_reg_kernel<M, C, true><<<(unsigned)bx, T, 0, s>>>(X, ld, m, d, rows, beta, out);
+    // the kernel works with 32-bit column offsets: wider matrices go in pieces of 2^30 columns
+    constexpr int64_t kMaxCols = (int64_t)1 << 30;
+    for (int64_t c0 = 0; c0 < d; c0 += kMaxCols) {
+        const int64_t dc = d - c0 < kMaxCols ? d - c0 : kMaxCols;
+        if (beta == 0) {
+            constexpr int T = reg_threads(M, C, false);
+            colselect_reg_kernel<M, C, false><<<(unsigned)ceil_div(dc, (int64_t)T * C), T, 0, s>>>(X + c0, ld, m, dc, rows, beta,
+                                                                                              out + c0);
+        } else {
+            constexpr int T = reg_threads(M, C, true);
+            colselect_reg_kernel<M, C, true><<<(unsigned)ceil_div(dc, (int64_t)T * C), T, 0, s>>>(X + c0, ld, m, dc, rows, beta,
+                                                                                             out + c0);
+        }
+        const detox_status st = launch_status();
+        if (st != DETOX_OK) return st;
     }
-    return launch_status();
+    return DETOX_OK;
 }
 
 template <int M>

@@ -39,23 +39,30 @@ colselect_pair_kernel(const float* __restrict__ X, int64_t ld, int m, int64_t d,
     const int extra = m - kHalf;                        // real rows held by lane 1
 
     int32_t key[kHalf];
+    // Lane 0 always holds kHalf rows.  Lane 1 holds `extra` rows, at least kSure of them when the median picks
+    // kHalf (half of m rounded up to 8), so only its top slots pay for the clamped row and the padding test.
+    constexpr int kSure = TRIM ? 0 : kHalf - 16;
     // the test for a row list is taken once, outside the loads: a per-load test would serialise them
-    auto load_all = [&](auto row_of) {
+    if (rows) {
 #pragma unroll
         for (int i = 0; i < kHalf; ++i) {
             int ri = hsel ? kHalf + i : i;
-            ri = ri < m ? ri : m - 1;
-            const int rr = row_of(ri);                // a negative entry of the row list stands for a zero row
+            if (i >= kSure) ri = ri < m ? ri : m - 1;
+            const int rr = srow[ri];                  // a negative entry of the row list stands for a zero row
             const uint32_t v = ld_stream_u1(X + (int64_t)(rr < 0 ? 0 : rr) * ld + col);
             key[i] = (int32_t)(rr < 0 ? 0u : v);
         }
-    };
-    if (rows) load_all([&](int ri) { return srow[ri]; });
-    else load_all([](int ri) { return ri; });
+    } else {
+        // this lane's first row at its column; row i of the lane is i * ld further (the same step for all lanes)
+        const float* base = X + (int64_t)(hsel ? kHalf : 0) * ld + col;
+        const int last = (hsel ? extra : kHalf) - 1;
+#pragma unroll
+        for (int i = 0; i < kHalf; ++i) key[i] = (int32_t)ld_stream_u1(base + (int64_t)(i < kSure ? i : (i < last ? i : last)) * ld);
+    }
 #pragma unroll
     for (int i = 0; i < kHalf; ++i) {
         int32_t k = key_of_bits((uint32_t)key[i]);
-        if (hsel && i >= extra) k = (i - extra < pad_lo) ? (int32_t)0x80000000 : 0x7fffffff;
+        if (i >= kSure && hsel && i >= extra) k = (i - extra < pad_lo) ? (int32_t)0x80000000 : 0x7fffffff;
         key[i] = k;
     }
     sort_registers<kHalf>(key);
