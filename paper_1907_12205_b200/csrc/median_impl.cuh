@@ -67,9 +67,7 @@ colselect_reg_kernel(const float* __restrict__ X, int64_t ld, int m, int64_t d, 
     const int pad = kPadded ? (M - m) >> 1 : 0;   // lowest keys added (and as many highest)
     int32_t key[C][M];
     const uint32_t col32 = (uint32_t)col0;        // the launcher keeps d below 2^31 per launch
-    auto load_piece = [&](const float* rowp, uint32_t keep, int i) {
-        // row pointer (the same for the whole warp) + 4 * column: one 32 x 32 + 64 bit multiply-add
-        const float* p = reinterpret_cast<const float*>(reinterpret_cast<const char*>(rowp) + (uint64_t)col32 * 4u);
+    auto load_piece = [&](const float* p, uint32_t keep, int i) {
         if (C == 4 && valid == 4) {
             uint4 v = ld_stream_u4(p);
             key[0][i] = (int32_t)(v.x & keep);
@@ -92,11 +90,15 @@ colselect_reg_kernel(const float* __restrict__ X, int64_t ld, int m, int64_t d, 
 #pragma unroll
         for (int i = 0; i < M; ++i) {
             const int rr = srow[i < kSure ? i : (i < m ? i : m - 1)];   // a negative entry stands for a zero row
-            load_piece(X + (int64_t)(rr < 0 ? 0 : rr) * ld, rr < 0 ? 0u : 0xFFFFFFFFu, i);
+            load_piece(X + (int64_t)(rr < 0 ? 0 : rr) * ld + col0, rr < 0 ? 0u : 0xFFFFFFFFu, i);
         }
     } else {
+        // row pointer (the same for the whole warp) + 4 * column: one 32 x 32 + 64 bit multiply-add per value
 #pragma unroll
-        for (int i = 0; i < M; ++i) load_piece(X + (int64_t)(i < kSure ? i : (i < m ? i : m - 1)) * ld, 0xFFFFFFFFu, i);
+        for (int i = 0; i < M; ++i) {
+            const float* rowp = X + (int64_t)(i < kSure ? i : (i < m ? i : m - 1)) * ld;
+            load_piece(reinterpret_cast<const float*>(reinterpret_cast<const char*>(rowp) + (uint64_t)col32 * 4u), 0xFFFFFFFFu, i);
+        }
     }
 #pragma unroll
     for (int i = 0; i < M; ++i) {
