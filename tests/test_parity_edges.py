@@ -65,6 +65,24 @@ def test_multikrum_fallback_paths(m, d, f, m_sel, odd):
     assert rel_l2(out.cpu().numpy(), out_o) <= TOL
 
 
+@pytest.mark.parametrize("m,d", [
+    (17, 63), (18, 64), (32, 65), (33, 4097), (63, 9473), (64, 129), (65, 4100), (80, 9472 + 31), (96, 2000),
+    (127, 3001), (128, 1000), (129, 1000), (144, 2049), (240, 777), (256, 640),
+    (20, 700_001), (100, 650_003), (140, 610_000)])       # last three: more than one 4096-column slab per CTA
+def test_tensor_core_distance_kernels_at_their_size_boundaries(m, d):
+    """Row counts on both sides of every switch of the tensor-core kernels (64 and 128 rows, tile sizes that are
+    multiples of 16) and column counts around the 32- and 64-column copies, with a ragged tail."""
+    f = max((m - 3) // 4, 0)
+    X = krum_inputs(m, d, seed=3 * m + d, copies=2 if m % 2 == 0 else 1, outliers=min(f, 3))
+    _, _, sc_o, _ = oracle.multikrum(X, f, 1)
+    _, _, sc = dx.agg_multikrum(padded(X), f, 1)
+    s = sc.cpu().numpy()
+    np.testing.assert_allclose(s, sc_o, rtol=2e-6, atol=1e-30)
+    if m % 2 == 0:                                   # bitwise-equal rows must get bitwise-equal scores
+        for i in range(0, m - 2 - min(f, 3), 2):
+            assert s[i] == s[i + 1]
+
+
 def test_bulyan_many_rows_through_the_shared_memory_stage_two():
     m, d, f = 400, 96, 20                      # theta = 360 rows enter stage 2: beyond the register kernels
     for attempt in range(8):
