@@ -196,6 +196,48 @@ def workload_label(name, spec, cfg):
             f"vote -> A0={a0} -> A1={ORACLE_A1[cfg['a1']]}(f={cfg['f']}, m_sel={cfg['m_sel']})")
 
 
+def median_minmax_ops(m: int) -> int:
+    """min/max operations per coordinate that a median over m rows needs on the register path.
+
+    The merge-exchange network on M inputs (M = m up to 32, else m rounded up to the next network size with an
+    even gap) is walked backwards from the middle output: a comparator costs one operation per output that
+    something later still reads.  Above 128 rows two lanes share a coordinate and no closed count is given."""
+    if m <= 32:
+        M = m
+    elif m <= 128:
+        step = 8 if m <= 64 else 16
+        M = (m + step - 1) // step * step
+        if (M - m) & 1:
+            M -= 1
+    else:
+        return 0
+    net = []
+    p = 1
+    while p < M:
+        k = p
+        while k >= 1:
+            j = k % p
+            while j <= M - 1 - k:
+                for i in range(min(k - 1, M - j - k - 1) + 1):
+                    if (i + j) // (2 * p) == (i + j + k) // (2 * p):
+                        net.append((i + j, i + j + k))
+                j += 2 * k
+            k //= 2
+        p *= 2
+    live = {M // 2} if M & 1 else {M // 2 - 1, M // 2}
+    ops = 0
+    for a, b in reversed(net):
+        used = (a in live) + (b in live)
+        if used:
+            ops += used
+            live.update((a, b))
+    return ops
+
+
+# Integer min/max issue on the plain-ALU pipe: 64 lanes per clock and SM, 148 SMs, at the sampled SM clock.
+ALU_LANES_PER_CLK_SM, N_SMS = 64, 148
+
+
 def run_sweep(args):
     """Config 5: every aggregator with and without the DETOX front end over n x d x attack.
 
@@ -246,6 +288,15 @@ def run_sweep(args):
         pipe_leg("detox_bulyan", dx.AGG_NONE, dx.AGG_BULYAN, fv, 1, (n + 2 * G + (G - 2 * fv) + 1) * d * 4)
         # direct legs on all n rows
         timed("direct_median", lambda: dx.agg_coord_median(X, out=out), (n + 1) * d * 4)
+        ops = median_minmax_ops(n)
+        if n > 16 and ops:
+            # beyond ~16 rows the register networks are bound by the plain ALUs, not by HBM: report that roof too
+            clk = float(peaks.get("sm_max_mhz", 1965.0))
+            peak = ALU_LANES_PER_CLK_SM * N_SMS * clk * 1e6 / 1e12
+            ach = ops * d / (legs["direct_median"]["ms"] * 1e-3) / 1e12
+            legs["direct_median"]["alu"] = {"bound": "alu", "minmax_per_coordinate": ops, "achieved": round(ach, 2),
+                                            "peak": round(peak, 2), "unit": "T min/max per s",
+                                            "frac": round(ach / peak, 3), "peak_kind": "64 lanes/clk/SM x 148 SMs x max SM clock"}
         ws = torch.empty(dx.agg_multikrum_workspace_bytes(n, d), dtype=torch.uint8, device=dev)
         sel = torch.empty(n, dtype=torch.int32, device=dev)
         sc = torch.empty(n, dtype=torch.float64, device=dev)

@@ -48,3 +48,13 @@ def test_single_process_is_passthrough():
     import bench
     assert bench.max_over_ranks(3.5) == 3.5
     assert abs(bench.whole_job_value(10**9, 1, 1.0) - 1000.0) < 1e-9
+
+
+def test_median_operation_count_of_small_networks():
+    """Three inputs: comparators (0,1), (0,2), (1,2); the middle output needs min of the last, max of the second and
+    both outputs of the first = 4 operations.  One input needs none; sizes beyond the register path report 0."""
+    import bench
+    assert bench.median_minmax_ops(1) == 0
+    assert bench.median_minmax_ops(3) == 4
+    assert bench.median_minmax_ops(200) == 0
+    assert bench.median_minmax_ops(45) < bench.median_minmax_ops(105)
