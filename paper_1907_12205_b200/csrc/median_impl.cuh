@@ -37,7 +37,7 @@ __device__ __forceinline__ int window_start(int theta, int beta, float med, KeyA
 
 __host__ __device__ constexpr int reg_threads(int M, int C, bool trim) {
     // the TRIM variant keeps M * C keys per thread in (static) shared memory, next to a staged row list
-    return (trim && M * C * kRegThreads * 4 + M * 4 > 48 * 1024) ? kRegThreads / 2 : kRegThreads;
+    return (trim && M * C * kRegThreads * 4 + M * 8 > 48 * 1024) ? kRegThreads / 2 : kRegThreads;
 }
 
 // M = network size, m = rows actually present (M - m even; the gap is filled with lowest / highest keys)
@@ -46,12 +46,19 @@ __global__ void __launch_bounds__(reg_threads(M, C, TRIM))
 colselect_reg_kernel(const float* __restrict__ X, int64_t ld, int m, int64_t d, const int32_t* __restrict__ rows,
                      int beta, float* __restrict__ out) {
     constexpr int kThreads = reg_threads(M, C, TRIM);
-    // a row list is staged in shared memory once per CTA: read from global memory it would put an index
-    // load in front of every data load
-    __shared__ int32_t srow[M];
+    // a row list is staged in shared memory once per CTA, as element offsets of the rows (-1 for a negative entry,
+    // which stands for a zero row): read from global memory it would put an index load and a 64-bit multiply in
+    // front of every data load
+    __shared__ int64_t soff[M];
+    bool any_zero_row = false;
     if (rows) {
-        for (int i = threadIdx.x; i < m; i += kThreads) srow[i] = rows[i];
-        __syncthreads();
+        int neg = 0;
+        for (int i = threadIdx.x; i < m; i += kThreads) {
+            const int rr = rows[i];
+            soff[i] = rr < 0 ? -1 : (int64_t)rr * ld;
+            neg |= rr < 0;
+        }
+        any_zero_row = __syncthreads_or(neg) != 0;
     }
     const int64_t col0 = ((int64_t)blockIdx.x * kThreads + threadIdx.x) * C;
     if (col0 >= d) return;
@@ -87,10 +94,16 @@ colselect_reg_kernel(const float* __restrict__ X, int64_t ld, int m, int64_t d, 
     // re-read the last row and are replaced by padding keys afterwards.  The test for a row list is
     // taken once, outside the loads: a per-load test would serialise them.
     if (rows) {
+        const float* base = X + col0;
+        if (!any_zero_row) {
 #pragma unroll
-        for (int i = 0; i < M; ++i) {
-            const int rr = srow[i < kSure ? i : (i < m ? i : m - 1)];   // a negative entry stands for a zero row
-            load_piece(X + (int64_t)(rr < 0 ? 0 : rr) * ld + col0, rr < 0 ? 0u : 0xFFFFFFFFu, i);
+            for (int i = 0; i < M; ++i) load_piece(base + soff[i < kSure ? i : (i < m ? i : m - 1)], 0xFFFFFFFFu, i);
+        } else {
+#pragma unroll
+            for (int i = 0; i < M; ++i) {
+                const int64_t off = soff[i < kSure ? i : (i < m ? i : m - 1)];
+                load_piece(base + (off < 0 ? 0 : off), off < 0 ? 0u : 0xFFFFFFFFu, i);
+            }
         }
     } else {
         // row pointer (the same for the whole warp) + 4 * column: one 32 x 32 + 64 bit multiply-add per value
@@ -129,11 +142,19 @@ colselect_reg_kernel(const float* __restrict__ X, int64_t ld, int m, int64_t d, 
             const int cnt = beta < 0 ? -beta : beta;
             const int L = pad + (beta < 0 ? (m - cnt) >> 1
                                           : window_start(m, beta, med, [&](int i) { return mine[(i + pad) * kThreads]; }));
-            // four interleaved partial sums (shorter dependency chains, smaller rounding error)
-            float acc[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-            for (int i = 0; i < M; ++i) acc[i & 3] += (i >= L && i < L + cnt) ? float_of_key(key[c][i]) : 0.f;
-            res[c] = ((acc[0] + acc[1]) + (acc[2] + acc[3])) / (float)cnt;
+            // the window is read back from the sorted keys in shared memory (a masked sum over all M registers costs
+            // more than that as soon as the window is short); four interleaved partial sums
+            const int32_t* win = mine + (size_t)L * kThreads;
+            float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+            int i = 0;
+            for (; i + 3 < cnt; i += 4) {
+                a0 += float_of_key(win[(i + 0) * kThreads]);
+                a1 += float_of_key(win[(i + 1) * kThreads]);
+                a2 += float_of_key(win[(i + 2) * kThreads]);
+                a3 += float_of_key(win[(i + 3) * kThreads]);
+            }
+            for (; i < cnt; ++i) a0 += float_of_key(win[i * kThreads]);
+            res[c] = ((a0 + a1) + (a2 + a3)) / (float)cnt;
         }
     }
     if (C == 4 && valid == 4) {
