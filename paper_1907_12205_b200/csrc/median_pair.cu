@@ -22,11 +22,15 @@ __global__ void __launch_bounds__(kPairThreads)
 colselect_pair_kernel(const float* __restrict__ X, int64_t ld, int m, int64_t d, const int32_t* __restrict__ rows,
                       int beta, float* __restrict__ out) {
     extern __shared__ int32_t sorted[];        // TRIM only: [2 * kHalf][kPairCols]
-    // a row list is staged in shared memory once per CTA: read from global memory it would put an index
-    // load in front of every data load
-    __shared__ int32_t srow[2 * kHalf];
+    // a row list is staged in shared memory once per CTA, as element offsets of the rows (-1 for a negative entry,
+    // which stands for a zero row): read from global memory it would put an index load and a 64-bit multiply in
+    // front of every data load
+    __shared__ int64_t soff[2 * kHalf];
     if (rows) {
-        for (int i = threadIdx.x; i < m; i += kPairThreads) srow[i] = rows[i];
+        for (int i = threadIdx.x; i < m; i += kPairThreads) {
+            const int rr = rows[i];
+            soff[i] = rr < 0 ? -1 : (int64_t)rr * ld;
+        }
         __syncthreads();
     }
     const int hsel = threadIdx.x & 1;
@@ -48,9 +52,9 @@ colselect_pair_kernel(const float* __restrict__ X, int64_t ld, int m, int64_t d,
         for (int i = 0; i < kHalf; ++i) {
             int ri = hsel ? kHalf + i : i;
             if (i >= kSure) ri = ri < m ? ri : m - 1;
-            const int rr = srow[ri];                  // a negative entry of the row list stands for a zero row
-            const uint32_t v = ld_stream_u1(X + (int64_t)(rr < 0 ? 0 : rr) * ld + col);
-            key[i] = (int32_t)(rr < 0 ? 0u : v);
+            const int64_t off = soff[ri];
+            const uint32_t v = ld_stream_u1(X + col + (off < 0 ? 0 : off));
+            key[i] = (int32_t)(off < 0 ? 0u : v);
         }
     } else {
         // this lane's first row at its column; row i of the lane is i * ld further (the same step for all lanes)
@@ -114,14 +118,23 @@ colselect_pair_kernel(const float* __restrict__ X, int64_t ld, int m, int64_t d,
     float med = float_of_key(at(kHalf - 1));
     if ((m & 1) == 0) med = (med + float_of_key(at(kHalf))) * 0.5f;
     const int cnt = beta < 0 ? -beta : beta;   // beta < 0: the middle -beta values (trimmed mean)
-    // both lanes of the pair find the same window; each adds the part of it that sits in its own registers
+    // both lanes of the pair find the same window
     const int L = pad_lo + (beta < 0 ? (m - cnt) >> 1
                                      : regselect::window_start(m, beta, med, [&](int i) { return at(i + pad_lo); }));
-    const int first = L - hsel * kHalf, last = first + cnt;     // window in this lane's positions
-    float acc[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-    for (int i = 0; i < kHalf; ++i) acc[i & 3] += (i >= first && i < last) ? float_of_key(key[i]) : 0.f;
-    float sum = (acc[0] + acc[1]) + (acc[2] + acc[3]);
+    // each lane adds the part of the window that lies in its own half of the sorted positions, read back from
+    // shared memory (cheaper than a masked sum over all of its registers); four interleaved partial sums
+    const int lo_p = hsel * kHalf, hi_p = lo_p + kHalf;
+    const int p0 = L > lo_p ? L : lo_p, p1 = L + cnt < hi_p ? L + cnt : hi_p;
+    float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+    int p = p0;
+    for (; p + 3 < p1; p += 4) {
+        a0 += float_of_key(at(p));
+        a1 += float_of_key(at(p + 1));
+        a2 += float_of_key(at(p + 2));
+        a3 += float_of_key(at(p + 3));
+    }
+    for (; p < p1; ++p) a0 += float_of_key(at(p));
+    float sum = (a0 + a1) + (a2 + a3);
     sum += __shfl_xor_sync(0xffffffffu, sum, 1);
     if (hsel == 0 && live) out[col] = sum / (float)cnt;
 }
