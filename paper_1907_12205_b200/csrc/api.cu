@@ -92,9 +92,9 @@ detox_status run_multikrum(const float* X, int64_t ld, int m, int64_t d, const i
     detox_status st;
     if (m >= 2 && m <= 16) {   // distance pass, then one small kernel for everything up to the chosen rows
         int nblocks = 0;
-        if ((st = launch_sqdist_partials(X, ld, m, d, rows, k.dist, &nblocks, s)) != DETOX_OK) return st;
+        if ((st = launch_sqdist_partials(X, ld, m, d, rows, k.dist, k.status, &nblocks, s)) != DETOX_OK) return st;
         st = launch_krum_small(false, static_cast<const double*>(k.dist), nblocks, m, f, m_sel, rows, sel_buf, k.mapped,
-                               scores, k.status, s);
+                               scores, sqdist_partials_use_status(m, X, ld, d) ? nullptr : k.status, s);
         if (st != DETOX_OK) return st;
         return launch_mean_rows(X, ld, d, rows ? k.mapped : sel_buf, m_sel, out, s);
     }
@@ -119,9 +119,9 @@ detox_status run_bulyan(const float* X, int64_t ld, int m, int64_t d, const int3
     detox_status st;
     if (m >= 2 && m <= 16) {   // distance pass, then one small kernel for everything up to the chosen rows
         int nblocks = 0;
-        if ((st = launch_sqdist_partials(X, ld, m, d, rows, k.dist, &nblocks, s)) != DETOX_OK) return st;
+        if ((st = launch_sqdist_partials(X, ld, m, d, rows, k.dist, k.status, &nblocks, s)) != DETOX_OK) return st;
         st = launch_krum_small(true, static_cast<const double*>(k.dist), nblocks, m, f, 0, rows, sel_buf, k.mapped, nullptr,
-                               k.status, s);
+                               sqdist_partials_use_status(m, X, ld, d) ? nullptr : k.status, s);
         if (st != DETOX_OK) return st;
         return launch_coord_select(X, ld, theta, d, rows ? k.mapped : sel_buf, beta, out, s);
     }

@@ -95,9 +95,12 @@ detox_status launch_sqdist(const float* X, int64_t ld, int m, int64_t d, const i
 // gram_tc.cu: the tcgen05 path for 16 < m <= 256 (needs 16-byte aligned rows)
 bool tc_supported(const float* X, int64_t ld, int m, int64_t d);
 size_t tc_ws_bytes(int m, int64_t d);
-// 2 <= m <= 16: the direct kernel's per-CTA pair partials only (consumed by launch_krum_small)
+// 2 <= m <= 16: the direct kernels' per-CTA pair partials only (consumed by launch_krum_small).  When
+// sqdist_partials_use_status() holds the kernel clears the device status word itself and may set it to
+// DETOX_ERR_TIMEOUT, so the consumer must leave it alone.
+bool sqdist_partials_use_status(int m, const float* X, int64_t ld, int64_t d);
 detox_status launch_sqdist_partials(const float* X, int64_t ld, int m, int64_t d, const int32_t* rows, void* ws,
-                                    int* nblocks, cudaStream_t s);
+                                    int* status, int* nblocks, cudaStream_t s);
 detox_status launch_sqdist_tc(const float* X, int64_t ld, int m, int64_t d, double* D, void* ws, int* status,
                               cudaStream_t s);
 

@@ -2,12 +2,14 @@
 // "Improved speed").  Output: D, m x m fp64, symmetric, zero diagonal.
 //
 //   m <= 16 : differences are formed directly, (x_i - x_j)^2, with one fp32 accumulator per pair in
-//             registers; HBM-bound (m*d*4 bytes read once).
+//             registers; HBM-bound (m*d*4 bytes read once).  From 9 rows on, long 16-byte aligned rows are
+//             streamed through shared memory with bulk copies so that the copies overlap the arithmetic.
 //   16 < m <= 256 with 16-byte aligned rows: the tensor-core Gram of gram_tc.cu.
 //   otherwise : CUDA-core Gram tiles G = X X^T over K-slabs, D_ij = G_ii + G_jj - 2 G_ij.
 // Both write per-CTA partial sums that a second kernel adds in a fixed order in fp64, so results
 // are deterministic and bitwise-equal rows get bitwise-equal distances.
 #include "common.cuh"
+#include "mbarrier.cuh"
 
 namespace detox {
 
@@ -97,6 +99,158 @@ sqdist_direct_kernel(const float* __restrict__ X, int64_t ld, int64_t d, const i
 #pragma unroll
         for (int w = 0; w < kDirWarps; ++w) v += red[w][p];
         partial[(int64_t)blockIdx.x * NP + p] = v;
+    }
+}
+
+// ------------------------------------------------------------------ 9 <= m <= 16, long rows: staged differences
+//
+// With 36 to 120 pair accumulators a thread has no registers left to keep the next columns in flight, and the
+// kernel above waits out the memory latency between its steps.  Here tiles of 1024 columns of all rows stream
+// into a ring of shared-memory stages with bulk copies (one per row and tile, issued by the first warp a few tiles
+// ahead of the arithmetic) while all eight warps form the differences from the stage that has landed.  One
+// persistent CTA per SM; eight warps, so that a thread may keep up to 255 registers.
+constexpr int kStgWarps = 8;
+constexpr int kStgThreads = kStgWarps * 32;
+constexpr int kStgPieces = kStgThreads;                   // 16-byte pieces per row and tile: one per thread
+constexpr int64_t kStgMinCols = (int64_t)kSMs * kStgPieces * 4 * 4;   // at least four tiles per CTA
+
+__host__ __device__ constexpr int stg_stages(int M) { return M <= 12 ? 4 : 3; }   // 16 rows x 4 KB x 3 = 192 KB
+
+__device__ __forceinline__ void bulk_copy_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar))
+                 : "memory");
+}
+
+// Rows must be 16-byte aligned (base and pitch).  `status` is cleared by the first CTA and set to
+// DETOX_ERR_TIMEOUT when a bounded wait runs out; the partials of that CTA are then NaN.
+template <int M>
+__global__ void __launch_bounds__(kStgThreads, 1)
+sqdist_staged_kernel(const float* __restrict__ X, int64_t ld, int64_t d, const int32_t* __restrict__ rows,
+                     double* __restrict__ partial, int* __restrict__ status) {
+    constexpr int NP = M * (M - 1) / 2;
+    constexpr int kStages = stg_stages(M), kAhead = kStages - 1;
+    extern __shared__ __align__(128) uint8_t stage_mem[];      // [kStages][M][kStgPieces] pieces of 16 bytes
+    __shared__ uint64_t full[kStages], empty[kStages];
+    __shared__ int64_t roff[M];                                // element offset of row i, -1 for a zero row
+    __shared__ int abort_word;
+    __shared__ double red[kStgWarps][NP];
+    volatile int* abort_flag = &abort_word;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+    if (tid == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(&full[s], 1);
+            mbar_init(&empty[s], kStgWarps);
+        }
+        abort_word = 0;
+        mbar_fence_init();
+        if (blockIdx.x == 0) *status = 0;
+    }
+    if (tid < M) {
+        const int r = rows ? rows[tid] : tid;      // a negative entry of the row list stands for a zero row
+        roff[tid] = r < 0 ? -1 : (int64_t)r * ld;
+    }
+    __syncthreads();
+    uint32_t zero_rows = 0;                         // bit i: row i is a zero row
+#pragma unroll
+    for (int i = 0; i < M; ++i) zero_rows |= roff[i] < 0 ? 1u << i : 0u;
+    const int nreal = M - __popc(zero_rows);
+
+    const int64_t npiece_all = d / 4;              // whole 16-byte pieces per row; the last d % 4 columns come below
+    const int64_t ntiles = (npiece_all + kStgPieces - 1) / kStgPieces;
+    // this CTA's tiles: b, b + G, ...; `it` counts them; tile `it` goes through stage it % kStages
+    const int64_t my_tiles = ntiles > blockIdx.x ? (ntiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
+    constexpr uint32_t kRowBytes = kStgPieces * 16u, kStageBytes = M * kRowBytes;
+
+    // first warp: copy this CTA's tile number `it` (lane i takes row i) once its stage has been read
+    auto issue = [&](int64_t it) -> bool {
+        const int s = (int)(it % kStages);
+        const uint32_t ph = (uint32_t)(it / kStages) & 1u;
+        int ok = 1;
+        if (lane == 0) ok = mbar_wait(&empty[s], ph ^ 1u, abort_flag, status) ? 1 : 0;
+        if (!__shfl_sync(0xffffffffu, ok, 0)) return false;
+        const int64_t t = blockIdx.x + it * gridDim.x;
+        const int64_t left = npiece_all - t * kStgPieces;
+        const uint32_t bytes = (uint32_t)(left < kStgPieces ? left : kStgPieces) * 16u;
+        if (lane == 0) mbar_expect_tx(&full[s], bytes * (uint32_t)nreal);
+        __syncwarp();
+        if (lane < M && roff[lane] >= 0)
+            bulk_copy_g2s(stage_mem + (size_t)s * kStageBytes + (size_t)lane * kRowBytes,
+                          X + roff[lane] + t * (int64_t)(kStgPieces * 4), bytes, &full[s]);
+        return true;
+    };
+
+    float acc[NP];
+#pragma unroll
+    for (int p = 0; p < NP; ++p) acc[p] = 0.f;
+
+    bool alive = true;
+    if (warp == 0)
+        for (int64_t it = 0; it < kAhead && it < my_tiles && alive; ++it) alive = issue(it);
+    int s = 0;
+    uint32_t ph = 0;
+    for (int64_t it = 0; it < my_tiles && alive; ++it) {
+        if (warp == 0 && it + kAhead < my_tiles) alive = issue(it + kAhead);
+        if (!alive || !mbar_wait(&full[s], ph, abort_flag, status)) break;
+        const int64_t t = blockIdx.x + it * gridDim.x;
+        if (t * kStgPieces + tid < npiece_all) {
+            const uint8_t* src = stage_mem + (size_t)s * kStageBytes + (size_t)tid * 16u;
+            float v[M][4];
+#pragma unroll
+            for (int i = 0; i < M; ++i) {
+                float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (!((zero_rows >> i) & 1u)) x = *reinterpret_cast<const float4*>(src + (size_t)i * kRowBytes);
+                v[i][0] = x.x; v[i][1] = x.y; v[i][2] = x.z; v[i][3] = x.w;
+            }
+            int p = 0;
+#pragma unroll
+            for (int i = 0; i < M; ++i)
+#pragma unroll
+                for (int j = i + 1; j < M; ++j, ++p) {
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const float a = v[i][e] - v[j][e];
+                        acc[p] = fmaf(a, a, acc[p]);
+                    }
+                }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&empty[s]);   // one arrival per warp: the stage may be refilled
+        if (++s == kStages) { s = 0; ph ^= 1u; }
+    }
+    if (blockIdx.x == 0 && tid == 0) {
+        for (int64_t c = npiece_all * 4; c < d; ++c) {
+            int p = 0;
+#pragma unroll
+            for (int i = 0; i < M; ++i)
+#pragma unroll
+                for (int j = i + 1; j < M; ++j, ++p) {
+                    const float a = (roff[i] < 0 ? 0.f : X[roff[i] + c]) - (roff[j] < 0 ? 0.f : X[roff[j] + c]);
+                    acc[p] = fmaf(a, a, acc[p]);
+                }
+        }
+    }
+    // block reduction in fp64, fixed order
+#pragma unroll
+    for (int p = 0; p < NP; ++p) {
+        double v = (double)acc[p];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) v += __shfl_down_sync(0xffffffffu, v, o);
+        if (lane == 0) red[warp][p] = v;
+    }
+    __syncthreads();
+    const bool bad = *abort_flag != 0;
+    // a CTA that gave up may still have copies in flight: give them a bounded time to land before it goes away
+    if (bad) {
+        for (int i = 0; i < 64; ++i) __nanosleep(2000);
+        __syncthreads();
+    }
+    for (int p = tid; p < NP; p += kStgThreads) {
+        double v = 0.0;
+#pragma unroll
+        for (int w = 0; w < kStgWarps; ++w) v += red[w][p];
+        partial[(int64_t)blockIdx.x * NP + p] = bad ? __longlong_as_double(0x7ff8000000000000LL) : v;
     }
 }
 
@@ -249,10 +403,29 @@ int direct_blocks(int64_t d) {
     return (int)(b < 1 ? 1 : b);
 }
 
+// 9 to 16 rows that are 16-byte aligned and long enough take the staged kernel (one CTA per SM).
+bool use_staged(int m, const float* X, int64_t ld, int64_t d) {
+    return m >= 9 && m <= 16 && aligned16(X) && ld % 4 == 0 && d >= kStgMinCols;
+}
+
+// Launches the pair-partial kernel for M rows; *nblocks = how many partial vectors it writes.  `status` (device)
+// is cleared and used by the staged kernel only.
 template <int M>
 detox_status launch_direct_partials(const float* X, int64_t ld, int64_t d, const int32_t* rows, double* partial,
-                                    cudaStream_t s) {
+                                    int* status, int* nblocks, cudaStream_t s) {
+    if constexpr (M >= 9) {
+        if (use_staged(M, X, ld, d)) {
+            constexpr size_t smem = (size_t)stg_stages(M) * M * kStgPieces * 16;
+            if (cudaFuncSetAttribute(sqdist_staged_kernel<M>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
+                cudaSuccess)
+                return DETOX_ERR_CUDA;
+            *nblocks = kSMs;
+            sqdist_staged_kernel<M><<<kSMs, kStgThreads, smem, s>>>(X, ld, d, rows, partial, status);
+            return launch_status();
+        }
+    }
     const int nb = direct_blocks(d);
+    *nblocks = nb;
     const uintptr_t addr = reinterpret_cast<uintptr_t>(X);
     if ((addr & 15u) == 0 && ld % 4 == 0) sqdist_direct_kernel<M, 4><<<nb, kDirThreads, 0, s>>>(X, ld, d, rows, partial);
     else if ((addr & 7u) == 0 && ld % 2 == 0) sqdist_direct_kernel<M, 2><<<nb, kDirThreads, 0, s>>>(X, ld, d, rows, partial);
@@ -262,9 +435,9 @@ detox_status launch_direct_partials(const float* X, int64_t ld, int64_t d, const
 
 template <int M>
 detox_status launch_direct(const float* X, int64_t ld, int64_t d, const int32_t* rows, double* D, double* partial,
-                           cudaStream_t s) {
-    const int nb = direct_blocks(d);
-    detox_status st = launch_direct_partials<M>(X, ld, d, rows, partial, s);
+                           int* status, cudaStream_t s) {
+    int nb = 0;
+    detox_status st = launch_direct_partials<M>(X, ld, d, rows, partial, status, &nb, s);
     if (st != DETOX_OK) return st;
     sqdist_direct_reduce_kernel<<<(M * (M - 1) / 2 + 3) / 4, 128, 0, s>>>(partial, nb, M, D);
     return launch_status();
@@ -280,15 +453,17 @@ size_t dist_ws_bytes(int m, int64_t d) {
     return simt > tc ? simt : tc;
 }
 
+bool sqdist_partials_use_status(int m, const float* X, int64_t ld, int64_t d) { return use_staged(m, X, ld, d); }
+
 // 2 <= m <= 16: only the per-CTA pair partials (ws: [nblocks][m (m-1) / 2] fp64, pairs in row-major order of
-// i < j); *nblocks says how many there are.
+// i < j); *nblocks says how many there are.  When sqdist_partials_use_status() holds, the kernel clears the device
+// status word itself and sets it to DETOX_ERR_TIMEOUT if a bounded wait runs out (its partials are then NaN).
 detox_status launch_sqdist_partials(const float* X, int64_t ld, int m, int64_t d, const int32_t* rows, void* ws,
-                                    int* nblocks, cudaStream_t s) {
+                                    int* status, int* nblocks, cudaStream_t s) {
     double* partial = static_cast<double*>(ws);
-    *nblocks = direct_blocks(d);
     switch (m) {
 #define DETOX_CASE(M) \
-    case M: return launch_direct_partials<M>(X, ld, d, rows, partial, s);
+    case M: return launch_direct_partials<M>(X, ld, d, rows, partial, status, nblocks, s);
         DETOX_CASE(2) DETOX_CASE(3) DETOX_CASE(4) DETOX_CASE(5) DETOX_CASE(6) DETOX_CASE(7) DETOX_CASE(8)
         DETOX_CASE(9) DETOX_CASE(10) DETOX_CASE(11) DETOX_CASE(12) DETOX_CASE(13) DETOX_CASE(14) DETOX_CASE(15)
         DETOX_CASE(16)
@@ -305,7 +480,7 @@ detox_status launch_sqdist(const float* X, int64_t ld, int m, int64_t d, const i
         case 1:
             return cudaMemsetAsync(D, 0, sizeof(double), s) == cudaSuccess ? DETOX_OK : DETOX_ERR_CUDA;
 #define DETOX_CASE(M) \
-    case M: return launch_direct<M>(X, ld, d, rows, D, partial, s);
+    case M: return launch_direct<M>(X, ld, d, rows, D, partial, status, s);
         DETOX_CASE(2) DETOX_CASE(3) DETOX_CASE(4) DETOX_CASE(5) DETOX_CASE(6) DETOX_CASE(7) DETOX_CASE(8)
         DETOX_CASE(9) DETOX_CASE(10) DETOX_CASE(11) DETOX_CASE(12) DETOX_CASE(13) DETOX_CASE(14) DETOX_CASE(15)
         DETOX_CASE(16)

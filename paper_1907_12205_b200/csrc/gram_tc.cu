@@ -30,6 +30,7 @@
 #include <cuda.h>
 
 #include "common.cuh"
+#include "mbarrier.cuh"
 
 namespace detox {
 
@@ -42,7 +43,6 @@ constexpr int kMmaWarps = 2;                   // two issuing threads, so one's 
 constexpr int kTmaWarps = 2;                   // copy-issuing threads (the kernel for m > 128 uses the first only)
 constexpr int kTcThreads = kProdThreads + 32 * (kMmaWarps + kTmaWarps);
 constexpr size_t kSmemBudget = 227 * 1024;     // dynamic shared memory one CTA may have
-constexpr long long kWaitLimitCycles = 2000000000LL;  // ~1 s at the SM clock
 constexpr int64_t kSlabCols = 4096;          // columns accumulated in tensor memory before a drain
 constexpr int kMinReduceChunks = 32, kMaxReduceChunks = 256;
 
@@ -58,53 +58,6 @@ int reduce_chunks(int m, int nitems) {
 }
 
 // ------------------------------------------------------------------------------------ PTX wrappers
-
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ bool mbar_test(uint64_t* bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(smem_u32(bar)), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-// Hardware-assisted wait: the thread is suspended until the phase completes or a short
-// implementation-defined time passes, whichever is first.
-__device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(smem_u32(bar)), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-// Bounded wait (about a second of SM clocks).  Returns false, and raises the CTA-wide abort flag,
-// when the limit is hit; returns false at once when another thread has already given up.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status) {
-    if (mbar_try(bar, parity)) return true;
-    const long long start = clock64();
-    for (;;) {
-        if (mbar_try(bar, parity)) return true;
-        if (*abort_flag) return false;
-        if (clock64() - start > kWaitLimitCycles) break;
-    }
-    *abort_flag = 1;
-    atomicExch(status, (int)DETOX_ERR_TIMEOUT);
-    return false;
-}
 
 __device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -156,9 +109,6 @@ __device__ __forceinline__ void tmem_load16(uint32_t taddr, uint32_t (&v)[16]) {
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
-__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
 // 2-D tiled TMA load (no multicast): box at (x = column, y = row) -> shared memory, completion on `bar`.
 __device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
     asm volatile(

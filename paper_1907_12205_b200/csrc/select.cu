@@ -225,7 +225,7 @@ bulyan_select_kernel(const double* __restrict__ sorted_d, const int32_t* __restr
 // the per-CTA pair partials of the direct distance kernel are added up (one warp per pair, lanes
 // round-robin over the partials, then a fixed shuffle tree), every row's distances are ranked, the
 // selection runs on the lists in shared memory, and the chosen indices are mapped through the row
-// list when there is one.  The device status word is cleared on the way.
+// list when there is one.  The device status word is cleared on the way (unless `status` is null).
 constexpr int kSmallRows = 16;
 constexpr int kSmallThreads = 1024;
 constexpr int kSmallPartialsPerLane = 19;   // covers the direct distance kernel's 4 CTAs per SM
@@ -240,7 +240,7 @@ krum_small_kernel(const double* __restrict__ partial, int nblocks, int m, int f,
     __shared__ int32_t s_sorted_j[kSmallRows * kSmallRows];
     __shared__ int32_t s_pos_t[kSmallRows * kSmallRows];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    if (tid == 0) *status = 0;
+    if (tid == 0 && status) *status = 0;   // null: the distance kernel before this one owns the status word
 
     const int np = m * (m - 1) / 2;
     for (int p = warp; p < np; p += kSmallThreads / 32) {

@@ -153,3 +153,22 @@ def test_pipeline_replays_from_a_cuda_graph(a1, f, m_sel):
                                      w0.set_offsets, w0.set_members, oname, f, m_sel)
         assert winner.cpu().numpy().tolist() == ref["winner"].tolist()
         assert rel_l2(out.cpu().numpy(), ref["out"]) <= TOL
+
+
+@pytest.mark.parametrize("a1,f,m_sel", [("multikrum", 2, 9), ("bulyan", 2, 1)])
+def test_pipeline_long_rows_with_a_zero_vote_through_the_staged_distance_kernel(a1, f, m_sel):
+    """Twelve votes read through winner[] at a length that takes the bulk-copy distance kernel (9 to 16 rows, at
+    least 606,208 columns), with one group that has no majority (its vote is the zero row) and d % 4 = 1."""
+    import workloads as wl
+    spec = wl.WorkloadSpec("p", n=36, r=3, d=640_001, sigma=1e-3, q=0, group_jitter=0.05, seed=11)
+    w = wl.make_workload(spec)
+    grp = w.members[3:6]
+    w.X[int(grp[0]), 5] += 1.0
+    w.X[int(grp[1]), 640_000] += 1.0                   # three different rows in group 1
+    code = dx.AGG_MULTIKRUM if a1 == "multikrum" else dx.AGG_BULYAN
+    pipe = dx.Pipeline(36, 3, spec.d, w.members, dx.AGG_NONE, None, None, code, f, m_sel)
+    res = dx.detox_aggregate(pipe, w.X.to("cuda:0")[:, :spec.d])
+    ref = oracle.detox_aggregate(w.data().numpy(), w.members, 3, "none", None, None, a1, f, m_sel)
+    assert ref["winner"][1] == -1 and res["winner"].cpu().numpy().tolist() == ref["winner"].tolist()
+    assert res["sel"].cpu().numpy().tolist() == ref["sel"].tolist()
+    assert rel_l2(res["out"].cpu().numpy(), ref["out"]) <= TOL
