@@ -6,7 +6,7 @@
 // leaves the H smallest keys in lane 0 and the H largest in lane 1; the median is then the
 // maximum of lane 0's keys (for an even count, averaged with the minimum of lane 1's).  Sorting
 // two halves and splitting costs about half the comparators of one network over all m values.
-// For Bulyan's second stage (H a power of two) both halves are sorted with a bitonic merge and
+// For Bulyan's second stage both halves are sorted with a bitonic merge (sortnet.cuh: any H) and
 // laid out in shared memory for the data-dependent window search.
 #include "median_impl.cuh"
 
@@ -45,7 +45,7 @@ colselect_pair_kernel(const float* __restrict__ X, int64_t ld, int m, int64_t d,
     int32_t key[kHalf];
     // Lane 0 always holds kHalf rows.  Lane 1 holds `extra` rows, at least kSure of them when the median picks
     // kHalf (half of m rounded up to 8), so only its top slots pay for the clamped row and the padding test.
-    constexpr int kSure = TRIM ? 0 : kHalf - 16;
+    constexpr int kSure = kHalf - 16;
     // the test for a row list is taken once, outside the loads: a per-load test would serialise them
     if (rows) {
 #pragma unroll
@@ -93,25 +93,23 @@ colselect_pair_kernel(const float* __restrict__ X, int64_t ld, int m, int64_t d,
         return;
     }
 
-    // each lane's 128 keys form a bitonic sequence: sort them ascending
+    // Lane 0's keys now rise and then fall, lane 1's fall and then rise.  Lane 1 complements its keys, which
+    // turns its sequence into a rise-then-fall one as well, so both lanes run the same merge network; lane 1's
+    // keys come out in descending order of the real values.
+    const int32_t flip = hsel ? -1 : 0;
 #pragma unroll
-    for (int s = kHalf / 2; s >= 1; s >>= 1) {
-#pragma unroll
-        for (int i = 0; i < kHalf; ++i) {
-            if ((i & s) == 0) {
-                const int32_t lo = min(key[i], key[i + s]);
-                const int32_t hi = max(key[i], key[i + s]);
-                key[i] = lo;
-                key[i + s] = hi;
-            }
-        }
-    }
-    // position p of the 256 sorted keys -> sorted[p * kPairCols + slot]; the slot is rotated by 16 for the
+    for (int i = 0; i < kHalf; ++i) key[i] ^= flip;
+    bitonic_merge_registers<kHalf>(key);
+    // position p of the 2 kHalf sorted keys -> sorted[p * kPairCols + slot]; the slot is rotated by 16 for the
     // upper half so that the two lanes of a pair never hit the same bank
     {
+        constexpr BitonicMergeNet<kHalf> net{};
         const int slot = (cidx + hsel * 16) & (kPairCols - 1);
 #pragma unroll
-        for (int i = 0; i < kHalf; ++i) sorted[(hsel * kHalf + i) * kPairCols + slot] = key[i];
+        for (int i = 0; i < kHalf; ++i) {
+            const int p = hsel ? 2 * kHalf - 1 - net.pos[i] : net.pos[i];
+            sorted[p * kPairCols + slot] = key[i] ^ flip;
+        }
     }
     __syncwarp();
     auto at = [&](int p) { return sorted[p * kPairCols + ((cidx + (p >= kHalf ? 16 : 0)) & (kPairCols - 1))]; };
@@ -147,25 +145,22 @@ detox_status launch_pair(const float* X, int64_t ld, int m, int64_t d, const int
     if (bx > 0x7fffffffLL) return DETOX_ERR_UNSUPPORTED;
     if (beta == 0) {
         colselect_pair_kernel<H, false><<<(unsigned)bx, kPairThreads, 0, s>>>(X, ld, m, d, rows, beta, out);
-    } else if constexpr ((H & (H - 1)) == 0) {
+    } else {
         const size_t smem = (size_t)2 * H * kPairCols * sizeof(int32_t);
         if (cudaFuncSetAttribute(colselect_pair_kernel<H, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)smem) != cudaSuccess)
             return DETOX_ERR_CUDA;
         colselect_pair_kernel<H, true><<<(unsigned)bx, kPairThreads, smem, s>>>(X, ld, m, d, rows, beta, out);
-    } else {
-        return DETOX_ERR_UNSUPPORTED;
     }
     return launch_status();
 }
 
 }  // namespace
 
-// 128 < m <= 256.  Median: H = half of m rounded up to 8; Bulyan stage 2: H = 128 (a power of two).
+// 128 < m <= 256.  H = half of m rounded up to 8.
 detox_status launch_pair_select(const float* X, int64_t ld, int m, int64_t d, const int32_t* rows, int beta,
                                 float* out, cudaStream_t s) {
-    int H = ((m + 1) / 2 + 7) / 8 * 8;
-    if (beta != 0) H = 128;
+    const int H = ((m + 1) / 2 + 7) / 8 * 8;
     switch (H) {
 #define DETOX_CASE(HH) \
     case HH: return launch_pair<HH>(X, ld, m, d, rows, beta, out, s);

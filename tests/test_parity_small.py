@@ -128,7 +128,11 @@ def test_coord_median_special_values(m):
 
 
 @pytest.mark.parametrize("m,trim", [(5, 1), (7, 0), (12, 3), (15, 7), (27, 6), (35, 8), (64, 16), (105, 26), (225, 56),
-                                    (300, 75)])
+                                    (300, 75),
+                                    # two lanes per coordinate: every network half size from 72 to 128, both parities
+                                    (129, 1), (130, 40), (144, 0), (145, 72), (159, 20), (160, 79), (176, 3), (181, 22),
+                                    (192, 50), (200, 99), (209, 10), (224, 100), (240, 1), (241, 120), (255, 60),
+                                    (256, 127)])
 def test_trimmed_mean_matches_oracle(m, trim):
     X = (np.random.default_rng(m).standard_normal((m, 2000 + m)) * 1e-3).astype(np.float32)
     X[0] *= -100
