@@ -14,12 +14,13 @@
 // and the transform warps write both MMA operands (see the staged kernel); above, the copies land directly in
 // the swizzled hi tile (see the wide kernel).
 // Column blocks are dealt round-robin to the CTAs and every 4096 columns of a CTA form a slab; at the end
-// of a slab the accumulator is drained to a per-slab fp32 partial in global memory and the slabs are
-// added in fp64 in a fixed order afterwards, so the long sum never lives in one fp32 accumulator and
+// of a slab the accumulator is drained into an fp32 partial in global memory (four consecutive slabs of a CTA
+// share one: the drain adds to what the slab before left there) and the partials are added in fp64 in a fixed
+// order afterwards, so the long sum never lives in one fp32 accumulator and
 // the result is deterministic.
 //
 // The tensor cores add into their fp32 accumulator by truncation, so a long same-sign sum (a row with
-// itself, or with a copy of itself) comes out low by a few 1e-5 relative per slab.  The producers
+// itself, or with a copy of itself) comes out low by about 1e-5 relative per 4096 columns.  The producers
 // therefore also accumulate each row's exact squared norm per slab on the CUDA cores; the final
 // reduction rescales every slab's T_ij by the mean of (exact norm / tensor-core norm) of rows i and
 // j.  The diagonal becomes exact, a pair of identical rows keeps distance zero, and entries
@@ -44,6 +45,7 @@ constexpr int kTmaWarps = 2;                   // copy-issuing threads (the kern
 constexpr int kTcThreads = kProdThreads + 32 * (kMmaWarps + kTmaWarps);
 constexpr size_t kSmemBudget = 227 * 1024;     // dynamic shared memory one CTA may have
 constexpr int64_t kSlabCols = 4096;          // columns accumulated in tensor memory before a drain
+constexpr int kItemSlabs = 4;                // consecutive slabs of a CTA that are added into one output slot
 constexpr int kMinReduceChunks = 32, kMaxReduceChunks = 256;
 
 // Slab slots are added up in `chunks` independent groups (one CTA per group and pair of 32-row blocks), enough
@@ -175,7 +177,7 @@ WidePlan wide_plan(int m, int64_t d) {
     p.nkb_total = (int)ceil_div(d, (int64_t)kKB);
     p.grid = p.nkb_total < kSMs ? p.nkb_total : kSMs;
     const int per_cta = (p.nkb_total + p.grid - 1) / p.grid;
-    p.nitems = p.grid * (int)ceil_div((int64_t)per_cta, kSlabCols / kKB);
+    p.nitems = p.grid * (int)ceil_div(ceil_div((int64_t)per_cta, kSlabCols / kKB), (int64_t)kItemSlabs);
     p.smem_bytes = (size_t)p.stage_bytes * p.stages + 1024 /*barriers*/ + 1024 /*alignment slack*/;
     return p;
 }
@@ -268,7 +270,9 @@ gram_wide_kernel(const __grid_constant__ CUtensorMap xmap, int m, uint32_t lo_of
                 if (lane == 0) mbar_arrive(&sm->full[s]);   // one arrival per transform warp
                 if (++s == stages) { s = 0; ph ^= 1u; }
             }
-            const int item = (int)blockIdx.x + li * (int)gridDim.x;
+            // output slot of this slab, and whether the slab opens / closes it
+            const int item = (int)blockIdx.x + (li / kItemSlabs) * (int)gridDim.x;
+            const bool opens = li % kItemSlabs == 0, closes = li % kItemSlabs == kItemSlabs - 1 || li == my_items - 1;
 
             // ---- end of a slab: exact squared norms (the 8 lanes that share a row add up) ...
 #pragma unroll
@@ -278,8 +282,10 @@ gram_wide_kernel(const __grid_constant__ CUtensorMap xmap, int m, uint32_t lo_of
                 v += __shfl_xor_sync(0xffffffffu, v, 2);
                 v += __shfl_xor_sync(0xffffffffu, v, 4);
                 const int row = row0 + (kProdThreads / 8) * j;
-                if (c == 0 && row < m) norms[(int64_t)item * m + row] = v;
-                sq[j] = 0ull;
+                if (closes) {
+                    if (c == 0 && row < m) norms[(int64_t)item * m + row] = v;
+                    sq[j] = 0ull;
+                }
             }
             // ... and the accumulator drain: warp w reads TMEM lanes 32*(w%4)..+31 (accumulator row i of a half sits
             // in lane i); the warps that share a lane quarter take 16-column chunks round-robin
@@ -295,10 +301,15 @@ gram_wide_kernel(const __grid_constant__ CUtensorMap xmap, int m, uint32_t lo_of
                     if (row < m) {
                         float* dstp = out_item + (int64_t)row * ncol + cc * 16;
 #pragma unroll
-                        for (int j = 0; j < 16; j += 4)
-                            *reinterpret_cast<float4*>(dstp + j) =
-                                make_float4(__uint_as_float(v[j]), __uint_as_float(v[j + 1]), __uint_as_float(v[j + 2]),
-                                            __uint_as_float(v[j + 3]));
+                        for (int j = 0; j < 16; j += 4) {
+                            float4 o = make_float4(__uint_as_float(v[j]), __uint_as_float(v[j + 1]), __uint_as_float(v[j + 2]),
+                                                   __uint_as_float(v[j + 3]));
+                            if (!opens) {   // this thread wrote the slot's earlier slabs itself
+                                const float4 e = *reinterpret_cast<const float4*>(dstp + j);
+                                o.x += e.x; o.y += e.y; o.z += e.z; o.w += e.w;
+                            }
+                            *reinterpret_cast<float4*>(dstp + j) = o;
+                        }
                     }
                 }
             }
@@ -307,7 +318,7 @@ gram_wide_kernel(const __grid_constant__ CUtensorMap xmap, int m, uint32_t lo_of
             if (lane == 0) mbar_arrive(&sm->accum_empty);
         }
         // slots of slabs this CTA does not have (it owns one K-block fewer than others) read as zero
-        for (int l2 = my_items; l2 * (int)gridDim.x < nitems; ++l2) {
+        for (int l2 = (my_items + kItemSlabs - 1) / kItemSlabs; l2 * (int)gridDim.x < nitems; ++l2) {
             const int64_t item = (int64_t)blockIdx.x + (int64_t)l2 * gridDim.x;
             for (int e = tid; e < m * ncol; e += kProdThreads) partial[item * m * ncol + e] = 0.f;
             for (int e = tid; e < m; e += kProdThreads) norms[item * m + e] = 0.f;
@@ -421,7 +432,7 @@ StagedPlan staged_plan(int m, int64_t d) {
     p.nst_total = (int)ceil_div(d, (int64_t)kStageCols);
     p.grid = p.nst_total < kSMs ? p.nst_total : kSMs;
     const int per_cta = (p.nst_total + p.grid - 1) / p.grid;
-    p.nitems = p.grid * (int)ceil_div((int64_t)per_cta, kSlabCols / kStageCols);
+    p.nitems = p.grid * (int)ceil_div(ceil_div((int64_t)per_cta, kSlabCols / kStageCols), (int64_t)kItemSlabs);
     p.smem_bytes = (size_t)p.nstg * p.stg_bytes + p.nmst * mst_bytes + 1024 /*barriers*/ + 1024 /*alignment slack*/;
     return p;
 }
@@ -539,7 +550,9 @@ gram_staged_kernel(const __grid_constant__ CUtensorMap xmap, int m, uint32_t stg
                 ms += LX;
                 if (ms >= nmst) { ms -= nmst; mph ^= 1u; }
             }
-            const int item = (int)blockIdx.x + li * (int)gridDim.x;
+            // output slot of this slab, and whether the slab opens / closes it
+            const int item = (int)blockIdx.x + (li / kItemSlabs) * (int)gridDim.x;
+            const bool opens = li % kItemSlabs == 0, closes = li % kItemSlabs == kItemSlabs - 1 || li == my_items - 1;
 
             // ---- end of a slab: this group's share of the exact squared norms (the 16 lanes that share a row
             // add up; the reduction kernel adds the groups) ...
@@ -551,8 +564,10 @@ gram_staged_kernel(const __grid_constant__ CUtensorMap xmap, int m, uint32_t stg
                 v += __shfl_xor_sync(0xffffffffu, v, 4);
                 v += __shfl_xor_sync(0xffffffffu, v, 8);
                 const int row = row0 + (kGroupThreads / 16) * j;
-                if (q == 0 && row < m) norms[((int64_t)item * LX + group) * m + row] = v;
-                sq[j] = 0ull;
+                if (closes) {
+                    if (q == 0 && row < m) norms[((int64_t)item * LX + group) * m + row] = v;
+                    sq[j] = 0ull;
+                }
             }
             // ... and the accumulator drain: warp w reads TMEM lanes 32*(w%4)..+31; the warps that share a
             // lane quarter take 16-column chunks round-robin
@@ -578,8 +593,14 @@ gram_staged_kernel(const __grid_constant__ CUtensorMap xmap, int m, uint32_t stg
                 if (row < m) {
                     float* dstp = out_item + (int64_t)row * ncol + cc * 16;
 #pragma unroll
-                    for (int j = 0; j < 16; j += 4)
-                        *reinterpret_cast<float4*>(dstp + j) = make_float4(acc[j], acc[j + 1], acc[j + 2], acc[j + 3]);
+                    for (int j = 0; j < 16; j += 4) {
+                        float4 o = make_float4(acc[j], acc[j + 1], acc[j + 2], acc[j + 3]);
+                        if (!opens) {   // this thread wrote the slot's earlier slabs itself
+                            const float4 e = *reinterpret_cast<const float4*>(dstp + j);
+                            o.x += e.x; o.y += e.y; o.z += e.z; o.w += e.w;
+                        }
+                        *reinterpret_cast<float4*>(dstp + j) = o;
+                    }
                 }
             }
             tc_fence_before();
@@ -587,7 +608,7 @@ gram_staged_kernel(const __grid_constant__ CUtensorMap xmap, int m, uint32_t stg
             if (lane == 0) mbar_arrive(&sm->accum_empty);
         }
         // slots of slabs this CTA does not have (it owns one stage fewer than others) read as zero
-        for (int l2 = my_items; l2 * (int)gridDim.x < nitems; ++l2) {
+        for (int l2 = (my_items + kItemSlabs - 1) / kItemSlabs; l2 * (int)gridDim.x < nitems; ++l2) {
             const int64_t item = (int64_t)blockIdx.x + (int64_t)l2 * gridDim.x;
             for (int e = tid; e < m * ncol; e += kProdThreads) partial[item * m * ncol + e] = 0.f;
             for (int e = tid; e < m * LX; e += kProdThreads) norms[item * LX * m + e] = 0.f;

@@ -68,7 +68,7 @@ def test_multikrum_fallback_paths(m, d, f, m_sel, odd):
 @pytest.mark.parametrize("m,d", [
     (17, 63), (18, 64), (32, 65), (33, 4097), (63, 9473), (64, 129), (65, 4100), (80, 9472 + 31), (96, 2000),
     (127, 3001), (128, 1000), (129, 1000), (144, 2049), (240, 777), (256, 640),
-    (20, 700_001), (100, 650_003), (140, 610_000)])       # last three: more than one 4096-column slab per CTA
+    (20, 2_500_001), (100, 2_450_003), (140, 2_430_000)])   # last three: more than one output slot (4 x 4096 columns) per CTA
 def test_tensor_core_distance_kernels_at_their_size_boundaries(m, d):
     """Row counts on both sides of every switch of the tensor-core kernels (64 and 128 rows, tile sizes that are
     multiples of 16) and column counts around the 32- and 64-column copies, with a ragged tail."""
