@@ -20,10 +20,11 @@
  *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
  *   - Workspace pointers must be 256-byte aligned; sizes come from the *_workspace_bytes helpers.
  *   - Errors: argument problems are reported before anything is launched; a failed launch returns
- *     DETOX_ERR_CUDA.  Nothing aborts or throws.  Multi-Krum and Bulyan on 17 to 256 rows run a
- *     tensor-core kernel whose device-side waits are bounded: should one run out, the first int32 of
- *     the workspace passed to agg_multikrum / agg_bulyan reads DETOX_ERR_TIMEOUT after the stream
- *     has been synchronised (0 otherwise) and the outputs are not valid.
+ *     DETOX_ERR_CUDA.  Nothing aborts or throws.  Multi-Krum and Bulyan run kernels that wait on
+ *     asynchronous copies (9 to 16 long rows) or on the tensor cores (17 to 256 rows); every such
+ *     device-side wait is bounded: should one run out, the first int32 of the workspace passed to
+ *     agg_multikrum / agg_bulyan reads DETOX_ERR_TIMEOUT after the stream has been synchronised
+ *     (0 otherwise) and the outputs are not valid.
  *   - Ranking of values (medians, "closest to the median") uses the total order
  *     -NaN < -Inf < ... < -0 < +0 < ... < +Inf < +NaN on fp32 bit patterns.
  */
