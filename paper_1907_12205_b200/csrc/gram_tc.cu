@@ -400,8 +400,12 @@ constexpr int kStageCols = 64;                       // columns per staging stag
 constexpr int kKbPerStage = kStageCols / kKB;
 constexpr int kMaxStg = 8, kMaxMst = 4;
 
+// Stages per slab: 4096 columns, a multiple of the transform groups and of the MMA-issuing threads.
+__host__ __device__ constexpr int staged_slab_stages(int) { return (int)(kSlabCols / kStageCols); }
+
 struct StagedPlan {
     int mrows, box_rows, ncol, tmem_cols;
+    int nmma;                    // MMA-issuing threads: four up to 64 rows, else two
     int groups;                  // groups of transform warps, each on a stage of its own
     int nstg, nmst;              // staging stages, MMA stages
     uint32_t stg_bytes;          // box_rows x 256 bytes
@@ -416,8 +420,9 @@ StagedPlan staged_plan(int m, int64_t d) {
     p.mrows = m <= 64 ? 64 : 128;
     p.box_rows = (m + 7) / 8 * 8;
     p.ncol = (m + 15) / 16 * 16;
+    p.nmma = m <= 64 ? 4 : 2;
     p.tmem_cols = 32;
-    while (p.tmem_cols < kMmaWarps * 2 * p.ncol) p.tmem_cols <<= 1;
+    while (p.tmem_cols < p.nmma * 2 * p.ncol) p.tmem_cols <<= 1;
     p.stg_bytes = (uint32_t)p.box_rows * (uint32_t)kStageCols * 4u;
     p.tile_bytes = 2u * (uint32_t)p.ncol * 128u;
     const size_t mst_bytes = (size_t)kKbPerStage * p.tile_bytes;
@@ -429,10 +434,13 @@ StagedPlan staged_plan(int m, int64_t d) {
     p.nstg = (int)(left / p.stg_bytes);
     if (p.nstg > kMaxStg) p.nstg = kMaxStg;
     while (p.nstg > 2 && (size_t)p.nstg * p.stg_bytes > 112 * 1024) --p.nstg;   // ~100 KB in flight saturates HBM
+    // With two transform groups a staging slot must always hold stages of the same group (an even slot count), so that
+    // each copy-issuing thread follows one group only: a parity wait cannot tell phases two apart.
+    if (p.groups == 2) p.nstg &= ~1;
     p.nst_total = (int)ceil_div(d, (int64_t)kStageCols);
     p.grid = p.nst_total < kSMs ? p.nst_total : kSMs;
     const int per_cta = (p.nst_total + p.grid - 1) / p.grid;
-    p.nitems = p.grid * (int)ceil_div(ceil_div((int64_t)per_cta, kSlabCols / kStageCols), (int64_t)kItemSlabs);
+    p.nitems = p.grid * (int)ceil_div(ceil_div((int64_t)per_cta, (int64_t)staged_slab_stages(p.nmma)), (int64_t)kItemSlabs);
     p.smem_bytes = (size_t)p.nstg * p.stg_bytes + p.nmst * mst_bytes + 1024 /*barriers*/ + 1024 /*alignment slack*/;
     return p;
 }
@@ -448,9 +456,15 @@ struct StagedSmem {
     int abort_flag;
 };
 
-// LX = groups of transform warps; J = 16-byte pieces per transform thread and stage (m * 16 / (512 / LX), rounded up)
-template <int J, int LX>
-__global__ void __launch_bounds__(kTcThreads, 1)
+// LX = groups of transform warps; J = 16-byte pieces per transform thread and stage (m * 16 / (512 / LX), rounded up);
+// NMMA = MMA-issuing threads, each with an accumulator of its own.  Up to 64 rows an MMA sits on its 59-cycle floor and
+// a stage's eight MMAs take less time than one thread's wait / fence / commit around them: four threads keep the
+// tensor pipe fed where two left it idle a quarter of the time.  NMMA must be a multiple of LX and divide the number
+// of MMA slots, so that a thread always serves the same slots and the same transform group: a parity wait tells two
+// consecutive phases of a barrier apart, no more, and a thread that followed one group's stages could otherwise get
+// more than a phase ahead of the other group's.
+template <int J, int LX, int NMMA>
+__global__ void __launch_bounds__(kProdThreads + 32 * (NMMA + kTmaWarps), 1)
 gram_staged_kernel(const __grid_constant__ CUtensorMap xmap, int m, uint32_t stg_bytes, uint32_t tile_bytes, int mrows,
                    int ncol, int tmem_cols, int nstg, int nmst, int nst_total, int nitems, float* __restrict__ partial,
                    float* __restrict__ norms, int* __restrict__ status) {
@@ -463,6 +477,7 @@ gram_staged_kernel(const __grid_constant__ CUtensorMap xmap, int m, uint32_t stg
     volatile int* abort_flag = &sm->abort_flag;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    constexpr int kThreads = kProdThreads + 32 * (NMMA + kTmaWarps);
     constexpr int kGroupThreads = kProdThreads / LX, kGroupWarps = kProdWarps / LX;
 
     if (tid == 0) {
@@ -474,13 +489,13 @@ gram_staged_kernel(const __grid_constant__ CUtensorMap xmap, int m, uint32_t stg
             mbar_init(&sm->mst_full[s], kGroupWarps);
             mbar_init(&sm->mst_empty[s], 1);
         }
-        mbar_init(&sm->accum_full, kMmaWarps);
+        mbar_init(&sm->accum_full, NMMA);
         mbar_init(&sm->accum_empty, kProdWarps);
         sm->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     // rows m .. 2 ncol of the MMA tiles are never written: clear the MMA stages once so that they read as zeros
-    for (uint32_t off = (uint32_t)tid * 16u; off < mst_bytes * (uint32_t)nmst; off += kTcThreads * 16u)
+    for (uint32_t off = (uint32_t)tid * 16u; off < mst_bytes * (uint32_t)nmst; off += kThreads * 16u)
         *reinterpret_cast<uint4*>(mst_base + off) = make_uint4(0u, 0u, 0u, 0u);
     fence_proxy_async_smem();
     if (warp == 0) tmem_alloc(&sm->tmem_base, (uint32_t)tmem_cols);
@@ -492,8 +507,9 @@ gram_staged_kernel(const __grid_constant__ CUtensorMap xmap, int m, uint32_t stg
     // This CTA owns the 64-column stages b, b + G, b + 2G, ... (b = blockIdx.x, G = gridDim.x), t = 0 .. total-1 in
     // its own count; stage t lands in staging slot t % nstg and is transformed into MMA slot t % nmst; a slab is
     // kStagesPerSlab consecutive ones (the last slab may be shorter) and goes to slot b + G * (slab number).
-    constexpr int kStagesPerSlab = (int)(kSlabCols / kStageCols);
-    static_assert(kStagesPerSlab % LX == 0 && kStagesPerSlab % kMmaWarps == 0, "slabs start at every role's own offset");
+    constexpr int kStagesPerSlab = staged_slab_stages(NMMA);
+    static_assert(kStagesPerSlab % LX == 0 && kStagesPerSlab % NMMA == 0, "slabs start at every role's own offset");
+    static_assert(NMMA % LX == 0 && kMaxMst % NMMA == 0, "an MMA-issuing thread serves the same slots and group throughout");
     const int total = (nst_total - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
     const int my_items = (total + kStagesPerSlab - 1) / kStagesPerSlab;
     const int last_nst = total - (my_items - 1) * kStagesPerSlab;
@@ -579,7 +595,7 @@ gram_staged_kernel(const __grid_constant__ CUtensorMap xmap, int m, uint32_t stg
             const int row = mrows == 64 ? (lane < 16 ? quarter * 16 + lane : m) : quarter * 32 + lane;
             // the hi.hi and hi.2lo parts of every issuing thread's accumulator (a slab of a single stage leaves the
             // second thread's accumulator untouched: skip it)
-            const int nparts = 2 * (nst < kMmaWarps ? nst : kMmaWarps);
+            const int nparts = 2 * (nst < NMMA ? nst : NMMA);
             for (int cc = warp >> 2; cc * 16 < ncol; cc += kProdWarps / 4) {   // ncol is a multiple of 16
                 float acc[16];
 #pragma unroll
@@ -613,10 +629,10 @@ gram_staged_kernel(const __grid_constant__ CUtensorMap xmap, int m, uint32_t stg
             for (int e = tid; e < m * ncol; e += kProdThreads) partial[item * m * ncol + e] = 0.f;
             for (int e = tid; e < m * LX; e += kProdThreads) norms[item * LX * m + e] = 0.f;
         }
-    } else if (warp >= kProdWarps + kMmaWarps) {
+    } else if (warp >= kProdWarps + NMMA) {
         // ------------------------------------------------ the TMA threads: thread l issues the stages l, l + kTmaWarps, ...
         if (lane == 0) {
-            const int l = warp - (kProdWarps + kMmaWarps);
+            const int l = warp - (kProdWarps + NMMA);
             int last = -1;
             int s = l % nstg;
             uint32_t ph = (uint32_t)(l / nstg) & 1u;
@@ -640,8 +656,8 @@ gram_staged_kernel(const __grid_constant__ CUtensorMap xmap, int m, uint32_t stg
             }
         }
     } else if (lane == 0) {
-        // ------------------------------------------------ the MMA threads (lane 0 of the two warps after the
-        // transform warps): they alternate stages and own one accumulator of 2 ncol columns each
+        // ------------------------------------------------ the MMA threads (lane 0 of the NMMA warps after the
+        // transform warps): they take the stages in turn and own one accumulator of 2 ncol columns each
         const int g = warp - kProdWarps;
         const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)((2 * ncol) >> 3) << 17) | ((uint32_t)(mrows >> 4) << 24);
         const uint32_t dcol = tmem_base + (uint32_t)(g * 2 * ncol);
@@ -657,7 +673,7 @@ gram_staged_kernel(const __grid_constant__ CUtensorMap xmap, int m, uint32_t stg
                 const uint32_t my_ph = ph;
                 const bool skip = turn != g;
                 if (++s == nmst) { s = 0; ph ^= 1u; }
-                turn ^= 1;
+                if (++turn == NMMA) turn = 0;
                 if (skip) continue;
                 mbar_wait(&sm->mst_full[my_s], my_ph, abort_flag, status);
                 tc_fence_after();
@@ -835,15 +851,16 @@ detox_status launch_wide(const WidePlan& p, const CUtensorMap& xmap, int m, floa
     return launch_status();
 }
 
-template <int J, int LX>
+template <int J, int LX, int NMMA>
 detox_status launch_staged(const StagedPlan& p, const CUtensorMap& xmap, int m, float* partial, float* norms, int* status,
                            cudaStream_t s) {
-    if (cudaFuncSetAttribute(gram_staged_kernel<J, LX>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem_bytes) !=
-        cudaSuccess)
+    if (cudaFuncSetAttribute(gram_staged_kernel<J, LX, NMMA>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)p.smem_bytes) != cudaSuccess)
         return DETOX_ERR_CUDA;
-    gram_staged_kernel<J, LX><<<p.grid, kTcThreads, p.smem_bytes, s>>>(xmap, m, p.stg_bytes, p.tile_bytes, p.mrows, p.ncol,
-                                                                       p.tmem_cols, p.nstg, p.nmst, p.nst_total, p.nitems,
-                                                                       partial, norms, status);
+    constexpr int kThreads = kProdThreads + 32 * (NMMA + kTmaWarps);
+    gram_staged_kernel<J, LX, NMMA><<<p.grid, kThreads, p.smem_bytes, s>>>(xmap, m, p.stg_bytes, p.tile_bytes, p.mrows, p.ncol,
+                                                                          p.tmem_cols, p.nstg, p.nmst, p.nst_total,
+                                                                          p.nitems, partial, norms, status);
     return launch_status();
 }
 
@@ -896,14 +913,14 @@ detox_status launch_sqdist_tc(const float* X, int64_t ld, int m, int64_t d, doub
         // 16-byte pieces per transform thread and stage: m * 16 / (threads of a group), rounded up
         const int gt = kProdThreads / p.groups;
         const int per_thread = (m * (kStageCols / 4) + gt - 1) / gt;
-        if (p.groups == 2) {
-            if (per_thread <= 2) st = launch_staged<2, 2>(p, xmap, m, partial, norms, status, s);
-            else if (per_thread <= 3) st = launch_staged<3, 2>(p, xmap, m, partial, norms, status, s);
-            else st = launch_staged<4, 2>(p, xmap, m, partial, norms, status, s);
+        if (p.groups == 2) {   // up to 64 rows: two transform groups, four MMA-issuing threads
+            if (per_thread <= 2) st = launch_staged<2, 2, 4>(p, xmap, m, partial, norms, status, s);
+            else if (per_thread <= 3) st = launch_staged<3, 2, 4>(p, xmap, m, partial, norms, status, s);
+            else st = launch_staged<4, 2, 4>(p, xmap, m, partial, norms, status, s);
         } else {
-            if (per_thread <= 2) st = launch_staged<2, 1>(p, xmap, m, partial, norms, status, s);
-            else if (per_thread <= 3) st = launch_staged<3, 1>(p, xmap, m, partial, norms, status, s);
-            else st = launch_staged<4, 1>(p, xmap, m, partial, norms, status, s);
+            if (per_thread <= 2) st = launch_staged<2, 1, 2>(p, xmap, m, partial, norms, status, s);
+            else if (per_thread <= 3) st = launch_staged<3, 1, 2>(p, xmap, m, partial, norms, status, s);
+            else st = launch_staged<4, 1, 2>(p, xmap, m, partial, norms, status, s);
         }
     } else {
         const WidePlan p = wide_plan(m, d);
