@@ -116,6 +116,13 @@ constexpr int64_t kStgMinCols = (int64_t)kSMs * kStgPieces * 4 * 4;   // at leas
 
 __host__ __device__ constexpr int stg_stages(int M) { return M <= 12 ? 4 : 3; }   // 16 rows x 4 KB x 3 = 192 KB
 
+// Two fp32 differences in one instruction (same rounding as the scalar subtraction).
+__device__ __forceinline__ uint64_t sub_f32x2(uint64_t a, uint64_t b) {
+    uint64_t r;
+    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+
 __device__ __forceinline__ void bulk_copy_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar))
@@ -196,23 +203,21 @@ sqdist_staged_kernel(const float* __restrict__ X, int64_t ld, int64_t d, const i
         const int64_t t = blockIdx.x + it * gridDim.x;
         if (t * kStgPieces + tid < npiece_all) {
             const uint8_t* src = stage_mem + (size_t)s * kStageBytes + (size_t)tid * 16u;
-            float v[M][4];
+            ulonglong2 v[M];                        // four columns of every row as two packed pairs
 #pragma unroll
             for (int i = 0; i < M; ++i) {
-                float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (!((zero_rows >> i) & 1u)) x = *reinterpret_cast<const float4*>(src + (size_t)i * kRowBytes);
-                v[i][0] = x.x; v[i][1] = x.y; v[i][2] = x.z; v[i][3] = x.w;
+                v[i] = make_ulonglong2(0ull, 0ull);
+                if (!((zero_rows >> i) & 1u)) v[i] = *reinterpret_cast<const ulonglong2*>(src + (size_t)i * kRowBytes);
             }
             int p = 0;
 #pragma unroll
             for (int i = 0; i < M; ++i)
 #pragma unroll
                 for (int j = i + 1; j < M; ++j, ++p) {
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const float a = v[i][e] - v[j][e];
-                        acc[p] = fmaf(a, a, acc[p]);
-                    }
+                    const uint64_t d01 = sub_f32x2(v[i].x, v[j].x), d23 = sub_f32x2(v[i].y, v[j].y);
+                    const float a0 = __uint_as_float((uint32_t)d01), a1 = __uint_as_float((uint32_t)(d01 >> 32));
+                    const float a2 = __uint_as_float((uint32_t)d23), a3 = __uint_as_float((uint32_t)(d23 >> 32));
+                    acc[p] = fmaf(a3, a3, fmaf(a2, a2, fmaf(a1, a1, fmaf(a0, a0, acc[p]))));
                 }
         }
         __syncwarp();
