@@ -302,6 +302,26 @@ def test_pipeline_no_majority_group_becomes_zero_vote():
     assert rel_l2(res["out"].cpu().numpy(), ref["out"]) <= TOL
 
 
+@pytest.mark.parametrize("a1,f", [(dx.AGG_COORD_MEDIAN, 0), (dx.AGG_TRIMMED_MEAN, 1), (dx.AGG_TRIMMED_MEAN, 3)])
+@pytest.mark.parametrize("n", [15, 27, 105])
+def test_pipeline_order_statistics_over_votes_with_a_zero_vote(a1, f, n):
+    """The order-statistic kernels read the votes through winner[]; a group without a majority is a zero row there
+    (the row list holds -1), which takes the masked loads instead of the plain ones."""
+    if 2 * f >= n // 3:
+        pytest.skip("nothing would be left of the votes")
+    spec = wl.WorkloadSpec("p", n=n, r=3, d=5003, sigma=1e-2, q=0, seed=n)
+    w = wl.make_workload(spec)
+    grp = w.members[3:6]
+    w.X[int(grp[0]), 0] += 1.0
+    w.X[int(grp[2]), 5002] -= 1.0                      # three different rows in group 1
+    res, ref = run_pipeline(w, dx.AGG_NONE, a1, f)
+    assert ref["winner"][1] == -1 and res["winner"].cpu().numpy().tolist() == ref["winner"].tolist()
+    if a1 == dx.AGG_COORD_MEDIAN:
+        assert np.array_equal(bits(res["out"]), ref["out"].view(np.uint32))
+    else:
+        assert rel_l2(res["out"].cpu().numpy(), ref["out"]) <= TOL
+
+
 @pytest.mark.parametrize("r,G,set_size,d", [(3, 15, 5, 20_003), (3, 15, 7, 4097), (5, 6, 2, 3001), (1, 8, 3, 1000),
                                             (7, 4, None, 2500)])
 def test_pipeline_fused_vote_mean_handles_no_majority_and_uneven_sets(r, G, set_size, d):
