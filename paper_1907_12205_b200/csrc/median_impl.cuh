@@ -193,7 +193,7 @@ detox_status launch_reg(const float* X, int64_t ld, int m, int64_t d, const int3
 template <int M>
 detox_status launch_reg_m(const float* X, int64_t ld, int m, int64_t d, const int32_t* rows, int beta, float* out,
                           bool vec, cudaStream_t s) {
-    constexpr int C = M <= 12 ? 4 : (M <= 16 ? 2 : 1);
+    constexpr int C = M <= 12 ? 4 : (M <= 28 ? 2 : 1);
     if (vec && C > 1) return launch_reg<M, C>(X, ld, m, d, rows, beta, out, s);
     return launch_reg<M, 1>(X, ld, m, d, rows, beta, out, s);
 }
