@@ -9,8 +9,8 @@
 // One persistent CTA per SM: copy-issuing threads stream column blocks of all m rows into shared memory with
 // TMA (rows and columns outside the matrix arrive as zeros), warps 0-15 form 2 lo = 2 (x - (x with its low 13
 // bits cleared)) -- the raw fp32 values themselves serve as `hi`, because a TF32 MMA reads only the upper 19
-// bits of each word -- and lane 0 of warps 16, 17 issues the MMAs; mbarriers form rings of stages between the
-// roles.  Two kernels share this scheme: up to 128 rows the copies are 64 columns wide, land in a staging ring
+// bits of each word -- and lane 0 of the warps after them (two, or four up to 64 rows) issues the MMAs;
+// mbarriers form rings of stages between the roles.  Two kernels share this scheme: up to 128 rows the copies are 64 columns wide, land in a staging ring
 // and the transform warps write both MMA operands (see the staged kernel); above, the copies land directly in
 // the swizzled hi tile (see the wide kernel).
 // Column blocks are dealt round-robin to the CTAs and every 4096 columns of a CTA form a slab; at the end
@@ -40,7 +40,8 @@ namespace {
 constexpr int kKB = 32;                      // fp32 columns per K-block: one 128-byte swizzle row
 constexpr int kProdWarps = 16;
 constexpr int kProdThreads = kProdWarps * 32;
-constexpr int kMmaWarps = 2;                   // two issuing threads, so one's bookkeeping overlaps the other's MMAs
+constexpr int kMmaWarps = 2;                   // issuing threads of the wide kernel (the staged kernel has two or four):
+                                               // one's bookkeeping overlaps the other's MMAs
 constexpr int kTmaWarps = 2;                   // copy-issuing threads (the kernel for m > 128 uses the first only)
 constexpr int kTcThreads = kProdThreads + 32 * (kMmaWarps + kTmaWarps);
 constexpr size_t kSmemBudget = 227 * 1024;     // dynamic shared memory one CTA may have
