@@ -1,11 +1,13 @@
 #!/usr/bin/env python
 """Benchmark of the DETOX aggregation step (vote -> hierarchical mean -> robust aggregator) on B200.
 
-Default workload: n = 45 workers, r = 3, d = 11,173,962 (ResNet-18-sized), q = 5 ALIE attackers placed
-worst-case; one step = detox_aggregate(vote -> mean over 3 sets of 5 -> Multi-Krum(f=1, m_sel=1)).
-The metric is aggregation input throughput n*d*4 bytes per second.  Prints ONE JSON line.
+Default workload: the largest named single-GPU configuration, n = 105 workers, r = 3, d = 28,000,000 (VGG-class),
+q = 15 ALIE attackers; one step = detox_aggregate(vote -> mean over 7 sets of 5 -> coordinate median over the 7).
+The metric is aggregation input throughput n*d*4 bytes per second.  Prints ONE JSON line, which also carries the
+direct (non-DETOX) aggregators on the same buffer, each with the roofline that bounds its dominant kernel.
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload cfg2|cfg1|cfg3|cfg4]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload cfg4|cfg1|cfg2|cfg3]
+  python bench.py --sweep            (one JSON line per point of the n x d x attack sweep)
 
 With N > 1 (launched by torch.distributed.run) every rank aggregates its own independent copy of the
 workload (replicas; the path has no exchange step) and rank 0 reports the sum over ranks.
@@ -31,27 +33,42 @@ UNIT = "GB/s"
 CLOCK_QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
                "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
                "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+# Dense TF32 tensor throughput is nominally 1.1 / 2.25 of the bf16 one; the tensor roof is the measured bf16 peak
+# times that ratio.
+TF32_OVER_BF16 = 1.1 / 2.25
 
 
 def pipeline_for(name, w, dx):
-    """The DETOX leg and the direct (non-DETOX) leg of each named configuration."""
+    """The DETOX leg and the direct (non-DETOX) legs of each named configuration."""
     s = w.spec
-    G = s.n // s.r
     if name == "cfg1":
-        return (dict(a0=dx.AGG_NONE, a1=dx.AGG_COORD_MEDIAN, f=0, m_sel=1), ("coord_median", {}))
+        return (dict(a0=dx.AGG_NONE, a1=dx.AGG_COORD_MEDIAN, f=0, m_sel=1), [("coord_median", {})])
     if name == "cfg2":
-        return (dict(a0=dx.AGG_MEAN, a1=dx.AGG_MULTIKRUM, f=1, m_sel=1), ("multikrum", dict(f=5, m_sel=s.n - 5)))
+        return (dict(a0=dx.AGG_MEAN, a1=dx.AGG_MULTIKRUM, f=1, m_sel=1), [("multikrum", dict(f=5, m_sel=s.n - 5))])
     if name == "cfg3":
-        return (dict(a0=dx.AGG_NONE, a1=dx.AGG_BULYAN, f=3, m_sel=1), ("bulyan", dict(f=9)))
+        return (dict(a0=dx.AGG_NONE, a1=dx.AGG_BULYAN, f=3, m_sel=1), [("bulyan", dict(f=9))])
     if name == "cfg4":
-        return (dict(a0=dx.AGG_MEAN, a1=dx.AGG_COORD_MEDIAN, f=0, m_sel=1), ("coord_median", {}))
+        return (dict(a0=dx.AGG_MEAN, a1=dx.AGG_COORD_MEDIAN, f=0, m_sel=1),
+                [("coord_median", {}), ("multikrum", dict(f=15, m_sel=s.n - 15))])
     raise ValueError(name)
+
+
+def paper_pairings(name, w, dx):
+    """The pairings the paper found most resilient (Section 5.2, setups 2 and 3; vote-set shapes of Appendix B.1):
+    the Krum-type aggregator inside every vote set, then the mean of the set results."""
+    G = w.G
+    if name in ("cfg2", "cfg3"):   # 15 votes: Multi-Krum in sets of 7 and 8 (f = 2); Bulyan on one set of 15 (f = 3)
+        return [("vote_multikrum_in_sets_7_8_mean", dx.AGG_MULTIKRUM, [0, 7, G], 2, 0),
+                ("vote_bulyan_in_one_set_mean", dx.AGG_BULYAN, [0, G], 3, 0)]
+    if name == "cfg4":             # 35 votes: Multi-Krum (f = 1, all but one kept) inside the 7 sets of 5
+        return [("vote_multikrum_in_sets_of_5_mean", dx.AGG_MULTIKRUM, [int(x) for x in w.set_offsets], 1, 0)]
+    return []
 
 
 ORACLE_A1 = {1: "mean", 2: "coord_median", 3: "multikrum", 4: "bulyan"}
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu captures summarised in
-# profiles/vote_kernels_cfg2.md (same kernel code; reset an entry to None when its kernel changes).
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel of the DETOX step, from ncu captures of
+# the same kernel code (reset an entry to None when its kernel changes).
 NCU_TRAFFIC_BYTES = {
     ("cfg2", "vote_mean_kernel"): 2_011_333_000 + 117_863_424,
     ("cfg3", "vote_kernel (winners only)"): 2_011_344_896 + 3_232_768,
@@ -70,7 +87,7 @@ class ClockSampler:
     def __enter__(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={CLOCK_QUERY}",
-                                          "--format=csv,noheader,nounits", "-lms", "50"],
+                                          "--format=csv,noheader,nounits", "-lms", "20"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -121,7 +138,7 @@ def measured_peaks():
     if os.path.exists(path):
         with open(path) as fh:
             return json.load(fh), "measured"
-    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0}, "fallback"
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "sm_max_mhz": 1965.0}, "fallback"
 
 
 def time_calls(torch, fn, steps, warmup):
@@ -161,8 +178,22 @@ def oracle_step(w, cfg, X_host):
                                   w.set_members, ORACLE_A1[cfg["a1"]], cfg["f"], cfg["m_sel"])
 
 
+def workload_label(name, spec, cfg):
+    a0 = {0: "none", 1: "mean"}[cfg["a0"]]
+    return (f"{name}: n={spec.n} r={spec.r} d={spec.d} q={spec.q} {spec.attack}/{spec.placement}; "
+            f"vote -> A0={a0} -> A1={ORACLE_A1[cfg['a1']]}(f={cfg['f']}, m_sel={cfg['m_sel']})")
+
+
+def config_entry(name, spec, cfg, world):
+    """The `config` object of the JSON line; both arms print the same one."""
+    in_bytes = spec.n * spec.d * 4
+    return {"workload": workload_label(name, spec, cfg),
+            "l2": "inputs larger than L2" if in_bytes > 2 * 126e6 else "inputs fit in L2 (warm)", "replicas": world}
+
+
 def run_reference(args, rank, world):
-    """The reference arm: the CPU oracle, as it stands, on the host cores (rank 0 only)."""
+    """The reference arm: the CPU oracle, as it stands, on the host cores (rank 0 only).  A step is the whole
+    workload when K such steps end within a few minutes, else its first d' columns (all rows)."""
     if rank != 0:
         return
     import oracle
@@ -172,45 +203,37 @@ def run_reference(args, rank, world):
     w = wl.make_workload(spec)
     cfg, _ = pipeline_for(args.workload, w, dx)
     X = w.data().numpy()
-    for _ in range(min(args.warmup, 1)):
-        oracle_step(w, cfg, X)
-    steps = max(1, min(args.steps, 5))
+    t0 = time.perf_counter()
+    oracle_step(w, cfg, X)                       # first touch + a full-size estimate
+    full_s = time.perf_counter() - t0
+    budget_s = 150.0
+    steps, warmup = max(1, args.steps), max(0, args.warmup)
+    d_s, sample = spec.d, "full workload, every step"
+    if full_s * (steps + warmup) > budget_s:
+        d_s = max(1024, int(spec.d * budget_s / (full_s * (steps + warmup))))
+        sample = f"first {d_s} of {spec.d} columns of all {spec.n} rows, every step"
+    Xs = np.ascontiguousarray(X[:, :d_s]) if d_s < spec.d else X
+    for _ in range(warmup):
+        oracle_step(w, cfg, Xs)
     t0 = time.perf_counter()
     for _ in range(steps):
-        oracle_step(w, cfg, X)
+        oracle_step(w, cfg, Xs)
     ms = (time.perf_counter() - t0) * 1e3 / steps
-    val = spec.n * spec.d * 4 / (ms * 1e-3) / 1e9
+    val = spec.n * d_s * 4 / (ms * 1e-3) / 1e9
     line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
-            "warmup": min(args.warmup, 1), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+            "warmup": warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": workload_label(args.workload, spec, cfg)},
+            "config": config_entry(args.workload, spec, cfg, world),
             "cpu_baseline": {"value": val, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
-                             "sample": "full workload, every step"},
+                             "sample": sample},
             "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line))
 
 
-def workload_label(name, spec, cfg):
-    a0 = {0: "none", 1: "mean"}[cfg["a0"]]
-    return (f"{name}: n={spec.n} r={spec.r} d={spec.d} q={spec.q} {spec.attack}/{spec.placement}; "
-            f"vote -> A0={a0} -> A1={ORACLE_A1[cfg['a1']]}(f={cfg['f']}, m_sel={cfg['m_sel']})")
+# ------------------------------------------------------------------------------------------- rooflines
 
-
-def median_minmax_ops(m: int) -> int:
-    """min/max operations per coordinate that a median over m rows needs on the register path.
-
-    The merge-exchange network on M inputs (M = m up to 32, else m rounded up to the next network size with an
-    even gap) is walked backwards from the middle output: a comparator costs one operation per output that
-    something later still reads.  Above 128 rows two lanes share a coordinate and no closed count is given."""
-    if m <= 32:
-        M = m
-    elif m <= 128:
-        step = 8 if m <= 64 else 16
-        M = (m + step - 1) // step * step
-        if (M - m) & 1:
-            M -= 1
-    else:
-        return 0
+def merge_exchange_net(M: int):
+    """Comparators of Batcher's merge-exchange network on M inputs, in network order."""
     net = []
     p = 1
     while p < M:
@@ -224,9 +247,33 @@ def median_minmax_ops(m: int) -> int:
                 j += 2 * k
             k //= 2
         p *= 2
+    return net
+
+
+def median_minmax_ops(m: int) -> int:
+    """min/max operations per coordinate that a median over m rows costs in the library's kernels.
+
+    Up to 128 rows (one thread per coordinate): the merge-exchange network on M inputs (M = m up to 32, else m
+    rounded up to the next network size with an even gap) is walked backwards from the middle output; a comparator
+    costs one operation per output that something later still reads.  129 to 256 rows (two lanes per coordinate, H
+    keys each, H = half of m rounded up to 8): each lane sorts its H keys completely (two operations per
+    comparator), takes H operations in the split against its partner's keys and H - 1 to reduce its half to the
+    extreme value.  Beyond 256 rows (shared-memory path) no count is given."""
+    if m > 256:
+        return 0
+    if m > 128:
+        H = ((m + 1) // 2 + 7) // 8 * 8
+        return 2 * (2 * len(merge_exchange_net(H)) + H + H - 1)
+    if m <= 32:
+        M = m
+    else:
+        step = 8 if m <= 64 else 16
+        M = (m + step - 1) // step * step
+        if (M - m) & 1:
+            M -= 1
     live = {M // 2} if M & 1 else {M // 2 - 1, M // 2}
     ops = 0
-    for a, b in reversed(net):
+    for a, b in reversed(merge_exchange_net(M)):
         used = (a in live) + (b in live)
         if used:
             ops += used
@@ -234,12 +281,54 @@ def median_minmax_ops(m: int) -> int:
     return ops
 
 
-# Integer min/max issue on the plain-ALU pipe: 64 lanes per clock and SM, 148 SMs, at the sampled SM clock.
+# Integer min/max issue on the plain-ALU pipe: 64 lanes per clock and SM, 148 SMs, at the maximum SM clock.
 ALU_LANES_PER_CLK_SM, N_SMS = 64, 148
 
 
+def median_alu_roofline(m, d, ms, peaks):
+    """The plain-ALU roof of a coordinate median over m rows (bound by integer min/max issue beyond ~16 rows)."""
+    ops = median_minmax_ops(m)
+    if m <= 16 or not ops:
+        return None
+    clk = float(peaks.get("sm_max_mhz", 1965.0))
+    peak = ALU_LANES_PER_CLK_SM * N_SMS * clk * 1e6 / 1e12
+    ach = ops * d / (ms * 1e-3) / 1e12
+    return {"kernel": "colselect_reg_kernel" if m <= 128 else "colselect_pair_kernel", "bound": "alu",
+            "minmax_per_coordinate": ops, "achieved": round(ach, 3), "peak": round(peak, 2), "unit": "T min/max per s",
+            "frac": round(ach / peak, 3), "peak_kind": "64 lanes/clk/SM x 148 SMs x max SM clock",
+            "hbm_frac": round((m + 1) * d * 4 / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"], 3), "ms_per_launch": ms,
+            "traffic": None}
+
+
+def gram_roofline(m, d, ms, peaks, peak_kind):
+    """Roofline of the distance pass of Multi-Krum / Bulyan over m rows, timed through agg_pairwise_sqdist (the
+    streaming kernel plus two small reduction kernels).
+
+    17 to 256 aligned rows run on the tensor cores: `achieved` is the 3xTF32-equivalent rate 2 m^2 d / t (the
+    flops of the Gram matrix the split products stand for); `issued` is what the tensor pipe was given, counting
+    the padding to the MMA shape (rows to 64 / 128 / 256, columns to twice m rounded up to 16, for the hi and the
+    2 lo operand); `frac` = issued / TF32 peak, the tensor-pipe utilisation; the HBM fraction is beside it."""
+    hbm = m * d * 4 / (ms * 1e-3) / 1e9
+    if m <= 16:
+        return {"kernel": "sqdist_staged_kernel / sqdist_direct_kernel", "bound": "hbm", "achieved": round(hbm, 1),
+                "peak": peaks["hbm_gbs"], "peak_kind": f"of {peak_kind}", "unit": "GB/s",
+                "frac": round(hbm / peaks["hbm_gbs"], 3), "ms_per_launch": ms, "algorithmic_bytes": m * d * 4,
+                "traffic": None}
+    ncol = (m + 15) // 16 * 16
+    mrows = 64 if m <= 64 else (128 if m <= 128 else 256)
+    useful = 2.0 * m * m * d / (ms * 1e-3) / 1e12
+    issued = 2.0 * mrows * (2 * ncol) * d / (ms * 1e-3) / 1e12
+    peak = peaks["bf16_tflops"] * TF32_OVER_BF16
+    return {"kernel": "gram_staged_kernel" if m <= 128 else "gram_wide_kernel", "bound": "tensor",
+            "achieved": round(useful, 1), "issued": round(issued, 1), "peak": round(peak, 1),
+            "peak_kind": f"{peak_kind} bf16 burst peak x nominal TF32/bf16 ratio {TF32_OVER_BF16:.3f}",
+            "unit": "TFLOP/s", "frac": round(issued / peak, 3), "useful_frac": round(useful / peak, 3),
+            "hbm_GBps": round(hbm, 1), "hbm_frac": round(hbm / peaks["hbm_gbs"], 3), "ms_per_launch": ms,
+            "algorithmic_flops": 2.0 * m * m * d, "traffic": None}
+
+
 def run_sweep(args):
-    """Config 5: every aggregator with and without the DETOX front end over n x d x attack.
+    """The sweep: every aggregator with and without the DETOX front end over n x d x attack.
 
     One JSON line per point (not the headline line).  Times are CUDA-event means on one stream after
     warm-up; GB/s is n*d*4 / t; "alg" is the algorithmic bytes of the leg over the same time."""
@@ -253,6 +342,8 @@ def run_sweep(args):
     peaks, peak_kind = measured_peaks()
     ns = [int(x) for x in args.sweep_n.split(",")]
     ds = [int(x) for x in args.sweep_d.split(",")]
+    code = {"none": dx.AGG_NONE, "mean": dx.AGG_MEAN, "coord_median": dx.AGG_COORD_MEDIAN,
+            "multikrum": dx.AGG_MULTIKRUM, "bulyan": dx.AGG_BULYAN}
     for spec in wl.sweep_specs(ns=ns, ds=ds, attacks=tuple(args.sweep_attacks.split(","))):
         w = wl.make_workload(spec, device=dev)
         n, r, d, G, S, q = spec.n, spec.r, spec.d, w.G, w.S, spec.q
@@ -267,48 +358,43 @@ def run_sweep(args):
             legs[name] = {"ms": round(ms, 4), "GBps": round(in_bytes / ms / 1e6, 1),
                           "alg_GBps": round(alg_bytes / ms / 1e6, 1),
                           "alg_frac_of_hbm": round(alg_bytes / ms / 1e6 / peaks["hbm_gbs"], 3)}
+            return ms
 
-        def pipe_leg(name, a0, a1, f, m_sel, alg_bytes):
-            p = dx.Pipeline(n, r, d, w.members, a0, w.set_offsets if a0 == dx.AGG_MEAN else None,
-                            w.set_members if a0 == dx.AGG_MEAN else None, a1, f, m_sel)
-            ws = torch.empty(p.workspace_bytes(), dtype=torch.uint8, device=dev)
-            win = torch.empty(G, dtype=torch.int32, device=dev)
-            sel = torch.empty(max(p.n_selected, 1), dtype=torch.int32, device=dev)
-            timed(name, lambda: dx.detox_aggregate(p, X, out=out, winner=win, sel=sel, ws=ws), alg_bytes)
-            del ws
-
-        # DETOX legs.  Median: vote -> mean over sets of 5 -> median over the S means (S >= 3), else over the votes.
-        if S >= 3:
-            pipe_leg("detox_median", dx.AGG_MEAN, dx.AGG_COORD_MEDIAN, 0, 1, (n + 2 * S + 1) * d * 4)
-        else:
-            pipe_leg("detox_median", dx.AGG_NONE, dx.AGG_COORD_MEDIAN, 0, 1, (n + 2 * G + 1) * d * 4)
-        # Krum family: vote -> aggregator over the G votes, tolerance for the few Byzantine votes that survive
-        fv = min(2, max((G - 3) // 4, 0))
-        pipe_leg("detox_multikrum", dx.AGG_NONE, dx.AGG_MULTIKRUM, fv, G - fv, (n + 2 * G + (G - fv) + 1) * d * 4)
-        pipe_leg("detox_bulyan", dx.AGG_NONE, dx.AGG_BULYAN, fv, 1, (n + 2 * G + (G - 2 * fv) + 1) * d * 4)
-        # direct legs on all n rows
-        timed("direct_median", lambda: dx.agg_coord_median(X, out=out), (n + 1) * d * 4)
-        ops = median_minmax_ops(n)
-        if n > 16 and ops:
-            # beyond ~16 rows the register networks are bound by the plain ALUs, not by HBM: report that roof too
-            clk = float(peaks.get("sm_max_mhz", 1965.0))
-            peak = ALU_LANES_PER_CLK_SM * N_SMS * clk * 1e6 / 1e12
-            ach = ops * d / (legs["direct_median"]["ms"] * 1e-3) / 1e12
-            legs["direct_median"]["alu"] = {"bound": "alu", "minmax_per_coordinate": ops, "achieved": round(ach, 2),
-                                            "peak": round(peak, 2), "unit": "T min/max per s",
-                                            "frac": round(ach / peak, 3), "peak_kind": "64 lanes/clk/SM x 148 SMs x max SM clock"}
         ws = torch.empty(dx.agg_multikrum_workspace_bytes(n, d), dtype=torch.uint8, device=dev)
         sel = torch.empty(n, dtype=torch.int32, device=dev)
         sc = torch.empty(n, dtype=torch.float64, device=dev)
-        timed("direct_multikrum", lambda: dx.agg_multikrum(X, q, n - q, out=out, sel=sel[: n - q], scores=sc, ws=ws),
-              (n + (n - q) + 1) * d * 4)
-        if n >= 4 * q + 3:
-            timed("direct_bulyan", lambda: dx.agg_bulyan(X, q, out=out, sel=sel[: n - 2 * q], ws=ws),
-                  (n + (n - 2 * q) + 1) * d * 4)
+        plan = wl.sweep_legs(spec, G, S)
+        for name, leg in plan.items():
+            if name.startswith("detox_"):
+                mean0 = leg["a0"] == "mean"
+                rows1 = S if mean0 else G
+                p = dx.Pipeline(n, r, d, w.members, code[leg["a0"]], w.set_offsets if mean0 else None,
+                                w.set_members if mean0 else None, code[leg["a1"]], leg["f"], leg["m_sel"])
+                pws = torch.empty(p.workspace_bytes(), dtype=torch.uint8, device=dev)
+                win = torch.empty(G, dtype=torch.int32, device=dev)
+                psel = torch.empty(max(p.n_selected, 1), dtype=torch.int32, device=dev)
+                second = {"coord_median": 0, "multikrum": leg["m_sel"], "bulyan": rows1 - 2 * leg["f"]}[leg["a1"]]
+                timed(name, lambda: dx.detox_aggregate(p, X, out=out, winner=win, sel=psel, ws=pws),
+                      (n + 2 * rows1 + second + 1) * d * 4)
+                del pws
+            elif leg["a1"] == "coord_median":
+                ms = timed(name, lambda: dx.agg_coord_median(X, out=out), (n + 1) * d * 4)
+                roof = median_alu_roofline(n, d, ms, peaks)
+                if roof:
+                    legs[name]["alu"] = roof
+            elif leg["a1"] == "multikrum":
+                timed(name, lambda: dx.agg_multikrum(X, leg["f"], leg["m_sel"], out=out, sel=sel[: leg["m_sel"]],
+                                                     scores=sc, ws=ws), (n + leg["m_sel"] + 1) * d * 4)
+                D = torch.empty((n, n), dtype=torch.float64, device=dev)
+                gms = time_calls(torch, lambda: dx.agg_pairwise_sqdist(X, D=D, ws=ws), reps, 3)
+                legs[name]["distance_pass"] = gram_roofline(n, d, gms, peaks, peak_kind)
+            else:
+                timed(name, lambda: dx.agg_bulyan(X, leg["f"], out=out, sel=sel[: n - 2 * leg["f"]], ws=ws),
+                      (n + (n - 2 * leg["f"]) + 1) * d * 4)
         del ws
         line = {"sweep_point": spec.name, "n": n, "r": r, "d": d, "q": q, "q_hat": w.q_hat, "attack": spec.attack,
-                "sets": S, "f_votes": fv, "unit": "GB/s = n*d*4/t", "hbm_peak": peaks["hbm_gbs"],
-                "peak_kind": peak_kind, "legs": legs,
+                "sets": S, "f_votes": plan["detox_multikrum"]["f"], "unit": "GB/s = n*d*4/t",
+                "hbm_peak": peaks["hbm_gbs"], "peak_kind": peak_kind, "legs": legs,
                 "speedup": {k: round(legs["direct_" + k]["ms"] / legs["detox_" + k]["ms"], 2)
                             for k in ("median", "multikrum", "bulyan") if "direct_" + k in legs}}
         print(json.dumps(line), flush=True)
@@ -319,12 +405,12 @@ def run_sweep(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="detox", choices=["detox", "reference"])
-    ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4"])
+    ap.add_argument("--workload", default="cfg4", choices=["cfg1", "cfg2", "cfg3", "cfg4"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--sweep", action="store_true", help="config 5: one JSON line per (n, d, attack) point")
+    ap.add_argument("--sweep", action="store_true", help="one JSON line per (n, d, attack) point of the sweep")
     ap.add_argument("--sweep-n", default="15,45,105,225")
     ap.add_argument("--sweep-d", default="1000000,11173962,25557032")
     ap.add_argument("--sweep-attacks", default="reverse,alie")
@@ -359,7 +445,7 @@ def main():
         import dataclasses
         spec = dataclasses.replace(spec, seed=spec.seed + rank)
     w = wl.make_workload(spec, device=dev)
-    cfg, (direct_name, direct_args) = pipeline_for(args.workload, w, dx)
+    cfg, direct_legs = pipeline_for(args.workload, w, dx)
     X = w.X[:, : spec.d]
     pipe = dx.Pipeline(spec.n, spec.r, spec.d, w.members, cfg["a0"], w.set_offsets, w.set_members, cfg["a1"],
                        cfg["f"], cfg["m_sel"])
@@ -387,11 +473,13 @@ def main():
         for _ in range(3):
             step()
         torch.cuda.synchronize()
+        launches_before = dx.kernel_launch_count()
         e0.record(st)
         for _ in range(args.steps):
             step()
         e1.record(st)
         barrier()
+        gpu_launches = dx.kernel_launch_count() - launches_before   # counted by the library at every launch
         # the dominant kernel alone, same inputs, same stream: the vote (reads n*d*4, writes G*d*4), or the vote
         # fused with the set means when A_0 is the mean (reads n*d*4, writes S*d*4)
         vws = torch.empty(dx.detox_vote_workspace_bytes(spec.n, spec.r), dtype=torch.uint8, device=dev)
@@ -427,30 +515,52 @@ def main():
     e2e_steps = max(2, min(args.steps, 5))
     barrier()
     e2e_ms = max_over_ranks(time_calls(torch, e2e_step, e2e_steps, 1), dev)
+    del Xd
 
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
         return
 
-    # ---- other legs on the same inputs (rank 0, N = 1 reporting only) ----
-    legs = {"detox_pipeline": {"ms": ms_per_step, "GBps": in_bytes / ms_per_step / 1e6}}
-    if direct_name == "multikrum":
-        dws = torch.empty(dx.agg_multikrum_workspace_bytes(spec.n, spec.d), dtype=torch.uint8, device=dev)
-        dsel = torch.empty(direct_args["m_sel"], dtype=torch.int32, device=dev)
-        dsc = torch.empty(spec.n, dtype=torch.float64, device=dev)
-        fn = lambda: dx.agg_multikrum(X, direct_args["f"], direct_args["m_sel"], out=out, sel=dsel, scores=dsc, ws=dws)
-    elif direct_name == "bulyan":
-        dws = torch.empty(dx.agg_bulyan_workspace_bytes(spec.n, spec.d), dtype=torch.uint8, device=dev)
-        dsel = torch.empty(spec.n - 2 * direct_args["f"], dtype=torch.int32, device=dev)
-        fn = lambda: dx.agg_bulyan(X, direct_args["f"], out=out, sel=dsel, ws=dws)
-    else:
-        fn = lambda: dx.agg_coord_median(X, out=out)
-    dms = time_calls(torch, fn, max(3, min(args.steps, 10)), 3)
-    legs[f"direct_{direct_name}"] = {"ms": dms, "GBps": in_bytes / dms / 1e6, "args": direct_args}
-    legs["detox_speedup_vs_direct"] = dms / ms_per_step
-
+    # ---- other legs on the same inputs (rank 0 reporting only) ----
     peaks, peak_kind = measured_peaks()
+    reps = max(3, min(args.steps, 10))
+    legs = {"detox_pipeline": {"ms": ms_per_step, "GBps": in_bytes / ms_per_step / 1e6}}
+    for direct_name, direct_args in direct_legs:
+        leg = {"args": direct_args}
+        if direct_name in ("multikrum", "bulyan"):
+            dws = torch.empty(dx.agg_multikrum_workspace_bytes(spec.n, spec.d), dtype=torch.uint8, device=dev)
+            if direct_name == "multikrum":
+                dsel = torch.empty(direct_args["m_sel"], dtype=torch.int32, device=dev)
+                dsc = torch.empty(spec.n, dtype=torch.float64, device=dev)
+                fn = lambda: dx.agg_multikrum(X, direct_args["f"], direct_args["m_sel"], out=out, sel=dsel, scores=dsc,
+                                              ws=dws)
+            else:
+                dsel = torch.empty(spec.n - 2 * direct_args["f"], dtype=torch.int32, device=dev)
+                fn = lambda: dx.agg_bulyan(X, direct_args["f"], out=out, sel=dsel, ws=dws)
+            dms = time_calls(torch, fn, reps, 3)
+            D = torch.empty((spec.n, spec.n), dtype=torch.float64, device=dev)
+            gms = time_calls(torch, lambda: dx.agg_pairwise_sqdist(X, D=D, ws=dws), reps, 3)
+            leg["roofline"] = gram_roofline(spec.n, spec.d, gms, peaks, peak_kind)
+            del dws
+        else:
+            dms = time_calls(torch, lambda: dx.agg_coord_median(X, out=out), reps, 3)
+            hbm = (spec.n + 1) * spec.d * 4 / (dms * 1e-3) / 1e9
+            leg["roofline"] = median_alu_roofline(spec.n, spec.d, dms, peaks) or {
+                "kernel": "colselect_reg_kernel", "bound": "hbm", "achieved": hbm, "peak": peaks["hbm_gbs"],
+                "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": hbm / peaks["hbm_gbs"], "ms_per_launch": dms,
+                "traffic": None}
+        leg.update(ms=dms, GBps=in_bytes / dms / 1e6, detox_speedup=dms / ms_per_step)
+        legs[f"direct_{direct_name}"] = leg
+    legs["detox_speedup_vs_direct"] = legs[f"direct_{direct_legs[0][0]}"]["ms"] / ms_per_step
+    for name, a0, offsets, f, m_sel in paper_pairings(args.workload, w, dx):
+        p2 = dx.Pipeline(spec.n, spec.r, spec.d, w.members, a0, offsets, w.set_members, dx.AGG_MEAN, f, m_sel)
+        ws2 = torch.empty(p2.workspace_bytes(), dtype=torch.uint8, device=dev)
+        sel2 = torch.empty(max(p2.n_selected, 1), dtype=torch.int32, device=dev)
+        ms2 = time_calls(torch, lambda: dx.detox_aggregate(p2, X, out=out, winner=winner, sel=sel2, ws=ws2), reps, 3)
+        legs[name] = {"ms": ms2, "GBps": in_bytes / ms2 / 1e6, "f": f, "sets": offsets}
+        del ws2
+
     vote_bytes = (spec.n + dom_rows_out) * spec.d * 4
     achieved = vote_bytes / (vote_ms * 1e-3) / 1e9
     roofline = {"kernel": dom_name, "bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"],
@@ -473,20 +583,19 @@ def main():
         o = out.cpu().numpy().astype(np.float64)
         den = np.linalg.norm(ref["out"].astype(np.float64))
         parity = {"winner_exact": winner.cpu().numpy().tolist() == ref["winner"].tolist(),
-                  "out_rel_l2": float(np.linalg.norm(o - ref["out"]) / (den if den else 1.0))}
+                  "out_rel_l2": float(np.linalg.norm(o - ref["out"]) / (den if den else 1.0)),
+                  "status_word": dx.read_status(ws)}
         if ref["sel"] is not None:
             parity["sel_exact"] = sel.cpu().numpy()[: len(ref["sel"])].tolist() == ref["sel"].tolist()
 
-    kernels_per_step = {"cfg1": 3, "cfg2": 6, "cfg3": 6, "cfg4": 4}[args.workload]
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": workload_label(args.workload, spec, cfg), "l2": "inputs larger than L2"
-                       if in_bytes > 2 * 126e6 else "inputs fit in L2 (warm)", "replicas": world},
+            "config": config_entry(args.workload, spec, cfg, world),
             "clocks": clocks.summary(),
             "e2e": {"value": whole_job_value(in_bytes, world, e2e_ms), "unit": UNIT, "ms_per_step": e2e_ms,
                     "h2d_bytes_per_step": int(Xh.numel() * 4), "d2h_bytes_per_step": int(outh.numel() * 4)},
-            "gpu_launches": kernels_per_step * args.steps, "kernels_per_step": kernels_per_step,
+            "gpu_launches": gpu_launches, "kernels_per_step": gpu_launches / args.steps,
             "roofline": roofline, "cpu_baseline": cpu_baseline, "legs": legs, "parity": parity}
     print(json.dumps(line))
     if world > 1:

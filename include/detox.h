@@ -22,9 +22,14 @@
  *   - Errors: argument problems are reported before anything is launched; a failed launch returns
  *     DETOX_ERR_CUDA.  Nothing aborts or throws.  Multi-Krum and Bulyan run kernels that wait on
  *     asynchronous copies (9 to 16 long rows) or on the tensor cores (17 to 256 rows); every such
- *     device-side wait is bounded: should one run out, the first int32 of the workspace passed to
- *     agg_multikrum / agg_bulyan reads DETOX_ERR_TIMEOUT after the stream has been synchronised
- *     (0 otherwise) and the outputs are not valid.
+ *     device-side wait is bounded.  Device status word: the first int32 of the workspace passed to
+ *     agg_multikrum, agg_bulyan or detox_aggregate.  The call clears it; should a wait run out in any
+ *     stage of the call it reads DETOX_ERR_TIMEOUT once the stream has been synchronised (0 otherwise),
+ *     the outputs are then not valid (the index outputs still hold in-range indices), and nothing
+ *     hangs or faults.
+ *   - Non-finite values: the vote and the order statistics are fully defined on them (bit patterns).
+ *     In Multi-Krum / Bulyan a row with an Inf or NaN entry is infinitely far from every other row
+ *     (a NaN distance counts as +Inf), so it is never preferred to a finite row.
  *   - Ranking of values (medians, "closest to the median") uses the total order
  *     -NaN < -Inf < ... < -0 < +0 < ... < +Inf < +NaN on fp32 bit patterns.
  */
@@ -131,7 +136,9 @@ detox_status detox_vote_hier_mean(const float* X, int64_t ld, int n, int r, int6
 /* ---------------------------------------------------------------------------------------------
  * Coordinate-wise median (Section 4; Appendix B.1): out[c] = median_i X[i][c] over the m rows.
  * Odd m: the middle value, bit for bit one of the inputs.  Even m: fp32 (lo + hi) * 0.5f.
- *   out  dev, d.   ws: agg_coord_median_workspace_bytes(m, d) bytes (may be 0, then ws may be NULL).
+ *   out  dev, d.   ws: agg_coord_median_workspace_bytes(m, d) bytes.  Every size built so far works in
+ *   registers or shared memory, so that is 0 and ws is not touched (pass NULL); the arguments keep the
+ *   signature of the other aggregators.
  * ------------------------------------------------------------------------------------------- */
 size_t agg_coord_median_workspace_bytes(int m, int64_t d);
 detox_status agg_coord_median(const float* X, int64_t ld, int m, int64_t d, float* out, void* ws,
@@ -146,7 +153,7 @@ detox_status agg_coord_median(const float* X, int64_t ld, int m, int64_t d, floa
 detox_status agg_trimmed_mean(const float* X, int64_t ld, int m, int64_t d, int trim, float* out, void* stream);
 
 /* ---------------------------------------------------------------------------------------------
- * Coordinate-wise sign majority, the aggregator of signSGD with majority vote (Section 5.1, setup 4:
+ * Coordinate-wise sign majority, the aggregator of signSGD with majority vote (Section 5.2, setup 4:
  * A_0 = A_1 = coordinate-wise majority): out[c] = sign(sum_i sign(X[i][c])), one of -1, 0, +1
  * (sign(0) = sign(NaN) = 0; a tie gives 0).
  *   out  dev, d.   No workspace.
@@ -164,6 +171,17 @@ detox_status agg_sign_majority(const float* X, int64_t ld, int m, int64_t d, flo
 size_t agg_geometric_median_workspace_bytes(int m, int64_t d);
 detox_status agg_geometric_median(const float* X, int64_t ld, int m, int64_t d, int iters, float eps, float* out,
                                   void* ws, size_t ws_bytes, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * Pairwise squared Euclidean distances between the m rows, the O(p^2 d) step that Section 4 ("Improved
+ * speed") names as the cost of Krum, Multi-Krum and Bulyan: D[i][j] = sum_c (X[i][c] - X[j][c])^2.
+ * This is the first stage of agg_multikrum / agg_bulyan on its own (same kernels, same results).
+ *   D   dev, m x m fp64, row-major, symmetric, zero diagonal (8-byte aligned)
+ *   ws  agg_pairwise_sqdist_workspace_bytes(m, d) bytes; its first int32 is the device status word
+ * ------------------------------------------------------------------------------------------- */
+size_t agg_pairwise_sqdist_workspace_bytes(int m, int64_t d);
+detox_status agg_pairwise_sqdist(const float* X, int64_t ld, int m, int64_t d, double* D, void* ws, size_t ws_bytes,
+                                 void* stream);
 
 /* ---------------------------------------------------------------------------------------------
  * Multi-Krum (cited in Section 4 "Improved speed" as the O(p^2 d) aggregator; requirement
@@ -203,7 +221,7 @@ detox_status agg_bulyan(const float* X, int64_t ld, int m, int64_t d, int f, flo
  *   a0 = DETOX_AGG_MEAN : the S set means go to A_1
  *   a0 = DETOX_AGG_SIGN_MAJORITY : the S coordinate-wise sign majorities of the sets go to A_1
  *   a0 = DETOX_AGG_MULTIKRUM | DETOX_AGG_BULYAN : the aggregator runs inside every vote set (the pairings the
- *        paper found most resilient, Section 5.1 setups 2 and 3; set shapes as in Appendix B.1, e.g. 7 + 8 or
+ *        paper found most resilient, Section 5.2, setups 2 and 3; set shapes as in Appendix B.1, e.g. 7 + 8 or
  *        one set of 15) and its S results go to A_1, which must then be MEAN or COORD_MEDIAN.  f and m_sel
  *        belong to A_0: every set of k votes averages its m_sel best (m_sel = 0: its k - f best), or, for
  *        Bulyan, needs k >= 4f+3.
@@ -217,7 +235,8 @@ detox_status agg_bulyan(const float* X, int64_t ld, int m, int64_t d, int f, flo
  *                              Krum-type stage; vote (group) indices, set after set, when A_0 is; may be NULL
  *   sel_workers  dev           out, the same rows as worker ids (winner[vote]), meaningful whenever sel
  *                              indexes votes (a0 = NONE, MULTIKRUM or BULYAN); may be NULL
- *   ws           detox_aggregate_workspace_bytes(desc) bytes (holds the votes and set means too)
+ *   ws           detox_aggregate_workspace_bytes(desc) bytes (holds the votes and set means too); its first
+ *                int32 is the device status word of the whole step (see "Errors" above)
  * ------------------------------------------------------------------------------------------- */
 typedef struct {
     int32_t n;                   /* compute nodes */
@@ -239,6 +258,20 @@ size_t detox_aggregate_workspace_bytes(const detox_pipeline_desc* desc);
 detox_status detox_aggregate(const detox_pipeline_desc* desc, const float* X, int64_t ld, float* out,
                              int32_t* winner, int32_t* sel, int32_t* sel_workers, void* ws,
                              size_t ws_bytes, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * Self-test of the bounded device-side waits (no counterpart in the paper; a diagnostic).  Launches one
+ * warp that waits, with the same wait routine the distance kernels use, on a barrier that nothing will
+ * ever complete, for at most `limit_cycles` SM clocks (1 .. 2e9).  The wait must give up by itself: after
+ * the stream has been synchronised *status reads DETOX_ERR_TIMEOUT (any other value is a failure of the
+ * wait routine), the kernel has exited normally and the context is intact.
+ *   status  dev, one int32 (cleared by the call)
+ * ------------------------------------------------------------------------------------------- */
+detox_status detox_selftest_bounded_wait(int32_t* status, int64_t limit_cycles, void* stream);
+
+/* Number of kernels this library has launched in this process so far (a diagnostic counter, no counterpart in
+ * the paper; the one piece of state the library keeps, besides the scratch of detox_vote_noalloc). */
+unsigned long long detox_kernel_launch_count(void);
 
 #ifdef __cplusplus
 }

@@ -239,7 +239,7 @@ def detox_aggregate(X, members, r: int, a0: str, set_offsets, set_members, a1: s
     sel = None
     sel_votes = None
     if a0 in ("multikrum", "bulyan"):
-        # Section 5.1, setups 2 and 3: the robust aggregator inside every vote group, then A_1 over the results.
+        # Section 5.2, setups 2 and 3: the robust aggregator inside every vote group, then A_1 over the results.
         # f and m_sel belong to A_0; m_sel = 0 means "all but f" of each group.
         so, sm = np.asarray(set_offsets), np.asarray(set_members)
         outs, sel_votes = [], []

@@ -369,7 +369,7 @@ int oracle_geometric_median(const float* X, int64_t ld, int m, int64_t d, int it
 }
 
 /* ---------------------------------------------------------------------------------------------
- * Coordinate-wise sign majority (signSGD with majority vote; Section 5.1, setup 4):
+ * Coordinate-wise sign majority (signSGD with majority vote; Section 5.2, setup 4):
  * out[c] = sign(sum_i sign(x_ic)); sign(0) = sign(NaN) = 0.  rows == NULL means rows 0..m-1.
  * ------------------------------------------------------------------------------------------- */
 int oracle_sign_majority(const float* X, int64_t ld, int m, int64_t d, const int32_t* rows, float* out) {

@@ -25,6 +25,8 @@ EXPORTS = (
     "detox_vote_hier_mean",
     "agg_coord_median_workspace_bytes", "agg_coord_median", "agg_trimmed_mean", "agg_sign_majority", "agg_geometric_median_workspace_bytes", "agg_geometric_median", "agg_multikrum_workspace_bytes", "agg_multikrum",
     "agg_bulyan_workspace_bytes", "agg_bulyan", "detox_aggregate_workspace_bytes", "detox_aggregate",
+    "detox_selftest_bounded_wait", "agg_pairwise_sqdist_workspace_bytes", "agg_pairwise_sqdist",
+    "detox_kernel_launch_count",
 )
 
 
@@ -82,6 +84,12 @@ def load() -> ctypes.CDLL:
     lib.detox_aggregate_workspace_bytes.restype = _sz
     lib.detox_aggregate_workspace_bytes.argtypes = [ctypes.POINTER(PipelineDesc)]
     lib.detox_aggregate.argtypes = [ctypes.POINTER(PipelineDesc), _vp, _i64, _vp, _vp, _vp, _vp, _vp, _sz, _vp]
+    lib.detox_selftest_bounded_wait.argtypes = [_vp, _i64, _vp]
+    lib.agg_pairwise_sqdist_workspace_bytes.restype = _sz
+    lib.agg_pairwise_sqdist_workspace_bytes.argtypes = [_int, _i64]
+    lib.agg_pairwise_sqdist.argtypes = [_vp, _i64, _int, _i64, _vp, _vp, _sz, _vp]
+    lib.detox_kernel_launch_count.restype = ctypes.c_ulonglong
+    lib.detox_kernel_launch_count.argtypes = []
     _lib = lib
     return lib
 
@@ -118,6 +126,29 @@ def _ws(nbytes: int, ws: Optional[torch.Tensor], device):
     if ws is None:
         ws = torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
     return ws, ws.data_ptr(), ws.numel() * ws.element_size()
+
+
+def read_status(ws: torch.Tensor, stream=None) -> int:
+    """The device status word of a finished call: the first int32 of the workspace that was passed to agg_multikrum,
+    agg_bulyan or detox_aggregate.  Synchronises the stream.  0, or 5 (DETOX_ERR_TIMEOUT) when a bounded device-side
+    wait ran out and the call's outputs are not valid."""
+    (torch.cuda.current_stream() if stream is None else stream).synchronize()
+    return int(ws[:4].view(torch.int32).item())
+
+
+def check_status(ws: torch.Tensor, what: str = "device status", stream=None):
+    """Raises DetoxError if the device status word of a finished call is not 0 (synchronises the stream)."""
+    _check(read_status(ws, stream), what)
+
+
+def detox_selftest_bounded_wait(limit_cycles: int = 100_000, status: Optional[torch.Tensor] = None, stream=None):
+    """Runs the library's bounded wait on a barrier that nothing completes; returns the int32 status tensor, which
+    reads 5 (DETOX_ERR_TIMEOUT) once the stream has been synchronised."""
+    if status is None:
+        status = torch.empty(1, dtype=torch.int32, device="cuda")
+    _check(load().detox_selftest_bounded_wait(status.data_ptr(), int(limit_cycles), _stream(stream)),
+           "detox_selftest_bounded_wait")
+    return status
 
 
 def _ptr(t: Optional[torch.Tensor]):
@@ -242,6 +273,26 @@ def agg_geometric_median(X, iters: int = 32, eps: float = 1e-12, out: Optional[t
     _check(lib.agg_geometric_median(xp, ld, m, d, iters, eps, out.data_ptr(), wp, wb, _stream(stream)),
            "agg_geometric_median")
     return out
+
+
+def kernel_launch_count() -> int:
+    """Kernels launched by the library in this process so far."""
+    return int(load().detox_kernel_launch_count())
+
+
+def agg_pairwise_sqdist_workspace_bytes(m: int, d: int) -> int:
+    return int(load().agg_pairwise_sqdist_workspace_bytes(m, d))
+
+
+def agg_pairwise_sqdist(X, D: Optional[torch.Tensor] = None, ws: Optional[torch.Tensor] = None, stream=None):
+    """Squared distances between the rows: D [m, m] float64, symmetric, zero diagonal."""
+    lib = load()
+    xp, ld, m, d = _mat(X)
+    if D is None:
+        D = torch.empty((m, m), dtype=torch.float64, device=X.device)
+    ws, wp, wb = _ws(lib.agg_pairwise_sqdist_workspace_bytes(m, d), ws, X.device)
+    _check(lib.agg_pairwise_sqdist(xp, ld, m, d, D.data_ptr(), wp, wb, _stream(stream)), "agg_pairwise_sqdist")
+    return D
 
 
 def agg_multikrum_workspace_bytes(m: int, d: int) -> int:

@@ -2,11 +2,25 @@
 // Nothing here touches gradient data on the host, allocates, or synchronises.
 #include <string.h>
 
+#include <atomic>
+
 #include "common.cuh"
 
 using namespace detox;
 
+namespace detox {
 namespace {
+std::atomic<unsigned long long> g_kernel_launches{0};
+}
+detox_status launch_status() {
+    g_kernel_launches.fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError() == cudaSuccess ? DETOX_OK : DETOX_ERR_CUDA;
+}
+}  // namespace detox
+
+namespace {
+
+constexpr size_t kStatusBytes = 256;   // the device status word has an aligned slot of its own
 
 bool ws_ok(const void* ws, size_t have, size_t need) {
     if (need == 0) return true;
@@ -68,7 +82,7 @@ KrumWs krum_ws(void* ws, int m, int64_t d) {
     char* p = static_cast<char*>(ws);
     size_t off = 0;
     k.status = reinterpret_cast<int*>(p + off);   // first word of the workspace: device-side status
-    off += 256;
+    off += kStatusBytes;
     k.D = reinterpret_cast<double*>(p + off);
     off += align_up((size_t)m * m * sizeof(double));
     k.dist = p + off;
@@ -85,21 +99,27 @@ KrumWs krum_ws(void* ws, int m, int64_t d) {
 
 // `rows` (optional, device, m <= 16): the m rows are X[rows[i]], a negative entry standing for a zero row
 // (this is how the votes are consumed straight from the workers' rows through winner[], without a copy).
+//
+// `status` (device): the word that a bounded device-side wait sets to DETOX_ERR_TIMEOUT when it runs out.  NULL: the
+// first word of `ws`, cleared here (the stand-alone aggregators).  Otherwise the caller's word, which the caller has
+// cleared and which is only ever set, never cleared, from here on (the pipeline: one word for all its stages).
 detox_status run_multikrum(const float* X, int64_t ld, int m, int64_t d, const int32_t* rows, int f, int m_sel,
-                           float* out, int32_t* sel, double* scores, void* ws, cudaStream_t s) {
+                           float* out, int32_t* sel, double* scores, void* ws, int* status, cudaStream_t s) {
     KrumWs k = krum_ws(ws, m, d);
+    const bool own_status = status == nullptr;
+    if (own_status) status = k.status;
     int32_t* sel_buf = sel ? sel : k.sel;
     detox_status st;
     if (m >= 2 && m <= 16) {   // distance pass, then one small kernel for everything up to the chosen rows
         int nblocks = 0;
-        if ((st = launch_sqdist_partials(X, ld, m, d, rows, k.dist, k.status, &nblocks, s)) != DETOX_OK) return st;
+        if ((st = launch_sqdist_partials(X, ld, m, d, rows, k.dist, status, own_status, &nblocks, s)) != DETOX_OK) return st;
         st = launch_krum_small(false, static_cast<const double*>(k.dist), nblocks, m, f, m_sel, rows, sel_buf, k.mapped,
-                               scores, sqdist_partials_use_status(m, X, ld, d) ? nullptr : k.status, s);
+                               scores, own_status && !sqdist_partials_use_status(m, X, ld, d) ? status : nullptr, s);
         if (st != DETOX_OK) return st;
         return launch_mean_rows(X, ld, d, rows ? k.mapped : sel_buf, m_sel, out, s);
     }
-    if (cudaMemsetAsync(k.status, 0, sizeof(int), s) != cudaSuccess) return DETOX_ERR_CUDA;
-    st = launch_sqdist(X, ld, m, d, rows, k.D, k.dist, k.status, s);
+    if (own_status && cudaMemsetAsync(status, 0, sizeof(int), s) != cudaSuccess) return DETOX_ERR_CUDA;
+    st = launch_sqdist(X, ld, m, d, rows, k.D, k.dist, status, s);
     if (st != DETOX_OK) return st;
     st = launch_multikrum_select(k.D, m, f, m_sel, sel_buf, scores, k.select, s);
     if (st != DETOX_OK) return st;
@@ -112,21 +132,23 @@ detox_status run_multikrum(const float* X, int64_t ld, int m, int64_t d, const i
 }
 
 detox_status run_bulyan(const float* X, int64_t ld, int m, int64_t d, const int32_t* rows, int f, float* out,
-                        int32_t* sel, void* ws, cudaStream_t s) {
+                        int32_t* sel, void* ws, int* status, cudaStream_t s) {
     KrumWs k = krum_ws(ws, m, d);
+    const bool own_status = status == nullptr;
+    if (own_status) status = k.status;
     int32_t* sel_buf = sel ? sel : k.sel;
     const int theta = m - 2 * f, beta = theta - 2 * f;
     detox_status st;
     if (m >= 2 && m <= 16) {   // distance pass, then one small kernel for everything up to the chosen rows
         int nblocks = 0;
-        if ((st = launch_sqdist_partials(X, ld, m, d, rows, k.dist, k.status, &nblocks, s)) != DETOX_OK) return st;
+        if ((st = launch_sqdist_partials(X, ld, m, d, rows, k.dist, status, own_status, &nblocks, s)) != DETOX_OK) return st;
         st = launch_krum_small(true, static_cast<const double*>(k.dist), nblocks, m, f, 0, rows, sel_buf, k.mapped, nullptr,
-                               sqdist_partials_use_status(m, X, ld, d) ? nullptr : k.status, s);
+                               own_status && !sqdist_partials_use_status(m, X, ld, d) ? status : nullptr, s);
         if (st != DETOX_OK) return st;
         return launch_coord_select(X, ld, theta, d, rows ? k.mapped : sel_buf, beta, out, s);
     }
-    if (cudaMemsetAsync(k.status, 0, sizeof(int), s) != cudaSuccess) return DETOX_ERR_CUDA;
-    st = launch_sqdist(X, ld, m, d, rows, k.D, k.dist, k.status, s);
+    if (own_status && cudaMemsetAsync(status, 0, sizeof(int), s) != cudaSuccess) return DETOX_ERR_CUDA;
+    st = launch_sqdist(X, ld, m, d, rows, k.D, k.dist, status, s);
     if (st != DETOX_OK) return st;
     st = launch_bulyan_select(k.D, m, f, sel_buf, k.select, s);
     if (st != DETOX_OK) return st;
@@ -167,6 +189,7 @@ bool votes_by_index(const detox_pipeline_desc* p) {
 }
 
 struct PipeWs {
+    int* status;                 // first word of the workspace: DETOX_ERR_TIMEOUT if a bounded device-side wait ran out
     int32_t* winner_set_order;   // Krum-type A_0: winners in set order
     int32_t* sel_local;          // Krum-type A_0: rows chosen inside the current set
     void* vote;
@@ -185,7 +208,9 @@ PipeWs pipe_ws(void* ws, const detox_pipeline_desc* p) {
     const int rows1 = p->a0 != DETOX_AGG_NONE ? p->n_sets : G;
     size_t off = 0;
     w.ldz = pad_ld(p->d);
-    w.vote = base + off;
+    w.status = reinterpret_cast<int*>(base);
+    off += kStatusBytes;
+    w.vote = base + off;         // directly behind the status word: the vote's clearing memset takes both
     off += vote_ws_bytes(p->n, p->r);
     w.winner = reinterpret_cast<int32_t*>(base + off);
     off += align_up((size_t)G * sizeof(int32_t));
@@ -202,12 +227,15 @@ PipeWs pipe_ws(void* ws, const detox_pipeline_desc* p) {
     if (krum_type(p->a1)) off += krum_ws(nullptr, rows1, p->d).total;
     if (p->a1 == DETOX_AGG_GEOMETRIC_MEDIAN) off += geomed_ws_bytes(p->d);
     if (krum_type(p->a0)) {
-        int kmax = 1;
+        // the sets run one after another in the same region; its size is the largest any set needs (the need is not
+        // monotone in the set size: the distance kernels change plan with the row count)
+        size_t need = 0;
         for (int s = 0; s < p->n_sets; ++s) {
             const int k = p->set_offsets[s + 1] - p->set_offsets[s];
-            kmax = k > kmax ? k : kmax;
+            const size_t t = krum_ws(nullptr, k, p->d).total;
+            need = t > need ? t : need;
         }
-        off += krum_ws(nullptr, kmax, p->d).total;
+        off += need;
     }
     w.total = off;
     return w;
@@ -366,7 +394,7 @@ detox_status agg_multikrum(const float* X, int64_t ld, int m, int64_t d, int f, 
     if ((st = check_multikrum(m, f, m_sel)) != DETOX_OK) return st;
     if (!out || (reinterpret_cast<uintptr_t>(out) & 3u)) return DETOX_ERR_BAD_ARG;
     if (!ws_ok(ws, ws_bytes, krum_ws(nullptr, m, d).total)) return DETOX_ERR_WORKSPACE;
-    return run_multikrum(X, ld, m, d, nullptr, f, m_sel, out, sel, scores, ws, static_cast<cudaStream_t>(stream));
+    return run_multikrum(X, ld, m, d, nullptr, f, m_sel, out, sel, scores, ws, nullptr, static_cast<cudaStream_t>(stream));
 }
 
 size_t agg_bulyan_workspace_bytes(int m, int64_t d) {
@@ -381,8 +409,27 @@ detox_status agg_bulyan(const float* X, int64_t ld, int m, int64_t d, int f, flo
     if ((st = check_bulyan(m, f)) != DETOX_OK) return st;
     if (!out || (reinterpret_cast<uintptr_t>(out) & 3u)) return DETOX_ERR_BAD_ARG;
     if (!ws_ok(ws, ws_bytes, krum_ws(nullptr, m, d).total)) return DETOX_ERR_WORKSPACE;
-    return run_bulyan(X, ld, m, d, nullptr, f, out, sel, ws, static_cast<cudaStream_t>(stream));
+    return run_bulyan(X, ld, m, d, nullptr, f, out, sel, ws, nullptr, static_cast<cudaStream_t>(stream));
 }
+
+size_t agg_pairwise_sqdist_workspace_bytes(int m, int64_t d) {
+    if (m < 1 || m > kMaxRows || d < 1) return 0;
+    return kStatusBytes + dist_ws_bytes(m, d);
+}
+
+detox_status agg_pairwise_sqdist(const float* X, int64_t ld, int m, int64_t d, double* D, void* ws, size_t ws_bytes,
+                                 void* stream) {
+    detox_status st = check_matrix(X, ld, m, d);
+    if (st != DETOX_OK) return st;
+    if (!D || (reinterpret_cast<uintptr_t>(D) & 7u)) return DETOX_ERR_BAD_ARG;
+    if (!ws_ok(ws, ws_bytes, kStatusBytes + dist_ws_bytes(m, d))) return DETOX_ERR_WORKSPACE;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    int* status = static_cast<int*>(ws);
+    if (cudaMemsetAsync(status, 0, sizeof(int), s) != cudaSuccess) return DETOX_ERR_CUDA;
+    return launch_sqdist(X, ld, m, d, nullptr, D, static_cast<char*>(ws) + kStatusBytes, status, s);
+}
+
+unsigned long long detox_kernel_launch_count(void) { return g_kernel_launches.load(std::memory_order_relaxed); }
 
 size_t detox_aggregate_workspace_bytes(const detox_pipeline_desc* desc) {
     if (check_desc(desc) != DETOX_OK) return 0;
@@ -413,25 +460,25 @@ detox_status detox_aggregate(const detox_pipeline_desc* p, const float* X, int64
     const int32_t* row_list = nullptr;
     int m = G;
     if (p->a0 == DETOX_AGG_MEAN) {
-        if ((st = launch_vote_mean(X, ld, p->n, p->r, p->d, groups, sets, p->n_sets, w.M, w.ldz, win, w.vote, s)) !=
+        if ((st = launch_vote_mean(X, ld, p->n, p->r, p->d, groups, sets, p->n_sets, w.M, w.ldz, win, w.vote, s, kStatusBytes)) !=
             DETOX_OK)
             return st;
         rows = w.M;
         m = p->n_sets;
     } else if (p->a0 == DETOX_AGG_SIGN_MAJORITY) {
-        // signSGD pairing (Section 5.1, setup 4): coordinate-wise sign majority inside every vote set
-        if ((st = launch_vote(X, ld, p->n, p->r, p->d, groups, w.Z, w.ldz, win, w.vote, s)) != DETOX_OK) return st;
+        // signSGD pairing (Section 5.2, setup 4): coordinate-wise sign majority inside every vote set
+        if ((st = launch_vote(X, ld, p->n, p->r, p->d, groups, w.Z, w.ldz, win, w.vote, s, kStatusBytes)) != DETOX_OK) return st;
         if ((st = launch_hier_mean(w.Z, w.ldz, p->d, sets, p->n_sets, w.M, w.ldz, s, true)) != DETOX_OK) return st;
         rows = w.M;
         m = p->n_sets;
     } else if (krum_type(p->a0)) {
-        // The paper's preferred pairings (Section 5.1, setups 2 and 3): Multi-Krum or Bulyan inside every
+        // The paper's preferred pairings (Section 5.2, setups 2 and 3): Multi-Krum or Bulyan inside every
         // vote set, then A_1.  The vote runs over the groups in set order, so each set's votes are
         // consecutive rows of Z and the aggregators take them as ordinary matrices.
         IdTable in_set_order;
         for (int k = 0; k < G; ++k)
             for (int a = 0; a < p->r; ++a) in_set_order.id[k * p->r + a] = groups.id[sets.member[k] * p->r + a];
-        if ((st = launch_vote(X, ld, p->n, p->r, p->d, in_set_order, w.Z, w.ldz, w.winner_set_order, w.vote, s)) !=
+        if ((st = launch_vote(X, ld, p->n, p->r, p->d, in_set_order, w.Z, w.ldz, w.winner_set_order, w.vote, s, kStatusBytes)) !=
             DETOX_OK)
             return st;
         if ((st = launch_scatter_by_set_order(w.winner_set_order, sets, G, win, s)) != DETOX_OK) return st;
@@ -442,8 +489,8 @@ detox_status detox_aggregate(const detox_pipeline_desc* p, const float* X, int64
             const float* rows_t = w.Z + (int64_t)b * w.ldz;
             float* out_t = w.M + (int64_t)t * w.ldz;
             st = p->a0 == DETOX_AGG_MULTIKRUM
-                     ? run_multikrum(rows_t, w.ldz, k, p->d, nullptr, p->f, keep, out_t, w.sel_local, nullptr, w.agg, s)
-                     : run_bulyan(rows_t, w.ldz, k, p->d, nullptr, p->f, out_t, w.sel_local, w.agg, s);
+                     ? run_multikrum(rows_t, w.ldz, k, p->d, nullptr, p->f, keep, out_t, w.sel_local, nullptr, w.agg, w.status, s)
+                     : run_bulyan(rows_t, w.ldz, k, p->d, nullptr, p->f, out_t, w.sel_local, w.agg, w.status, s);
             if (st != DETOX_OK) return st;
             st = launch_map_set_selection(w.sel_local, keep, sets, b, w.winner_set_order, sel ? sel + emitted : nullptr,
                                           sel_workers ? sel_workers + emitted : nullptr, s);
@@ -455,11 +502,11 @@ detox_status detox_aggregate(const detox_pipeline_desc* p, const float* X, int64
     } else if (votes_by_index(p)) {
         // The votes are rows of X: only winner[] is produced and A_1 reads the winners' rows through it
         // (a group without a majority has winner -1, which the consumers take as a zero row).
-        if ((st = launch_vote(X, ld, p->n, p->r, p->d, groups, nullptr, 0, win, w.vote, s)) != DETOX_OK) return st;
+        if ((st = launch_vote(X, ld, p->n, p->r, p->d, groups, nullptr, 0, win, w.vote, s, kStatusBytes)) != DETOX_OK) return st;
         rows = X;
         row_ld = ld;
         row_list = win;
-    } else if ((st = launch_vote(X, ld, p->n, p->r, p->d, groups, w.Z, w.ldz, win, w.vote, s)) != DETOX_OK) {
+    } else if ((st = launch_vote(X, ld, p->n, p->r, p->d, groups, w.Z, w.ldz, win, w.vote, s, kStatusBytes)) != DETOX_OK) {
         return st;
     }
     int cnt = 0;
@@ -477,12 +524,12 @@ detox_status detox_aggregate(const detox_pipeline_desc* p, const float* X, int64
         case DETOX_AGG_MULTIKRUM:
             cnt = p->m_sel;
             sel_buf = sel ? sel : krum_ws(w.agg, m, p->d).sel;
-            st = run_multikrum(rows, row_ld, m, p->d, row_list, p->f, p->m_sel, out, sel_buf, nullptr, w.agg, s);
+            st = run_multikrum(rows, row_ld, m, p->d, row_list, p->f, p->m_sel, out, sel_buf, nullptr, w.agg, w.status, s);
             break;
         case DETOX_AGG_BULYAN:
             cnt = m - 2 * p->f;
             sel_buf = sel ? sel : krum_ws(w.agg, m, p->d).sel;
-            st = run_bulyan(rows, row_ld, m, p->d, row_list, p->f, out, sel_buf, w.agg, s);
+            st = run_bulyan(rows, row_ld, m, p->d, row_list, p->f, out, sel_buf, w.agg, w.status, s);
             break;
         default: st = DETOX_ERR_BAD_ARG;
     }

@@ -53,21 +53,22 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
 inline size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
 
-inline detox_status launch_status() {
-    return cudaGetLastError() == cudaSuccess ? DETOX_OK : DETOX_ERR_CUDA;
-}
+// Called once after every kernel launch: the launch's error status; also counts the launch (api.cu).
+detox_status launch_status();
 
 // ---- launchers (each enqueues on `s`; none synchronises) ------------------------------------
 
 // vote.cu
 size_t vote_ws_bytes(int n, int r);
+// clear_before: bytes directly in front of `ws` that the launcher's clearing memset zeroes along with the words it
+// uses itself (the pipeline keeps its device status word there)
 detox_status launch_vote(const float* X, int64_t ld, int n, int r, int64_t d, const IdTable& members,
-                         float* Z, int64_t ldz, int32_t* winner, void* ws, cudaStream_t s);
+                         float* Z, int64_t ldz, int32_t* winner, void* ws, cudaStream_t s, size_t clear_before = 0);
 
 // vote + A_0 = mean in one pass: M[s] = mean of the votes of set s; the votes themselves are not stored
 detox_status launch_vote_mean(const float* X, int64_t ld, int n, int r, int64_t d, const IdTable& members,
                               const SetTable& sets, int S, float* M, int64_t ldm, int32_t* winner, void* ws,
-                              cudaStream_t s);
+                              cudaStream_t s, size_t clear_before = 0);
 
 // mean.cu
 // (sign = true: coordinate-wise sign majority sign(sum sign(x)) instead of the mean, in both launchers)
@@ -99,8 +100,9 @@ size_t tc_ws_bytes(int m, int64_t d);
 // sqdist_partials_use_status() holds the kernel clears the device status word itself and may set it to
 // DETOX_ERR_TIMEOUT, so the consumer must leave it alone.
 bool sqdist_partials_use_status(int m, const float* X, int64_t ld, int64_t d);
+// clear_status: whether that kernel clears the word first (false: the word is shared with other stages and only ever set)
 detox_status launch_sqdist_partials(const float* X, int64_t ld, int m, int64_t d, const int32_t* rows, void* ws,
-                                    int* status, int* nblocks, cudaStream_t s);
+                                    int* status, bool clear_status, int* nblocks, cudaStream_t s);
 detox_status launch_sqdist_tc(const float* X, int64_t ld, int m, int64_t d, double* D, void* ws, int* status,
                               cudaStream_t s);
 

@@ -129,12 +129,12 @@ __device__ __forceinline__ void bulk_copy_g2s(void* dst, const void* src, uint32
                  : "memory");
 }
 
-// Rows must be 16-byte aligned (base and pitch).  `status` is cleared by the first CTA and set to
+// Rows must be 16-byte aligned (base and pitch).  `status` is cleared by the first CTA (if clear_status) and set to
 // DETOX_ERR_TIMEOUT when a bounded wait runs out; the partials of that CTA are then NaN.
 template <int M>
 __global__ void __launch_bounds__(kStgThreads, 1)
 sqdist_staged_kernel(const float* __restrict__ X, int64_t ld, int64_t d, const int32_t* __restrict__ rows,
-                     double* __restrict__ partial, int* __restrict__ status) {
+                     double* __restrict__ partial, int* __restrict__ status, int clear_status) {
     constexpr int NP = M * (M - 1) / 2;
     constexpr int kStages = stg_stages(M), kAhead = kStages - 1;
     extern __shared__ __align__(128) uint8_t stage_mem[];      // [kStages][M][kStgPieces] pieces of 16 bytes
@@ -152,7 +152,7 @@ sqdist_staged_kernel(const float* __restrict__ X, int64_t ld, int64_t d, const i
         }
         abort_word = 0;
         mbar_fence_init();
-        if (blockIdx.x == 0) *status = 0;
+        if (blockIdx.x == 0 && clear_status) *status = 0;
     }
     if (tid < M) {
         const int r = rows ? rows[tid] : tid;      // a negative entry of the row list stands for a zero row
@@ -275,7 +275,7 @@ __global__ void sqdist_direct_reduce_kernel(const double* __restrict__ partial, 
             int i = 0, rem = p;
             while (rem >= m - 1 - i) { rem -= m - 1 - i; ++i; }
             const int j = i + 1 + rem;
-            D[i * m + j] = v;
+            D[i * m + j] = v;   // may be NaN (two rows with non-finite entries); the ranking kernels take NaN as +Inf
             D[j * m + i] = v;
         }
     }
@@ -380,7 +380,8 @@ __global__ void dist_from_gram_kernel(const double* __restrict__ gram, int m, do
         if (i == j) { D[e] = 0.0; continue; }
         const int a = i < j ? i : j, b = i < j ? j : i;
         const double v = gram[(int64_t)a * m + a] + gram[(int64_t)b * m + b] - 2.0 * gram[(int64_t)a * m + b];
-        D[e] = v > 0.0 ? v : 0.0;
+        // a NaN (rows with non-finite entries: Inf - Inf) must not turn into "distance zero": it is as far as it gets
+        D[e] = v > 0.0 ? v : (v != v ? __longlong_as_double(0x7ff0000000000000LL) : 0.0);
     }
 }
 
@@ -417,7 +418,7 @@ bool use_staged(int m, const float* X, int64_t ld, int64_t d) {
 // is cleared and used by the staged kernel only.
 template <int M>
 detox_status launch_direct_partials(const float* X, int64_t ld, int64_t d, const int32_t* rows, double* partial,
-                                    int* status, int* nblocks, cudaStream_t s) {
+                                    int* status, bool clear_status, int* nblocks, cudaStream_t s) {
     if constexpr (M >= 9) {
         if (use_staged(M, X, ld, d)) {
             constexpr size_t smem = (size_t)stg_stages(M) * M * kStgPieces * 16;
@@ -425,7 +426,7 @@ detox_status launch_direct_partials(const float* X, int64_t ld, int64_t d, const
                 cudaSuccess)
                 return DETOX_ERR_CUDA;
             *nblocks = kSMs;
-            sqdist_staged_kernel<M><<<kSMs, kStgThreads, smem, s>>>(X, ld, d, rows, partial, status);
+            sqdist_staged_kernel<M><<<kSMs, kStgThreads, smem, s>>>(X, ld, d, rows, partial, status, clear_status ? 1 : 0);
             return launch_status();
         }
     }
@@ -442,7 +443,7 @@ template <int M>
 detox_status launch_direct(const float* X, int64_t ld, int64_t d, const int32_t* rows, double* D, double* partial,
                            int* status, cudaStream_t s) {
     int nb = 0;
-    detox_status st = launch_direct_partials<M>(X, ld, d, rows, partial, status, &nb, s);
+    detox_status st = launch_direct_partials<M>(X, ld, d, rows, partial, status, false, &nb, s);   // the caller cleared it
     if (st != DETOX_OK) return st;
     sqdist_direct_reduce_kernel<<<(M * (M - 1) / 2 + 3) / 4, 128, 0, s>>>(partial, nb, M, D);
     return launch_status();
@@ -464,11 +465,11 @@ bool sqdist_partials_use_status(int m, const float* X, int64_t ld, int64_t d) { 
 // i < j); *nblocks says how many there are.  When sqdist_partials_use_status() holds, the kernel clears the device
 // status word itself and sets it to DETOX_ERR_TIMEOUT if a bounded wait runs out (its partials are then NaN).
 detox_status launch_sqdist_partials(const float* X, int64_t ld, int m, int64_t d, const int32_t* rows, void* ws,
-                                    int* status, int* nblocks, cudaStream_t s) {
+                                    int* status, bool clear_status, int* nblocks, cudaStream_t s) {
     double* partial = static_cast<double*>(ws);
     switch (m) {
 #define DETOX_CASE(M) \
-    case M: return launch_direct_partials<M>(X, ld, d, rows, partial, status, nblocks, s);
+    case M: return launch_direct_partials<M>(X, ld, d, rows, partial, status, clear_status, nblocks, s);
         DETOX_CASE(2) DETOX_CASE(3) DETOX_CASE(4) DETOX_CASE(5) DETOX_CASE(6) DETOX_CASE(7) DETOX_CASE(8)
         DETOX_CASE(9) DETOX_CASE(10) DETOX_CASE(11) DETOX_CASE(12) DETOX_CASE(13) DETOX_CASE(14) DETOX_CASE(15)
         DETOX_CASE(16)

@@ -702,17 +702,21 @@ gram_staged_kernel(const __grid_constant__ CUtensorMap xmap, int m, uint32_t stg
     if (warp == 0) tmem_dealloc(tmem_base, (uint32_t)tmem_cols);
 }
 
-// For one chunk of slabs: gpart[chunk][i*m+j] (i < j) = sum_s sym(T(s))_ij * (r_i(s) + r_j(s)) / 2 with
-// r_i(s) = exact norm / tensor-core norm of row i in slab s; gpart[chunk][i*m+i] = sum_s exact norm
-// (the exact norm of a slab comes in `ngroups` shares, added here in a fixed order).
-// One CTA per pair of 32-row blocks (bi <= bj) and chunk: per slab it reads the tile T[bi][bj] and the
+// For one chunk of slab slots: dpart[chunk][i*m+j] (i < j) = sum over the slots s of the squared distance that slot
+// contributes,
+//     r_i T_ii + r_j T_jj - (r_i + r_j) sym(T)_ij,     sym(T)_ij = (T_ij + T_ji) / 2,
+// with r_i(s) = exact norm / tensor-core norm of row i in slot s (the exact norm comes in `ngroups` shares, added
+// here in a fixed order): the slot's exact norms n_i = r_i T_ii and n_j, minus twice the rescaled inner product.
+// Every product and sum is rounded on its own (no fused multiply-add), so that two bitwise-equal rows, for which
+// T_ii = T_jj = T_ij = T_ji and r_i = r_j, get exactly zero from every slot.
+// One CTA per pair of 32-row blocks (bi <= bj) and chunk: per slot it reads the tile T[bi][bj] and the
 // mirrored tile T[bj][bi] row by row (coalesced) and transposes the second through shared memory.
 constexpr int kRT = 32;
 __global__ void __launch_bounds__(kRT * 8)
 tc_reduce_kernel(const float* __restrict__ partial, const float* __restrict__ norms, int ngroups, int nitems, int m,
-                 int ncol, double* __restrict__ gpart) {
+                 int ncol, double* __restrict__ dpart) {
     __shared__ float mirror[kRT][kRT + 1];
-    __shared__ double ratio_i[kRT], ratio_j[kRT];
+    __shared__ double ratio_i[kRT], ratio_j[kRT], diag_i[kRT], diag_j[kRT];
     const int nt = (m + kRT - 1) / kRT;
     int bi = 0, rem = blockIdx.x;
     while (rem >= nt - bi) { rem -= nt - bi; ++bi; }
@@ -726,7 +730,6 @@ tc_reduce_kernel(const float* __restrict__ partial, const float* __restrict__ no
     double acc[kRT / 8];
 #pragma unroll
     for (int k = 0; k < kRT / 8; ++k) acc[k] = 0.0;
-    double nsum = 0.0;                       // ty == 0 on a diagonal tile: exact norm of row bi*32 + tx
     const int j = bj * kRT + tx;             // this thread's column of the tile
 
     for (int s = s0; s < s1; ++s) {
@@ -734,15 +737,16 @@ tc_reduce_kernel(const float* __restrict__ partial, const float* __restrict__ no
         const float* nrm = norms + (int64_t)s * ngroups * m;   // one share per group of transform warps
         if (ty < 2) {
             const int r = (ty == 0 ? bi : bj) * kRT + tx;
-            double ratio = 1.0;
+            double ratio = 1.0, t = 0.0;
             if (r < m) {
-                const double t = (double)T[(int64_t)r * ncol + r];
+                t = (double)T[(int64_t)r * ncol + r];
                 double nv = 0.0;
                 for (int g = 0; g < ngroups; ++g) nv += (double)nrm[g * m + r];
                 if (t > 0.0) ratio = nv / t;
-                if (ty == 0 && bi == bj) nsum += nv;
+                else t = nv;   // an all-zero row (or a non-finite one): its norm as it is
             }
             (ty == 0 ? ratio_i : ratio_j)[tx] = ratio;
+            (ty == 0 ? diag_i : diag_j)[tx] = t;
         }
         float a[kRT / 8];
 #pragma unroll
@@ -757,7 +761,9 @@ tc_reduce_kernel(const float* __restrict__ partial, const float* __restrict__ no
         for (int k = 0; k < kRT / 8; ++k) {
             const int il = ty + 8 * k;
             const double tij = 0.5 * ((double)a[k] + (double)mirror[tx][il]);
-            acc[k] += tij * (0.5 * (ratio_i[il] + ratio_j[tx]));
+            const double ri = ratio_i[il], rj = ratio_j[tx];
+            const double norms_ij = __dadd_rn(__dmul_rn(ri, diag_i[il]), __dmul_rn(rj, diag_j[tx]));
+            acc[k] += __dadd_rn(norms_ij, -__dmul_rn(__dadd_rn(ri, rj), tij));
         }
         __syncthreads();
     }
@@ -765,14 +771,14 @@ tc_reduce_kernel(const float* __restrict__ partial, const float* __restrict__ no
 #pragma unroll
     for (int k = 0; k < kRT / 8; ++k) {
         const int i = bi * kRT + ty + 8 * k;
-        if (i < m && j < m && i < j) gpart[(int64_t)chunk * total + (int64_t)i * m + j] = acc[k];
+        if (i < m && j < m && i < j) dpart[(int64_t)chunk * total + (int64_t)i * m + j] = acc[k];
     }
-    if (ty == 0 && bi == bj && j < m) gpart[(int64_t)chunk * total + (int64_t)j * m + j] = nsum;
 }
 
-// D_ij = n_i + n_j - 2 G_ij (never negative, zero diagonal); status != 0 -> NaN.
+// D_ij = sum of the chunks' contributions (never negative, zero diagonal); a NaN (rows with non-finite entries)
+// reads as +Inf, "as far as it gets", never as zero; status != 0 -> NaN.
 // One warp per pair i < j: the lanes add the chunks round-robin, then a fixed butterfly.
-__global__ void tc_dist_kernel(const double* __restrict__ gpart, int nchunks, int m, const int* __restrict__ status,
+__global__ void tc_dist_kernel(const double* __restrict__ dpart, int nchunks, int m, const int* __restrict__ status,
                                double* __restrict__ D) {
     const bool bad = *status != 0;
     const int64_t total = (int64_t)m * m;
@@ -785,22 +791,12 @@ __global__ void tc_dist_kernel(const double* __restrict__ gpart, int nchunks, in
         if (lane == 0) D[warp] = bad ? __longlong_as_double(0x7ff8000000000000LL) : 0.0;
         return;
     }
-    double gii = 0.0, gjj = 0.0, gij = 0.0;
-    for (int c = lane; c < nchunks; c += 32) {
-        const double* g = gpart + (int64_t)c * total;
-        gii += g[(int64_t)i * m + i];
-        gjj += g[(int64_t)j * m + j];
-        gij += g[(int64_t)i * m + j];
-    }
+    double v = 0.0;
+    for (int c = lane; c < nchunks; c += 32) v += dpart[(int64_t)c * total + (int64_t)i * m + j];
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-        gii += __shfl_xor_sync(0xffffffffu, gii, o);
-        gjj += __shfl_xor_sync(0xffffffffu, gjj, o);
-        gij += __shfl_xor_sync(0xffffffffu, gij, o);
-    }
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
     if (lane == 0) {
-        double v = gii + gjj - 2.0 * gij;
-        v = v > 0.0 ? v : 0.0;
+        v = v > 0.0 ? v : (v != v ? __longlong_as_double(0x7ff0000000000000LL) : 0.0);
         if (bad) v = __longlong_as_double(0x7ff8000000000000LL);
         D[(int64_t)i * m + j] = v;
         D[(int64_t)j * m + i] = v;

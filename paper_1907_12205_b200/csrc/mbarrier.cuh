@@ -40,15 +40,16 @@ __device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
-// Bounded wait (about a second of SM clocks).  Returns false, and raises the CTA-wide abort flag,
-// when the limit is hit; returns false at once when another thread has already given up.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status) {
+// Bounded wait (`limit` SM clocks, about a second by default).  Returns false, and raises the CTA-wide abort
+// flag, when the limit is hit; returns false at once when another thread has already given up.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status,
+                                          long long limit = kWaitLimitCycles) {
     if (mbar_try(bar, parity)) return true;
     const long long start = clock64();
     for (;;) {
         if (mbar_try(bar, parity)) return true;
         if (*abort_flag) return false;
-        if (clock64() - start > kWaitLimitCycles) break;
+        if (clock64() - start > limit) break;
     }
     *abort_flag = 1;
     atomicExch(status, (int)DETOX_ERR_TIMEOUT);

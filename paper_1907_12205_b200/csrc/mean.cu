@@ -1,7 +1,7 @@
 // Streaming means: A_0 = mean over each vote group (Algorithm 2, step 3) and the average of the rows
 // selected by Multi-Krum.  One pass: k*d*4 bytes read, d*4 bytes written per output row.
 // The same kernels, with SIGN set, give the coordinate-wise sign majority used with signSGD
-// (Section 5.1, setup 4): sign(sum_i sign(x_i)), in {-1, 0, +1}.
+// (Section 5.2, setup 4): sign(sum_i sign(x_i)), in {-1, 0, +1}.
 #include "common.cuh"
 
 namespace detox {

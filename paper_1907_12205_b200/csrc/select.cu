@@ -22,6 +22,9 @@ namespace {
 
 constexpr int kFreshSumBelow = 8;   // Bulyan rounds with at most this many neighbours re-add them from scratch
 
+// NaN compares false with everything, which would break the ranking below: it is ranked as +Inf.
+__device__ __forceinline__ double nan_to_inf(double v) { return v != v ? CUDART_INF : v; }
+
 struct SelectWs {
     double* sorted_d;    // m x m, row i ascending, self at the end (+inf)
     int32_t* sorted_j;   // m x m, matching column indices
@@ -47,7 +50,9 @@ rank_rows_kernel(const double* __restrict__ D, int m, double* __restrict__ sorte
                  int32_t* __restrict__ pos_t) {
     extern __shared__ double rowv[];  // m
     const int i = blockIdx.x;
-    for (int j = threadIdx.x; j < m; j += blockDim.x) rowv[j] = (j == i) ? CUDART_INF : D[(int64_t)i * m + j];
+    // a NaN distance (a row with non-finite entries, or a distance pass that gave up) counts as +Inf, so that the
+    // ranks below are always a permutation of 0..m-1 and every slot of the lists is written
+    for (int j = threadIdx.x; j < m; j += blockDim.x) rowv[j] = (j == i) ? CUDART_INF : nan_to_inf(D[(int64_t)i * m + j]);
     __syncthreads();
     for (int j = threadIdx.x; j < m; j += blockDim.x) {
         int rank;
@@ -138,7 +143,8 @@ __device__ __forceinline__ void bulyan_select_body(const double* sorted_d, const
     const int theta = m - 2 * f;
     for (int round = 0; round < theta; ++round) {
         // argmin over (score, index) among the remaining rows
-        double s = (mine && alive[i]) ? sum : CUDART_INF;
+        // (Inf - Inf from a non-finite row gives a NaN sum: it competes as +Inf, so the winner is always a remaining row)
+        double s = (mine && alive[i]) ? nan_to_inf(sum) : CUDART_INF;
         int idx = (mine && alive[i]) ? i : 0x7fffffff;
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) {
@@ -262,8 +268,8 @@ krum_small_kernel(const double* __restrict__ partial, int nblocks, int m, int f,
             int i = 0, rem = p;
             while (rem >= m - 1 - i) { rem -= m - 1 - i; ++i; }
             const int j = i + 1 + rem;
-            dmat[i][j] = v;
-            dmat[j][i] = v;
+            dmat[i][j] = nan_to_inf(v);   // non-finite rows: Inf - Inf between two of them is as far as it gets
+            dmat[j][i] = nan_to_inf(v);
         }
     }
     if (tid < m) dmat[tid][tid] = CUDART_INF;   // a row never counts itself: it goes to the end of its own list

@@ -361,10 +361,11 @@ size_t vote_ws_bytes(int n, int r) {
 }
 
 detox_status launch_vote(const float* X, int64_t ld, int n, int r, int64_t d, const IdTable& members,
-                         float* Z, int64_t ldz, int32_t* winner, void* ws, cudaStream_t s) {
+                         float* Z, int64_t ldz, int32_t* winner, void* ws, cudaStream_t s, size_t clear_before) {
     const int G = n / r;
     uint32_t* pairdiff = static_cast<uint32_t*>(ws);
-    if (cudaMemsetAsync(pairdiff, 0, (size_t)G * kPairWords * sizeof(uint32_t), s) != cudaSuccess)
+    if (cudaMemsetAsync(static_cast<char*>(ws) - clear_before, 0,
+                        clear_before + (size_t)G * kPairWords * sizeof(uint32_t), s) != cudaSuccess)
         return DETOX_ERR_CUDA;
     const bool vec = aligned16(X) && ld % 4 == 0 && (!Z || (aligned16(Z) && ldz % 4 == 0));
     detox_status st = vec ? launch_vote_vec<4>(X, ld, G, r, d, members, Z, ldz, pairdiff, s)
@@ -382,10 +383,11 @@ detox_status launch_vote(const float* X, int64_t ld, int n, int r, int64_t d, co
 
 detox_status launch_vote_mean(const float* X, int64_t ld, int n, int r, int64_t d, const IdTable& members,
                               const SetTable& sets, int S, float* M, int64_t ldm, int32_t* winner, void* ws,
-                              cudaStream_t s) {
+                              cudaStream_t s, size_t clear_before) {
     const int G = n / r;
     uint32_t* pairdiff = static_cast<uint32_t*>(ws);
-    if (cudaMemsetAsync(pairdiff, 0, (size_t)G * kPairWords * sizeof(uint32_t), s) != cudaSuccess)
+    if (cudaMemsetAsync(static_cast<char*>(ws) - clear_before, 0,
+                        clear_before + (size_t)G * kPairWords * sizeof(uint32_t), s) != cudaSuccess)
         return DETOX_ERR_CUDA;
     const bool vec = aligned16(X) && ld % 4 == 0 && aligned16(M) && ldm % 4 == 0;
     detox_status st = vec ? launch_vote_mean_vec<4>(X, ld, r, d, members, sets, S, M, ldm, pairdiff, s)

@@ -40,3 +40,23 @@ def bulyan_min_gap(D: np.ndarray, f: int) -> float:
         pick = min((i for i in range(m) if alive[i]), key=lambda i: (sc[i], i))
         alive[pick] = 0
     return worst
+
+
+def check_bulyan_selection(D: np.ndarray, f: int, sel, tol: float) -> bool:
+    """Checks a Bulyan selection sequence against the oracle's scores, round by round, following the sequence
+    itself: every pick must be a remaining row whose fp64 score is the minimum (ties: the lowest index) or, at a
+    near-tie, within `tol` (relative) of the minimum.  Returns True when every pick was the oracle's own."""
+    m = D.shape[0]
+    alive = np.ones(m, np.uint8)
+    exact = True
+    assert len(sel) == m - 2 * f
+    for rnd, pick in enumerate(int(x) for x in sel):
+        sc = oracle.krum_scores(D, f, alive)
+        best = min((i for i in range(m) if alive[i]), key=lambda i: (sc[i], i))
+        assert 0 <= pick < m and alive[pick], f"round {rnd}: row {pick} is not a remaining row"
+        if pick != best:
+            exact = False
+            gap = abs(sc[pick] - sc[best]) / max(abs(sc[best]), 1e-300)
+            assert gap <= tol, f"round {rnd}: picked row {pick} (score {sc[pick]}) over row {best} ({sc[best]})"
+        alive[pick] = 0
+    return exact

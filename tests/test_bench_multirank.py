@@ -52,9 +52,12 @@ def test_single_process_is_passthrough():
 
 def test_median_operation_count_of_small_networks():
     """Three inputs: comparators (0,1), (0,2), (1,2); the middle output needs min of the last, max of the second and
-    both outputs of the first = 4 operations.  One input needs none; sizes beyond the register path report 0."""
+    both outputs of the first = 4 operations.  One input needs none; 129 to 256 rows are counted for the two-lane
+    scheme (two full sorts of half the rows, the split and the reduction); larger sizes report 0."""
     import bench
     assert bench.median_minmax_ops(1) == 0
     assert bench.median_minmax_ops(3) == 4
-    assert bench.median_minmax_ops(200) == 0
+    assert bench.median_minmax_ops(300) == 0
+    H = 104                                   # 200 rows: two lanes of 104 keys
+    assert bench.median_minmax_ops(200) == 2 * (2 * len(bench.merge_exchange_net(H)) + 2 * H - 1)
     assert bench.median_minmax_ops(45) < bench.median_minmax_ops(105)

@@ -285,6 +285,24 @@ def test_bulyan_hand_worked_scalar_example():
     assert sel.tolist() == brute_bulyan_select(D, 1)
 
 
+def test_bulyan_selection_order_worked_by_hand():
+    # The same column, every round written out (squared distances; ties go to the lower index):
+    #   round 1, 7 rows, 4 neighbours: scores 30 15 10 10 15 30 37254      -> row 2 (ties with row 3)
+    #   round 2, 6 rows, 3 neighbours: rows 0 1 3 4 5 6: 26 14 9 11 21 27650 -> row 3
+    #   round 3, 5 rows, 2 neighbours: rows 0 1 4 5 6: 17 10 10 17 18241    -> row 1 (ties with row 4)
+    #   round 4, 4 rows, 1 neighbour : rows 0 4 5 6: 16 1 1 9025            -> row 4 (ties with row 5)
+    #   round 5, 3 rows, 3 - 1 - 2 = 0 neighbours, clamped to 1: rows 0 5 6: 25 25 9025 -> row 0 (ties with row 5)
+    # Selected values 2 3 1 4 0: median 2, the three closest are 1 2 3, mean 2.
+    X = np.array([[0.0], [1.0], [2.0], [3.0], [4.0], [5.0], [100.0]], np.float32)
+    out, sel, D = oracle.bulyan(X, f=1)
+    assert sel.tolist() == [2, 3, 1, 4, 0]
+    assert out.tolist() == [2.0]
+    alive = np.ones(7, np.uint8)
+    assert oracle.krum_scores(D, 1, alive).tolist() == [30.0, 15.0, 10.0, 10.0, 15.0, 30.0, 37254.0]
+    alive[[2, 3]] = 0
+    assert oracle.krum_scores(D, 1, alive)[[0, 1, 4, 5, 6]].tolist() == [17.0, 10.0, 10.0, 17.0, 18241.0]
+
+
 def test_trimmed_around_median_reductions_and_brute_force():
     g = rng(18)
     theta, d = 9, 200
@@ -359,7 +377,7 @@ def test_pipeline_honest_majority_equals_aggregator_on_true_gradients():
 
 
 def test_pipeline_krum_family_inside_vote_sets():
-    # Section 5.1, setups 2 and 3: the aggregator inside every vote group, then the mean.
+    # Section 5.2, setups 2 and 3: the aggregator inside every vote group, then the mean.
     G, r, d = 15, 3, 128
     honest = rng(30).standard_normal((G, d)).astype(np.float32)
     members = rng(31).permutation(G * r).astype(np.int32)
@@ -447,3 +465,13 @@ def test_sign_majority_against_numpy_and_hand_worked_column():
     assert oracle.sign_majority(col).tolist() == [0.0]
     assert oracle.sign_majority(col[:3]).tolist() == [-1.0]
     assert np.array_equal(oracle.sign_majority(X, [2, 5, 7]), np.sign(np.sign(X[[2, 5, 7]]).sum(0)).astype(np.float32))
+
+
+def test_selection_checker_accepts_the_oracles_own_sequence_and_rejects_a_wrong_one():
+    from helpers import check_bulyan_selection
+    X = np.array([[0.0], [1.0], [2.0], [3.0], [4.0], [5.0], [100.0]], np.float32)
+    D = oracle.sqdist(X)
+    assert check_bulyan_selection(D, 1, [2, 3, 1, 4, 0], 1e-9) is True
+    assert check_bulyan_selection(D, 1, [3, 2, 1, 4, 0], 1e-9) is False     # rows 2 and 3 tie exactly in round 1
+    with pytest.raises(AssertionError):
+        check_bulyan_selection(D, 1, [6, 3, 1, 4, 0], 1e-9)

@@ -172,3 +172,53 @@ def test_pipeline_long_rows_with_a_zero_vote_through_the_staged_distance_kernel(
     assert ref["winner"][1] == -1 and res["winner"].cpu().numpy().tolist() == ref["winner"].tolist()
     assert res["sel"].cpu().numpy().tolist() == ref["sel"].tolist()
     assert rel_l2(res["out"].cpu().numpy(), ref["out"]) <= TOL
+
+
+@pytest.mark.parametrize("M", list(range(9, 17)))
+def test_bulk_copy_distance_kernel_for_every_row_count(M):
+    """9 to 16 rows of just over 606,208 columns take the bulk-copy ring (one template instance per row count):
+    a ragged last tile, a length that is not a multiple of four, and, through the pipeline, a zero vote."""
+    d = 606_208 + 4 * 37 + 1
+    for attempt in range(8):
+        X = krum_inputs(M, d, seed=50 * M + 1000 * attempt, copies=1, outliers=2)
+        out_o, sel_o, sc_o, _ = oracle.multikrum(X, 2, M - 3)
+        if multikrum_min_gap(sc_o, M - 3) > 1e-5:
+            break
+    out, sel, sc = dx.agg_multikrum(padded(X), 2, M - 3)
+    assert sel.cpu().numpy().tolist() == sel_o.tolist()
+    np.testing.assert_allclose(sc.cpu().numpy(), sc_o, rtol=2e-6, atol=1e-30)
+    assert rel_l2(out.cpu().numpy(), out_o) <= TOL
+    # the same rows as the votes of M groups of three, the second group without a majority (its vote is zero)
+    import workloads as wl
+    spec = wl.WorkloadSpec("p", n=3 * M, r=3, d=d, sigma=1e-3, q=0, group_jitter=0.2, seed=M)
+    w = wl.make_workload(spec)
+    grp = w.members[3:6]
+    w.X[int(grp[0]), 7] += 1.0
+    w.X[int(grp[1]), d - 1] += 1.0
+    pipe = dx.Pipeline(3 * M, 3, d, w.members, dx.AGG_NONE, None, None, dx.AGG_MULTIKRUM, 1, M - 2)
+    res = dx.detox_aggregate(pipe, w.X.to("cuda:0")[:, :d])
+    ref = oracle.detox_aggregate(w.data().numpy(), w.members, 3, "none", None, None, "multikrum", 1, M - 2)
+    assert ref["winner"][1] == -1 and res["winner"].cpu().numpy().tolist() == ref["winner"].tolist()
+    assert res["sel"].cpu().numpy().tolist() == ref["sel"].tolist()
+    assert rel_l2(res["out"].cpu().numpy(), ref["out"]) <= TOL
+
+
+@pytest.mark.parametrize("m,d", [(9, 5001), (20, 5001), (140, 3000), (9, 700_001)])
+def test_a_row_with_an_infinite_entry_is_never_selected(m, d):
+    """A Byzantine row may hold anything.  One +Inf makes the row infinitely far from every other row on both
+    sides (direct differences give Inf; the Gram path's NaN counts as Inf), so Multi-Krum and Bulyan leave it out
+    and the selections match the oracle."""
+    f = 2 if m >= 11 else 1
+    for attempt in range(8):
+        X = krum_inputs(m, d, seed=9 * m + 1000 * attempt, copies=1, outliers=1)
+        X[3, d // 2] = np.inf
+        _, sel_o, sc_o, D_o = oracle.multikrum(X, f, m - f, want_out=False)
+        if multikrum_min_gap(sc_o[np.isfinite(sc_o)], m - f) > 1e-5 and bulyan_min_gap(D_o, f) > 5e-6:
+            break
+    assert 3 not in sel_o.tolist()
+    out, sel, sc = dx.agg_multikrum(padded(X), f, m - f)
+    assert sel.cpu().numpy().tolist() == sel_o.tolist()
+    assert torch.isfinite(out).all()
+    _, bsel = dx.agg_bulyan(padded(X), f)
+    bsel_o = oracle.bulyan_select(D_o, f)
+    assert 3 not in bsel_o.tolist() and bsel.cpu().numpy().tolist() == bsel_o.tolist()

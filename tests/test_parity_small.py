@@ -163,7 +163,7 @@ def test_sign_majority_bit_exact(m, d):
 
 
 def test_pipeline_signsgd_pairing():
-    # Section 5.1, setup 4: sign majority inside the vote sets and over their results; constant attack (-1)
+    # Section 5.2, setup 4: sign majority inside the vote sets and over their results; constant attack (-1)
     spec = wl.WorkloadSpec("p", n=45, r=3, d=30_001, sigma=1.0, q=5, attack="constant", placement="worst", set_size=5,
                            seed=8)
     w = wl.make_workload(spec)
@@ -354,7 +354,7 @@ def test_pipeline_fused_vote_mean_handles_no_majority_and_uneven_sets(r, G, set_
 @pytest.mark.parametrize("a0,f,m_sel,offs,a1", [("multikrum", 1, 0, [0, 7, 15], "mean"), ("bulyan", 2, 0, [0, 15], "mean"),
                                                  ("multikrum", 1, 3, [0, 5, 10, 15], "coord_median")])
 def test_pipeline_krum_family_inside_vote_sets(a0, f, m_sel, offs, a1):
-    # the paper's preferred pairings (Section 5.1, setups 2 and 3; set shapes of Appendix B.1)
+    # the paper's preferred pairings (Section 5.2, setups 2 and 3; set shapes of Appendix B.1)
     code = {"multikrum": dx.AGG_MULTIKRUM, "bulyan": dx.AGG_BULYAN, "mean": dx.AGG_MEAN,
             "coord_median": dx.AGG_COORD_MEDIAN}
     for attempt in range(16):

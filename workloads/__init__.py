@@ -4,6 +4,9 @@ The CUDA library and the CPU oracle are both fed from this module and from nothi
 """
 from .gen import (  # noqa: F401
     CONFIGS,
+    RESNET18_D,
+    RESNET50_D,
+    VGG_D,
     Workload,
     WorkloadSpec,
     expected_byzantine_votes,
@@ -12,5 +15,6 @@ from .gen import (  # noqa: F401
     make_workload,
     padded_ld,
     place_byzantine,
+    sweep_legs,
     sweep_specs,
 )

@@ -252,3 +252,23 @@ def sweep_specs(ns=(15, 45, 105, 225), ds=(1_000_000, RESNET18_D, RESNET50_D),
                                         attack=a, placement="random", set_size=5,
                                         group_jitter=0.02, seed=seed))
     return out
+
+
+def sweep_legs(spec: WorkloadSpec, G: int, S: int) -> dict:
+    """Which aggregations a sweep point runs (configuration only: names and parameters, no arithmetic).
+
+    DETOX legs: the median of the set means (of the votes when there are fewer than three sets), and
+    Multi-Krum / Bulyan over the G votes with a tolerance f_votes for the few Byzantine votes that survive the
+    filter.  Direct legs: the same aggregators over all n rows with f = q.  Bulyan only where rows >= 4 f + 3."""
+    fv = min(2, max((G - 3) // 4, 0))
+    n, q = spec.n, spec.q
+    legs = {
+        "detox_median": dict(a0="mean" if S >= 3 else "none", a1="coord_median", f=0, m_sel=1),
+        "detox_multikrum": dict(a0="none", a1="multikrum", f=fv, m_sel=G - fv),
+        "detox_bulyan": dict(a0="none", a1="bulyan", f=fv, m_sel=1),
+        "direct_median": dict(a1="coord_median"),
+        "direct_multikrum": dict(a1="multikrum", f=q, m_sel=n - q),
+    }
+    if n >= 4 * q + 3:
+        legs["direct_bulyan"] = dict(a1="bulyan", f=q)
+    return legs
