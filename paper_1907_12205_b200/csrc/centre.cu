@@ -1,13 +1,16 @@
-// Choice of a centring row for the tensor-core distance pass.
+// Choice of the centring rows for the tensor-core distance pass.
 //
 // The tensor-core path forms D_ij = |a_i|^2 + |a_j|^2 - 2 a_i.a_j from inner products, which loses accuracy when the
 // rows share a large common vector (honest gradients of one loss at one model do): the three terms are then much
-// larger than their difference.  Distances do not change when one vector is subtracted from every row, so the pass
-// may work on a_i = x_i - x_k for a row k that lies in the middle of the rows.  Here k is found on a sample of the
-// columns: squared distances between all rows over a few evenly spaced column blocks (formed as differences, so
-// they are accurate whatever the rows share), then for every row the median of its distances to the others; k is
-// the row whose median is smallest.  Centring is switched on only when it at least halves the typical squared norm
-// (the rows' own sample norms against their sample distances to k); rows that hover around zero are left as they are.
+// larger than their difference, and the tensor cores' fp32 accumulation loses most on long sums of one sign.
+// Distances do not change when one vector is subtracted from every row, so the pass may work on a_i = x_i - c with c
+// in the middle of the rows; it forms c, column by column, as the mean of a few rows that are listed here.  The rows
+// are found on a sample of the columns: squared distances between all rows over a few evenly spaced column blocks
+// (formed as differences, so they are accurate whatever the rows share), then for every row the median of its
+// distances to the others; the rows are ranked by that median and every s-th of the more central half is taken (so
+// that a group of colluding rows that sit in the very middle cannot fill the list).  Centring is switched on only
+// when the most central row is closer to the typical row than the origin is by a clear margin; rows that hover around
+// zero are left as they are.
 //
 // Everything is deterministic: per-block partial sums are added in a fixed order and ties go to the lower index.
 #include <math_constants.h>
@@ -19,6 +22,7 @@ namespace detox {
 namespace {
 
 constexpr int kPickThreads = 256;
+constexpr int kMaxCentreRows = 16;   // as in the distance kernels
 
 struct CentrePlan {
     int cols;      // columns per sampled block
@@ -43,7 +47,8 @@ struct CentreWs {
     float* part;        // [nblk][m*m]: entry i*m+j (i < j) = squared distance over the block; i*m+i = squared norm
     float* key;         // [m] median sample distance of row i to the others
     float* nrm;         // [m] sample squared norm
-    unsigned* counter;  // [2] CTAs of the pick kernel / of the check kernel that have finished
+    unsigned* counter;  // [2] CTAs of the pick kernel / of the check kernel that have finished; behind them one float:
+                        // the typical squared norm of a row as the sample predicts it for all d columns
 };
 
 CentreWs centre_carve(void* ws, int m, int nblk) {
@@ -100,8 +105,8 @@ centre_sample_kernel(const float* __restrict__ X, int64_t ld, int m, int64_t d, 
 // One CTA per row: the median of the row's sample distances to the other rows and its sample norm; the CTA that
 // finishes last picks the row with the smallest median and decides whether centring pays.
 __global__ void __launch_bounds__(kPickThreads)
-centre_pick_kernel(const float* __restrict__ part, int nblk, int m, float* __restrict__ key, float* __restrict__ nrm,
-                   unsigned* __restrict__ counter, int* __restrict__ centre) {
+centre_pick_kernel(const float* __restrict__ part, int nblk, int m, float scale, float* __restrict__ key,
+                   float* __restrict__ nrm, unsigned* __restrict__ counter, int* __restrict__ centre) {
     extern __shared__ float rowv[];   // [m]
     __shared__ float s_val[kPickThreads];
     __shared__ int s_idx[kPickThreads];
@@ -157,7 +162,6 @@ centre_pick_kernel(const float* __restrict__ part, int nblk, int m, float* __res
         __syncthreads();
     }
     const float best_key = s_val[0];
-    const int best_row = s_idx[0];
     __syncthreads();
     // median of the sample norms (rank counting again; rowv is free now)
     for (int r = threadIdx.x; r < m; r += kPickThreads) rowv[r] = __ldcg(nrm + r);
@@ -170,67 +174,79 @@ centre_pick_kernel(const float* __restrict__ part, int nblk, int m, float* __res
             const float u = rowv[k];
             rank += (u < v || (u == v && k < r)) ? 1 : 0;
         }
-        if (rank == hm) *centre = (best_row < m && best_key < 0.5f * v) ? best_row : -1;
+        if (rank == hm) s_val[0] = v;
+    }
+    __syncthreads();
+    // on when the most central row's typical distance to the others is clearly below what two rows that hover around
+    // zero have (twice the typical squared norm)
+    const int want = m / 2 < kMaxCentreRows ? m / 2 : kMaxCentreRows;
+    const bool on = best_key < 1.5f * s_val[0] && want >= 1;
+    // the rows at ranks 0, s, 2s, ... of the ordering by median distance, inside its more central half
+    const int stride = (m / 2) / (want > 0 ? want : 1) > 1 ? (m / 2) / want : 1;
+    for (int r = threadIdx.x; r < m; r += kPickThreads) rowv[r] = __ldcg(key + r);
+    __syncthreads();
+    for (int r = threadIdx.x; r < m; r += kPickThreads) {
+        const float v = rowv[r];
+        int rank = 0;
+        for (int k = 0; k < m; ++k) {
+            const float u = rowv[k];
+            rank += (u < v || (u == v && k < r)) ? 1 : 0;
+        }
+        if (rank % stride == 0 && rank / stride < want) centre[2 + rank / stride] = r;
+    }
+    if (threadIdx.x == 0) {
+        centre[0] = on ? want : 0;
+        *reinterpret_cast<float*>(counter + 2) = s_val[0] * scale;   // for the check after the pass
     }
 }
 
-// After the distance pass: is the centred data really smaller?  norms / xnorms hold, per output slot and group of
-// transform warps, every row's exact squared norm after and before the subtraction.  One CTA per row adds its two
-// norms up; the last one compares the medians over the rows.  If the typical row did not get smaller the centre is
-// withdrawn (*centre = -1) and *redo = 1 asks for the pass to be repeated without it.
+// After the distance pass: did the subtraction leave the rows small?  The listed rows were chosen on a sample of the
+// columns; a row that is central there and holds huge values elsewhere would, once subtracted, swamp the differences
+// between the other rows.  `norms` holds, per output slot and group of transform warps, every row's exact squared
+// norm after the subtraction.  One CTA per row adds its shares up; the last one takes the median over the rows and
+// compares it with what the sample predicted for the rows as they came.  If the typical row is more than 16 times
+// larger than that, the centring is withdrawn (centre[0] = 0) and *redo = 1 asks for the pass to be repeated without it.
+constexpr float kCentreSlack = 16.f;
 __global__ void __launch_bounds__(128)
-centre_check_kernel(const float* __restrict__ norms, const float* __restrict__ xnorms, int nshares, int m,
-                    float* __restrict__ na, float* __restrict__ nx, unsigned* __restrict__ counter,
-                    int* __restrict__ centre, int* __restrict__ redo) {
-    __shared__ double red[2][4];
+centre_check_kernel(const float* __restrict__ norms, int nshares, int m, float* __restrict__ na,
+                    unsigned* __restrict__ counter, int* __restrict__ centre, int* __restrict__ redo) {
+    __shared__ double red[4];
     __shared__ bool s_last;
     const int i = blockIdx.x;
-    if (*centre < 0) {
+    if (*centre <= 0) {
         if (i == 0 && threadIdx.x == 0) *redo = 0;
         return;
     }
-    double a = 0.0, x = 0.0;
-    for (int s = threadIdx.x; s < nshares; s += 128) {
-        a += (double)norms[(int64_t)s * m + i];
-        x += (double)xnorms[(int64_t)s * m + i];
-    }
+    double a = 0.0;
+    for (int s = threadIdx.x; s < nshares; s += 128) a += (double)norms[(int64_t)s * m + i];
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-        a += __shfl_xor_sync(0xffffffffu, a, o);
-        x += __shfl_xor_sync(0xffffffffu, x, o);
-    }
-    if ((threadIdx.x & 31) == 0) { red[0][threadIdx.x >> 5] = a; red[1][threadIdx.x >> 5] = x; }
+    for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = a;
     __syncthreads();
     if (threadIdx.x == 0) {
-        na[i] = nan_to_inf((float)(red[0][0] + red[0][1] + red[0][2] + red[0][3]));
-        nx[i] = nan_to_inf((float)(red[1][0] + red[1][1] + red[1][2] + red[1][3]));
+        na[i] = nan_to_inf((float)(red[0] + red[1] + red[2] + red[3]));
         __threadfence();
-        s_last = atomicAdd(counter, 1u) == (unsigned)(m - 1);
+        s_last = atomicAdd(counter + 1, 1u) == (unsigned)(m - 1);
     }
     __syncthreads();
     if (!s_last) return;
     __threadfence();
-    // medians by rank counting, one thread per row (m <= 256 on this path: two rows per thread at most)
-    __shared__ float med[2];
+    // median by rank counting (m <= 256 on this path: two rows per thread at most)
     const int hm = (m - 1) / 2;
-    for (int which = 0; which < 2; ++which) {
-        const float* v = which == 0 ? na : nx;
-        for (int r = threadIdx.x; r < m; r += 128) {
-            const float mine = __ldcg(v + r);
-            int rank = 0;
-            for (int k = 0; k < m; ++k) {
-                const float u = __ldcg(v + k);
-                rank += (u < mine || (u == mine && k < r)) ? 1 : 0;
-            }
-            if (rank == hm) med[which] = mine;
+    const float ref = *reinterpret_cast<const float*>(counter + 2);
+    for (int r = threadIdx.x; r < m; r += 128) {
+        const float mine = __ldcg(na + r);
+        int rank = 0;
+        for (int k = 0; k < m; ++k) {
+            const float u = __ldcg(na + k);
+            rank += (u < mine || (u == mine && k < r)) ? 1 : 0;
         }
-    }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        const bool keep = med[0] <= med[1];
-        *redo = keep ? 0 : 1;
-        if (!keep) *centre = -1;
-        *counter = 0u;
+        if (rank == hm) {
+            const bool keep = mine <= kCentreSlack * ref;
+            *redo = keep ? 0 : 1;
+            if (!keep) *centre = 0;
+            counter[1] = 0u;
+        }
     }
 }
 
@@ -238,7 +254,7 @@ centre_check_kernel(const float* __restrict__ norms, const float* __restrict__ x
 
 size_t centre_ws_bytes(int m, int64_t d) {
     const CentrePlan p = centre_plan(m, d);
-    return align_up((size_t)p.nblk * m * m * sizeof(float)) + 2 * align_up((size_t)m * sizeof(float)) + 256;
+    return align_up((size_t)p.nblk * m * m * sizeof(float)) + 2 * align_up((size_t)m * sizeof(float)) + 256;   // counters, float
 }
 
 detox_status launch_pick_centre(const float* X, int64_t ld, int m, int64_t d, void* ws, int* centre, cudaStream_t s) {
@@ -251,17 +267,21 @@ detox_status launch_pick_centre(const float* X, int64_t ld, int m, int64_t d, vo
                                                                                           w.counter);
     detox_status st = launch_status();
     if (st != DETOX_OK) return st;
-    centre_pick_kernel<<<m, kPickThreads, (size_t)m * sizeof(float), s>>>(w.part, p.nblk, m, w.key, w.nrm, w.counter, centre);
+    // the sample's squared norms are scaled up to all d columns for the check after the pass
+    const int64_t sampled = (int64_t)p.nblk * p.cols < d ? (int64_t)p.nblk * p.cols : d;
+    const float scale = (float)((double)d / (double)sampled);
+    centre_pick_kernel<<<m, kPickThreads, (size_t)m * sizeof(float), s>>>(w.part, p.nblk, m, scale, w.key, w.nrm, w.counter,
+                                                                         centre);
     return launch_status();
 }
 
-detox_status launch_check_centre(const float* norms, const float* xnorms, int nshares, int m, void* ws, int64_t d,
-                                 int* centre, int* redo, cudaStream_t s) {
+detox_status launch_check_centre(const float* norms, int nshares, int m, void* ws, int64_t d, int* centre, int* redo,
+                                 cudaStream_t s) {
     const CentrePlan p = centre_plan(m, d);
     CentreWs w = centre_carve(ws, m, p.nblk);
-    // the pick kernel is done with key / nrm: they hold the two exact norms now; the second counter word was
-    // cleared by the sample kernel
-    centre_check_kernel<<<m, 128, 0, s>>>(norms, xnorms, nshares, m, w.key, w.nrm, w.counter + 1, centre, redo);
+    // the pick kernel is done with `key`: it holds the exact norms now; the second counter word was cleared by the
+    // sample kernel
+    centre_check_kernel<<<m, 128, 0, s>>>(norms, nshares, m, w.key, w.counter, centre, redo);
     return launch_status();
 }
 

@@ -106,6 +106,17 @@ detox_status launch_sqdist_partials(const float* X, int64_t ld, int m, int64_t d
 detox_status launch_sqdist_tc(const float* X, int64_t ld, int m, int64_t d, double* D, void* ws, int* status,
                               cudaStream_t s);
 
+// centre.cu: the centring rows for the tensor-core distance pass (m <= 256), chosen on a sample of the columns
+//   centre[0] = how many rows are averaged into the vector that is subtracted from every row (0 when the rows hover
+//   around zero anyway), centre[1] = redo flag (below), centre[2..17] = the rows
+size_t centre_ws_bytes(int m, int64_t d);
+detox_status launch_pick_centre(const float* X, int64_t ld, int m, int64_t d, void* ws, int* centre, cudaStream_t s);
+//   after the pass: norms = the rows' exact squared norms after the subtraction, in nshares x m shares; withdraws
+//   the centring (centre[0] = 0, *redo = 1) when the typical row came out far larger than the sample predicted for the
+//   rows as they were (*redo = 0 otherwise)
+detox_status launch_check_centre(const float* norms, int nshares, int m, void* ws, int64_t d, int* centre, int* redo,
+                                 cudaStream_t s);
+
 // geomed.cu: Weiszfeld iterations for the geometric median of m <= 32 rows
 size_t geomed_ws_bytes(int64_t d);
 detox_status launch_geometric_median(const float* X, int64_t ld, int m, int64_t d, int iters, float eps, float* out,

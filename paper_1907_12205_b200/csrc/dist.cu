@@ -5,8 +5,9 @@
 //             registers; HBM-bound (m*d*4 bytes read once).  From 9 rows on, long 16-byte aligned rows are
 //             streamed through shared memory with bulk copies so that the copies overlap the arithmetic.
 //   16 < m <= 256 with 16-byte aligned rows: the tensor-core Gram of gram_tc.cu.
-//   otherwise : CUDA-core Gram tiles G = X X^T over K-slabs, D_ij = G_ii + G_jj - 2 G_ij.
-// Both write per-CTA partial sums that a second kernel adds in a fixed order in fp64, so results
+//   otherwise : CUDA-core tiles of squared differences over K-slabs (rows that are not 16-byte aligned, more than
+//             256 rows).
+// All write per-CTA partial sums that a second kernel adds in a fixed order in fp64, so results
 // are deterministic and bitwise-equal rows get bitwise-equal distances.
 #include "common.cuh"
 #include "mbarrier.cuh"
@@ -283,14 +284,17 @@ __global__ void sqdist_direct_reduce_kernel(const double* __restrict__ partial, 
         for (int i = threadIdx.x; i < m; i += blockDim.x) D[i * m + i] = 0.0;
 }
 
-// ------------------------------------------------------------------ m > 16: CUDA-core Gram tiles
+// ------------------------------------------------------------------ m > 16: CUDA-core tiles of squared differences
+//
+// Differences are formed before squaring, as in the small kernels: nothing cancels when the rows share a large
+// common vector, and bitwise-equal rows are at distance exactly zero.
 
 constexpr int kGT = 64;          // output tile edge
 constexpr int kGK = 32;          // columns per shared-memory step
 constexpr int kGramThreads = 256;  // 16 x 16 threads, 4 x 4 outputs each
 
 __global__ void __launch_bounds__(kGramThreads)
-gram_simt_kernel(const float* __restrict__ X, int64_t ld, int m, int64_t d, int ntile, int nslab,
+sqdist_simt_kernel(const float* __restrict__ X, int64_t ld, int m, int64_t d, int ntile, int nslab,
                  int64_t slab_cols, double* __restrict__ partial) {
     __shared__ float As[kGT][kGK + 1];
     __shared__ float Bs[kGT][kGK + 1];
@@ -339,7 +343,10 @@ gram_simt_kernel(const float* __restrict__ X, int64_t ld, int m, int64_t d, int 
 #pragma unroll
             for (int a = 0; a < 4; ++a)
 #pragma unroll
-                for (int b = 0; b < 4; ++b) part[a][b] = fmaf(av[a], bv[b], part[a][b]);
+                for (int b = 0; b < 4; ++b) {
+                    const float t = av[a] - bv[b];
+                    part[a][b] = fmaf(t, t, part[a][b]);
+                }
         }
 #pragma unroll
         for (int a = 0; a < 4; ++a)
@@ -355,33 +362,22 @@ gram_simt_kernel(const float* __restrict__ X, int64_t ld, int m, int64_t d, int 
         for (int b = 0; b < 4; ++b) out[(ty + 16 * a) * kGT + (tx + 16 * b)] = acc[a][b];
 }
 
-// Gram entry (i <= j) = sum over slabs of the tile partials, in slab order
-__global__ void gram_reduce_kernel(const double* __restrict__ partial, int m, int ntile, int nslab,
-                                   double* __restrict__ gram) {
+// D_ij (i < j) = sum over slabs of the tile partials, in slab order; mirrored; zero diagonal
+__global__ void sqdist_simt_reduce_kernel(const double* __restrict__ partial, int m, int ntile, int nslab,
+                                          double* __restrict__ D) {
     const int64_t total = (int64_t)m * m;
     for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
         const int i = (int)(e / m), j = (int)(e - (int64_t)i * m);
         if (i > j) continue;
+        if (i == j) { D[e] = 0.0; continue; }
         const int bi = i / kGT, bj = j / kGT;
         const int pair = bi * ntile - bi * (bi - 1) / 2 + (bj - bi);
         const double* p = partial + (int64_t)pair * nslab * (kGT * kGT) + (i % kGT) * kGT + (j % kGT);
         double v = 0.0;
 #pragma unroll 8
         for (int s = 0; s < nslab; ++s) v += p[(int64_t)s * (kGT * kGT)];
-        gram[e] = v;
-    }
-}
-
-// D_ij = G_ii + G_jj - 2 G_ij from the upper triangle; never negative; exact zero on the diagonal
-__global__ void dist_from_gram_kernel(const double* __restrict__ gram, int m, double* __restrict__ D) {
-    const int64_t total = (int64_t)m * m;
-    for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
-        const int i = (int)(e / m), j = (int)(e - (int64_t)i * m);
-        if (i == j) { D[e] = 0.0; continue; }
-        const int a = i < j ? i : j, b = i < j ? j : i;
-        const double v = gram[(int64_t)a * m + a] + gram[(int64_t)b * m + b] - 2.0 * gram[(int64_t)a * m + b];
-        // a NaN (rows with non-finite entries: Inf - Inf) must not turn into "distance zero": it is as far as it gets
-        D[e] = v > 0.0 ? v : (v != v ? __longlong_as_double(0x7ff0000000000000LL) : 0.0);
+        D[e] = v;   // may be NaN (two rows with non-finite entries); the ranking kernels take NaN as +Inf
+        D[(int64_t)j * m + i] = v;
     }
 }
 
@@ -454,7 +450,7 @@ detox_status launch_direct(const float* X, int64_t ld, int64_t d, const int32_t*
 size_t dist_ws_bytes(int m, int64_t d) {
     if (m <= 16) return align_up((size_t)direct_blocks(d) * (size_t)(m * (m - 1) / 2 + 1) * sizeof(double));
     GramPlan g = gram_plan(m, d);
-    size_t simt = align_up((size_t)g.npair * g.nslab * kGT * kGT * sizeof(double)) + align_up((size_t)m * m * sizeof(double));
+    size_t simt = align_up((size_t)g.npair * g.nslab * kGT * kGT * sizeof(double));
     size_t tc = m <= 256 ? tc_ws_bytes(m, d) : 0;
     return simt > tc ? simt : tc;
 }
@@ -495,14 +491,10 @@ detox_status launch_sqdist(const float* X, int64_t ld, int m, int64_t d, const i
     }
     if (tc_supported(X, ld, m, d)) return launch_sqdist_tc(X, ld, m, d, D, ws, status, s);
     GramPlan g = gram_plan(m, d);
-    double* gram = reinterpret_cast<double*>(static_cast<char*>(ws) +
-                                             align_up((size_t)g.npair * g.nslab * kGT * kGT * sizeof(double)));
-    gram_simt_kernel<<<g.npair * g.nslab, kGramThreads, 0, s>>>(X, ld, m, d, g.ntile, g.nslab, g.slab_cols, partial);
+    sqdist_simt_kernel<<<g.npair * g.nslab, kGramThreads, 0, s>>>(X, ld, m, d, g.ntile, g.nslab, g.slab_cols, partial);
     detox_status st = launch_status();
     if (st != DETOX_OK) return st;
-    gram_reduce_kernel<<<64, 256, 0, s>>>(partial, m, g.ntile, g.nslab, gram);
-    if ((st = launch_status()) != DETOX_OK) return st;
-    dist_from_gram_kernel<<<64, 256, 0, s>>>(gram, m, D);
+    sqdist_simt_reduce_kernel<<<64, 256, 0, s>>>(partial, m, g.ntile, g.nslab, D);
     return launch_status();
 }
 

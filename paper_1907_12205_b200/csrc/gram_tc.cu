@@ -42,8 +42,14 @@ constexpr int kProdWarps = 16;
 constexpr int kProdThreads = kProdWarps * 32;
 constexpr int kMmaWarps = 2;                   // issuing threads of the wide kernel (the staged kernel has two or four):
                                                // one's bookkeeping overlaps the other's MMAs
-constexpr int kTmaWarps = 2;                   // copy-issuing threads (the kernel for m > 128 uses the first only)
-constexpr int kTcThreads = kProdThreads + 32 * (kMmaWarps + kTmaWarps);
+constexpr int kTmaWarps = 2;                   // copy-issuing warps of the wide kernel (it uses the first only; the second
+                                               // one does the centring)
+// copy-issuing threads of the staged kernel: one per group of transform warps (above 64 rows a stage takes HBM longer
+// than one thread's wait / expect / copy loop, so one thread keeps up)
+__host__ __device__ constexpr int staged_tma_warps(int lx) { return lx; }
+constexpr int kCentreWarps = 1;                // forms the vector that is subtracted from every row (when one is)
+constexpr int kTcThreads = kProdThreads + 32 * (kMmaWarps + kTmaWarps);   // wide kernel: its second copy warp does the centring
+constexpr int kMaxCentreRows = 16;             // the subtracted vector is the mean of at most this many rows
 constexpr size_t kSmemBudget = 227 * 1024;     // dynamic shared memory one CTA may have
 constexpr int64_t kSlabCols = 4096;          // columns accumulated in tensor memory before a drain
 constexpr int kItemSlabs = 4;                // consecutive slabs of a CTA that are added into one output slot
@@ -143,6 +149,18 @@ __device__ __forceinline__ uint64_t lo2_of(uint64_t x2) {
     return add2(t, t);
 }
 
+// A packed pair of fp32 with every Inf / NaN replaced by zero (the centring row must not spread its non-finite
+// entries to the other rows: at such a coordinate nothing is subtracted).
+__device__ __forceinline__ uint64_t finite_or_zero2(uint64_t v) {
+    const uint32_t lo = (uint32_t)v, hi = (uint32_t)(v >> 32);
+    const uint32_t lo_ok = (lo & 0x7f800000u) != 0x7f800000u ? lo : 0u;
+    const uint32_t hi_ok = (hi & 0x7f800000u) != 0x7f800000u ? hi : 0u;
+    return (uint64_t)lo_ok | ((uint64_t)hi_ok << 32);
+}
+__device__ __forceinline__ float finite_or_zero(float v) {
+    return (__float_as_uint(v) & 0x7f800000u) != 0x7f800000u ? v : 0.f;
+}
+
 // ------------------------------------------------------------------------------------ 128 < m <= 256: wide kernel
 //
 // The accumulator has two halves of 128 rows, one per MMA-issuing thread; per K-step each thread issues
@@ -189,8 +207,11 @@ struct WideSmem {
     uint64_t empty[kMaxWideStages];
     uint64_t accum_full;
     uint64_t accum_empty;
+    uint64_t c_full[kMaxWideStages];   // the subtracted vector's piece for this stage is written
     uint32_t tmem_base;
     int abort_flag;
+    int crow[kMaxCentreRows];
+    __align__(16) float cring[kMaxWideStages][kKB];
 };
 
 // J = 16-byte pieces per transform thread and K-block (m * 8 / 512, rounded up)
@@ -198,7 +219,13 @@ template <int J>
 __global__ void __launch_bounds__(kTcThreads, 1)
 gram_wide_kernel(const __grid_constant__ CUtensorMap xmap, int m, uint32_t lo_off, uint32_t stage_bytes, int box_rows,
                  int ncol, int tmem_cols, int stages, int nkb_total, int nitems, float* __restrict__ partial,
-                 float* __restrict__ norms, int* __restrict__ status) {
+                 float* __restrict__ norms, const int* __restrict__ centre_ptr,
+                 const int* __restrict__ redo_ptr, int* __restrict__ status) {
+    // second launch of a call: only runs when the first one's centring was withdrawn
+    if (redo_ptr != nullptr && *redo_ptr == 0) return;
+    // Centring: centre_ptr[0] rows, listed from centre_ptr[2] on, are averaged column by column and the average is
+    // subtracted from every row before the products (distances do not change; 0 rows: nothing is subtracted).
+    const int ncentre = *centre_ptr;
     extern __shared__ uint8_t smem_raw[];
     // tiles need 1024-byte alignment for the 128-byte swizzle pattern
     const uint32_t raw = smem_u32(smem_raw);
@@ -213,12 +240,14 @@ gram_wide_kernel(const __grid_constant__ CUtensorMap xmap, int m, uint32_t lo_of
             mbar_init(&sm->landed[s], 1);
             mbar_init(&sm->full[s], kProdWarps);
             mbar_init(&sm->empty[s], kMmaWarps);
+            mbar_init(&sm->c_full[s], 1);
         }
         mbar_init(&sm->accum_full, kMmaWarps);
         mbar_init(&sm->accum_empty, kProdWarps);
         sm->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+    if (tid < ncentre) sm->crow[tid] = centre_ptr[2 + tid];
     // rows beyond the TMA box are never written: clear all tiles once so the padded rows are zeros
     for (uint32_t off = (uint32_t)tid * 16u; off < stage_bytes * (uint32_t)stages; off += kTcThreads * 16u)
         *reinterpret_cast<uint4*>(base + off) = make_uint4(0u, 0u, 0u, 0u);
@@ -245,7 +274,7 @@ gram_wide_kernel(const __grid_constant__ CUtensorMap xmap, int m, uint32_t lo_of
         const int row0 = tid >> 3, c = tid & 7;
         const uint32_t off0 = (uint32_t)(row0 >> 3) * 1024u + (uint32_t)(row0 & 7) * 128u + (uint32_t)((c ^ (row0 & 7)) << 4);
         constexpr uint32_t kOffStep = (uint32_t)(kProdThreads / 64) * 1024u;
-        uint64_t sq[J];   // packed pair of partial sums of squares per piece
+        uint64_t sq[J];   // packed pair of partial sums of squares per piece (of the centred values)
 #pragma unroll
         for (int j = 0; j < J; ++j) sq[j] = 0ull;
 
@@ -256,14 +285,31 @@ gram_wide_kernel(const __grid_constant__ CUtensorMap xmap, int m, uint32_t lo_of
             const int t_end = li * kBlocksPerSlab + nkb;
             for (; t < t_end; ++t) {
                 mbar_wait(&sm->landed[s], ph, abort_flag, status);
-                const uint8_t* hi_tile = base + (size_t)s * stage_bytes + off0;
+                uint8_t* hi_tile = base + (size_t)s * stage_bytes + off0;
                 uint8_t* lo_tile = base + (size_t)s * stage_bytes + lo_off + off0;
+                if (ncentre == 0) {
 #pragma unroll
-                for (int j = 0; j < J; ++j) {
-                    if (tid + j * kProdThreads < npieces) {
-                        const ulonglong2 x = *reinterpret_cast<const ulonglong2*>(hi_tile + j * kOffStep);
-                        sq[j] = fma2(x.x, x.x, fma2(x.y, x.y, sq[j]));
-                        *reinterpret_cast<ulonglong2*>(lo_tile + j * kOffStep) = make_ulonglong2(lo2_of(x.x), lo2_of(x.y));
+                    for (int j = 0; j < J; ++j) {
+                        if (tid + j * kProdThreads < npieces) {
+                            const ulonglong2 x = *reinterpret_cast<const ulonglong2*>(hi_tile + j * kOffStep);
+                            sq[j] = fma2(x.x, x.x, fma2(x.y, x.y, sq[j]));
+                            *reinterpret_cast<ulonglong2*>(lo_tile + j * kOffStep) = make_ulonglong2(lo2_of(x.x), lo2_of(x.y));
+                        }
+                    }
+                } else {
+                    // the hi tile is rewritten in place with the centred values; the warp that forms the subtracted
+                    // vector has read its rows by the time c_full completes
+                    mbar_wait(&sm->c_full[s], ph, abort_flag, status);
+                    const ulonglong2 ck = *reinterpret_cast<const ulonglong2*>(&sm->cring[s][c * 4]);
+#pragma unroll
+                    for (int j = 0; j < J; ++j) {
+                        if (tid + j * kProdThreads < npieces) {
+                            const ulonglong2 x = *reinterpret_cast<const ulonglong2*>(hi_tile + j * kOffStep);
+                            const ulonglong2 a = make_ulonglong2(sub2(x.x, ck.x), sub2(x.y, ck.y));
+                            sq[j] = fma2(a.x, a.x, fma2(a.y, a.y, sq[j]));
+                            *reinterpret_cast<ulonglong2*>(hi_tile + j * kOffStep) = a;
+                            *reinterpret_cast<ulonglong2*>(lo_tile + j * kOffStep) = make_ulonglong2(lo2_of(a.x), lo2_of(a.y));
+                        }
                     }
                 }
                 fence_proxy_async_smem();   // make the generic-proxy stores visible to the MMA's reads
@@ -350,6 +396,37 @@ gram_wide_kernel(const __grid_constant__ CUtensorMap xmap, int m, uint32_t lo_of
                 }
             }
         }
+    } else if (warp == kProdWarps + kMmaWarps + 1) {
+        // ------------------------------------------------ the centring warp: lane l averages column l of the listed
+        // rows of every K-block as it lands (non-finite entries count as zero) and hands the 32 averages on
+        if (ncentre > 0) {
+            const float inv = 1.f / (float)ncentre;
+            // byte offset of this lane's column in every listed row (swizzled layout); all loads of a K-block are
+            // issued together
+            uint32_t off[kMaxCentreRows];
+#pragma unroll
+            for (int k = 0; k < kMaxCentreRows; ++k) {
+                const int r = sm->crow[k < ncentre ? k : 0];
+                off[k] = (uint32_t)(r >> 3) * 1024u + (uint32_t)(r & 7) * 128u + (uint32_t)(((lane >> 2) ^ (r & 7)) << 4) +
+                         (uint32_t)(lane & 3) * 4u;
+            }
+            int s = 0;
+            uint32_t ph = 0;
+            for (int t = 0; t < total; ++t) {
+                if (!mbar_wait(&sm->landed[s], ph, abort_flag, status)) break;
+                const uint8_t* tile = base + (size_t)s * stage_bytes;
+                float v[kMaxCentreRows];
+#pragma unroll
+                for (int k = 0; k < kMaxCentreRows; ++k) v[k] = *reinterpret_cast<const float*>(tile + off[k]);
+                float acc = 0.f;
+#pragma unroll
+                for (int k = 0; k < kMaxCentreRows; ++k) acc += k < ncentre ? finite_or_zero(v[k]) : 0.f;
+                sm->cring[s][lane] = acc * inv;
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sm->c_full[s]);
+                if (++s == stages) { s = 0; ph ^= 1u; }
+            }
+        }
     } else if (warp < kProdWarps + kMmaWarps && lane == 0) {
         // ------------------------------------------------ the MMA threads (lane 0 of the two warps after the
         // transform warps): thread g owns the accumulator half of rows 128 g .. 128 g + 127
@@ -431,7 +508,7 @@ StagedPlan staged_plan(int m, int64_t d) {
     // tensor cores read the others; above, two MMA stages and one group
     p.nmst = m <= 64 ? 4 : 2;
     p.groups = m <= 64 ? 2 : 1;
-    const size_t left = kSmemBudget - 2048 - p.nmst * mst_bytes;
+    const size_t left = kSmemBudget - 4096 - p.nmst * mst_bytes;
     p.nstg = (int)(left / p.stg_bytes);
     if (p.nstg > kMaxStg) p.nstg = kMaxStg;
     while (p.nstg > 2 && (size_t)p.nstg * p.stg_bytes > 112 * 1024) --p.nstg;   // ~100 KB in flight saturates HBM
@@ -442,7 +519,7 @@ StagedPlan staged_plan(int m, int64_t d) {
     p.grid = p.nst_total < kSMs ? p.nst_total : kSMs;
     const int per_cta = (p.nst_total + p.grid - 1) / p.grid;
     p.nitems = p.grid * (int)ceil_div(ceil_div((int64_t)per_cta, (int64_t)staged_slab_stages(p.nmma)), (int64_t)kItemSlabs);
-    p.smem_bytes = (size_t)p.nstg * p.stg_bytes + p.nmst * mst_bytes + 1024 /*barriers*/ + 1024 /*alignment slack*/;
+    p.smem_bytes = (size_t)p.nstg * p.stg_bytes + p.nmst * mst_bytes + 3072 /*barriers, centring ring*/ + 1024 /*alignment slack*/;
     return p;
 }
 
@@ -453,9 +530,13 @@ struct StagedSmem {
     uint64_t mst_empty[kMaxMst];   // the MMAs that read them are done
     uint64_t accum_full;
     uint64_t accum_empty;
+    uint64_t c_full[kMaxStg];      // the subtracted vector's piece for this staging stage is written
     uint32_t tmem_base;
     int abort_flag;
+    int crow[kMaxCentreRows];
+    __align__(16) float cring[kMaxStg][kStageCols];
 };
+static_assert(sizeof(StagedSmem) <= 3072, "fits the shared memory reserved behind the tiles");
 
 // LX = groups of transform warps; J = 16-byte pieces per transform thread and stage (m * 16 / (512 / LX), rounded up);
 // NMMA = MMA-issuing threads, each with an accumulator of its own.  Up to 64 rows an MMA sits on its 59-cycle floor and
@@ -465,10 +546,16 @@ struct StagedSmem {
 // consecutive phases of a barrier apart, no more, and a thread that followed one group's stages could otherwise get
 // more than a phase ahead of the other group's.
 template <int J, int LX, int NMMA>
-__global__ void __launch_bounds__(kProdThreads + 32 * (NMMA + kTmaWarps), 1)
+__global__ void __launch_bounds__(kProdThreads + 32 * (NMMA + staged_tma_warps(LX) + kCentreWarps), 1)
 gram_staged_kernel(const __grid_constant__ CUtensorMap xmap, int m, uint32_t stg_bytes, uint32_t tile_bytes, int mrows,
                    int ncol, int tmem_cols, int nstg, int nmst, int nst_total, int nitems, float* __restrict__ partial,
-                   float* __restrict__ norms, int* __restrict__ status) {
+                   float* __restrict__ norms, const int* __restrict__ centre_ptr,
+                   const int* __restrict__ redo_ptr, int* __restrict__ status) {
+    // second launch of a call: only runs when the first one's centring was withdrawn
+    if (redo_ptr != nullptr && *redo_ptr == 0) return;
+    // Centring: centre_ptr[0] rows, listed from centre_ptr[2] on, are averaged column by column and the average is
+    // subtracted from every row before the products (distances do not change; 0 rows: nothing is subtracted).
+    const int ncentre = *centre_ptr;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     uint8_t* stg_base = smem_raw + ((1024u - (raw & 1023u)) & 1023u);       // MMA tiles need 1024-byte alignment
@@ -478,13 +565,15 @@ gram_staged_kernel(const __grid_constant__ CUtensorMap xmap, int m, uint32_t stg
     volatile int* abort_flag = &sm->abort_flag;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    constexpr int kThreads = kProdThreads + 32 * (NMMA + kTmaWarps);
+    constexpr int kTma = staged_tma_warps(LX);
+    constexpr int kThreads = kProdThreads + 32 * (NMMA + kTma + kCentreWarps);
     constexpr int kGroupThreads = kProdThreads / LX, kGroupWarps = kProdWarps / LX;
 
     if (tid == 0) {
         for (int s = 0; s < nstg; ++s) {
             mbar_init(&sm->stg_full[s], 1);
             mbar_init(&sm->stg_empty[s], kGroupWarps);
+            mbar_init(&sm->c_full[s], 1);
         }
         for (int s = 0; s < nmst; ++s) {
             mbar_init(&sm->mst_full[s], kGroupWarps);
@@ -495,6 +584,7 @@ gram_staged_kernel(const __grid_constant__ CUtensorMap xmap, int m, uint32_t stg
         sm->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+    if (tid < ncentre) sm->crow[tid] = centre_ptr[2 + tid];
     // rows m .. 2 ncol of the MMA tiles are never written: clear the MMA stages once so that they read as zeros
     for (uint32_t off = (uint32_t)tid * 16u; off < mst_bytes * (uint32_t)nmst; off += kThreads * 16u)
         *reinterpret_cast<uint4*>(mst_base + off) = make_uint4(0u, 0u, 0u, 0u);
@@ -529,7 +619,7 @@ gram_staged_kernel(const __grid_constant__ CUtensorMap xmap, int m, uint32_t stg
                               (uint32_t)((cq ^ (row0 & 7)) << 4);
         constexpr uint32_t kDstStep = (uint32_t)(kGroupThreads / 128) * 1024u;
         const uint32_t lo_off = (uint32_t)ncol * 128u;      // the 2lo rows follow the hi rows inside a tile
-        uint64_t sq[J];   // packed pair of partial sums of squares per piece
+        uint64_t sq[J];   // packed pair of partial sums of squares per piece (of the centred values)
 #pragma unroll
         for (int j = 0; j < J; ++j) sq[j] = 0ull;
 
@@ -546,6 +636,13 @@ gram_staged_kernel(const __grid_constant__ CUtensorMap xmap, int m, uint32_t stg
 #pragma unroll
                 for (int j = 0; j < J; ++j)
                     if (gtid + j * kGroupThreads < npieces) x[j] = *reinterpret_cast<const ulonglong2*>(src + j * kSrcStep);
+                if (ncentre > 0) {
+                    mbar_wait(&sm->c_full[ss], sph, abort_flag, status);
+                    const ulonglong2 ck = *reinterpret_cast<const ulonglong2*>(&sm->cring[ss][q * 4]);
+#pragma unroll
+                    for (int j = 0; j < J; ++j)
+                        if (gtid + j * kGroupThreads < npieces) x[j] = make_ulonglong2(sub2(x[j].x, ck.x), sub2(x[j].y, ck.y));
+                }
                 mbar_wait(&sm->mst_empty[ms], mph ^ 1u, abort_flag, status);   // the MMAs that read this slot are done
                 uint8_t* dst = mst_base + (size_t)ms * mst_bytes + dst0;
 #pragma unroll
@@ -630,26 +727,56 @@ gram_staged_kernel(const __grid_constant__ CUtensorMap xmap, int m, uint32_t stg
             for (int e = tid; e < m * ncol; e += kProdThreads) partial[item * m * ncol + e] = 0.f;
             for (int e = tid; e < m * LX; e += kProdThreads) norms[item * LX * m + e] = 0.f;
         }
+    } else if (warp == kProdWarps + NMMA + kTma) {
+        // ------------------------------------------------ the centring warp: lane l averages columns 2l and 2l+1 of the
+        // listed rows of every stage as it lands (non-finite entries count as zero) and hands the 64 averages on
+        if (ncentre > 0) {
+            const float inv = 1.f / (float)ncentre;
+            // byte offset of this lane's two columns in every listed row; all loads of a stage are issued together
+            uint32_t off[kMaxCentreRows];
+#pragma unroll
+            for (int k = 0; k < kMaxCentreRows; ++k)
+                off[k] = (uint32_t)sm->crow[k < ncentre ? k : 0] * (uint32_t)(kStageCols * 4) + (uint32_t)lane * 8u;
+            int s = 0;
+            uint32_t ph = 0;
+            for (int t = 0; t < total; ++t) {
+                if (!mbar_wait(&sm->stg_full[s], ph, abort_flag, status)) break;
+                const uint8_t* stg = stg_base + (size_t)s * stg_bytes;
+                float2 v[kMaxCentreRows];
+#pragma unroll
+                for (int k = 0; k < kMaxCentreRows; ++k) v[k] = *reinterpret_cast<const float2*>(stg + off[k]);
+                float2 acc = make_float2(0.f, 0.f);
+#pragma unroll
+                for (int k = 0; k < kMaxCentreRows; ++k) {
+                    acc.x += k < ncentre ? finite_or_zero(v[k].x) : 0.f;
+                    acc.y += k < ncentre ? finite_or_zero(v[k].y) : 0.f;
+                }
+                *reinterpret_cast<float2*>(&sm->cring[s][2 * lane]) = make_float2(acc.x * inv, acc.y * inv);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sm->c_full[s]);
+                if (++s == nstg) { s = 0; ph ^= 1u; }
+            }
+        }
     } else if (warp >= kProdWarps + NMMA) {
-        // ------------------------------------------------ the TMA threads: thread l issues the stages l, l + kTmaWarps, ...
+        // ------------------------------------------------ the TMA threads: thread l issues the stages l, l + kTma, ...
         if (lane == 0) {
             const int l = warp - (kProdWarps + NMMA);
             int last = -1;
             int s = l % nstg;
             uint32_t ph = (uint32_t)(l / nstg) & 1u;
             int64_t c0 = ((int64_t)blockIdx.x + (int64_t)l * gridDim.x) * kStageCols;   // first column of the stage
-            for (int t = l; t < total; t += kTmaWarps) {
+            for (int t = l; t < total; t += kTma) {
                 if (!mbar_wait(&sm->stg_empty[s], ph ^ 1u, abort_flag, status)) break;   // the slot has been read
                 mbar_expect_tx(&sm->stg_full[s], stg_bytes);
                 tma_load_2d(stg_base + (size_t)s * stg_bytes, &xmap, (int)c0, 0, &sm->stg_full[s]);
                 last = t;
-                s += kTmaWarps;
+                s += kTma;
                 while (s >= nstg) { s -= nstg; ph ^= 1u; }
-                c0 += (int64_t)kTmaWarps * gridDim.x * kStageCols;
+                c0 += (int64_t)kTma * gridDim.x * kStageCols;
             }
             if (*abort_flag) {
                 // give this thread's copies still in flight a bounded time to land before the CTA goes away
-                for (int tt = last; tt >= 0 && tt > last - nstg; tt -= kTmaWarps) {
+                for (int tt = last; tt >= 0 && tt > last - nstg; tt -= kTma) {
                     const int s2 = (int)((uint32_t)tt % (uint32_t)nstg);
                     const uint32_t ph2 = ((uint32_t)tt / (uint32_t)nstg) & 1u;
                     for (uint32_t spin = 0; spin < (1u << 16) && !mbar_test(&sm->stg_full[s2], ph2); ++spin) __nanosleep(64);
@@ -836,28 +963,37 @@ detox_status make_xmap(CUtensorMap* map, const float* X, int64_t ld, int m, int6
     return r == CUDA_SUCCESS ? DETOX_OK : DETOX_ERR_CUDA;
 }
 
+// What a launch of either kernel is given besides its plan.  redo: null for the first launch of a call; for the second
+// the flag the check of the first one's centring has set (the kernel returns at once when it reads 0).
+struct TcBuffers {
+    float* partial;
+    float* norms;
+    const int* centre;
+    const int* redo;
+    int* status;
+};
+
 template <int J>
-detox_status launch_wide(const WidePlan& p, const CUtensorMap& xmap, int m, float* partial, float* norms, int* status,
-                         cudaStream_t s) {
+detox_status launch_wide(const WidePlan& p, const CUtensorMap& xmap, int m, const TcBuffers& b, cudaStream_t s) {
     if (cudaFuncSetAttribute(gram_wide_kernel<J>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem_bytes) !=
         cudaSuccess)
         return DETOX_ERR_CUDA;
     gram_wide_kernel<J><<<p.grid, kTcThreads, p.smem_bytes, s>>>(xmap, m, p.lo_off, p.stage_bytes, p.box_rows, p.ncol,
-                                                                 p.tmem_cols, p.stages, p.nkb_total, p.nitems, partial,
-                                                                 norms, status);
+                                                                 p.tmem_cols, p.stages, p.nkb_total, p.nitems, b.partial,
+                                                                 b.norms, b.centre, b.redo, b.status);
     return launch_status();
 }
 
 template <int J, int LX, int NMMA>
-detox_status launch_staged(const StagedPlan& p, const CUtensorMap& xmap, int m, float* partial, float* norms, int* status,
-                           cudaStream_t s) {
+detox_status launch_staged(const StagedPlan& p, const CUtensorMap& xmap, int m, const TcBuffers& b, cudaStream_t s) {
     if (cudaFuncSetAttribute(gram_staged_kernel<J, LX, NMMA>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)p.smem_bytes) != cudaSuccess)
         return DETOX_ERR_CUDA;
-    constexpr int kThreads = kProdThreads + 32 * (NMMA + kTmaWarps);
+    constexpr int kThreads = kProdThreads + 32 * (NMMA + staged_tma_warps(LX) + kCentreWarps);
     gram_staged_kernel<J, LX, NMMA><<<p.grid, kThreads, p.smem_bytes, s>>>(xmap, m, p.stg_bytes, p.tile_bytes, p.mrows, p.ncol,
                                                                           p.tmem_cols, p.nstg, p.nmst, p.nst_total,
-                                                                          p.nitems, partial, norms, status);
+                                                                          p.nitems, b.partial, b.norms, b.centre, b.redo,
+                                                                          b.status);
     return launch_status();
 }
 
@@ -886,22 +1022,42 @@ bool tc_supported(const float* X, int64_t ld, int m, int64_t d) {
     return m > 16 && m <= 256 && aligned16(X) && ld % 4 == 0 && d < (int64_t)1 << 31 && encode_tiled_fn() != nullptr;
 }
 
-size_t tc_ws_bytes(int m, int64_t d) {
-    const TcShape o = tc_shape(m, d);
+// workspace: slab partials | norms | per-chunk distance sums | centring rows, redo flag |
+// scratch of the centre choice
+struct TcWs {
+    float* partial;
+    float* norms;
+    double* dpart;
+    int* centre;     // [0] how many rows are averaged into the subtracted vector (0: none), [1] the redo flag, [2..] the rows
+    void* pick;
+    size_t total;
+};
+TcWs tc_carve(void* ws, int m, int64_t d, const TcShape& o) {
+    TcWs w;
+    char* p = static_cast<char*>(ws);
+    size_t off = 0;
     const size_t elems = (size_t)m * o.ncol;
-    return align_up((size_t)o.nitems * elems * sizeof(float)) + align_up((size_t)o.nitems * o.groups * m * sizeof(float)) +
-           align_up((size_t)reduce_chunks(m, o.nitems) * m * m * sizeof(double));
+    w.partial = reinterpret_cast<float*>(p + off);
+    off += align_up((size_t)o.nitems * elems * sizeof(float));
+    w.norms = reinterpret_cast<float*>(p + off);
+    off += align_up((size_t)o.nitems * o.groups * m * sizeof(float));
+    w.dpart = reinterpret_cast<double*>(p + off);
+    off += align_up((size_t)reduce_chunks(m, o.nitems) * m * m * sizeof(double));
+    w.centre = reinterpret_cast<int*>(p + off);
+    off += 256;
+    w.pick = p + off;
+    off += centre_ws_bytes(m, d);
+    w.total = off;
+    return w;
 }
 
-detox_status launch_sqdist_tc(const float* X, int64_t ld, int m, int64_t d, double* D, void* ws, int* status,
-                              cudaStream_t s) {
-    const TcShape o = tc_shape(m, d);
-    const int64_t elems = (int64_t)m * o.ncol;
-    char* base = static_cast<char*>(ws);
-    float* partial = reinterpret_cast<float*>(base);
-    float* norms = reinterpret_cast<float*>(base + align_up((size_t)o.nitems * elems * sizeof(float)));
-    double* gpart = reinterpret_cast<double*>(base + align_up((size_t)o.nitems * elems * sizeof(float)) +
-                                              align_up((size_t)o.nitems * o.groups * m * sizeof(float)));
+size_t tc_ws_bytes(int m, int64_t d) { return tc_carve(nullptr, m, d, tc_shape(m, d)).total; }
+
+namespace {
+
+// One launch of the streaming kernel that fits m.
+detox_status launch_tc_gram(const float* X, int64_t ld, int m, int64_t d, const TcShape& o, const TcBuffers& b,
+                            cudaStream_t s) {
     CUtensorMap xmap;
     detox_status st;
     if (o.staged) {
@@ -911,28 +1067,45 @@ detox_status launch_sqdist_tc(const float* X, int64_t ld, int m, int64_t d, doub
         const int gt = kProdThreads / p.groups;
         const int per_thread = (m * (kStageCols / 4) + gt - 1) / gt;
         if (p.groups == 2) {   // up to 64 rows: two transform groups, four MMA-issuing threads
-            if (per_thread <= 2) st = launch_staged<2, 2, 4>(p, xmap, m, partial, norms, status, s);
-            else if (per_thread <= 3) st = launch_staged<3, 2, 4>(p, xmap, m, partial, norms, status, s);
-            else st = launch_staged<4, 2, 4>(p, xmap, m, partial, norms, status, s);
-        } else {
-            if (per_thread <= 2) st = launch_staged<2, 1, 2>(p, xmap, m, partial, norms, status, s);
-            else if (per_thread <= 3) st = launch_staged<3, 1, 2>(p, xmap, m, partial, norms, status, s);
-            else st = launch_staged<4, 1, 2>(p, xmap, m, partial, norms, status, s);
+            if (per_thread <= 2) return launch_staged<2, 2, 4>(p, xmap, m, b, s);
+            if (per_thread <= 3) return launch_staged<3, 2, 4>(p, xmap, m, b, s);
+            return launch_staged<4, 2, 4>(p, xmap, m, b, s);
         }
-    } else {
-        const WidePlan p = wide_plan(m, d);
-        if ((st = make_xmap(&xmap, X, ld, m, d, kKB, p.box_rows, CU_TENSOR_MAP_SWIZZLE_128B)) != DETOX_OK) return st;
-        // 16-byte pieces per transform thread and K-block: m * 8 / 512, rounded up
-        if (m * 8 <= 3 * kProdThreads) st = launch_wide<3>(p, xmap, m, partial, norms, status, s);
-        else st = launch_wide<4>(p, xmap, m, partial, norms, status, s);
+        if (per_thread <= 2) return launch_staged<2, 1, 2>(p, xmap, m, b, s);
+        if (per_thread <= 3) return launch_staged<3, 1, 2>(p, xmap, m, b, s);
+        return launch_staged<4, 1, 2>(p, xmap, m, b, s);
     }
-    if (st != DETOX_OK) return st;
+    const WidePlan p = wide_plan(m, d);
+    if ((st = make_xmap(&xmap, X, ld, m, d, kKB, p.box_rows, CU_TENSOR_MAP_SWIZZLE_128B)) != DETOX_OK) return st;
+    // 16-byte pieces per transform thread and K-block: m * 8 / 512, rounded up
+    if (m * 8 <= 3 * kProdThreads) return launch_wide<3>(p, xmap, m, b, s);
+    return launch_wide<4>(p, xmap, m, b, s);
+}
+
+}  // namespace
+
+// Sequence: choose the centring rows on a column sample (or none) -> streaming pass -> check that the centred rows
+// really got smaller, else withdraw the centring -> the streaming pass again, which returns at once unless the
+// centring was withdrawn -> reduction of the slab partials to distances.
+detox_status launch_sqdist_tc(const float* X, int64_t ld, int m, int64_t d, double* D, void* ws, int* status,
+                              cudaStream_t s) {
+    const TcShape o = tc_shape(m, d);
+    const TcWs w = tc_carve(ws, m, d, o);
+    detox_status st;
+    if ((st = launch_pick_centre(X, ld, m, d, w.pick, w.centre, s)) != DETOX_OK) return st;
+    TcBuffers b{w.partial, w.norms, w.centre, nullptr, status};
+    if ((st = launch_tc_gram(X, ld, m, d, o, b, s)) != DETOX_OK) return st;
+    if ((st = launch_check_centre(w.norms, o.nitems * o.groups, m, w.pick, d, w.centre, w.centre + 1, s)) !=
+        DETOX_OK)
+        return st;
+    b.redo = w.centre + 1;
+    if ((st = launch_tc_gram(X, ld, m, d, o, b, s)) != DETOX_OK) return st;
     const int nt = (m + kRT - 1) / kRT;
     const int nchunks = reduce_chunks(m, o.nitems);
-    tc_reduce_kernel<<<dim3((unsigned)(nt * (nt + 1) / 2), (unsigned)nchunks), kRT * 8, 0, s>>>(partial, norms, o.groups,
-                                                                                           o.nitems, m, o.ncol, gpart);
+    tc_reduce_kernel<<<dim3((unsigned)(nt * (nt + 1) / 2), (unsigned)nchunks), kRT * 8, 0, s>>>(w.partial, w.norms, o.groups,
+                                                                                           o.nitems, m, o.ncol, w.dpart);
     if ((st = launch_status()) != DETOX_OK) return st;
-    tc_dist_kernel<<<(unsigned)ceil_div((int64_t)m * m * 32, 256), 256, 0, s>>>(gpart, nchunks, m, status, D);
+    tc_dist_kernel<<<(unsigned)ceil_div((int64_t)m * m * 32, 256), 256, 0, s>>>(w.dpart, nchunks, m, status, D);
     return launch_status();
 }
 

@@ -222,3 +222,61 @@ def test_a_row_with_an_infinite_entry_is_never_selected(m, d):
     _, bsel = dx.agg_bulyan(padded(X), f)
     bsel_o = oracle.bulyan_select(D_o, f)
     assert 3 not in bsel_o.tolist() and bsel.cpu().numpy().tolist() == bsel_o.tolist()
+
+
+def correlated_rows(m, d, ratio, seed, copies=1, outliers=0):
+    """x_i = mu + eps_i: a common vector of `ratio` times the length of the individual parts (honest gradients of one
+    loss at one model share a direction)."""
+    rng = np.random.default_rng(seed)
+    eps = krum_inputs(m, d, seed=seed + 1, copies=copies, outliers=0)
+    mu = (rng.standard_normal(d) * 1e-3 * ratio).astype(np.float32)
+    X = eps + mu
+    for i in range(outliers):
+        X[m - 1 - i] = -100 * X[m - 1 - i]
+    return X
+
+
+@pytest.mark.parametrize("ratio", [1, 10, 100])
+@pytest.mark.parametrize("m", [45, 105, 225])
+def test_tensor_core_distances_on_rows_that_share_a_large_common_vector(m, ratio):
+    d = 150_003
+    f = m // 10
+    for attempt in range(8):
+        X = correlated_rows(m, d, ratio, seed=31 * m + ratio + 1000 * attempt, copies=3 if m == 105 else 1, outliers=f)
+        out_o, sel_o, sc_o, D_o = oracle.multikrum(X, f, m - f)
+        if multikrum_min_gap(sc_o, m - f) > 1e-5:
+            break
+    out, sel, sc = dx.agg_multikrum(padded(X), f, m - f)
+    assert sel.cpu().numpy().tolist() == sel_o.tolist()
+    np.testing.assert_allclose(sc.cpu().numpy(), sc_o, rtol=2e-6, atol=1e-30)
+    assert rel_l2(out.cpu().numpy(), out_o) <= TOL
+    D = dx.agg_pairwise_sqdist(padded(X)).cpu().numpy()
+    honest = m - f
+    np.testing.assert_allclose(D[:honest, :honest], D_o[:honest, :honest], rtol=2e-6, atol=0)
+    if m == 105:                                     # bitwise-equal rows: distance exactly zero, equal scores
+        s = sc.cpu().numpy()
+        for i in range(0, honest - 3, 3):
+            assert D[i, i + 1] == 0.0 and D[i, i + 2] == 0.0 and s[i] == s[i + 1] == s[i + 2]
+
+
+@pytest.mark.parametrize("m", [45, 140])
+def test_a_centring_row_that_is_only_central_where_it_is_sampled_is_withdrawn(m):
+    """The row subtracted from all rows is chosen on 32 evenly spaced blocks of 64 columns.  A Byzantine row that sits
+    in the middle of the others there and holds huge values everywhere else would, once subtracted, wipe out the
+    differences between the honest rows.  The library checks the exact norms after the pass and repeats it without
+    that row; distances and selection must come out right."""
+    d, ratio, f = 100_000, 3, 4
+    X = correlated_rows(m, d, ratio, seed=5 * m, outliers=0)
+    nb_all = (d + 63) // 64
+    sampled = np.zeros(d, bool)
+    for b in range(32):
+        c0 = (nb_all * b // 32) * 64
+        sampled[c0:c0 + 64] = True
+    bad = X[: m - 1].astype(np.float64).mean(axis=0).astype(np.float32)   # the centre of the others where sampled ...
+    bad[~sampled] = 1e30                                                   # ... and far away everywhere else
+    X[m - 1] = bad
+    _, sel_o, sc_o, D_o = oracle.multikrum(X, f, m - f, want_out=False)
+    assert m - 1 not in sel_o.tolist()
+    _, sel, sc = dx.agg_multikrum(padded(X), f, m - f)
+    assert sel.cpu().numpy().tolist() == sel_o.tolist()
+    np.testing.assert_allclose(sc.cpu().numpy()[: m - 1], sc_o[: m - 1], rtol=2e-5)
