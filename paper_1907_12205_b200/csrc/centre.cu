@@ -4,13 +4,14 @@
 // rows share a large common vector (honest gradients of one loss at one model do): the three terms are then much
 // larger than their difference, and the tensor cores' fp32 accumulation loses most on long sums of one sign.
 // Distances do not change when one vector is subtracted from every row, so the pass may work on a_i = x_i - c with c
-// in the middle of the rows; it forms c, column by column, as the mean of a few rows that are listed here.  The rows
-// are found on a sample of the columns: squared distances between all rows over a few evenly spaced column blocks
-// (formed as differences, so they are accurate whatever the rows share), then for every row the median of its
-// distances to the others; the rows are ranked by that median and every s-th of the more central half is taken (so
-// that a group of colluding rows that sit in the very middle cannot fill the list).  Centring is switched on only
-// when the most central row is closer to the typical row than the origin is by a clear margin; rows that hover around
-// zero are left as they are.
+// in the middle of the rows; it forms c, column by column, as the mean of a few rows that are listed here.
+//
+// The rows are found on a sample of the columns (16 evenly spaced blocks of 64), at a cost linear in the number of
+// rows: per column the median of seven rows at fixed, evenly spaced positions gives a first centre that a minority of
+// outlying rows cannot move; every row's squared distance to it and squared norm are added up over the sample; the
+// rows are ranked by that distance and every s-th of the closer half is listed (so that a group of colluding rows
+// that sit in the very middle cannot fill the list).  Centring is switched on only when the typical row is closer to
+// the first centre than to the origin; rows that hover around zero are left as they are.
 //
 // Everything is deterministic: per-block partial sums are added in a fixed order and ties go to the lower index.
 #include <math_constants.h>
@@ -23,180 +24,130 @@ namespace {
 
 constexpr int kPickThreads = 256;
 constexpr int kMaxCentreRows = 16;   // as in the distance kernels
+constexpr int kSampleCols = 64;      // columns per sampled block
+constexpr int kSampleBlocks = 16;
+constexpr int kFirstRows = 7;        // rows whose column-wise median is the first centre
 
-struct CentrePlan {
-    int cols;      // columns per sampled block
-    int nblk;      // sampled blocks
-    int nsplit;    // CTAs per block (they share the pairs)
-};
-
-CentrePlan centre_plan(int m, int64_t d) {
-    CentrePlan p;
-    p.cols = 64;           // (the tensor-core path, the only user, has at most 256 rows: a tile is at most 66.5 KB)
-    const int64_t avail = ceil_div(d, (int64_t)p.cols);
-    p.nblk = 32;
-    if (p.nblk > avail) p.nblk = (int)avail;
-    const int64_t want = ceil_div((int64_t)m * m, 4 * kPickThreads);
-    int64_t ns = (2 * kSMs) / p.nblk;
-    if (ns > want) ns = want;
-    p.nsplit = (int)(ns < 1 ? 1 : ns);
-    return p;
+int sample_blocks(int64_t d) {
+    const int64_t avail = ceil_div(d, (int64_t)kSampleCols);
+    return (int)(avail < kSampleBlocks ? avail : kSampleBlocks);
 }
 
 struct CentreWs {
-    float* part;        // [nblk][m*m]: entry i*m+j (i < j) = squared distance over the block; i*m+i = squared norm
-    float* key;         // [m] median sample distance of row i to the others
-    float* nrm;         // [m] sample squared norm
-    unsigned* counter;  // [2] CTAs of the pick kernel / of the check kernel that have finished; behind them one float:
+    float* part;        // [nblk][2][m]: per block, every row's squared distance to the first centre, then its squared norm
+    float* key;         // [m] scratch of the check after the pass
+    unsigned* counter;  // [2] unused / CTAs of the check kernel that have finished; behind them one float:
                         // the typical squared norm of a row as the sample predicts it for all d columns
 };
 
-CentreWs centre_carve(void* ws, int m, int nblk) {
+CentreWs centre_carve(void* ws, int m) {
     CentreWs w;
     char* p = static_cast<char*>(ws);
     w.part = reinterpret_cast<float*>(p);
-    p += align_up((size_t)nblk * m * m * sizeof(float));
+    p += align_up((size_t)kSampleBlocks * 2 * m * sizeof(float));
     w.key = reinterpret_cast<float*>(p);
-    p += align_up((size_t)m * sizeof(float));
-    w.nrm = reinterpret_cast<float*>(p);
     p += align_up((size_t)m * sizeof(float));
     w.counter = reinterpret_cast<unsigned*>(p);
     return w;
 }
 
 __device__ __forceinline__ float nan_to_inf(float v) { return v != v ? CUDART_INF_F : v; }
+__device__ __forceinline__ float finite_or_zero(float v) {
+    return (__float_as_uint(v) & 0x7f800000u) != 0x7f800000u ? v : 0.f;
+}
+__device__ __forceinline__ void order2(float& a, float& b) {
+    const float lo = fminf(a, b), hi = fmaxf(a, b);
+    a = lo;
+    b = hi;
+}
 
-// grid (nblk, nsplit): block b covers columns [c0, c0 + cols), the blocks evenly spaced over d
+// One CTA per sampled block of 64 columns (evenly spaced over d).
 __global__ void __launch_bounds__(kPickThreads)
-centre_sample_kernel(const float* __restrict__ X, int64_t ld, int m, int64_t d, int cols, float* __restrict__ part,
+centre_sample_kernel(const float* __restrict__ X, int64_t ld, int m, int64_t d, float* __restrict__ part,
                      unsigned* __restrict__ counter) {
-    extern __shared__ float tile[];   // [m][cols + 1]
+    extern __shared__ float tile[];   // [m][kSampleCols + 1], then the first centre [kSampleCols]
+    constexpr int pitch = kSampleCols + 1;
+    float* first = tile + (size_t)m * pitch;
     const int b = blockIdx.x, nblk = gridDim.x;
-    const int64_t nb_all = (d + cols - 1) / cols;
-    const int64_t c0 = (nb_all * b / nblk) * cols;
-    const int pitch = cols + 1;
-    if (b == 0 && blockIdx.y == 0 && threadIdx.x == 0) counter[0] = counter[1] = 0u;   // for the kernels that follow
-    for (int e = threadIdx.x; e < m * cols; e += kPickThreads) {
-        const int r = e / cols, c = e - r * cols;
+    const int64_t nb_all = (d + kSampleCols - 1) / kSampleCols;
+    const int64_t c0 = (nb_all * b / nblk) * kSampleCols;
+    if (b == 0 && threadIdx.x == 0) counter[0] = counter[1] = 0u;   // for the kernels that follow
+    for (int e = threadIdx.x; e < m * kSampleCols; e += kPickThreads) {
+        const int r = e / kSampleCols, c = e - r * kSampleCols;
         const int64_t col = c0 + c;
-        tile[r * pitch + c] = col < d ? X[(int64_t)r * ld + col] : 0.f;
+        tile[r * pitch + c] = col < d ? finite_or_zero(X[(int64_t)r * ld + col]) : 0.f;
     }
     __syncthreads();
-    float* out = part + (int64_t)b * m * m;
-    const int total = m * m;
-    for (int e = blockIdx.y * kPickThreads + threadIdx.x; e < total; e += gridDim.y * kPickThreads) {
-        const int i = e / m, j = e - i * m;
-        if (j < i) continue;
-        const float* ti = tile + i * pitch;
-        const float* tj = tile + j * pitch;
-        float s = 0.f;
-        if (i == j) {
-            for (int c = 0; c < cols; ++c) s = fmaf(ti[c], ti[c], s);
-        } else {
-            for (int c = 0; c < cols; ++c) {
-                const float t = ti[c] - tj[c];
-                s = fmaf(t, t, s);
-            }
+    if (threadIdx.x < kSampleCols) {
+        // median of the rows at positions (2k + 1) m / 14, k = 0..6: the 16-comparator sorting network on seven values
+        const int c = threadIdx.x;
+        float v[kFirstRows];
+#pragma unroll
+        for (int k = 0; k < kFirstRows; ++k) v[k] = tile[(((2 * k + 1) * m) / (2 * kFirstRows)) * pitch + c];
+        order2(v[0], v[6]); order2(v[2], v[3]); order2(v[4], v[5]);
+        order2(v[0], v[2]); order2(v[1], v[4]); order2(v[3], v[6]);
+        order2(v[0], v[1]); order2(v[2], v[5]); order2(v[3], v[4]);
+        order2(v[1], v[2]); order2(v[4], v[6]);
+        order2(v[2], v[3]); order2(v[4], v[5]);
+        order2(v[1], v[2]); order2(v[3], v[4]); order2(v[5], v[6]);
+        first[c] = v[3];
+    }
+    __syncthreads();
+    float* out = part + (size_t)b * 2 * m;
+    for (int r = threadIdx.x; r < m; r += kPickThreads) {
+        const float* row = tile + r * pitch;
+        float dist = 0.f, nrm = 0.f;
+#pragma unroll 8
+        for (int c = 0; c < kSampleCols; ++c) {
+            const float x = row[c], t = x - first[c];
+            dist = fmaf(t, t, dist);
+            nrm = fmaf(x, x, nrm);
         }
-        out[e] = s;
+        out[r] = dist;
+        out[m + r] = nrm;
     }
 }
 
-// One CTA per row: the median of the row's sample distances to the other rows and its sample norm; the CTA that
-// finishes last picks the row with the smallest median and decides whether centring pays.
+// One CTA: adds the blocks' partial sums, ranks the rows by their distance to the first centre, lists the centring
+// rows and decides whether centring pays.
 __global__ void __launch_bounds__(kPickThreads)
-centre_pick_kernel(const float* __restrict__ part, int nblk, int m, float scale, float* __restrict__ key,
-                   float* __restrict__ nrm, unsigned* __restrict__ counter, int* __restrict__ centre) {
-    extern __shared__ float rowv[];   // [m]
-    __shared__ float s_val[kPickThreads];
-    __shared__ int s_idx[kPickThreads];
-    __shared__ bool s_last;
-    const int i = blockIdx.x;
-    const int64_t mm = (int64_t)m * m;
-    for (int j = threadIdx.x; j < m; j += kPickThreads) {
-        const int a = i < j ? i : j, b2 = i < j ? j : i;
-        float v = 0.f;
-        for (int b = 0; b < nblk; ++b) v += part[(int64_t)b * mm + (int64_t)a * m + b2];
-        v = nan_to_inf(v);
-        if (j == i) nrm[i] = v;
-        rowv[j] = j == i ? CUDART_INF_F : v;
-    }
-    __syncthreads();
-    const int h = (m - 2) / 2;   // middle of the m - 1 distances to the other rows
-    for (int j = threadIdx.x; j < m; j += kPickThreads) {
-        if (j == i) continue;
-        const float v = rowv[j];
-        int rank = 0;
-        for (int k = 0; k < m; ++k) {
-            if (k == i) continue;
-            const float u = rowv[k];
-            rank += (u < v || (u == v && k < j)) ? 1 : 0;
-        }
-        if (rank == h) key[i] = v;
-    }
-    __threadfence();
-    __syncthreads();
-    if (threadIdx.x == 0) s_last = atomicAdd(counter, 1u) == (unsigned)(m - 1);
-    __syncthreads();
-    if (!s_last) return;
-    __threadfence();
-    // smallest key, ties to the lower row
-    float best = CUDART_INF_F;
-    int arg = 0x7fffffff;
+centre_pick_kernel(const float* __restrict__ part, int nblk, int m, float scale, unsigned* __restrict__ counter,
+                   int* __restrict__ centre) {
+    extern __shared__ float sh[];   // dist [m], norm [m]
+    float* dist = sh;
+    float* nrm = sh + m;
+    __shared__ float med[2];
     for (int r = threadIdx.x; r < m; r += kPickThreads) {
-        const float v = __ldcg(key + r);
-        if (v < best || (v == best && r < arg)) { best = v; arg = r; }
-    }
-    s_val[threadIdx.x] = best;
-    s_idx[threadIdx.x] = arg;
-    __syncthreads();
-    for (int o = kPickThreads / 2; o > 0; o >>= 1) {
-        if (threadIdx.x < o) {
-            const float v = s_val[threadIdx.x + o];
-            const int r = s_idx[threadIdx.x + o];
-            if (v < s_val[threadIdx.x] || (v == s_val[threadIdx.x] && r < s_idx[threadIdx.x])) {
-                s_val[threadIdx.x] = v;
-                s_idx[threadIdx.x] = r;
-            }
+        float a = 0.f, n = 0.f;
+        for (int b = 0; b < nblk; ++b) {
+            a += part[(size_t)b * 2 * m + r];
+            n += part[(size_t)b * 2 * m + m + r];
         }
-        __syncthreads();
+        dist[r] = nan_to_inf(a);
+        nrm[r] = nan_to_inf(n);
     }
-    const float best_key = s_val[0];
     __syncthreads();
-    // median of the sample norms (rank counting again; rowv is free now)
-    for (int r = threadIdx.x; r < m; r += kPickThreads) rowv[r] = __ldcg(nrm + r);
-    __syncthreads();
+    const int want = m / 2 < kMaxCentreRows ? m / 2 : kMaxCentreRows;
+    // the rows at ranks 0, s, 2s, ... of the ordering by distance, inside its closer half
+    const int stride = (m / 2) / (want > 0 ? want : 1) > 1 ? (m / 2) / want : 1;
     const int hm = (m - 1) / 2;
     for (int r = threadIdx.x; r < m; r += kPickThreads) {
-        const float v = rowv[r];
-        int rank = 0;
+        const float v = dist[r], w = nrm[r];
+        int rank = 0, rank_n = 0;
         for (int k = 0; k < m; ++k) {
-            const float u = rowv[k];
+            const float u = dist[k], un = nrm[k];
             rank += (u < v || (u == v && k < r)) ? 1 : 0;
-        }
-        if (rank == hm) s_val[0] = v;
-    }
-    __syncthreads();
-    // on when the most central row's typical distance to the others is clearly below what two rows that hover around
-    // zero have (twice the typical squared norm)
-    const int want = m / 2 < kMaxCentreRows ? m / 2 : kMaxCentreRows;
-    const bool on = best_key < 1.5f * s_val[0] && want >= 1;
-    // the rows at ranks 0, s, 2s, ... of the ordering by median distance, inside its more central half
-    const int stride = (m / 2) / (want > 0 ? want : 1) > 1 ? (m / 2) / want : 1;
-    for (int r = threadIdx.x; r < m; r += kPickThreads) rowv[r] = __ldcg(key + r);
-    __syncthreads();
-    for (int r = threadIdx.x; r < m; r += kPickThreads) {
-        const float v = rowv[r];
-        int rank = 0;
-        for (int k = 0; k < m; ++k) {
-            const float u = rowv[k];
-            rank += (u < v || (u == v && k < r)) ? 1 : 0;
+            rank_n += (un < w || (un == w && k < r)) ? 1 : 0;
         }
         if (rank % stride == 0 && rank / stride < want) centre[2 + rank / stride] = r;
+        if (rank == hm) med[0] = v;
+        if (rank_n == hm) med[1] = w;
     }
+    __syncthreads();
     if (threadIdx.x == 0) {
-        centre[0] = on ? want : 0;
-        *reinterpret_cast<float*>(counter + 2) = s_val[0] * scale;   // for the check after the pass
+        // on when the typical row is closer to the first centre than to the origin
+        centre[0] = (want >= 1 && med[0] < med[1]) ? want : 0;
+        *reinterpret_cast<float*>(counter + 2) = med[1] * scale;   // for the check after the pass
     }
 }
 
@@ -253,34 +204,31 @@ centre_check_kernel(const float* __restrict__ norms, int nshares, int m, float* 
 }  // namespace
 
 size_t centre_ws_bytes(int m, int64_t d) {
-    const CentrePlan p = centre_plan(m, d);
-    return align_up((size_t)p.nblk * m * m * sizeof(float)) + 2 * align_up((size_t)m * sizeof(float)) + 256;   // counters, float
+    (void)d;
+    return align_up((size_t)kSampleBlocks * 2 * m * sizeof(float)) + align_up((size_t)m * sizeof(float)) + 256;   // counters, float
 }
 
 detox_status launch_pick_centre(const float* X, int64_t ld, int m, int64_t d, void* ws, int* centre, cudaStream_t s) {
-    const CentrePlan p = centre_plan(m, d);
-    CentreWs w = centre_carve(ws, m, p.nblk);
-    const size_t smem = (size_t)m * (p.cols + 1) * sizeof(float);
+    CentreWs w = centre_carve(ws, m);
+    const int nblk = sample_blocks(d);
+    const size_t smem = ((size_t)m * (kSampleCols + 1) + kSampleCols) * sizeof(float);
     if (cudaFuncSetAttribute(centre_sample_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return DETOX_ERR_CUDA;
-    centre_sample_kernel<<<dim3((unsigned)p.nblk, (unsigned)p.nsplit), kPickThreads, smem, s>>>(X, ld, m, d, p.cols, w.part,
-                                                                                          w.counter);
+    centre_sample_kernel<<<nblk, kPickThreads, smem, s>>>(X, ld, m, d, w.part, w.counter);
     detox_status st = launch_status();
     if (st != DETOX_OK) return st;
     // the sample's squared norms are scaled up to all d columns for the check after the pass
-    const int64_t sampled = (int64_t)p.nblk * p.cols < d ? (int64_t)p.nblk * p.cols : d;
+    const int64_t sampled = (int64_t)nblk * kSampleCols < d ? (int64_t)nblk * kSampleCols : d;
     const float scale = (float)((double)d / (double)sampled);
-    centre_pick_kernel<<<m, kPickThreads, (size_t)m * sizeof(float), s>>>(w.part, p.nblk, m, scale, w.key, w.nrm, w.counter,
-                                                                         centre);
+    centre_pick_kernel<<<1, kPickThreads, (size_t)2 * m * sizeof(float), s>>>(w.part, nblk, m, scale, w.counter, centre);
     return launch_status();
 }
 
 detox_status launch_check_centre(const float* norms, int nshares, int m, void* ws, int64_t d, int* centre, int* redo,
                                  cudaStream_t s) {
-    const CentrePlan p = centre_plan(m, d);
-    CentreWs w = centre_carve(ws, m, p.nblk);
-    // the pick kernel is done with `key`: it holds the exact norms now; the second counter word was cleared by the
-    // sample kernel
+    (void)d;
+    CentreWs w = centre_carve(ws, m);
+    // the second counter word was cleared by the sample kernel
     centre_check_kernel<<<m, 128, 0, s>>>(norms, nshares, m, w.key, w.counter, centre, redo);
     return launch_status();
 }

@@ -149,14 +149,8 @@ __device__ __forceinline__ uint64_t lo2_of(uint64_t x2) {
     return add2(t, t);
 }
 
-// A packed pair of fp32 with every Inf / NaN replaced by zero (the centring row must not spread its non-finite
-// entries to the other rows: at such a coordinate nothing is subtracted).
-__device__ __forceinline__ uint64_t finite_or_zero2(uint64_t v) {
-    const uint32_t lo = (uint32_t)v, hi = (uint32_t)(v >> 32);
-    const uint32_t lo_ok = (lo & 0x7f800000u) != 0x7f800000u ? lo : 0u;
-    const uint32_t hi_ok = (hi & 0x7f800000u) != 0x7f800000u ? hi : 0u;
-    return (uint64_t)lo_ok | ((uint64_t)hi_ok << 32);
-}
+// An Inf / NaN replaced by zero (the subtracted vector must not spread a listed row's non-finite entries to the
+// other rows: at such a coordinate nothing is subtracted).
 __device__ __forceinline__ float finite_or_zero(float v) {
     return (__float_as_uint(v) & 0x7f800000u) != 0x7f800000u ? v : 0.f;
 }
@@ -420,8 +414,9 @@ gram_wide_kernel(const __grid_constant__ CUtensorMap xmap, int m, uint32_t lo_of
                 for (int k = 0; k < kMaxCentreRows; ++k) v[k] = *reinterpret_cast<const float*>(tile + off[k]);
                 float acc = 0.f;
 #pragma unroll
-                for (int k = 0; k < kMaxCentreRows; ++k) acc += k < ncentre ? finite_or_zero(v[k]) : 0.f;
-                sm->cring[s][lane] = acc * inv;
+                for (int k = 0; k < kMaxCentreRows; ++k)
+                    if (k < ncentre) acc += v[k];
+                sm->cring[s][lane] = finite_or_zero(acc) * inv;   // a column whose sum is not finite is left uncentred
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&sm->c_full[s]);
                 if (++s == stages) { s = 0; ph ^= 1u; }
@@ -630,14 +625,23 @@ gram_staged_kernel(const __grid_constant__ CUtensorMap xmap, int m, uint32_t stg
             const int nst = li == my_items - 1 ? last_nst : kStagesPerSlab;
             const int t_end = li * kStagesPerSlab + nst;
             for (; t < t_end; t += LX) {
-                mbar_wait(&sm->stg_full[ss], sph, abort_flag, status);
+                // (the centring warp works ahead of the transform warps, so its barrier has usually completed; waiting
+                // for it first lets the load of the subtracted vector travel with the loads of the rows)
+                if (ncentre > 0) {
+                    const bool c_ok = mbar_try(&sm->c_full[ss], sph), x_ok = mbar_try(&sm->stg_full[ss], sph);
+                    if (!(c_ok && x_ok)) {
+                        mbar_wait(&sm->c_full[ss], sph, abort_flag, status);
+                        mbar_wait(&sm->stg_full[ss], sph, abort_flag, status);
+                    }
+                } else {
+                    mbar_wait(&sm->stg_full[ss], sph, abort_flag, status);
+                }
                 const uint8_t* src = stg_base + (size_t)ss * stg_bytes + src0;
                 ulonglong2 x[J];
 #pragma unroll
                 for (int j = 0; j < J; ++j)
                     if (gtid + j * kGroupThreads < npieces) x[j] = *reinterpret_cast<const ulonglong2*>(src + j * kSrcStep);
                 if (ncentre > 0) {
-                    mbar_wait(&sm->c_full[ss], sph, abort_flag, status);
                     const ulonglong2 ck = *reinterpret_cast<const ulonglong2*>(&sm->cring[ss][q * 4]);
 #pragma unroll
                     for (int j = 0; j < J; ++j)
@@ -728,30 +732,43 @@ gram_staged_kernel(const __grid_constant__ CUtensorMap xmap, int m, uint32_t stg
             for (int e = tid; e < m * LX; e += kProdThreads) norms[item * LX * m + e] = 0.f;
         }
     } else if (warp == kProdWarps + NMMA + kTma) {
-        // ------------------------------------------------ the centring warp: lane l averages columns 2l and 2l+1 of the
-        // listed rows of every stage as it lands (non-finite entries count as zero) and hands the 64 averages on
+        // ------------------------------------------------ the centring warp: averages the listed rows of every stage as
+        // it lands and hands the 64 averages on.  Lanes 0-15 add the first eight listed rows, lanes 16-31 the others,
+        // four columns (16 bytes) a lane; the halves meet through shuffles.  A column whose sum is not finite is left
+        // uncentred (zero is subtracted there).  The warp shares its scheduler with transform warps that are always
+        // ready, so it is kept to a few dozen instructions a stage.
         if (ncentre > 0) {
             const float inv = 1.f / (float)ncentre;
-            // byte offset of this lane's two columns in every listed row; all loads of a stage are issued together
-            uint32_t off[kMaxCentreRows];
+            const int half = lane >> 4;
+            constexpr int kPerHalf = kMaxCentreRows / 2;
+            uint32_t off[kPerHalf];
 #pragma unroll
-            for (int k = 0; k < kMaxCentreRows; ++k)
-                off[k] = (uint32_t)sm->crow[k < ncentre ? k : 0] * (uint32_t)(kStageCols * 4) + (uint32_t)lane * 8u;
+            for (int k = 0; k < kPerHalf; ++k) {
+                const int kk = half * kPerHalf + k;
+                off[k] = (uint32_t)sm->crow[kk < ncentre ? kk : 0] * (uint32_t)(kStageCols * 4) + (uint32_t)(lane & 15) * 16u;
+            }
+            const int mine = ncentre - half * kPerHalf;   // listed rows in this half (may be <= 0)
             int s = 0;
             uint32_t ph = 0;
             for (int t = 0; t < total; ++t) {
                 if (!mbar_wait(&sm->stg_full[s], ph, abort_flag, status)) break;
                 const uint8_t* stg = stg_base + (size_t)s * stg_bytes;
-                float2 v[kMaxCentreRows];
+                float4 v[kPerHalf];
 #pragma unroll
-                for (int k = 0; k < kMaxCentreRows; ++k) v[k] = *reinterpret_cast<const float2*>(stg + off[k]);
-                float2 acc = make_float2(0.f, 0.f);
+                for (int k = 0; k < kPerHalf; ++k) v[k] = *reinterpret_cast<const float4*>(stg + off[k]);
+                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-                for (int k = 0; k < kMaxCentreRows; ++k) {
-                    acc.x += k < ncentre ? finite_or_zero(v[k].x) : 0.f;
-                    acc.y += k < ncentre ? finite_or_zero(v[k].y) : 0.f;
+                for (int k = 0; k < kPerHalf; ++k) {
+                    if (k < mine) { acc.x += v[k].x; acc.y += v[k].y; acc.z += v[k].z; acc.w += v[k].w; }
                 }
-                *reinterpret_cast<float2*>(&sm->cring[s][2 * lane]) = make_float2(acc.x * inv, acc.y * inv);
+                acc.x += __shfl_xor_sync(0xffffffffu, acc.x, 16);
+                acc.y += __shfl_xor_sync(0xffffffffu, acc.y, 16);
+                acc.z += __shfl_xor_sync(0xffffffffu, acc.z, 16);
+                acc.w += __shfl_xor_sync(0xffffffffu, acc.w, 16);
+                if (lane < 16)
+                    *reinterpret_cast<float4*>(&sm->cring[s][4 * lane]) =
+                        make_float4(finite_or_zero(acc.x) * inv, finite_or_zero(acc.y) * inv, finite_or_zero(acc.z) * inv,
+                                    finite_or_zero(acc.w) * inv);
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&sm->c_full[s]);
                 if (++s == nstg) { s = 0; ph ^= 1u; }

@@ -116,8 +116,9 @@ __device__ __forceinline__ void multikrum_select_body(const double* sorted_d, in
     }
 }
 
-template <bool ONE_WARP>
-__device__ __forceinline__ void bulyan_select_body(const double* sorted_d, const int32_t* sorted_j, const int32_t* pos_t,
+// Idx: the type the column and position tables are held in (int32 in global memory; uint8 when cached in shared memory)
+template <bool ONE_WARP, typename Idx>
+__device__ __forceinline__ void bulyan_select_body(const double* sorted_d, const Idx* sorted_j, const Idx* pos_t,
                                                    int m, int f, int32_t* sel) {
     __shared__ unsigned char alive[kMaxRows];
     __shared__ double best_s[32];
@@ -129,7 +130,7 @@ __device__ __forceinline__ void bulyan_select_body(const double* sorted_d, const
     const bool mine = i < m;
     if (i < kMaxRows) alive[i] = mine ? 1 : 0;
     const double* dist = sorted_d + (int64_t)i * m;   // row i's other rows, closest first (self last)
-    const int32_t* col = sorted_j + (int64_t)i * m;
+    const Idx* col = sorted_j + (int64_t)i * m;
 
     // round 0: the nb closest rows, added in ascending order
     int nb = krum_neighbours(m, f);
@@ -225,6 +226,25 @@ __global__ void __launch_bounds__(1024)
 bulyan_select_kernel(const double* __restrict__ sorted_d, const int32_t* __restrict__ sorted_j,
                      const int32_t* __restrict__ pos_t, int m, int f, int32_t* __restrict__ sel) {
     bulyan_select_body<false>(sorted_d, sorted_j, pos_t, m, f, sel);
+}
+
+// Up to 256 rows the two index tables fit in shared memory as bytes (2 m^2 <= 128 KB).  A round is a chain of
+// dependent look-ups (which position did the removed row have in my list? which is my next remaining neighbour?);
+// from shared memory each costs tens of cycles instead of a trip to L2, and only the distances themselves, one or
+// two per row and round, still come from global memory.
+constexpr int kCachedSelectRows = 256;
+__global__ void __launch_bounds__(kCachedSelectRows)
+bulyan_select_cached_kernel(const double* __restrict__ sorted_d, const int32_t* __restrict__ sorted_j,
+                            const int32_t* __restrict__ pos_t, int m, int f, int32_t* __restrict__ sel) {
+    extern __shared__ uint8_t tables[];   // [m*m] columns, then [m*m] positions
+    uint8_t* col8 = tables;
+    uint8_t* pos8 = tables + m * m;
+    for (int e = threadIdx.x; e < m * m; e += blockDim.x) {
+        col8[e] = (uint8_t)sorted_j[e];
+        pos8[e] = (uint8_t)pos_t[e];
+    }
+    __syncthreads();
+    bulyan_select_body<false>(sorted_d, col8, pos8, m, f, sel);
 }
 
 // m <= 16: everything between the distance pass and the final mean / order statistics in one CTA:
@@ -356,7 +376,15 @@ detox_status launch_bulyan_select(const double* D, int m, int f, int32_t* sel_de
     rank_rows_kernel<<<m, 256, (size_t)m * sizeof(double), s>>>(D, m, w.sorted_d, w.sorted_j, w.pos_t);
     detox_status st = launch_status();
     if (st != DETOX_OK) return st;
-    bulyan_select_kernel<<<1, round_up_warp(m), 0, s>>>(w.sorted_d, w.sorted_j, w.pos_t, m, f, sel_dev);
+    if (m <= kCachedSelectRows) {
+        const size_t smem = (size_t)2 * m * m;
+        if (cudaFuncSetAttribute(bulyan_select_cached_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
+            cudaSuccess)
+            return DETOX_ERR_CUDA;
+        bulyan_select_cached_kernel<<<1, round_up_warp(m), smem, s>>>(w.sorted_d, w.sorted_j, w.pos_t, m, f, sel_dev);
+    } else {
+        bulyan_select_kernel<<<1, round_up_warp(m), 0, s>>>(w.sorted_d, w.sorted_j, w.pos_t, m, f, sel_dev);
+    }
     return launch_status();
 }
 
