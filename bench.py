@@ -8,6 +8,7 @@ direct (non-DETOX) aggregators on the same buffer, each with the roofline that b
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload cfg4|cfg1|cfg2|cfg3]
   python bench.py --sweep            (one JSON line per point of the n x d x attack sweep)
+  python bench.py --mean-estimation  (the synthetic experiment with 220,000 nodes: one JSON line per dimension)
 
 With N > 1 (launched by torch.distributed.run) every rank aggregates its own independent copy of the
 workload (replicas; the path has no exchange step) and rank 0 reports the sum over ranks.
@@ -402,6 +403,65 @@ def run_sweep(args):
         torch.cuda.empty_cache()
 
 
+def run_mean_estimation(args):
+    """The paper's synthetic experiment (Section 5.3, "Mean estimation on synthetic data"): p = 220,000 nodes, r = 11,
+    q = floor(e^r / 3) Byzantine nodes sending a constant vector of norm 100, d = 20 .. 100.  DETOX = vote -> mean
+    inside 25 vote sets -> geometric median (or coordinate median) of the 25 means; the error is the l2 norm of the
+    estimate (the true mean is zero).  One JSON line per d; times are CUDA-event means after warm-up."""
+    import torch
+
+    import oracle
+    import paper_1907_12205_b200 as dx
+    import workloads as wl
+
+    dev = "cuda:0"
+    torch.cuda.set_device(0)
+    reps = max(3, min(args.steps, 20))
+    for d in range(20, 101, 10):
+        w = wl.make_mean_estimation(d=d, seed=d, device=dev)
+        X = w.X
+        members = torch.as_tensor(w.members, device=dev)
+        G, S = w.p // w.r, len(w.set_offsets) - 1
+        M = torch.empty((S, (d + 31) // 32 * 32), dtype=torch.float32, device=dev)[:, :d]
+        win = torch.empty(G, dtype=torch.int32, device=dev)
+        out = torch.empty(d, dtype=torch.float32, device=dev)
+        gws = torch.empty(max(int(dx.load().agg_geometric_median_workspace_bytes(S, d)), 256), dtype=torch.uint8, device=dev)
+
+        def step_gm():
+            dx.detox_vote_hier_mean_many(X, w.r, members, w.set_offsets, M=M, winner=win)
+            dx.agg_geometric_median(M, iters=32, out=out, ws=gws)
+
+        def step_med():
+            dx.detox_vote_hier_mean_many(X, w.r, members, w.set_offsets, M=M, winner=win)
+            dx.agg_coord_median(M, out=out)
+
+        ms_gm = time_calls(torch, step_gm, reps, 3)
+        step_gm(); torch.cuda.synchronize()
+        err_gm = float(torch.linalg.vector_norm(out))
+        ms_med = time_calls(torch, step_med, reps, 3)
+        step_med(); torch.cuda.synchronize()
+        err_med = float(torch.linalg.vector_norm(out))
+        ms_front = time_calls(torch, lambda: dx.detox_vote_hier_mean_many(X, w.r, members, w.set_offsets, M=M, winner=win),
+                              reps, 3)
+        Xh = X.cpu().numpy()
+        t0 = time.perf_counter()
+        Zo, wo = oracle.vote(Xh, w.members, w.r)
+        Mo = oracle.hier_mean(Zo, w.set_offsets, np.arange(G, dtype=np.int32))
+        go = oracle.geometric_median(Mo, iters=32)
+        cpu_ms = (time.perf_counter() - t0) * 1e3
+        in_bytes = w.p * d * 4
+        print(json.dumps({"mean_estimation": True, "p": w.p, "r": w.r, "q": w.q, "q_hat": w.q_hat, "d": d, "sets": S,
+                          "detox_geometric_median": {"ms": round(ms_gm, 4), "l2_error": err_gm,
+                                                     "GBps": round(in_bytes / ms_gm / 1e6, 1)},
+                          "detox_coord_median": {"ms": round(ms_med, 4), "l2_error": err_med,
+                                                 "GBps": round(in_bytes / ms_med / 1e6, 1)},
+                          "vote_and_set_means": {"ms": round(ms_front, 4), "GBps": round(in_bytes / ms_front / 1e6, 1)},
+                          "oracle": {"ms": round(cpu_ms, 1), "cores": oracle.num_threads(),
+                                     "l2_error_geometric_median": float(np.linalg.norm(go)),
+                                     "winners_equal": win.cpu().numpy().tolist() == wo.tolist()}}), flush=True)
+        del w, X
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -414,6 +474,8 @@ def main():
     ap.add_argument("--sweep-n", default="15,45,105,225")
     ap.add_argument("--sweep-d", default="1000000,11173962,25557032")
     ap.add_argument("--sweep-attacks", default="reverse,alie")
+    ap.add_argument("--mean-estimation", action="store_true",
+                    help="the synthetic mean-estimation experiment: one JSON line per dimension")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "detox" else args.warmup
 
@@ -426,6 +488,10 @@ def main():
     if args.sweep:
         if rank == 0:
             run_sweep(args)
+        return
+    if args.mean_estimation:
+        if rank == 0:
+            run_mean_estimation(args)
         return
 
     import torch

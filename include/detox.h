@@ -134,6 +134,28 @@ detox_status detox_vote_hier_mean(const float* X, int64_t ld, int n, int r, int6
                                   int64_t ldm, int32_t* winner, void* ws, size_t ws_bytes, void* stream);
 
 /* ---------------------------------------------------------------------------------------------
+ * The same two steps for very many nodes with short vectors - the regime of the paper's synthetic
+ * experiment (Section 5.3, "Mean estimation on synthetic data": p = 220,000 nodes, r = 11, d <= 100), where
+ * the tables above (at most DETOX_MAX_ROWS nodes) do not reach.  One warp votes per node group; the
+ * group table lives in device memory; a vote set is a run of consecutive groups (the group table is a
+ * random partition already, so consecutive groups are a random set).  The S set means then go to
+ * agg_geometric_median / agg_coord_median as ordinary rows.
+ *
+ *   X            dev, n x ld     n <= 2^30 nodes, d <= DETOX_MANY_MAX_D
+ *   members      dev, n          worker ids, group j owns members[j*r .. j*r+r-1]; must be a partition of
+ *                                0..n-1 (not checked; a group holding an id outside 0..n-1 gets no vote)
+ *   set_offsets  host, S+1       set s owns the groups set_offsets[s] .. set_offsets[s+1]-1; S <= DETOX_MAX_ROWS
+ *   M            dev, S x ldm    out: mean of the votes of each set (a group without a majority counts as a
+ *                                zero vote); may be NULL, then only `winner` is produced and sets are ignored
+ *   winner       dev, n / r      out, as in detox_vote
+ * No workspace.
+ * ------------------------------------------------------------------------------------------- */
+#define DETOX_MANY_MAX_D 1024
+detox_status detox_vote_hier_mean_many(const float* X, int64_t ld, int64_t n, int r, int d, const int32_t* members,
+                                       const int32_t* set_offsets, int S, float* M, int64_t ldm, int32_t* winner,
+                                       void* stream);
+
+/* ---------------------------------------------------------------------------------------------
  * Coordinate-wise median (Section 4; Appendix B.1): out[c] = median_i X[i][c] over the m rows.
  * Odd m: the middle value, bit for bit one of the inputs.  Even m: fp32 (lo + hi) * 0.5f.
  *   out  dev, d.   ws: agg_coord_median_workspace_bytes(m, d) bytes.  Every size built so far works in

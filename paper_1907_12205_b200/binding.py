@@ -26,7 +26,7 @@ EXPORTS = (
     "agg_coord_median_workspace_bytes", "agg_coord_median", "agg_trimmed_mean", "agg_sign_majority", "agg_geometric_median_workspace_bytes", "agg_geometric_median", "agg_multikrum_workspace_bytes", "agg_multikrum",
     "agg_bulyan_workspace_bytes", "agg_bulyan", "detox_aggregate_workspace_bytes", "detox_aggregate",
     "detox_selftest_bounded_wait", "agg_pairwise_sqdist_workspace_bytes", "agg_pairwise_sqdist",
-    "detox_kernel_launch_count",
+    "detox_kernel_launch_count", "detox_vote_hier_mean_many",
 )
 
 
@@ -88,6 +88,7 @@ def load() -> ctypes.CDLL:
     lib.agg_pairwise_sqdist_workspace_bytes.restype = _sz
     lib.agg_pairwise_sqdist_workspace_bytes.argtypes = [_int, _i64]
     lib.agg_pairwise_sqdist.argtypes = [_vp, _i64, _int, _i64, _vp, _vp, _sz, _vp]
+    lib.detox_vote_hier_mean_many.argtypes = [_vp, _i64, _i64, _int, _int, _vp, _ip, _int, _vp, _i64, _vp, _vp]
     lib.detox_kernel_launch_count.restype = ctypes.c_ulonglong
     lib.detox_kernel_launch_count.argtypes = []
     _lib = lib
@@ -225,6 +226,30 @@ def detox_vote_hier_mean(X, r: int, members, set_offsets, set_members, M: Option
     _check(lib.detox_vote_hier_mean(xp, ld, n, r, d, mem.ctypes.data_as(_ip), so.ctypes.data_as(_ip),
                                     sm.ctypes.data_as(_ip), S, M.data_ptr(), ldm, winner.data_ptr(), wp, wb,
                                     _stream(stream)), "detox_vote_hier_mean")
+    return M, winner
+
+
+def detox_vote_hier_mean_many(X, r: int, members_dev: torch.Tensor, set_offsets=None, M: Optional[torch.Tensor] = None,
+                              winner: Optional[torch.Tensor] = None, stream=None):
+    """Vote and set means for very many nodes with short vectors.  members_dev: int32 CUDA tensor [n];
+    set_offsets: host, in groups (None: votes only).  Returns (M [S, d] or None, winner [n / r])."""
+    lib = load()
+    xp, ld, n, d = _mat(X)
+    if not (members_dev.is_cuda and members_dev.dtype == torch.int32 and members_dev.numel() == n):
+        raise TypeError("members_dev: int32 CUDA tensor with one entry per node")
+    G = n // max(r, 1)
+    if winner is None:
+        winner = torch.empty(max(G, 1), dtype=torch.int32, device=X.device)[:G]
+    so, S, mp, ldm = None, 0, None, 0
+    if set_offsets is not None:
+        so = _host_i32(set_offsets)
+        S = len(so) - 1
+        if M is None:
+            M = torch.empty((max(S, 1), (d + 31) // 32 * 32), dtype=torch.float32, device=X.device)[:S, :d]
+        mp, ldm = M.data_ptr(), (M.stride(0) if M.shape[0] > 1 else max(M.stride(0), d))
+    _check(lib.detox_vote_hier_mean_many(xp, ld, n, r, d, members_dev.data_ptr(),
+                                         None if so is None else so.ctypes.data_as(_ip), S, mp, ldm, winner.data_ptr(),
+                                         _stream(stream)), "detox_vote_hier_mean_many")
     return M, winner
 
 

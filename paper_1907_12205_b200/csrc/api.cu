@@ -184,6 +184,12 @@ int a0_selected(const detox_pipeline_desc* p, int k) {
 // written: always for the per-coordinate aggregators, and for the Krum type up to 16 votes (the
 // direct-difference distance kernel takes a row list; the tensor-core Gram wants consecutive rows).
 bool votes_by_index(const detox_pipeline_desc* p) {
+    if (krum_type(p->a0)) {
+        // Multi-Krum / Bulyan inside the vote sets: every set of at most 16 votes is read through its winners
+        for (int s = 0; s < p->n_sets; ++s)
+            if (p->set_offsets[s + 1] - p->set_offsets[s] > 16) return false;
+        return true;
+    }
     if (p->a0 != DETOX_AGG_NONE || p->a1 == DETOX_AGG_GEOMETRIC_MEDIAN) return false;
     return !krum_type(p->a1) || p->n / p->r <= 16;
 }
@@ -478,19 +484,24 @@ detox_status detox_aggregate(const detox_pipeline_desc* p, const float* X, int64
         IdTable in_set_order;
         for (int k = 0; k < G; ++k)
             for (int a = 0; a < p->r; ++a) in_set_order.id[k * p->r + a] = groups.id[sets.member[k] * p->r + a];
-        if ((st = launch_vote(X, ld, p->n, p->r, p->d, in_set_order, w.Z, w.ldz, w.winner_set_order, w.vote, s, kStatusBytes)) !=
-            DETOX_OK)
+        // Sets of at most 16 votes take the distance kernels that read rows through a list: the votes are then the
+        // winners' rows of X (a negative entry: the zero row) and no vote matrix is written.
+        const bool by_index = votes_by_index(p);
+        if ((st = launch_vote(X, ld, p->n, p->r, p->d, in_set_order, by_index ? nullptr : w.Z, w.ldz, w.winner_set_order,
+                              w.vote, s, kStatusBytes)) != DETOX_OK)
             return st;
         if ((st = launch_scatter_by_set_order(w.winner_set_order, sets, G, win, s)) != DETOX_OK) return st;
         int emitted = 0;
         for (int t = 0; t < p->n_sets; ++t) {
             const int b = sets.offset[t], k = sets.offset[t + 1] - b;
             const int keep = a0_selected(p, k);
-            const float* rows_t = w.Z + (int64_t)b * w.ldz;
+            const float* rows_t = by_index ? X : w.Z + (int64_t)b * w.ldz;
+            const int64_t ld_t = by_index ? ld : w.ldz;
+            const int32_t* list_t = by_index ? w.winner_set_order + b : nullptr;
             float* out_t = w.M + (int64_t)t * w.ldz;
             st = p->a0 == DETOX_AGG_MULTIKRUM
-                     ? run_multikrum(rows_t, w.ldz, k, p->d, nullptr, p->f, keep, out_t, w.sel_local, nullptr, w.agg, w.status, s)
-                     : run_bulyan(rows_t, w.ldz, k, p->d, nullptr, p->f, out_t, w.sel_local, w.agg, w.status, s);
+                     ? run_multikrum(rows_t, ld_t, k, p->d, list_t, p->f, keep, out_t, w.sel_local, nullptr, w.agg, w.status, s)
+                     : run_bulyan(rows_t, ld_t, k, p->d, list_t, p->f, out_t, w.sel_local, w.agg, w.status, s);
             if (st != DETOX_OK) return st;
             st = launch_map_set_selection(w.sel_local, keep, sets, b, w.winner_set_order, sel ? sel + emitted : nullptr,
                                           sel_workers ? sel_workers + emitted : nullptr, s);

@@ -96,3 +96,24 @@ def test_named_configs_shapes():
     assert (c["cfg3"].q, c["cfg3"].attack) == (9, "reverse")
     assert (c["cfg4"].n, c["cfg4"].d, c["cfg4"].q, c["cfg4"].coord_scales) == (105, 28_000_000, 15, True)
     assert len(wl.sweep_specs()) == 4 * 3 * 2
+
+
+def test_mean_estimation_inputs_follow_the_papers_recipe():
+    # Section 5.3, "Mean estimation on synthetic data": p = 220000, r = 11, q = floor(e^11 / 3) = 19958
+    import math
+    w = wl.make_mean_estimation(d=20, p=22_000, r=11, seed=1)
+    assert w.q == math.floor(math.exp(11) / 3) == 19958                   # q does not depend on p
+    w = wl.make_mean_estimation(d=30, p=2200, r=11, q=200, n_sets=7, seed=1)
+    X = w.X.numpy()
+    assert X.shape == (2200, 30) and sorted(w.members.tolist()) == list(range(2200))
+    assert int(w.byzantine.sum()) == 200
+    np.testing.assert_allclose(np.linalg.norm(X[w.byzantine], axis=1), 100.0, rtol=1e-6)
+    groups = w.members.reshape(-1, 11)
+    for grp in groups[:20]:
+        hon = [i for i in grp if not w.byzantine[i]]
+        assert all(np.array_equal(X[hon[0]], X[i]) for i in hon)          # bitwise copies inside a group
+    # honest vectors are means of 20 draws of N(0, I): variance 1/20 per coordinate
+    hon_rows = X[~w.byzantine]
+    assert abs(hon_rows.var() - 1 / 20) < 0.005
+    assert w.set_offsets[0] == 0 and w.set_offsets[-1] == 200 and len(w.set_offsets) == 8
+    assert set(np.diff(w.set_offsets).tolist()) <= {28, 29}

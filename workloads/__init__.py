@@ -10,7 +10,9 @@ from .gen import (  # noqa: F401
     Workload,
     WorkloadSpec,
     expected_byzantine_votes,
+    MeanEstimation,
     make_groups,
+    make_mean_estimation,
     make_sets,
     make_workload,
     padded_ld,

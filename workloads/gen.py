@@ -272,3 +272,55 @@ def sweep_legs(spec: WorkloadSpec, G: int, S: int) -> dict:
     if n >= 4 * q + 3:
         legs["direct_bulyan"] = dict(a1="bulyan", f=q)
     return legs
+
+
+@dataclasses.dataclass
+class MeanEstimation:
+    """Inputs of the synthetic mean-estimation experiment (Section 5.3, "Mean estimation on synthetic data")."""
+    X: torch.Tensor             # [p, d] float32
+    members: np.ndarray         # int32 [p]; group j owns members[j*r:(j+1)*r]
+    set_offsets: np.ndarray     # int32 [S+1], in groups: set s owns the groups set_offsets[s] .. set_offsets[s+1]-1
+    byzantine: np.ndarray       # bool [p]
+    p: int
+    r: int
+    q: int
+    d: int
+    q_hat: int                  # groups in which Byzantine members outnumber honest ones
+
+
+def make_mean_estimation(d: int, p: int = 220_000, r: int = 11, samples: int = 20, n_sets: int = 25, seed: int = 0,
+                         q: Optional[int] = None, device: str = "cpu") -> MeanEstimation:
+    """p nodes in p / r groups; q = floor(e^r / 3) of them Byzantine, placed uniformly at random.
+
+    The paper says that 20 samples are drawn iid from N(0, I_d); the reading taken here is that every group's batch
+    holds `samples` such draws and the group's honest vector is their mean (an estimate of the true mean, zero),
+    copied bitwise to its r members.  Byzantine nodes send the constant vector of l2 norm 100.  The votes are
+    grouped into `n_sets` runs of consecutive groups (the group table is a random partition already)."""
+    if p % r != 0:
+        raise ValueError("r must divide p")
+    G = p // r
+    q = int(math.floor(math.exp(r) / 3.0)) if q is None else q
+    rng = np.random.default_rng(seed)
+    members = rng.permutation(p).astype(np.int32)
+    byz = np.zeros(p, dtype=bool)
+    byz[rng.choice(p, size=q, replace=False)] = True
+    tg = torch.Generator(device=device)
+    tg.manual_seed(seed)
+    g = torch.empty((G, d), dtype=torch.float32, device=device)
+    chunk = max(1, (1 << 24) // (samples * d))
+    for j0 in range(0, G, chunk):
+        j1 = min(G, j0 + chunk)
+        draws = torch.randn((j1 - j0, samples, d), generator=tg, device=device, dtype=torch.float32)
+        g[j0:j1] = draws.mean(dim=1)
+    X = torch.empty((p, d), dtype=torch.float32, device=device)
+    group_of = torch.empty(p, dtype=torch.long, device=device)
+    group_of[torch.as_tensor(members, dtype=torch.long, device=device)] = torch.arange(G, device=device).repeat_interleave(r)
+    X.copy_(g.index_select(0, group_of))
+    X[torch.as_tensor(byz, device=device)] = 100.0 / math.sqrt(d)
+    byz_in_group = byz[members].reshape(G, r).sum(axis=1)
+    base, extra = divmod(G, n_sets)
+    sizes = [base + (1 if s >= n_sets - extra else 0) for s in range(n_sets)]
+    offsets = np.zeros(n_sets + 1, dtype=np.int32)
+    offsets[1:] = np.cumsum(sizes)
+    return MeanEstimation(X=X, members=members, set_offsets=offsets, byzantine=byz, p=p, r=r, q=q, d=d,
+                          q_hat=int((2 * byz_in_group > r).sum()))
