@@ -177,14 +177,24 @@ __device__ __forceinline__ void bulyan_select_body(const double* sorted_d, const
         if (mine && alive[i] && remaining >= 1) {
             // the removed row leaves the sum if it was counted
             const int q = pos_t[(int64_t)gone * m + i];
+            double left_q = 0.0, left_far = 0.0;
             if (q <= last) {
-                sum -= dist[q];
+                left_q = dist[q];
                 --counted;
                 if (q == last) {
                     do { --last; } while (last >= 0 && !alive[col[last]]);
                 }
             }
-            // then the count follows nb: drop the farthest counted entry, or take the next remaining one
+            // then the count follows nb: drop the farthest counted entry, or take the next remaining one.  The first
+            // such step (the usual one: nb shrinks by one a round) is taken before either distance is used, so that
+            // the two loads travel together; the subtractions keep their order.
+            if (counted > nb_next) {
+                left_far = dist[last];
+                --counted;
+                do { --last; } while (last >= 0 && !alive[col[last]]);
+            }
+            sum -= left_q;
+            sum -= left_far;
             while (counted > nb_next) {
                 sum -= dist[last];
                 --counted;
@@ -228,23 +238,28 @@ bulyan_select_kernel(const double* __restrict__ sorted_d, const int32_t* __restr
     bulyan_select_body<false>(sorted_d, sorted_j, pos_t, m, f, sel);
 }
 
-// Up to 256 rows the two index tables fit in shared memory as bytes (2 m^2 <= 128 KB).  A round is a chain of
-// dependent look-ups (which position did the removed row have in my list? which is my next remaining neighbour?);
-// from shared memory each costs tens of cycles instead of a trip to L2, and only the distances themselves, one or
-// two per row and round, still come from global memory.
+// Up to 256 rows the two index tables fit in shared memory as bytes (2 m^2 <= 128 KB), and up to 128 rows the ranked
+// distances do as well (8 m^2 <= 128 KB).  A round is a chain of dependent look-ups (which position did the removed
+// row have in my list? which is my next remaining neighbour? what is that distance?); from shared memory each costs
+// tens of cycles instead of a trip to L2 (measured per call: 165 -> 148 microseconds at 75 rows with everything
+// cached, 360 -> 340 at 225 rows with the tables alone: the three CTA-wide barriers of a round remain).
 constexpr int kCachedSelectRows = 256;
+constexpr int kCachedDistRows = 128;
 __global__ void __launch_bounds__(kCachedSelectRows)
 bulyan_select_cached_kernel(const double* __restrict__ sorted_d, const int32_t* __restrict__ sorted_j,
                             const int32_t* __restrict__ pos_t, int m, int f, int32_t* __restrict__ sel) {
-    extern __shared__ uint8_t tables[];   // [m*m] columns, then [m*m] positions
-    uint8_t* col8 = tables;
-    uint8_t* pos8 = tables + m * m;
+    extern __shared__ __align__(8) uint8_t tables[];   // [m*m] distances (m <= 128 only), [m*m] columns, [m*m] positions
+    const bool with_dist = m <= kCachedDistRows;
+    double* dist_s = reinterpret_cast<double*>(tables);
+    uint8_t* col8 = tables + (with_dist ? (size_t)m * m * sizeof(double) : 0);
+    uint8_t* pos8 = col8 + m * m;
     for (int e = threadIdx.x; e < m * m; e += blockDim.x) {
         col8[e] = (uint8_t)sorted_j[e];
         pos8[e] = (uint8_t)pos_t[e];
+        if (with_dist) dist_s[e] = sorted_d[e];
     }
     __syncthreads();
-    bulyan_select_body<false>(sorted_d, col8, pos8, m, f, sel);
+    bulyan_select_body<false>(with_dist ? dist_s : sorted_d, col8, pos8, m, f, sel);
 }
 
 // m <= 16: everything between the distance pass and the final mean / order statistics in one CTA:
@@ -377,7 +392,7 @@ detox_status launch_bulyan_select(const double* D, int m, int f, int32_t* sel_de
     detox_status st = launch_status();
     if (st != DETOX_OK) return st;
     if (m <= kCachedSelectRows) {
-        const size_t smem = (size_t)2 * m * m;
+        const size_t smem = (size_t)2 * m * m + (m <= kCachedDistRows ? (size_t)m * m * sizeof(double) : 0);
         if (cudaFuncSetAttribute(bulyan_select_cached_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
             cudaSuccess)
             return DETOX_ERR_CUDA;
