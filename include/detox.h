@@ -291,6 +291,25 @@ detox_status detox_aggregate(const detox_pipeline_desc* desc, const float* X, in
  * ------------------------------------------------------------------------------------------- */
 detox_status detox_selftest_bounded_wait(int32_t* status, int64_t limit_cycles, void* stream);
 
+/* ---------------------------------------------------------------------------------------------
+ * Which operand split the tensor-core distance pass (17 .. 256 aligned rows; Section 4, "Improved speed": the
+ * O(p^2 d) part of Multi-Krum and Bulyan) tries first.  Process-wide; returns the previous mode; any other value of
+ * `mode` only queries.
+ *   DETOX_SPLIT_AUTO  (default) every entry as two fp16 numbers after a per-row power-of-two scale; a check after the
+ *                     pass repeats it with the split-TF32 kernels when an entry left the fp16 range (distances are
+ *                     the same to within the accuracy both give; only the time differs)
+ *   DETOX_SPLIT_TF32  the split-TF32 kernels (three-product TF32 with the cross terms folded) from the start
+ * A switch for measurements and tests; not meant to be flipped while calls are in flight on other threads.
+ * ------------------------------------------------------------------------------------------- */
+enum { DETOX_SPLIT_AUTO = 0, DETOX_SPLIT_TF32 = 1 };
+int detox_tc_split_mode(int mode);
+
+/* How many calls on the current device have had their tensor-core distance pass repeated so far in this process:
+ * by the split-TF32 kernels after an entry left the fp16 range, or without the common vector after the check
+ * withdrew it (a diagnostic counter, no counterpart in the paper).  Waits for the device's pending work;
+ * ~0 on a CUDA error. */
+unsigned long long detox_tc_repeated_passes(void);
+
 /* Number of kernels this library has launched in this process so far (a diagnostic counter, no counterpart in
  * the paper; the one piece of state the library keeps, besides the scratch of detox_vote_noalloc). */
 unsigned long long detox_kernel_launch_count(void);

@@ -26,7 +26,7 @@ EXPORTS = (
     "agg_coord_median_workspace_bytes", "agg_coord_median", "agg_trimmed_mean", "agg_sign_majority", "agg_geometric_median_workspace_bytes", "agg_geometric_median", "agg_multikrum_workspace_bytes", "agg_multikrum",
     "agg_bulyan_workspace_bytes", "agg_bulyan", "detox_aggregate_workspace_bytes", "detox_aggregate",
     "detox_selftest_bounded_wait", "agg_pairwise_sqdist_workspace_bytes", "agg_pairwise_sqdist",
-    "detox_kernel_launch_count", "detox_vote_hier_mean_many",
+    "detox_kernel_launch_count", "detox_vote_hier_mean_many", "detox_tc_split_mode", "detox_tc_repeated_passes",
 )
 
 
@@ -89,6 +89,10 @@ def load() -> ctypes.CDLL:
     lib.agg_pairwise_sqdist_workspace_bytes.argtypes = [_int, _i64]
     lib.agg_pairwise_sqdist.argtypes = [_vp, _i64, _int, _i64, _vp, _vp, _sz, _vp]
     lib.detox_vote_hier_mean_many.argtypes = [_vp, _i64, _i64, _int, _int, _vp, _ip, _int, _vp, _i64, _vp, _vp]
+    lib.detox_tc_split_mode.argtypes = [_int]
+    lib.detox_tc_split_mode.restype = _int
+    lib.detox_tc_repeated_passes.restype = ctypes.c_ulonglong
+    lib.detox_tc_repeated_passes.argtypes = []
     lib.detox_kernel_launch_count.restype = ctypes.c_ulonglong
     lib.detox_kernel_launch_count.argtypes = []
     _lib = lib
@@ -298,6 +302,20 @@ def agg_geometric_median(X, iters: int = 32, eps: float = 1e-12, out: Optional[t
     _check(lib.agg_geometric_median(xp, ld, m, d, iters, eps, out.data_ptr(), wp, wb, _stream(stream)),
            "agg_geometric_median")
     return out
+
+
+SPLIT_AUTO, SPLIT_TF32 = 0, 1
+
+
+def tc_split_mode(mode: int = -1) -> int:
+    """Sets which operand split the tensor-core distance pass tries first (SPLIT_AUTO: fp16 pairs, SPLIT_TF32);
+    returns the previous mode; without an argument only queries."""
+    return int(load().detox_tc_split_mode(int(mode)))
+
+
+def tc_repeated_passes() -> int:
+    """Calls on the current device whose tensor-core distance pass had to be repeated so far (synchronises)."""
+    return int(load().detox_tc_repeated_passes())
 
 
 def kernel_launch_count() -> int:

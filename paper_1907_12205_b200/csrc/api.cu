@@ -435,6 +435,10 @@ detox_status agg_pairwise_sqdist(const float* X, int64_t ld, int m, int64_t d, d
     return launch_sqdist(X, ld, m, d, nullptr, D, static_cast<char*>(ws) + kStatusBytes, status, s);
 }
 
+int detox_tc_split_mode(int mode) { return tc_split_mode(mode); }
+
+unsigned long long detox_tc_repeated_passes(void) { return tc_repeated_passes(); }
+
 unsigned long long detox_kernel_launch_count(void) { return g_kernel_launches.load(std::memory_order_relaxed); }
 
 size_t detox_aggregate_workspace_bytes(const detox_pipeline_desc* desc) {

@@ -10,20 +10,20 @@
 // rows: per column the median of seven rows at fixed, evenly spaced positions gives a first centre that a minority of
 // outlying rows cannot move; every row's squared distance to it and squared norm are added up over the sample; the
 // rows are ranked by that distance and every s-th of the closer half is listed (so that a group of colluding rows
-// that sit in the very middle cannot fill the list).  Centring is switched on only when the typical row is closer to
-// the first centre than to the origin; rows that hover around zero are left as they are.
+// that sit in the very middle cannot fill the list).  Centring is switched on only when the typical row is clearly
+// closer to the first centre than to the origin; rows that hover around zero are left as they are.
 //
 // Everything is deterministic: per-block partial sums are added in a fixed order and ties go to the lower index.
 #include <math_constants.h>
 
 #include "common.cuh"
+#include "gram_tc.cuh"
 
 namespace detox {
 
 namespace {
 
 constexpr int kPickThreads = 256;
-constexpr int kMaxCentreRows = 16;   // as in the distance kernels
 constexpr int kSampleCols = 64;      // columns per sampled block
 constexpr int kSampleBlocks = 16;
 constexpr int kFirstRows = 7;        // rows whose column-wise median is the first centre
@@ -36,8 +36,8 @@ int sample_blocks(int64_t d) {
 struct CentreWs {
     float* part;        // [nblk][2][m]: per block, every row's squared distance to the first centre, then its squared norm
     float* key;         // [m] scratch of the check after the pass
-    unsigned* counter;  // [2] unused / CTAs of the check kernel that have finished; behind them one float:
-                        // the typical squared norm of a row as the sample predicts it for all d columns
+    unsigned* counter;  // [2] "a row failed the check" / CTAs of the check kernel that have finished; behind them one
+                        // float: the typical squared norm of a centred row as the sample predicts it for all d columns
 };
 
 CentreWs centre_carve(void* ws, int m) {
@@ -109,14 +109,17 @@ centre_sample_kernel(const float* __restrict__ X, int64_t ld, int m, int64_t d, 
 }
 
 // One CTA: adds the blocks' partial sums, ranks the rows by their distance to the first centre, lists the centring
-// rows and decides whether centring pays.
+// rows, decides whether centring pays, and gives every row its power-of-two scale for the split-fp16 pass:
+// expo[r] = kTargetRmsLog2 - floor(log2(rms of row r's sampled entries after the subtraction)), so that 2^expo[r] times
+// the row has its typical entry in [2^6, 2^7).  A row whose sample is zero or not finite takes the typical row's scale.
 __global__ void __launch_bounds__(kPickThreads)
-centre_pick_kernel(const float* __restrict__ part, int nblk, int m, float scale, unsigned* __restrict__ counter,
-                   int* __restrict__ centre) {
+centre_pick_kernel(const float* __restrict__ part, int nblk, int m, float scale, float inv_sampled,
+                   unsigned* __restrict__ counter, int* __restrict__ centre, int* __restrict__ expo) {
     extern __shared__ float sh[];   // dist [m], norm [m]
     float* dist = sh;
     float* nrm = sh + m;
     __shared__ float med[2];
+    __shared__ int centring_on;
     for (int r = threadIdx.x; r < m; r += kPickThreads) {
         float a = 0.f, n = 0.f;
         for (int b = 0; b < nblk; ++b) {
@@ -145,59 +148,120 @@ centre_pick_kernel(const float* __restrict__ part, int nblk, int m, float scale,
     }
     __syncthreads();
     if (threadIdx.x == 0) {
-        // on when the typical row is closer to the first centre than to the origin
-        centre[0] = (want >= 1 && med[0] < med[1]) ? want : 0;
-        *reinterpret_cast<float*>(counter + 2) = med[1] * scale;   // for the check after the pass
+        // on when the typical row is clearly closer to the first centre than to the origin.  Rows that hover around
+        // zero have a ratio of squared distances of 0.8 .. 1.2 (the seven rows behind the first centre are a little
+        // closer to it than the others) and gain nothing; rows that share a vector as long as their individual parts
+        // have 0.6, and their sums of products, all of one sign, already lose to the tensor cores' truncation.
+        centring_on = (want >= 1 && med[0] < 0.7f * med[1]) ? 1 : 0;
+        centre[0] = centring_on ? want : 0;
+        // for the check after the pass: the typical squared norm the sample predicts for the centred rows
+        *reinterpret_cast<float*>(counter + 2) = med[0] * scale;
+    }
+    __syncthreads();
+    const float typical = (centring_on ? med[0] : med[1]) * inv_sampled;
+    for (int r = threadIdx.x; r < m; r += kPickThreads) {
+        float v = (centring_on ? dist[r] : nrm[r]) * inv_sampled;   // mean square of the sampled entries
+        if (!(v > 0.f && v < CUDART_INF_F)) v = typical;
+        int e = 0;
+        if (v > 0.f && v < CUDART_INF_F) e = kTargetRmsLog2 - (ilogbf(v) >> 1);
+        expo[r] = e < -100 ? -100 : (e > 100 ? 100 : e);
     }
 }
 
-// After the distance pass: did the subtraction leave the rows small?  The listed rows were chosen on a sample of the
-// columns; a row that is central there and holds huge values elsewhere would, once subtracted, swamp the differences
-// between the other rows.  `norms` holds, per output slot and group of transform warps, every row's exact squared
-// norm after the subtraction.  One CTA per row adds its shares up; the last one takes the median over the rows and
-// compares it with what the sample predicted for the rows as they came.  If the typical row is more than 16 times
-// larger than that, the centring is withdrawn (centre[0] = 0) and *redo = 1 asks for the pass to be repeated without it.
-constexpr float kCentreSlack = 16.f;
+// After the distance pass, two questions.
+//
+// Did the subtraction leave the rows small?  The listed rows were chosen on a sample of the columns; a row that is
+// central there and holds huge values elsewhere would, once subtracted, swamp the differences between the other rows.
+// `norms` holds, per output slot and group of transform warps, every row's exact squared norm after the subtraction
+// (and after the row's scale 2^expo, when the split-fp16 pass ran).  One CTA per row adds its shares up; the last one
+// takes the median over the rows and compares it with what the sample predicted for the centred rows.  If the
+// typical row is more than 4 times larger than that, the centring is withdrawn (centre[0] = 0): a listed row with
+// one large entry outside the sample is enough to put that entry into every row, and the distances would then be
+// small differences of large norms.
+//
+// Did the split-fp16 pass (expo != null) see every entry?  In every slot the tensor cores' own squared norm of the
+// row, the diagonal entry of the slot's partial, must be finite and within 1/256 of the exact one (an fp16 overflow
+// makes it Inf or NaN), and the scaled row as a whole must not have come out far below the range its scale aimed at
+// (its entries would have lost their low bits).  A row whose exact norm is not finite also sends the call to the other
+// pass, which sees the row unscaled.
+//
+// *redo = 1 asks for the split-TF32 pass (with the centring that is left) when either answer is no.
+constexpr float kCentreSlack = 4.f;
+__device__ unsigned long long g_repeated_passes;   // calls whose check asked for the pass to be repeated (a diagnostic)
 __global__ void __launch_bounds__(128)
-centre_check_kernel(const float* __restrict__ norms, int nshares, int m, float* __restrict__ na,
+centre_check_kernel(const float* __restrict__ norms, const float* __restrict__ partial, int nitems, int groups, int m,
+                    int ncol, float min_scaled_norm, const int* __restrict__ expo, float* __restrict__ na,
                     unsigned* __restrict__ counter, int* __restrict__ centre, int* __restrict__ redo) {
     __shared__ double red[4];
+    __shared__ int red_bad[4];
     __shared__ bool s_last;
+    __shared__ int s_keep;
     const int i = blockIdx.x;
-    if (*centre <= 0) {
+    const bool fast = expo != nullptr;
+    const int ncentre = *centre;
+    if (!fast && ncentre <= 0) {
         if (i == 0 && threadIdx.x == 0) *redo = 0;
         return;
     }
     double a = 0.0;
-    for (int s = threadIdx.x; s < nshares; s += 128) a += (double)norms[(int64_t)s * m + i];
+    int bad = 0;
+    for (int it = threadIdx.x; it < nitems; it += 128) {
+        float n = 0.f;
+        for (int g = 0; g < groups; ++g) n += norms[((int64_t)it * groups + g) * m + i];
+        a += (double)n;
+        if (fast) {
+            if (!(n < CUDART_INF_F)) {
+                bad = 1;   // Inf or NaN: an entry of the row itself, or one that its scale pushed out of fp32
+            } else if (n > 0.f) {
+                const float t = partial[((int64_t)it * m + i) * ncol + i];
+                if (!(fabsf(n - t) <= n * (1.f / 256.f))) bad = 1;
+            }
+        }
+    }
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
-    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = a;
+    for (int o = 16; o > 0; o >>= 1) {
+        a += __shfl_xor_sync(0xffffffffu, a, o);
+        bad |= __shfl_xor_sync(0xffffffffu, bad, o);
+    }
+    if ((threadIdx.x & 31) == 0) { red[threadIdx.x >> 5] = a; red_bad[threadIdx.x >> 5] = bad; }
+    if (threadIdx.x == 0) s_keep = 1;
     __syncthreads();
     if (threadIdx.x == 0) {
-        na[i] = nan_to_inf((float)(red[0] + red[1] + red[2] + red[3]));
+        float total = nan_to_inf((float)(red[0] + red[1] + red[2] + red[3]));
+        bad = red_bad[0] | red_bad[1] | red_bad[2] | red_bad[3];
+        if (fast) {
+            if (total > 0.f && total < min_scaled_norm) bad = 1;
+            total = total < CUDART_INF_F ? ldexpf(total, -2 * expo[i]) : total;   // back to the row's own units
+        }
+        na[i] = total;
+        if (bad) atomicOr(counter, 1u);
         __threadfence();
         s_last = atomicAdd(counter + 1, 1u) == (unsigned)(m - 1);
     }
     __syncthreads();
     if (!s_last) return;
     __threadfence();
-    // median by rank counting (m <= 256 on this path: two rows per thread at most)
-    const int hm = (m - 1) / 2;
-    const float ref = *reinterpret_cast<const float*>(counter + 2);
-    for (int r = threadIdx.x; r < m; r += 128) {
-        const float mine = __ldcg(na + r);
-        int rank = 0;
-        for (int k = 0; k < m; ++k) {
-            const float u = __ldcg(na + k);
-            rank += (u < mine || (u == mine && k < r)) ? 1 : 0;
+    if (ncentre > 0) {
+        // median by rank counting (m <= 256 on this path: two rows per thread at most)
+        const int hm = (m - 1) / 2;
+        const float ref = *reinterpret_cast<const float*>(counter + 2);
+        for (int r = threadIdx.x; r < m; r += 128) {
+            const float mine = __ldcg(na + r);
+            int rank = 0;
+            for (int k = 0; k < m; ++k) {
+                const float u = __ldcg(na + k);
+                rank += (u < mine || (u == mine && k < r)) ? 1 : 0;
+            }
+            if (rank == hm && !(mine <= kCentreSlack * ref)) s_keep = 0;
         }
-        if (rank == hm) {
-            const bool keep = mine <= kCentreSlack * ref;
-            *redo = keep ? 0 : 1;
-            if (!keep) *centre = 0;
-            counter[1] = 0u;
-        }
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const bool any_bad = __ldcg(counter) != 0u;
+        *redo = (!s_keep || any_bad) ? 1 : 0;
+        if (!s_keep || any_bad) atomicAdd(&g_repeated_passes, 1ull);
+        if (!s_keep) *centre = 0;
+        counter[0] = counter[1] = 0u;
     }
 }
 
@@ -208,7 +272,8 @@ size_t centre_ws_bytes(int m, int64_t d) {
     return align_up((size_t)kSampleBlocks * 2 * m * sizeof(float)) + align_up((size_t)m * sizeof(float)) + 256;   // counters, float
 }
 
-detox_status launch_pick_centre(const float* X, int64_t ld, int m, int64_t d, void* ws, int* centre, cudaStream_t s) {
+detox_status launch_pick_centre(const float* X, int64_t ld, int m, int64_t d, void* ws, int* centre, int* expo,
+                                cudaStream_t s) {
     CentreWs w = centre_carve(ws, m);
     const int nblk = sample_blocks(d);
     const size_t smem = ((size_t)m * (kSampleCols + 1) + kSampleCols) * sizeof(float);
@@ -220,17 +285,26 @@ detox_status launch_pick_centre(const float* X, int64_t ld, int m, int64_t d, vo
     // the sample's squared norms are scaled up to all d columns for the check after the pass
     const int64_t sampled = (int64_t)nblk * kSampleCols < d ? (int64_t)nblk * kSampleCols : d;
     const float scale = (float)((double)d / (double)sampled);
-    centre_pick_kernel<<<1, kPickThreads, (size_t)2 * m * sizeof(float), s>>>(w.part, nblk, m, scale, w.counter, centre);
+    centre_pick_kernel<<<1, kPickThreads, (size_t)2 * m * sizeof(float), s>>>(w.part, nblk, m, scale, 1.f / (float)sampled,
+                                                                            w.counter, centre, expo);
     return launch_status();
 }
 
-detox_status launch_check_centre(const float* norms, int nshares, int m, void* ws, int64_t d, int* centre, int* redo,
-                                 cudaStream_t s) {
-    (void)d;
+detox_status launch_check_centre(const float* norms, const float* partial, int nitems, int groups, int m, int ncol,
+                                 void* ws, int64_t d, int* centre, int* redo, const int* expo, cudaStream_t s) {
     CentreWs w = centre_carve(ws, m);
-    // the second counter word was cleared by the sample kernel
-    centre_check_kernel<<<m, 128, 0, s>>>(norms, nshares, m, w.key, w.counter, centre, redo);
+    // a scaled row aims at a typical entry of 2^6 or more; below 2^2 its scale was far off
+    const float min_scaled_norm = (float)((double)d * 16.0);
+    // both counter words were cleared by the sample kernel
+    centre_check_kernel<<<m, 128, 0, s>>>(norms, partial, nitems, groups, m, ncol, min_scaled_norm, expo, w.key, w.counter,
+                                          centre, redo);
     return launch_status();
+}
+
+unsigned long long tc_repeated_passes() {
+    unsigned long long v = 0;
+    if (cudaMemcpyFromSymbol(&v, g_repeated_passes, sizeof(v)) != cudaSuccess) return ~0ull;
+    return v;
 }
 
 }  // namespace detox

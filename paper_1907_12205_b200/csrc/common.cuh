@@ -96,6 +96,10 @@ detox_status launch_sqdist(const float* X, int64_t ld, int m, int64_t d, const i
 // gram_tc.cu: the tcgen05 path for 16 < m <= 256 (needs 16-byte aligned rows)
 bool tc_supported(const float* X, int64_t ld, int m, int64_t d);
 size_t tc_ws_bytes(int m, int64_t d);
+// which operand split the pass tries first (DETOX_SPLIT_*); returns the previous mode
+int tc_split_mode(int mode);
+// how many calls on the current device had their tensor-core pass repeated so far (synchronises the device)
+unsigned long long tc_repeated_passes();
 // 2 <= m <= 16: the direct kernels' per-CTA pair partials only (consumed by launch_krum_small).  When
 // sqdist_partials_use_status() holds the kernel clears the device status word itself and may set it to
 // DETOX_ERR_TIMEOUT, so the consumer must leave it alone.
@@ -108,14 +112,18 @@ detox_status launch_sqdist_tc(const float* X, int64_t ld, int m, int64_t d, doub
 
 // centre.cu: the centring rows for the tensor-core distance pass (m <= 256), chosen on a sample of the columns
 //   centre[0] = how many rows are averaged into the vector that is subtracted from every row (0 when the rows hover
-//   around zero anyway), centre[1] = redo flag (below), centre[2..17] = the rows
+//   around zero anyway), centre[1] = redo flag (below), centre[2..17] = the rows; expo[m] = every row's power-of-two
+//   scale for the split-fp16 pass
 size_t centre_ws_bytes(int m, int64_t d);
-detox_status launch_pick_centre(const float* X, int64_t ld, int m, int64_t d, void* ws, int* centre, cudaStream_t s);
-//   after the pass: norms = the rows' exact squared norms after the subtraction, in nshares x m shares; withdraws
-//   the centring (centre[0] = 0, *redo = 1) when the typical row came out far larger than the sample predicted for the
-//   rows as they were (*redo = 0 otherwise)
-detox_status launch_check_centre(const float* norms, int nshares, int m, void* ws, int64_t d, int* centre, int* redo,
-                                 cudaStream_t s);
+detox_status launch_pick_centre(const float* X, int64_t ld, int m, int64_t d, void* ws, int* centre, int* expo,
+                                cudaStream_t s);
+//   after the pass: norms = the rows' exact squared norms after the subtraction (nitems x groups x m), partial = the
+//   slots' sums of products (nitems x m x ncol).  Withdraws the centring (centre[0] = 0) when the typical row came out
+//   far larger than the sample predicted for the rows as they were; expo != null: the split-fp16 pass ran with these
+//   row scales, and its tensor-core norms are checked against the exact ones.  *redo = 1 when the pass has to be
+//   repeated (by the split-TF32 kernels), 0 otherwise.
+detox_status launch_check_centre(const float* norms, const float* partial, int nitems, int groups, int m, int ncol,
+                                 void* ws, int64_t d, int* centre, int* redo, const int* expo, cudaStream_t s);
 
 // geomed.cu: Weiszfeld iterations for the geometric median of m <= 32 rows
 size_t geomed_ws_bytes(int64_t d);

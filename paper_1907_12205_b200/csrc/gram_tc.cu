@@ -30,16 +30,18 @@
 // status word, stops waiting everywhere, frees its tensor memory and returns.
 #include <cuda.h>
 
+#include <atomic>
+
 #include "common.cuh"
 #include "mbarrier.cuh"
+#include "gram_tc.cuh"
+#include "tcgen05.cuh"
 
 namespace detox {
 
 namespace {
 
 constexpr int kKB = 32;                      // fp32 columns per K-block: one 128-byte swizzle row
-constexpr int kProdWarps = 16;
-constexpr int kProdThreads = kProdWarps * 32;
 constexpr int kMmaWarps = 2;                   // issuing threads of the wide kernel (the staged kernel has two or four):
                                                // one's bookkeeping overlaps the other's MMAs
 constexpr int kTmaWarps = 2;                   // copy-issuing warps of the wide kernel (it uses the first only; the second
@@ -49,10 +51,6 @@ constexpr int kTmaWarps = 2;                   // copy-issuing warps of the wide
 __host__ __device__ constexpr int staged_tma_warps(int lx) { return lx; }
 constexpr int kCentreWarps = 1;                // forms the vector that is subtracted from every row (when one is)
 constexpr int kTcThreads = kProdThreads + 32 * (kMmaWarps + kTmaWarps);   // wide kernel: its second copy warp does the centring
-constexpr int kMaxCentreRows = 16;             // the subtracted vector is the mean of at most this many rows
-constexpr size_t kSmemBudget = 227 * 1024;     // dynamic shared memory one CTA may have
-constexpr int64_t kSlabCols = 4096;          // columns accumulated in tensor memory before a drain
-constexpr int kItemSlabs = 4;                // consecutive slabs of a CTA that are added into one output slot
 constexpr int kMinReduceChunks = 32, kMaxReduceChunks = 256;
 
 // Slab slots are added up in `chunks` independent groups (one CTA per group and pair of 32-row blocks), enough
@@ -64,95 +62,6 @@ int reduce_chunks(int m, int nitems) {
     if (c > kMaxReduceChunks) c = kMaxReduceChunks;
     if (c > nitems) c = nitems;
     return c;
-}
-
-// ------------------------------------------------------------------------------------ PTX wrappers
-
-__device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-__device__ __forceinline__ void tmem_alloc(uint32_t* slot, uint32_t ncols) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(slot)), "r"(ncols)
-                 : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
-}
-
-// Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, rows packed 128 bytes apart,
-// 8-row groups 1024 bytes apart.  `addr` must lie in a 1024-byte aligned tile.
-__device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
-    uint64_t desc = (uint64_t)((addr & 0x3FFFFu) >> 4);   // start address, 16-byte units
-    desc |= (uint64_t)1 << 16;                              // leading byte offset (unused for swizzled K-major)
-    desc |= (uint64_t)(1024 >> 4) << 32;                    // stride byte offset: next 8-row group
-    desc |= (uint64_t)1 << 46;                              // descriptor version of this architecture
-    desc |= (uint64_t)2 << 61;                              // 128-byte swizzle
-    return desc;
-}
-
-// D[tmem] (+)= A[smem] * B[smem]^T, TF32 inputs, fp32 accumulate; M and N come with the instruction descriptor.
-__device__ __forceinline__ void mma_tf32(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
-// Arrive on `bar` once every MMA issued so far by this thread has finished.
-__device__ __forceinline__ void mma_commit(uint64_t* bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
-                 : "memory");
-}
-
-__device__ __forceinline__ void tmem_load16(uint32_t taddr, uint32_t (&v)[16]) {
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
-          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
-        : "r"(taddr)
-        : "memory");
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-}
-
-// 2-D tiled TMA load (no multicast): box at (x = column, y = row) -> shared memory, completion on `bar`.
-__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-        ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(smem_u32(bar))
-        : "memory");
-}
-
-// Packed pairs of fp32 (one instruction for two lanes).
-__device__ __forceinline__ uint64_t sub2(uint64_t a, uint64_t b) {
-    uint64_t r;
-    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
-    return r;
-}
-__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
-    uint64_t r;
-    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
-    return r;
-}
-__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
-    uint64_t r;
-    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
-    return r;
-}
-// What a TF32 MMA sees of x is hi = x with the low 13 mantissa bits cleared; x - hi is exact in fp32
-// and so is its double.  (The MMA again reads only the upper 19 bits of 2 lo.)
-__device__ __forceinline__ uint64_t lo2_of(uint64_t x2) {
-    const uint64_t t = sub2(x2, x2 & 0xFFFFE000FFFFE000ull);
-    return add2(t, t);
-}
-
-// An Inf / NaN replaced by zero (the subtracted vector must not spread a listed row's non-finite entries to the
-// other rows: at such a coordinate nothing is subtracted).
-__device__ __forceinline__ float finite_or_zero(float v) {
-    return (__float_as_uint(v) & 0x7f800000u) != 0x7f800000u ? v : 0.f;
 }
 
 // ------------------------------------------------------------------------------------ 128 < m <= 256: wide kernel
@@ -857,10 +766,16 @@ gram_staged_kernel(const __grid_constant__ CUtensorMap xmap, int m, uint32_t stg
 // mirrored tile T[bj][bi] row by row (coalesced) and transposes the second through shared memory.
 constexpr int kRT = 32;
 __global__ void __launch_bounds__(kRT * 8)
-tc_reduce_kernel(const float* __restrict__ partial, const float* __restrict__ norms, int ngroups, int nitems, int m,
+tc_reduce_kernel(const float* __restrict__ partial, const float* __restrict__ norms, int ngroups, int nitems,
+                 int ngroups_redo, int nitems_redo, const int* __restrict__ expo, const int* __restrict__ redo, int m,
                  int ncol, double* __restrict__ dpart) {
     __shared__ float mirror[kRT][kRT + 1];
     __shared__ double ratio_i[kRT], ratio_j[kRT], diag_i[kRT], diag_j[kRT];
+    __shared__ int expo_i[kRT], expo_j[kRT];
+    // The slots hold the split-fp16 pass's sums (rows scaled by 2^expo) unless that pass was repeated by the
+    // split-TF32 kernels (*redo != 0), whose rows are unscaled and whose slot count may differ.
+    const bool scaled = expo != nullptr && *redo == 0;
+    if (expo != nullptr && !scaled) { ngroups = ngroups_redo; nitems = nitems_redo; }
     const int nt = (m + kRT - 1) / kRT;
     int bi = 0, rem = blockIdx.x;
     while (rem >= nt - bi) { rem -= nt - bi; ++bi; }
@@ -875,6 +790,10 @@ tc_reduce_kernel(const float* __restrict__ partial, const float* __restrict__ no
 #pragma unroll
     for (int k = 0; k < kRT / 8; ++k) acc[k] = 0.0;
     const int j = bj * kRT + tx;             // this thread's column of the tile
+    if (ty < 2) {
+        const int r = (ty == 0 ? bi : bj) * kRT + tx;
+        (ty == 0 ? expo_i : expo_j)[tx] = (scaled && r < m) ? expo[r] : 0;
+    }
 
     for (int s = s0; s < s1; ++s) {
         const float* T = partial + (int64_t)s * elems;
@@ -906,8 +825,10 @@ tc_reduce_kernel(const float* __restrict__ partial, const float* __restrict__ no
             const int il = ty + 8 * k;
             const double tij = 0.5 * ((double)a[k] + (double)mirror[tx][il]);
             const double ri = ratio_i[il], rj = ratio_j[tx];
-            const double norms_ij = __dadd_rn(__dmul_rn(ri, diag_i[il]), __dmul_rn(rj, diag_j[tx]));
-            acc[k] += __dadd_rn(norms_ij, -__dmul_rn(__dadd_rn(ri, rj), tij));
+            // (the rows' power-of-two scales come off exactly; for equal rows they are equal)
+            const int ei = expo_i[il], ej = expo_j[tx];
+            const double norms_ij = __dadd_rn(scalbn(__dmul_rn(ri, diag_i[il]), -2 * ei), scalbn(__dmul_rn(rj, diag_j[tx]), -2 * ej));
+            acc[k] += __dadd_rn(norms_ij, -scalbn(__dmul_rn(__dadd_rn(ri, rj), tij), -ei - ej));
         }
         __syncthreads();
     }
@@ -964,31 +885,24 @@ EncodeTiledFn encode_tiled_fn() {
     return fn;
 }
 
-// X as a 2-D fp32 tensor (d columns innermost, m rows, row pitch ld); box = 32 columns x box_rows rows,
-// 128-byte swizzle, zero fill outside.
-detox_status make_xmap(CUtensorMap* map, const float* X, int64_t ld, int m, int64_t d, int box_cols, int box_rows,
-                       CUtensorMapSwizzle swizzle) {
+}  // namespace
+
+// X as a 2-D fp32 tensor (d columns innermost, m rows, row pitch ld), zero fill outside the matrix.
+detox_status make_xmap(void* map, const float* X, int64_t ld, int m, int64_t d, int box_cols, int box_rows, bool swizzle128) {
     EncodeTiledFn enc = encode_tiled_fn();
     if (!enc) return DETOX_ERR_CUDA;
     const cuuint64_t gdim[2] = {(cuuint64_t)d, (cuuint64_t)m};
     const cuuint64_t gstride[1] = {(cuuint64_t)ld * sizeof(float)};
     const cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows};
     const cuuint32_t estride[2] = {1, 1};
-    CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(X), gdim, gstride, box, estride,
-                     CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+    CUresult r = enc(static_cast<CUtensorMap*>(map), CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(X), gdim, gstride,
+                     box, estride, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                     swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? DETOX_OK : DETOX_ERR_CUDA;
 }
 
-// What a launch of either kernel is given besides its plan.  redo: null for the first launch of a call; for the second
-// the flag the check of the first one's centring has set (the kernel returns at once when it reads 0).
-struct TcBuffers {
-    float* partial;
-    float* norms;
-    const int* centre;
-    const int* redo;
-    int* status;
-};
+namespace {
 
 template <int J>
 detox_status launch_wide(const WidePlan& p, const CUtensorMap& xmap, int m, const TcBuffers& b, cudaStream_t s) {
@@ -1014,10 +928,17 @@ detox_status launch_staged(const StagedPlan& p, const CUtensorMap& xmap, int m, 
     return launch_status();
 }
 
-// What the two kernels' outputs look like to the reduction: slab slots, shares of the norms per slot, row pitch.
+// What the kernels' outputs look like to the reduction: slab slots, shares of the norms per slot, row pitch -- of
+// the split-TF32 kernel that fits m, and of the split-fp16 kernel.
 struct TcShape {
     bool staged;
     int nitems, groups, ncol;
+    int nitems_f16, groups_f16;
+    int max_items() const { return nitems > nitems_f16 ? nitems : nitems_f16; }
+    int max_shares() const {
+        const int a = nitems * groups, b = nitems_f16 * groups_f16;
+        return a > b ? a : b;
+    }
 };
 TcShape tc_shape(int m, int64_t d) {
     TcShape o;
@@ -1029,8 +950,12 @@ TcShape tc_shape(int m, int64_t d) {
         const WidePlan p = wide_plan(m, d);
         o.nitems = p.nitems, o.groups = 1, o.ncol = p.ncol;
     }
+    o.nitems_f16 = f16_nitems(m, d);
+    o.groups_f16 = f16_groups(m);
     return o;
 }
+
+std::atomic<int> g_split_mode{DETOX_SPLIT_AUTO};
 
 }  // namespace
 
@@ -1039,13 +964,19 @@ bool tc_supported(const float* X, int64_t ld, int m, int64_t d) {
     return m > 16 && m <= 256 && aligned16(X) && ld % 4 == 0 && d < (int64_t)1 << 31 && encode_tiled_fn() != nullptr;
 }
 
-// workspace: slab partials | norms | per-chunk distance sums | centring rows, redo flag |
+int tc_split_mode(int mode) {
+    if (mode != DETOX_SPLIT_AUTO && mode != DETOX_SPLIT_TF32) return g_split_mode.load();
+    return g_split_mode.exchange(mode);
+}
+
+// workspace: slab partials | norms | per-chunk distance sums | centring rows, redo flag | row scales |
 // scratch of the centre choice
 struct TcWs {
     float* partial;
     float* norms;
     double* dpart;
     int* centre;     // [0] how many rows are averaged into the subtracted vector (0: none), [1] the redo flag, [2..] the rows
+    int* expo;       // [m] power-of-two scale of every row for the split-fp16 pass
     void* pick;
     size_t total;
 };
@@ -1055,13 +986,15 @@ TcWs tc_carve(void* ws, int m, int64_t d, const TcShape& o) {
     size_t off = 0;
     const size_t elems = (size_t)m * o.ncol;
     w.partial = reinterpret_cast<float*>(p + off);
-    off += align_up((size_t)o.nitems * elems * sizeof(float));
+    off += align_up((size_t)o.max_items() * elems * sizeof(float));
     w.norms = reinterpret_cast<float*>(p + off);
-    off += align_up((size_t)o.nitems * o.groups * m * sizeof(float));
+    off += align_up((size_t)o.max_shares() * m * sizeof(float));
     w.dpart = reinterpret_cast<double*>(p + off);
-    off += align_up((size_t)reduce_chunks(m, o.nitems) * m * m * sizeof(double));
+    off += align_up((size_t)reduce_chunks(m, o.max_items()) * m * m * sizeof(double));
     w.centre = reinterpret_cast<int*>(p + off);
     off += 256;
+    w.expo = reinterpret_cast<int*>(p + off);
+    off += align_up((size_t)m * sizeof(int));
     w.pick = p + off;
     off += centre_ws_bytes(m, d);
     w.total = off;
@@ -1079,7 +1012,7 @@ detox_status launch_tc_gram(const float* X, int64_t ld, int m, int64_t d, const 
     detox_status st;
     if (o.staged) {
         const StagedPlan p = staged_plan(m, d);
-        if ((st = make_xmap(&xmap, X, ld, m, d, kStageCols, p.box_rows, CU_TENSOR_MAP_SWIZZLE_NONE)) != DETOX_OK) return st;
+        if ((st = make_xmap(&xmap, X, ld, m, d, kStageCols, p.box_rows, false)) != DETOX_OK) return st;
         // 16-byte pieces per transform thread and stage: m * 16 / (threads of a group), rounded up
         const int gt = kProdThreads / p.groups;
         const int per_thread = (m * (kStageCols / 4) + gt - 1) / gt;
@@ -1093,7 +1026,7 @@ detox_status launch_tc_gram(const float* X, int64_t ld, int m, int64_t d, const 
         return launch_staged<4, 1, 2>(p, xmap, m, b, s);
     }
     const WidePlan p = wide_plan(m, d);
-    if ((st = make_xmap(&xmap, X, ld, m, d, kKB, p.box_rows, CU_TENSOR_MAP_SWIZZLE_128B)) != DETOX_OK) return st;
+    if ((st = make_xmap(&xmap, X, ld, m, d, kKB, p.box_rows, true)) != DETOX_OK) return st;
     // 16-byte pieces per transform thread and K-block: m * 8 / 512, rounded up
     if (m * 8 <= 3 * kProdThreads) return launch_wide<3>(p, xmap, m, b, s);
     return launch_wide<4>(p, xmap, m, b, s);
@@ -1101,26 +1034,34 @@ detox_status launch_tc_gram(const float* X, int64_t ld, int m, int64_t d, const 
 
 }  // namespace
 
-// Sequence: choose the centring rows on a column sample (or none) -> streaming pass -> check that the centred rows
-// really got smaller, else withdraw the centring -> the streaming pass again, which returns at once unless the
-// centring was withdrawn -> reduction of the slab partials to distances.
+// Sequence: choose the centring rows and the rows' scales on a column sample -> the split-fp16 pass -> check that the
+// centred rows really got smaller and that no entry left the fp16 range -> the split-TF32 pass, which returns at once
+// unless the check asked for it -> reduction of the slab partials to distances.  (DETOX_SPLIT_TF32: the split-TF32
+// pass runs first and the check only looks at the centring, as it did before there was an fp16 pass.)
 detox_status launch_sqdist_tc(const float* X, int64_t ld, int m, int64_t d, double* D, void* ws, int* status,
                               cudaStream_t s) {
     const TcShape o = tc_shape(m, d);
     const TcWs w = tc_carve(ws, m, d, o);
+    const bool fast = g_split_mode.load() == DETOX_SPLIT_AUTO;
     detox_status st;
-    if ((st = launch_pick_centre(X, ld, m, d, w.pick, w.centre, s)) != DETOX_OK) return st;
+    if ((st = launch_pick_centre(X, ld, m, d, w.pick, w.centre, w.expo, s)) != DETOX_OK) return st;
     TcBuffers b{w.partial, w.norms, w.centre, nullptr, status};
-    if ((st = launch_tc_gram(X, ld, m, d, o, b, s)) != DETOX_OK) return st;
-    if ((st = launch_check_centre(w.norms, o.nitems * o.groups, m, w.pick, d, w.centre, w.centre + 1, s)) !=
-        DETOX_OK)
-        return st;
+    if (fast) {
+        if ((st = launch_gram_f16(X, ld, m, d, b, w.expo, s)) != DETOX_OK) return st;
+        st = launch_check_centre(w.norms, w.partial, o.nitems_f16, o.groups_f16, m, o.ncol, w.pick, d, w.centre, w.centre + 1,
+                                 w.expo, s);
+    } else {
+        if ((st = launch_tc_gram(X, ld, m, d, o, b, s)) != DETOX_OK) return st;
+        st = launch_check_centre(w.norms, w.partial, o.nitems, o.groups, m, o.ncol, w.pick, d, w.centre, w.centre + 1, nullptr, s);
+    }
+    if (st != DETOX_OK) return st;
     b.redo = w.centre + 1;
     if ((st = launch_tc_gram(X, ld, m, d, o, b, s)) != DETOX_OK) return st;
     const int nt = (m + kRT - 1) / kRT;
-    const int nchunks = reduce_chunks(m, o.nitems);
-    tc_reduce_kernel<<<dim3((unsigned)(nt * (nt + 1) / 2), (unsigned)nchunks), kRT * 8, 0, s>>>(w.partial, w.norms, o.groups,
-                                                                                           o.nitems, m, o.ncol, w.dpart);
+    const int nchunks = reduce_chunks(m, o.max_items());
+    tc_reduce_kernel<<<dim3((unsigned)(nt * (nt + 1) / 2), (unsigned)nchunks), kRT * 8, 0, s>>>(
+        w.partial, w.norms, fast ? o.groups_f16 : o.groups, fast ? o.nitems_f16 : o.nitems, o.groups, o.nitems,
+        fast ? w.expo : nullptr, w.centre + 1, m, o.ncol, w.dpart);
     if ((st = launch_status()) != DETOX_OK) return st;
     tc_dist_kernel<<<(unsigned)ceil_div((int64_t)m * m * 32, 256), 256, 0, s>>>(w.dpart, nchunks, m, status, D);
     return launch_status();

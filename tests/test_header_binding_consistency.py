@@ -22,6 +22,11 @@ def test_aggregator_codes_match():
                      "DETOX_AGG_SIGN_MAJORITY": dx.AGG_SIGN_MAJORITY}
 
 
+def test_split_modes_match():
+    modes = {name: int(val) for name, val in re.findall(r"\b(DETOX_SPLIT_[A-Z0-9_]+)\s*=\s*(\d+)", HEADER)}
+    assert modes == {"DETOX_SPLIT_AUTO": dx.SPLIT_AUTO, "DETOX_SPLIT_TF32": dx.SPLIT_TF32}
+
+
 def test_limits_and_status_codes_match():
     defs = {k: int(v) for k, v in re.findall(r"#define\s+(DETOX_[A-Z_]+)\s+(\d+)", HEADER)}
     assert defs["DETOX_MAX_ROWS"] == binding.MAX_ROWS and defs["DETOX_MAX_R"] == binding.MAX_R

@@ -14,6 +14,15 @@ pytestmark = pytest.mark.gpu
 TOL = 1e-5
 
 
+@pytest.fixture(params=["auto", "tf32"])
+def split(request):
+    """Runs a test once with the default operand split of the tensor-core distance pass (fp16 pairs first) and once
+    with the split-TF32 kernels from the start."""
+    prev = dx.tc_split_mode(dx.SPLIT_TF32 if request.param == "tf32" else dx.SPLIT_AUTO)
+    yield request.param
+    dx.tc_split_mode(prev)
+
+
 @pytest.mark.parametrize("r,G,d", [(3, 341, 257), (15, 68, 130), (1, 1024, 33), (5, 204, 64)])
 def test_vote_largest_group_counts(r, G, d):
     rng = np.random.default_rng(G)
@@ -69,7 +78,7 @@ def test_multikrum_fallback_paths(m, d, f, m_sel, odd):
     (17, 63), (18, 64), (32, 65), (33, 4097), (63, 9473), (64, 129), (65, 4100), (80, 9472 + 31), (96, 2000),
     (127, 3001), (128, 1000), (129, 1000), (144, 2049), (240, 777), (256, 640),
     (20, 2_500_001), (100, 2_450_003), (140, 2_430_000)])   # last three: more than one output slot (4 x 4096 columns) per CTA
-def test_tensor_core_distance_kernels_at_their_size_boundaries(m, d):
+def test_tensor_core_distance_kernels_at_their_size_boundaries(m, d, split):
     """Row counts on both sides of every switch of the tensor-core kernels (64 and 128 rows, tile sizes that are
     multiples of 16) and column counts around the 32- and 64-column copies, with a ragged tail."""
     f = max((m - 3) // 4, 0)
@@ -204,7 +213,7 @@ def test_bulk_copy_distance_kernel_for_every_row_count(M):
 
 
 @pytest.mark.parametrize("m,d", [(9, 5001), (20, 5001), (140, 3000), (9, 700_001)])
-def test_a_row_with_an_infinite_entry_is_never_selected(m, d):
+def test_a_row_with_an_infinite_entry_is_never_selected(m, d, split):
     """A Byzantine row may hold anything.  One +Inf makes the row infinitely far from every other row on both
     sides (direct differences give Inf; the Gram path's NaN counts as Inf), so Multi-Krum and Bulyan leave it out
     and the selections match the oracle."""
@@ -238,7 +247,7 @@ def correlated_rows(m, d, ratio, seed, copies=1, outliers=0):
 
 @pytest.mark.parametrize("ratio", [1, 10, 100])
 @pytest.mark.parametrize("m", [45, 105, 225])
-def test_tensor_core_distances_on_rows_that_share_a_large_common_vector(m, ratio):
+def test_tensor_core_distances_on_rows_that_share_a_large_common_vector(m, ratio, split):
     d = 150_003
     f = m // 10
     for attempt in range(8):
@@ -260,7 +269,7 @@ def test_tensor_core_distances_on_rows_that_share_a_large_common_vector(m, ratio
 
 
 @pytest.mark.parametrize("m", [45, 140])
-def test_a_centring_row_that_is_only_central_where_it_is_sampled_is_withdrawn(m):
+def test_a_centring_row_that_is_only_central_where_it_is_sampled_is_withdrawn(m, split):
     """The row subtracted from all rows is chosen on 32 evenly spaced blocks of 64 columns.  A Byzantine row that sits
     in the middle of the others there and holds huge values everywhere else would, once subtracted, wipe out the
     differences between the honest rows.  The library checks the exact norms after the pass and repeats it without
