@@ -301,14 +301,22 @@ def median_alu_roofline(m, d, ms, peaks):
             "traffic": None}
 
 
-def gram_roofline(m, d, ms, peaks, peak_kind):
-    """Roofline of the distance pass of Multi-Krum / Bulyan over m rows, timed through agg_pairwise_sqdist (the
-    streaming kernel plus two small reduction kernels).
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the tensor-core distance kernel over the algorithmic
+# bytes m d 4, from ncu captures at d = 2.5 M (the kernel reads every row once, so its traffic grows with m d); reset an
+# entry to None when the kernel changes.
+NCU_GRAM_TRAFFIC_RATIO = {45: None, 105: None, 225: None}
 
-    17 to 256 aligned rows run on the tensor cores: `achieved` is the 3xTF32-equivalent rate 2 m^2 d / t (the
-    flops of the Gram matrix the split products stand for); `issued` is what the tensor pipe was given, counting
-    the padding to the MMA shape (rows to 64 / 128 / 256, columns to twice m rounded up to 16, for the hi and the
-    2 lo operand); `frac` = issued / TF32 peak, the tensor-pipe utilisation; the HBM fraction is beside it."""
+
+def gram_roofline(m, d, ms, peaks, peak_kind, ms_tf32=None):
+    """Roofline of the distance pass of Multi-Krum / Bulyan over m rows, timed through agg_pairwise_sqdist (the
+    streaming kernel plus the small kernels around it: sample, check, reduction).
+
+    17 to 256 aligned rows run on the tensor cores with every entry split into an fp16 pair.  The pass reads every
+    row once, so `hbm` is m d 4 / t.  `tensor.issued` is what the tensor pipe was given -- two fp16 products (hi.hi
+    and hi.lo), padded to the MMA shape (rows to 64 / 128 / 256, columns to m rounded up to 16) -- against the fp16
+    dense peak (= the measured bf16 one); `tensor.useful` = 2 m^2 d / t, the flops of the Gram matrix the split
+    products stand for, also as a multiple of what three-product TF32 could reach at most (TF32 peak / 3).  The bound
+    named is the one with the larger fraction.  ms_tf32: the same call with the split-TF32 kernels, for comparison."""
     hbm = m * d * 4 / (ms * 1e-3) / 1e9
     if m <= 16:
         return {"kernel": "sqdist_staged_kernel / sqdist_direct_kernel", "bound": "hbm", "achieved": round(hbm, 1),
@@ -319,13 +327,44 @@ def gram_roofline(m, d, ms, peaks, peak_kind):
     mrows = 64 if m <= 64 else (128 if m <= 128 else 256)
     useful = 2.0 * m * m * d / (ms * 1e-3) / 1e12
     issued = 2.0 * mrows * (2 * ncol) * d / (ms * 1e-3) / 1e12
-    peak = peaks["bf16_tflops"] * TF32_OVER_BF16
-    return {"kernel": "gram_staged_kernel" if m <= 128 else "gram_wide_kernel", "bound": "tensor",
-            "achieved": round(useful, 1), "issued": round(issued, 1), "peak": round(peak, 1),
-            "peak_kind": f"{peak_kind} bf16 burst peak x nominal TF32/bf16 ratio {TF32_OVER_BF16:.3f}",
-            "unit": "TFLOP/s", "frac": round(issued / peak, 3), "useful_frac": round(useful / peak, 3),
-            "hbm_GBps": round(hbm, 1), "hbm_frac": round(hbm / peaks["hbm_gbs"], 3), "ms_per_launch": ms,
-            "algorithmic_flops": 2.0 * m * m * d, "traffic": None}
+    peak_f16 = peaks["bf16_tflops"]
+    peak_3xtf32 = peaks["bf16_tflops"] * TF32_OVER_BF16 / 3.0
+    hbm_frac, tensor_frac = hbm / peaks["hbm_gbs"], issued / peak_f16
+    ratio = NCU_GRAM_TRAFFIC_RATIO.get(m)
+    out = {"kernel": "gram_f16_kernel", "bound": "hbm" if hbm_frac >= tensor_frac else "tensor",
+           "achieved": round(hbm, 1) if hbm_frac >= tensor_frac else round(issued, 1),
+           "peak": peaks["hbm_gbs"] if hbm_frac >= tensor_frac else round(peak_f16, 1),
+           "unit": "GB/s" if hbm_frac >= tensor_frac else "TFLOP/s", "peak_kind": f"of {peak_kind}",
+           "frac": round(max(hbm_frac, tensor_frac), 3),
+           "hbm": {"GBps": round(hbm, 1), "frac": round(hbm_frac, 3)},
+           "tensor": {"issued": round(issued, 1), "peak": round(peak_f16, 1), "frac": round(tensor_frac, 3),
+                      "peak_kind": f"{peak_kind} bf16 burst peak (fp16 runs at the same rate)",
+                      "useful": round(useful, 1), "peak_3xTF32": round(peak_3xtf32, 1),
+                      "useful_over_peak_3xTF32": round(useful / peak_3xtf32, 3), "unit": "TFLOP/s"},
+           "ms_per_launch": ms, "algorithmic_bytes": m * d * 4, "algorithmic_flops": 2.0 * m * m * d,
+           "traffic": None if ratio is None else int(ratio * m * d * 4)}
+    if ms_tf32 is not None:
+        issued32 = 2.0 * mrows * (2 * ncol) * d / (ms_tf32 * 1e-3) / 1e12
+        peak32 = peaks["bf16_tflops"] * TF32_OVER_BF16
+        out["split_tf32"] = {"kernel": "gram_staged_kernel" if m <= 128 else "gram_wide_kernel", "ms_per_launch": ms_tf32,
+                             "hbm_frac": round(m * d * 4 / (ms_tf32 * 1e-3) / 1e9 / peaks["hbm_gbs"], 3),
+                             "issued": round(issued32, 1), "peak": round(peak32, 1),
+                             "peak_kind": f"{peak_kind} bf16 burst peak x nominal TF32/bf16 ratio {TF32_OVER_BF16:.3f}",
+                             "frac": round(issued32 / peak32, 3)}
+    return out
+
+
+def time_distance_pass(torch, dx, X, D, ws, reps):
+    """agg_pairwise_sqdist with the default operand split and, for the tensor-core sizes, with the split-TF32 kernels."""
+    ms = time_calls(torch, lambda: dx.agg_pairwise_sqdist(X, D=D, ws=ws), reps, 3)
+    ms32 = None
+    if 16 < X.shape[0] <= 256:
+        prev = dx.tc_split_mode(dx.SPLIT_TF32)
+        try:
+            ms32 = time_calls(torch, lambda: dx.agg_pairwise_sqdist(X, D=D, ws=ws), reps, 3)
+        finally:
+            dx.tc_split_mode(prev)
+    return ms, ms32
 
 
 def run_sweep(args):
@@ -387,8 +426,8 @@ def run_sweep(args):
                 timed(name, lambda: dx.agg_multikrum(X, leg["f"], leg["m_sel"], out=out, sel=sel[: leg["m_sel"]],
                                                      scores=sc, ws=ws), (n + leg["m_sel"] + 1) * d * 4)
                 D = torch.empty((n, n), dtype=torch.float64, device=dev)
-                gms = time_calls(torch, lambda: dx.agg_pairwise_sqdist(X, D=D, ws=ws), reps, 3)
-                legs[name]["distance_pass"] = gram_roofline(n, d, gms, peaks, peak_kind)
+                gms, gms32 = time_distance_pass(torch, dx, X, D, ws, reps)
+                legs[name]["distance_pass"] = gram_roofline(n, d, gms, peaks, peak_kind, gms32)
             else:
                 timed(name, lambda: dx.agg_bulyan(X, leg["f"], out=out, sel=sel[: n - 2 * leg["f"]], ws=ws),
                       (n + (n - 2 * leg["f"]) + 1) * d * 4)
@@ -606,8 +645,8 @@ def main():
                 fn = lambda: dx.agg_bulyan(X, direct_args["f"], out=out, sel=dsel, ws=dws)
             dms = time_calls(torch, fn, reps, 3)
             D = torch.empty((spec.n, spec.n), dtype=torch.float64, device=dev)
-            gms = time_calls(torch, lambda: dx.agg_pairwise_sqdist(X, D=D, ws=dws), reps, 3)
-            leg["roofline"] = gram_roofline(spec.n, spec.d, gms, peaks, peak_kind)
+            gms, gms32 = time_distance_pass(torch, dx, X, D, dws, reps)
+            leg["roofline"] = gram_roofline(spec.n, spec.d, gms, peaks, peak_kind, gms32)
             del dws
         else:
             dms = time_calls(torch, lambda: dx.agg_coord_median(X, out=out), reps, 3)

@@ -33,10 +33,21 @@ namespace {
 
 constexpr int kStageCols = 64;                                  // fp32 columns per stage = one 128-byte row of fp16
 constexpr int kStagesPerSlab = (int)(kSlabCols / kStageCols);
-constexpr int kMaxStg = 12, kMaxMst = 4;
+constexpr int kMaxStg = 12, kMaxMst = 8;
 constexpr size_t kMaxInFlight = 112 * 1024;   // staging bytes beyond which HBM is no faster (a deeper ring measured no gain)
 constexpr size_t kSmemTail = 4096;   // barriers and the centring ring behind the tiles
 constexpr int kCentreWarps = 1;
+
+}  // namespace
+
+// Groups of transform warps, each on stages of its own.  A group starts its next stage only when it is through with
+// the chain  wait - read - convert - write - fence - arrive  of the current one, which takes several hundred cycles
+// whatever the row count; with few rows that chain, not HBM, sets the pace, so the fewer the rows, the more groups
+// share the warps (a thread handles at most four 16-byte pieces of a stage; with five the registers spill and
+// 33 .. 40 rows ran slower in four groups than in two).
+int f16_groups(int m) { return m <= 32 ? 4 : (m <= 64 ? 2 : 1); }
+
+namespace {
 
 struct F16Plan {
     bool wide;                   // more than 128 rows: two boxes per stage, two accumulator halves
@@ -61,19 +72,19 @@ F16Plan f16_plan(int m, int64_t d) {
     p.ncol = (m + 15) / 16 * 16;
     p.mrows = m <= 64 ? 64 : 128;
     p.nmma = m <= 64 ? 4 : 2;
-    p.groups = m <= 64 ? 2 : 1;
+    p.groups = f16_groups(m);
     p.lo_row = p.wide ? 256 : p.ncol;
     p.tile_bytes = (uint32_t)(p.lo_row + p.ncol) * 128u;
     p.stg_bytes = (uint32_t)p.box_rows * (uint32_t)kStageCols * 4u;
     p.tmem_cols = 32;
     while (p.tmem_cols < (p.wide ? 2 * p.ncol : p.nmma * 2 * p.ncol)) p.tmem_cols <<= 1;
-    p.nmst = m <= 64 ? 4 : 2;
+    p.nmst = 2 * p.groups;   // two MMA slots per transform group
     const size_t left = kSmemBudget - kSmemTail - 1024 - (size_t)p.nmst * p.tile_bytes;
     p.nstg = (int)(left / p.stg_bytes);
     if (p.nstg > kMaxStg) p.nstg = kMaxStg;
     while (p.nstg > 2 && (size_t)p.nstg * p.stg_bytes > kMaxInFlight) --p.nstg;
-    // two transform groups: a staging slot always holds stages of the same group (see the split-TF32 staged kernel)
-    if (p.groups == 2) p.nstg &= ~1;
+    // several transform groups: a staging slot always holds stages of the same group (see the split-TF32 staged kernel)
+    p.nstg -= p.nstg % p.groups;
     p.nst_total = (int)ceil_div(d, (int64_t)kStageCols);
     p.grid = p.nst_total < kSMs ? p.nst_total : kSMs;
     const int per_cta = (p.nst_total + p.grid - 1) / p.grid;
@@ -299,13 +310,10 @@ gram_f16_kernel(const __grid_constant__ CUtensorMap xmap, int m, int box_rows, u
                             float* dstp = out_item + (int64_t)row * ncol + cc * 16;
 #pragma unroll
                             for (int j = 0; j < 16; j += 4) {
-                                float4 o = make_float4(__uint_as_float(v[j]), __uint_as_float(v[j + 1]),
-                                                       __uint_as_float(v[j + 2]), __uint_as_float(v[j + 3]));
-                                if (!opens) {   // this thread wrote the slot's earlier slabs itself
-                                    const float4 e = *reinterpret_cast<const float4*>(dstp + j);
-                                    o.x += e.x; o.y += e.y; o.z += e.z; o.w += e.w;
-                                }
-                                *reinterpret_cast<float4*>(dstp + j) = o;
+                                const float4 o = make_float4(__uint_as_float(v[j]), __uint_as_float(v[j + 1]), __uint_as_float(v[j + 2]),
+                                                             __uint_as_float(v[j + 3]));
+                                if (opens) *reinterpret_cast<float4*>(dstp + j) = o;
+                                else red_add_f4(dstp + j, o);   // this thread wrote the slot's earlier slabs itself
                             }
                         }
                     }
@@ -331,12 +339,9 @@ gram_f16_kernel(const __grid_constant__ CUtensorMap xmap, int m, int box_rows, u
                         float* dstp = out_item + (int64_t)row * ncol + cc * 16;
 #pragma unroll
                         for (int j = 0; j < 16; j += 4) {
-                            float4 o = make_float4(acc[j], acc[j + 1], acc[j + 2], acc[j + 3]);
-                            if (!opens) {
-                                const float4 e = *reinterpret_cast<const float4*>(dstp + j);
-                                o.x += e.x; o.y += e.y; o.z += e.z; o.w += e.w;
-                            }
-                            *reinterpret_cast<float4*>(dstp + j) = o;
+                            const float4 o = make_float4(acc[j], acc[j + 1], acc[j + 2], acc[j + 3]);
+                            if (opens) *reinterpret_cast<float4*>(dstp + j) = o;
+                            else red_add_f4(dstp + j, o);   // this thread wrote the slot's earlier slabs itself
                         }
                     }
                 }
@@ -512,7 +517,6 @@ detox_status launch_f16(const F16Plan& p, const CUtensorMap& xmap, int m, const 
 }  // namespace
 
 int f16_nitems(int m, int64_t d) { return f16_plan(m, d).nitems; }
-int f16_groups(int m) { return m <= 64 ? 2 : 1; }
 
 detox_status launch_gram_f16(const float* X, int64_t ld, int m, int64_t d, const TcBuffers& b, const int* expo,
                              cudaStream_t s) {
@@ -527,8 +531,11 @@ detox_status launch_gram_f16(const float* X, int64_t ld, int m, int64_t d, const
         if (per_thread <= 3) return launch_f16<3, 1, 2, true>(p, xmap, m, b, expo, s);
         return launch_f16<4, 1, 2, true>(p, xmap, m, b, expo, s);
     }
+    if (p.groups == 4) {   // up to 32 rows: four transform groups, four MMA-issuing threads
+        if (per_thread <= 3) return launch_f16<3, 4, 4, false>(p, xmap, m, b, expo, s);
+        return launch_f16<4, 4, 4, false>(p, xmap, m, b, expo, s);
+    }
     if (p.groups == 2) {   // up to 64 rows: two transform groups, four MMA-issuing threads
-        if (per_thread <= 2) return launch_f16<2, 2, 4, false>(p, xmap, m, b, expo, s);
         if (per_thread <= 3) return launch_f16<3, 2, 4, false>(p, xmap, m, b, expo, s);
         return launch_f16<4, 2, 4, false>(p, xmap, m, b, expo, s);
     }

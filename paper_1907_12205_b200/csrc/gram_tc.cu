@@ -252,13 +252,10 @@ gram_wide_kernel(const __grid_constant__ CUtensorMap xmap, int m, uint32_t lo_of
                         float* dstp = out_item + (int64_t)row * ncol + cc * 16;
 #pragma unroll
                         for (int j = 0; j < 16; j += 4) {
-                            float4 o = make_float4(__uint_as_float(v[j]), __uint_as_float(v[j + 1]), __uint_as_float(v[j + 2]),
-                                                   __uint_as_float(v[j + 3]));
-                            if (!opens) {   // this thread wrote the slot's earlier slabs itself
-                                const float4 e = *reinterpret_cast<const float4*>(dstp + j);
-                                o.x += e.x; o.y += e.y; o.z += e.z; o.w += e.w;
-                            }
-                            *reinterpret_cast<float4*>(dstp + j) = o;
+                            const float4 o = make_float4(__uint_as_float(v[j]), __uint_as_float(v[j + 1]), __uint_as_float(v[j + 2]),
+                                                         __uint_as_float(v[j + 3]));
+                            if (opens) *reinterpret_cast<float4*>(dstp + j) = o;
+                            else red_add_f4(dstp + j, o);   // this thread wrote the slot's earlier slabs itself
                         }
                     }
                 }
@@ -621,12 +618,9 @@ gram_staged_kernel(const __grid_constant__ CUtensorMap xmap, int m, uint32_t stg
                     float* dstp = out_item + (int64_t)row * ncol + cc * 16;
 #pragma unroll
                     for (int j = 0; j < 16; j += 4) {
-                        float4 o = make_float4(acc[j], acc[j + 1], acc[j + 2], acc[j + 3]);
-                        if (!opens) {   // this thread wrote the slot's earlier slabs itself
-                            const float4 e = *reinterpret_cast<const float4*>(dstp + j);
-                            o.x += e.x; o.y += e.y; o.z += e.z; o.w += e.w;
-                        }
-                        *reinterpret_cast<float4*>(dstp + j) = o;
+                        const float4 o = make_float4(acc[j], acc[j + 1], acc[j + 2], acc[j + 3]);
+                        if (opens) *reinterpret_cast<float4*>(dstp + j) = o;
+                        else red_add_f4(dstp + j, o);   // this thread wrote the slot's earlier slabs itself
                     }
                 }
             }

@@ -75,6 +75,13 @@ __device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, i
         : "memory");
 }
 
+// p[0..3] += v as one reduction that returns nothing: the thread does not wait for the old values.  A slot of partial
+// sums is only ever touched by one thread, whose additions to one address happen in program order, so the result is
+// the same as read - add - write.
+__device__ __forceinline__ void red_add_f4(float* p, float4 v) {
+    asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(p), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
+}
+
 // Packed pairs of fp32 (one instruction for two lanes).
 __device__ __forceinline__ uint64_t sub2(uint64_t a, uint64_t b) {
     uint64_t r;

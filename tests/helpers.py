@@ -34,8 +34,8 @@ def bulyan_min_gap(D: np.ndarray, f: int) -> float:
         sc = oracle.krum_scores(D, f, alive)
         live = np.sort(sc[alive.astype(bool)])
         best = live[0]
-        others = live[live != best]
-        if len(others):
+        others = live[(live != best) & np.isfinite(live)]   # (rows at infinite distance never compete)
+        if len(others) and np.isfinite(best):
             worst = min(worst, abs(others[0] - best) / max(abs(others[0]), abs(best), 1e-300))
         pick = min((i for i in range(m) if alive[i]), key=lambda i: (sc[i], i))
         alive[pick] = 0
