@@ -95,3 +95,35 @@ def test_the_split_tf32_kernels_alone_match_the_oracle():
     finally:
         dx.tc_split_mode(prev)
     assert dx.tc_split_mode() == dx.SPLIT_AUTO
+
+
+@pytest.mark.parametrize("m,d", [(45, 20_011), (64, 4097), (105, 33_333), (140, 9001), (225, 12_345)])
+@pytest.mark.parametrize("factor", [-100.0, -1.0e4])
+def test_multikrum_average_with_huge_rejected_rows(m, d, factor):
+    """The rejected rows are up to 10^4 times longer than the kept ones: the average of the kept rows must not lose
+    digits to them, whichever way the second sweep forms it."""
+    f = m // 9
+    X = krum_inputs(m, d, seed=5 * m + d, copies=1, outliers=0)
+    X[m - f:] *= np.float32(factor)
+    out_o, sel_o, _, _ = oracle.multikrum(X, f, m - f)
+    assert sel_o.tolist() == list(range(m - f))
+    out, sel, _ = dx.agg_multikrum(padded(X), f, m - f)
+    assert sel.cpu().numpy().tolist() == sel_o.tolist()
+    err = np.linalg.norm(out.cpu().numpy().astype(np.float64) - out_o) / np.linalg.norm(out_o)
+    assert err <= 1e-5
+
+
+def test_multikrum_average_with_non_finite_rejected_rows():
+    """Rejected rows with Inf and NaN entries leave the average of the kept rows finite and exact."""
+    m, d, f = 105, 10_007, 10
+    X = krum_inputs(m, d, seed=99, copies=1, outliers=0)
+    X[m - f:] *= np.float32(-100.0)
+    X[m - 1, 5] = np.inf
+    X[m - 2, 5000] = -np.inf
+    X[m - 3, d - 1] = np.nan
+    out_o, sel_o, _, _ = oracle.multikrum(X, f, m - f)
+    out, sel, _ = dx.agg_multikrum(padded(X), f, m - f)
+    assert sel.cpu().numpy().tolist() == sel_o.tolist()
+    o = out.cpu().numpy()
+    assert np.isfinite(o).all()
+    assert np.linalg.norm(o.astype(np.float64) - out_o) / np.linalg.norm(out_o) <= 1e-5
