@@ -71,11 +71,11 @@ ORACLE_A1 = {1: "mean", 2: "coord_median", 3: "multikrum", 4: "bulyan"}
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel of the DETOX step, from ncu captures of
 # the same kernel code (reset an entry to None when its kernel changes).
 NCU_TRAFFIC_BYTES = {
-    ("cfg2", "vote_mean_kernel"): 2_011_333_000 + 117_863_424,
-    ("cfg3", "vote_kernel (winners only)"): 2_011_344_896 + 3_232_768,
+    ("cfg2", "vote_mean_kernel"): 2_011_332_000 + 118_065_152,
+    ("cfg3", "vote_kernel (winners only)"): 2_011_382_000 + 5_457_920,
     # config 4 holds 11.8 GB, too much for a multi-pass capture: config 2's traffic of the same streaming kernel,
     # scaled by the algorithmic bytes (12,544,000,000 / 2,145,400,704)
-    ("cfg4", "vote_mean_kernel"): int((2_011_333_000 + 117_863_424) * 12_544_000_000 / 2_145_400_704),
+    ("cfg4", "vote_mean_kernel"): int((2_011_332_000 + 118_065_152) * 12_544_000_000 / 2_145_400_704),
 }
 
 
@@ -304,7 +304,7 @@ def median_alu_roofline(m, d, ms, peaks):
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the tensor-core distance kernel over the algorithmic
 # bytes m d 4, from ncu captures at d = 2.5 M (the kernel reads every row once, so its traffic grows with m d); reset an
 # entry to None when the kernel changes.
-NCU_GRAM_TRAFFIC_RATIO = {45: None, 105: None, 225: None}
+NCU_GRAM_TRAFFIC_RATIO = {45: 1.025, 105: 1.043, 225: 1.096}
 
 
 def gram_roofline(m, d, ms, peaks, peak_kind, ms_tf32=None):
