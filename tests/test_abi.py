@@ -54,6 +54,31 @@ def test_workspace_sizes(lib):
     assert bad.workspace_bytes() == 0
 
 
+def test_distance_workspace_covers_every_row_count_of_the_tensor_core_path(lib):
+    """The workspace of the distance pass is planned on the host (slab slots of both operand splits, norms, row scales,
+    centre choice).  For every row count of the tensor-core path and column counts from one stage to ResNet-50 size the
+    plan must exist, hold at least the distance matrix and its slab partials, and grow with d."""
+    for m in list(range(17, 257, 7)) + [32, 33, 64, 65, 128, 129, 256]:
+        prev = 0
+        for d in (64, 4097, 1_000_000, 11_173_962, 25_557_032):
+            b = dx.agg_pairwise_sqdist_workspace_bytes(m, d)
+            assert b >= m * m * 8 + m * 4, (m, d)
+            assert b >= prev, (m, d)
+            prev = b
+        ncol = (m + 15) // 16 * 16
+        # at least one fp32 partial of m x ncol per CTA at full width
+        assert dx.agg_pairwise_sqdist_workspace_bytes(m, 25_557_032) >= 148 * m * ncol * 4
+        assert dx.agg_multikrum_workspace_bytes(m, 11_173_962) >= dx.agg_pairwise_sqdist_workspace_bytes(m, 11_173_962)
+
+
+def test_split_mode_switch_and_its_query(lib):
+    assert dx.tc_split_mode() == dx.SPLIT_AUTO
+    assert dx.tc_split_mode(dx.SPLIT_TF32) == dx.SPLIT_AUTO
+    assert dx.tc_split_mode(7) == dx.SPLIT_TF32          # an unknown value only queries
+    assert dx.tc_split_mode(dx.SPLIT_AUTO) == dx.SPLIT_TF32
+    assert dx.tc_split_mode() == dx.SPLIT_AUTO
+
+
 def test_bad_arguments_are_rejected_before_any_launch(lib):
     # Pointers are fake but never dereferenced: every call must fail in validation.
     fake = ctypes.c_void_p(0x1000)
