@@ -73,9 +73,9 @@ ORACLE_A1 = {1: "mean", 2: "coord_median", 3: "multikrum", 4: "bulyan"}
 NCU_TRAFFIC_BYTES = {
     ("cfg2", "vote_mean_kernel"): 2_011_332_000 + 118_065_152,
     ("cfg3", "vote_kernel (winners only)"): 2_011_382_000 + 5_457_920,
-    # config 4 holds 11.8 GB, too much for a multi-pass capture: config 2's traffic of the same streaming kernel,
-    # scaled by the algorithmic bytes (12,544,000,000 / 2,145,400,704)
-    ("cfg4", "vote_mean_kernel"): int((2_011_332_000 + 118_065_152) * 12_544_000_000 / 2_145_400_704),
+    # config 4 holds 11.8 GB, too much for a multi-pass capture: the traffic of the same streaming kernel on 105 rows of
+    # 2,500,000 columns, scaled by the algorithmic bytes (11,872,000,000 / 1,060,000,000)
+    ("cfg4", "vote_mean_select_kernel"): int((1_050_018_000 + 7_588_096) * 11_872_000_000 / 1_060_000_000),
 }
 
 
@@ -588,7 +588,13 @@ def main():
         # the dominant kernel alone, same inputs, same stream: the vote (reads n*d*4, writes G*d*4), or the vote
         # fused with the set means when A_0 is the mean (reads n*d*4, writes S*d*4)
         vws = torch.empty(dx.detox_vote_workspace_bytes(spec.n, spec.r), dtype=torch.uint8, device=dev)
-        if cfg["a0"] == dx.AGG_MEAN:
+        fused_a1 = cfg["a1"] in (dx.AGG_COORD_MEDIAN, dx.AGG_TRIMMED_MEAN, dx.AGG_MEAN)
+        if cfg["a0"] == dx.AGG_MEAN and fused_a1 and w.S <= 16 and spec.r in (1, 3, 5):
+            # vote, set means and the coordinate-wise A_1 are one kernel (reads n*d*4, writes d*4): the step itself,
+            # which only adds two ~3 us helper kernels
+            dom_name, dom_rows_out = "vote_mean_select_kernel", 1
+            dom = step
+        elif cfg["a0"] == dx.AGG_MEAN:
             Mbuf = torch.empty((w.S, w.ld), dtype=torch.float32, device=dev)[:, : spec.d]
             dom_name, dom_rows_out = "vote_mean_kernel", w.S
             dom = lambda: dx.detox_vote_hier_mean(X, spec.r, w.members, w.set_offsets, w.set_members, M=Mbuf,

@@ -470,6 +470,13 @@ detox_status detox_aggregate(const detox_pipeline_desc* p, const float* X, int64
     const int32_t* row_list = nullptr;
     int m = G;
     if (p->a0 == DETOX_AGG_MEAN) {
+        // A_1 that works coordinate by coordinate over at most 16 set means: everything in one pass over X
+        const bool coordwise = p->a1 == DETOX_AGG_COORD_MEDIAN || p->a1 == DETOX_AGG_TRIMMED_MEAN || p->a1 == DETOX_AGG_MEAN;
+        if (coordwise && vote_mean_select_supported(X, ld, p->r, p->n_sets, out)) {
+            const int beta = p->a1 == DETOX_AGG_TRIMMED_MEAN ? -(p->n_sets - 2 * p->f) : 0;
+            return launch_vote_mean_select(X, ld, p->n, p->r, p->d, groups, sets, p->n_sets, beta, p->a1 == DETOX_AGG_MEAN, out,
+                                           win, w.vote, s, kStatusBytes);
+        }
         if ((st = launch_vote_mean(X, ld, p->n, p->r, p->d, groups, sets, p->n_sets, w.M, w.ldz, win, w.vote, s, kStatusBytes)) !=
             DETOX_OK)
             return st;

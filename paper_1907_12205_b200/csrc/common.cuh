@@ -70,6 +70,14 @@ detox_status launch_vote_mean(const float* X, int64_t ld, int n, int r, int64_t 
                               const SetTable& sets, int S, float* M, int64_t ldm, int32_t* winner, void* ws,
                               cudaStream_t s, size_t clear_before = 0);
 
+// vote + A_0 = mean + a coordinate-wise A_1 over the S <= 16 set means in one pass: out = A_1(set means); neither votes
+// nor set means are stored.  beta as in launch_coord_select (0: median; <= -1: mean of the middle -beta values);
+// mean = true: the mean of the set means.  Needs 16-byte aligned rows and r in {1, 3, 5}.
+bool vote_mean_select_supported(const float* X, int64_t ld, int r, int S, const float* out);
+detox_status launch_vote_mean_select(const float* X, int64_t ld, int n, int r, int64_t d, const IdTable& members,
+                                     const SetTable& sets, int S, int beta, bool mean, float* out, int32_t* winner,
+                                     void* ws, cudaStream_t s, size_t clear_before = 0);
+
 // mean.cu
 // (sign = true: coordinate-wise sign majority sign(sum sign(x)) instead of the mean, in both launchers)
 detox_status launch_hier_mean(const float* Z, int64_t ldz, int64_t d, const SetTable& sets, int S,

@@ -8,6 +8,7 @@
 // whether a global majority exists; only groups without one have their Z row cleared again.
 // Traffic: n*d*4 bytes read, G*d*4 bytes written, once.
 #include "common.cuh"
+#include "sortnet.cuh"
 
 namespace detox {
 
@@ -305,6 +306,186 @@ __global__ void vote_mean_fix_kernel(const float* __restrict__ X, int64_t ld, in
     }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Vote, A_0 = mean and a coordinate-wise A_1 over the set means in one pass (Algorithm 1's filtering step + the
+// whole of Algorithm 2 when A_1 works coordinate by coordinate): a CTA covers ALL vote sets for its 128 columns, the
+// S set means meet in shared memory and A_1 is applied to them at once, so that neither the votes nor the set means
+// travel to memory (n*d*4 bytes read, d*4 written).  The set means are formed exactly as in vote_mean_kernel and
+// A_1 exactly as in the order-statistic kernels, so the result is bitwise the one of the separate kernels.
+//   mode == 0: median;  mode < 0: mean of the middle -mode values (S + mode even);  mode == kSelectMean: mean.
+// SM = size of the sorting network: S rounded up (same parity) with (SM - S) / 2 lowest and as many highest keys.
+// If a group turns out to have no majority, the output is recomputed from the winners' rows afterwards
+// (vote_mean_select_fix_kernel).
+// ---------------------------------------------------------------------------------------------
+constexpr int kSelectMean = 0x40000000;
+constexpr int kMaxFusedSets = 16;
+
+// A_1 over v[0..S-1] (SM >= S, SM - S even).
+template <int SM>
+__device__ __forceinline__ float select_over_sets(const float (&v)[SM], int S, int mode) {
+    if (mode == kSelectMean) {
+        float acc = 0.f;
+#pragma unroll
+        for (int i = 0; i < SM; ++i)
+            if (i < S) acc += v[i];
+        return acc / (float)S;
+    }
+    const int pad = (SM - S) >> 1;
+    int32_t key[SM];
+#pragma unroll
+    for (int i = 0; i < SM; ++i)
+        key[i] = i < S ? key_of_bits(__float_as_uint(v[i])) : (i - S < pad ? (int32_t)0x80000000 : 0x7fffffff);
+    sort_registers<SM>(key);
+    if (mode == 0) {
+        if (SM & 1) return float_of_key(key[SM / 2]);
+        return (float_of_key(key[SM / 2 > 0 ? SM / 2 - 1 : 0]) + float_of_key(key[SM / 2])) * 0.5f;
+    }
+    const int cnt = -mode, L = pad + ((S - cnt) >> 1);
+    float acc = 0.f;
+#pragma unroll
+    for (int i = 0; i < SM; ++i)
+        if (i >= L && i < L + cnt) acc += float_of_key(key[i]);
+    return acc / (float)cnt;
+}
+
+// CTA = 64 column pieces (256 columns) x S sets: the two warps of row y form set y's mean of the CTA's 256 columns exactly as
+// vote_mean_kernel does (few registers, all loads of a group in flight, full occupancy), leaves it in shared memory,
+// and after one barrier the first 256 threads apply A_1 to the S means of one column each.
+constexpr int kFusedPieces = 64;   // (32 pieces: 1.83 ms on the 105 x 28 M configuration, 64: 1.75 ms)
+template <int R, int SM>
+__global__ void __launch_bounds__(kFusedPieces * kMaxFusedSets)
+vote_mean_select_kernel(const float* __restrict__ X, int64_t ld, int64_t d, const __grid_constant__ IdTable members,
+                        const __grid_constant__ SetTable sets, int S, int mode, float* __restrict__ out,
+                        uint32_t* __restrict__ pairdiff) {
+    using Shape = VoteShape<R>;
+    __shared__ __align__(16) float means[kMaxFusedSets][kFusedPieces * 4];
+    const int s = threadIdx.y;
+    const int64_t col0 = (int64_t)blockIdx.x * (kFusedPieces * 4);
+    const int64_t col = col0 + threadIdx.x * 4;
+    const int64_t left = d - col;
+    const int valid = left >= 4 ? 4 : (left > 0 ? (int)left : 0);
+    // (with fewer than four sets the CTA still has four rows of threads: the spare ones only help with A_1)
+    const int b = s < S ? sets.offset[s] : 0, e = s < S ? sets.offset[s + 1] : 0;
+
+    PieceSum<4> sum;
+    sum.zero();
+#pragma unroll 2
+    for (int t = b; t < e; ++t) {
+        const int g = sets.member[t];
+        Piece<4> v[R];
+#pragma unroll
+        for (int a = 0; a < R; ++a) {
+            if (valid > 0) v[a].load(X + (int64_t)members.id[g * R + a] * ld + col, valid);
+            else v[a].clear();
+        }
+        uint32_t loc[Shape::kWords];
+#pragma unroll
+        for (int w = 0; w < Shape::kWords; ++w) loc[w] = 0u;
+#pragma unroll
+        for (int a = 0; a < R; ++a) {
+#pragma unroll
+            for (int c = a + 1; c < R; ++c) {
+                const int p = pair_index(R, a, c);
+                if (v[a].differs(v[c])) loc[p >> 5] |= 1u << (p & 31);
+            }
+        }
+        Piece<4> pick;
+        pick.clear();
+#pragma unroll
+        for (int a = R - 1; a >= 0; --a) {
+            int agree = 1;
+#pragma unroll
+            for (int c = 0; c < R; ++c) {
+                if (c == a) continue;
+                const int p = a < c ? pair_index(R, a, c) : pair_index(R, c, a);
+                agree += ((loc[p >> 5] >> (p & 31)) & 1u) ? 0 : 1;
+            }
+            if (2 * agree > R) pick = v[a];
+        }
+        sum.add(pick);
+#pragma unroll
+        for (int w = 0; w < Shape::kWords; ++w) {
+            const uint32_t bits = __reduce_or_sync(0xffffffffu, loc[w]);
+            if ((threadIdx.x & 31) == 0 && bits != 0u) {
+                uint32_t* word = pairdiff + (int64_t)g * kPairWords + w;
+                const uint32_t seen = *reinterpret_cast<volatile uint32_t*>(word);
+                if (bits & ~seen) atomicOr(word, bits);
+            }
+        }
+    }
+    const float k = (float)(e - b);
+    if (s < S)
+        *reinterpret_cast<float4*>(&means[s][threadIdx.x * 4]) = make_float4(sum.a.x / k, sum.a.y / k, sum.a.z / k, sum.a.w / k);
+    __syncthreads();
+    const int tid = threadIdx.y * kFusedPieces + threadIdx.x;
+    if (tid >= kFusedPieces * 4 || col0 + tid >= d) return;
+    float v[SM];
+#pragma unroll
+    for (int i = 0; i < SM; ++i) v[i] = i < S ? means[i][tid] : 0.f;
+    out[col0 + tid] = select_over_sets<SM>(v, S, mode);
+}
+
+// After the winners are known: nothing to do unless some group has no majority (rare).  Then every coordinate is
+// recomputed from the winners' rows: such a group counts as a zero row, the others contribute their winner's row
+// (bitwise the vote), with the same order of additions and the same A_1.
+template <int SM>
+__global__ void vote_mean_select_fix_kernel(const float* __restrict__ X, int64_t ld, int64_t d,
+                                            const __grid_constant__ SetTable sets, int S, int G,
+                                            const int32_t* __restrict__ winner, int mode, float* __restrict__ out) {
+    int broken = 0;
+    for (int g = threadIdx.x; g < G; g += blockDim.x) broken |= winner[g] < 0;
+    if (!__syncthreads_or(broken)) return;
+    for (int64_t c = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; c < d; c += (int64_t)gridDim.x * blockDim.x) {
+        float mean[SM];
+#pragma unroll
+        for (int s = 0; s < SM; ++s) {
+            mean[s] = 0.f;
+            if (s < S) {
+                const int b = sets.offset[s], e = sets.offset[s + 1];
+                float acc = 0.f;
+                for (int t = b; t < e; ++t) {
+                    const int w = winner[sets.member[t]];
+                    acc += w >= 0 ? X[(int64_t)w * ld + c] : 0.f;
+                }
+                mean[s] = acc / (float)(e - b);
+            }
+        }
+        out[c] = select_over_sets<SM>(mean, S, mode);
+    }
+}
+
+template <int R, int SM>
+detox_status launch_vote_mean_select_rs(const float* X, int64_t ld, int G, int64_t d, const IdTable& members,
+                                        const SetTable& sets, int S, int mode, float* out, int32_t* winner,
+                                        uint32_t* pairdiff, cudaStream_t s) {
+    const int64_t bx = ceil_div(d, (int64_t)kFusedPieces * 4);
+    if (bx > 0x7fffffffLL) return DETOX_ERR_UNSUPPORTED;
+    // at least four rows of threads, so that the 256 columns of a CTA all get their A_1
+    const int by = S < 4 ? 4 : S;
+    vote_mean_select_kernel<R, SM><<<(unsigned)bx, dim3(kFusedPieces, (unsigned)by), 0, s>>>(X, ld, d, members, sets, S, mode,
+                                                                                         out, pairdiff);
+    detox_status st = launch_status();
+    if (st != DETOX_OK) return st;
+    vote_finalize_kernel<<<(G + 127) / 128, 128, 0, s>>>(G, R, members, pairdiff, winner);
+    if ((st = launch_status()) != DETOX_OK) return st;
+    const unsigned fx = (unsigned)(ceil_div(d, 256) < 4 * kSMs ? ceil_div(d, 256) : 4 * kSMs);
+    vote_mean_select_fix_kernel<SM><<<fx, 256, 0, s>>>(X, ld, d, sets, S, G, winner, mode, out);
+    return launch_status();
+}
+
+template <int R>
+detox_status launch_vote_mean_select_r(const float* X, int64_t ld, int G, int64_t d, const IdTable& members,
+                                       const SetTable& sets, int S, int mode, float* out, int32_t* winner,
+                                       uint32_t* pairdiff, cudaStream_t s) {
+    // network sizes 7, 8, 15, 16: S rounded up with its parity kept
+    if (S <= 8) {
+        if (S & 1) return launch_vote_mean_select_rs<R, 7>(X, ld, G, d, members, sets, S, mode, out, winner, pairdiff, s);
+        return launch_vote_mean_select_rs<R, 8>(X, ld, G, d, members, sets, S, mode, out, winner, pairdiff, s);
+    }
+    if (S & 1) return launch_vote_mean_select_rs<R, 15>(X, ld, G, d, members, sets, S, mode, out, winner, pairdiff, s);
+    return launch_vote_mean_select_rs<R, 16>(X, ld, G, d, members, sets, S, mode, out, winner, pairdiff, s);
+}
+
 template <int VEC>
 detox_status launch_vote_mean_vec(const float* X, int64_t ld, int r, int64_t d, const IdTable& members,
                                   const SetTable& sets, int S, float* M, int64_t ldm, uint32_t* pairdiff,
@@ -398,6 +579,30 @@ detox_status launch_vote_mean(const float* X, int64_t ld, int n, int r, int64_t 
     unsigned bx = (unsigned)(ceil_div(d, 256 * 8) < 64 ? ceil_div(d, 256 * 8) : 64);
     vote_mean_fix_kernel<<<dim3(bx, (unsigned)S), 256, 0, s>>>(X, ld, d, sets, winner, M, ldm);
     return launch_status();
+}
+
+bool vote_mean_select_supported(const float* X, int64_t ld, int r, int S, const float* out) {
+    return (r == 1 || r == 3 || r == 5) && S >= 1 && S <= kMaxFusedSets && aligned16(X) && ld % 4 == 0 && aligned16(out);
+}
+
+detox_status launch_vote_mean_select(const float* X, int64_t ld, int n, int r, int64_t d, const IdTable& members,
+                                     const SetTable& sets, int S, int beta, bool mean, float* out, int32_t* winner,
+                                     void* ws, cudaStream_t s, size_t clear_before) {
+    if (!vote_mean_select_supported(X, ld, r, S, out)) return DETOX_ERR_UNSUPPORTED;
+    if (!mean && beta > 0) return DETOX_ERR_UNSUPPORTED;
+    if (!mean && beta < 0 && (-beta > S || ((S + beta) & 1))) return DETOX_ERR_BAD_ARG;
+    const int G = n / r;
+    const int mode = mean ? kSelectMean : beta;
+    uint32_t* pairdiff = static_cast<uint32_t*>(ws);
+    if (cudaMemsetAsync(static_cast<char*>(ws) - clear_before, 0,
+                        clear_before + (size_t)G * kPairWords * sizeof(uint32_t), s) != cudaSuccess)
+        return DETOX_ERR_CUDA;
+    switch (r) {
+        case 1: return launch_vote_mean_select_r<1>(X, ld, G, d, members, sets, S, mode, out, winner, pairdiff, s);
+        case 3: return launch_vote_mean_select_r<3>(X, ld, G, d, members, sets, S, mode, out, winner, pairdiff, s);
+        case 5: return launch_vote_mean_select_r<5>(X, ld, G, d, members, sets, S, mode, out, winner, pairdiff, s);
+        default: return DETOX_ERR_UNSUPPORTED;
+    }
 }
 
 }  // namespace detox

@@ -351,6 +351,45 @@ def test_pipeline_fused_vote_mean_handles_no_majority_and_uneven_sets(r, G, set_
     assert np.array_equal(bits(fused), bits(two_step))
 
 
+@pytest.mark.parametrize("r,set_size,S", [(3, 5, 1), (3, 3, 2), (3, 5, 3), (3, 2, 4), (3, 5, 5), (5, 1, 6), (3, 5, 7), (3, 4, 8),
+                                          (3, 3, 9), (1, 2, 12), (3, 5, 15), (3, 2, 16), (3, 1, 17)])
+@pytest.mark.parametrize("broken", [False, True])
+def test_pipeline_vote_set_means_and_coordinatewise_a1_in_one_pass(r, set_size, S, broken):
+    """With A_0 = mean and a coordinate-wise A_1 over at most 16 set means the whole step is one pass over X (set
+    means and A_1 in registers).  It must give, bit for bit, what the separate entry points give (fused vote + set
+    means, then the order-statistic or mean kernel over them), with and without a group that has no majority, and
+    match the oracle; 17 sets take the separate kernels."""
+    G = set_size * S
+    d = 4099 + 64 * S                                   # a ragged tail
+    spec = wl.WorkloadSpec("p", n=r * G, r=r, d=d, sigma=1e-2, q=0, set_size=set_size, seed=31 * S + r)
+    w = wl.make_workload(spec)
+    assert w.S == S
+    if broken and r >= 3:                               # the last group: nobody agrees -> zero vote inside its set
+        for t, i in enumerate(w.members[r * (G - 1):r * G]):
+            w.X[int(i), (t * 53) % d] += 1.0 + t
+    Xd = w.X.to(DEV)[:, :d]
+    M, _ = dx.detox_vote_hier_mean(Xd, r, w.members, w.set_offsets, w.set_members)
+    cases = [(dx.AGG_COORD_MEDIAN, 0), (dx.AGG_MEAN, 0)]
+    if S >= 3:
+        cases.append((dx.AGG_TRIMMED_MEAN, 1))
+    if S >= 7:
+        cases.append((dx.AGG_TRIMMED_MEAN, 3))
+    for a1, f in cases:
+        res, ref = run_pipeline(w, dx.AGG_MEAN, a1, f)
+        assert res["winner"].cpu().numpy().tolist() == ref["winner"].tolist()
+        if broken and r >= 3:
+            assert ref["winner"][G - 1] == -1
+        out = res["out"]
+        if a1 == dx.AGG_COORD_MEDIAN:
+            two_step = dx.agg_coord_median(M)
+            assert np.array_equal(bits(out), bits(two_step))
+            assert np.array_equal(bits(out), ref["out"].view(np.uint32)) or rel_l2(out.cpu().numpy(), ref["out"]) <= TOL
+        elif a1 == dx.AGG_MEAN:
+            two_step = dx.detox_aggregate(dx.Pipeline(S, 1, d, np.arange(S), dx.AGG_NONE, None, None, dx.AGG_MEAN), M)["out"]
+            assert np.array_equal(bits(out), bits(two_step))
+        assert rel_l2(out.cpu().numpy(), ref["out"]) <= TOL
+
+
 @pytest.mark.parametrize("a0,f,m_sel,offs,a1", [("multikrum", 1, 0, [0, 7, 15], "mean"), ("bulyan", 2, 0, [0, 15], "mean"),
                                                  ("multikrum", 1, 3, [0, 5, 10, 15], "coord_median")])
 def test_pipeline_krum_family_inside_vote_sets(a0, f, m_sel, offs, a1):
