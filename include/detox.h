@@ -240,7 +240,9 @@ detox_status agg_bulyan(const float* X, int64_t ld, int m, int64_t d, int f, flo
  * vote over the node groups, A_0 over each vote group, A_1 over the results.
  *
  *   a0 = DETOX_AGG_NONE : the G votes go to A_1 directly (sets are ignored)
- *   a0 = DETOX_AGG_MEAN : the S set means go to A_1
+ *   a0 = DETOX_AGG_MEAN : the S set means go to A_1 (with a1 = MEAN, COORD_MEDIAN or TRIMMED_MEAN over at most 16 sets,
+ *        r in {1, 3, 5} and 16-byte aligned rows of X and out, the whole step is one pass over X and the set means
+ *        are never stored; the result is bitwise the same either way)
  *   a0 = DETOX_AGG_SIGN_MAJORITY : the S coordinate-wise sign majorities of the sets go to A_1
  *   a0 = DETOX_AGG_MULTIKRUM | DETOX_AGG_BULYAN : the aggregator runs inside every vote set (the pairings the
  *        paper found most resilient, Section 5.2, setups 2 and 3; set shapes as in Appendix B.1, e.g. 7 + 8 or
