@@ -97,6 +97,17 @@ KrumWs krum_ws(void* ws, int m, int64_t d) {
     return k;
 }
 
+// The filtering step folded into the distance pass (more than 16 votes of groups of three): the m rows are the votes,
+// `rows` is winner[], which the pass fills in before anything reads it.
+struct VoteFuse {
+    const IdTable* members;
+    int n;
+    void* vote_ws;     // the vote's workspace words (cleared by the caller)
+    float* Z;          // where the votes go if the pass has to be repeated on stored rows
+    int64_t ldz;
+    int32_t* winner;
+};
+
 // `rows` (optional, device, m <= 16): the m rows are X[rows[i]], a negative entry standing for a zero row
 // (this is how the votes are consumed straight from the workers' rows through winner[], without a copy).
 //
@@ -104,7 +115,8 @@ KrumWs krum_ws(void* ws, int m, int64_t d) {
 // first word of `ws`, cleared here (the stand-alone aggregators).  Otherwise the caller's word, which the caller has
 // cleared and which is only ever set, never cleared, from here on (the pipeline: one word for all its stages).
 detox_status run_multikrum(const float* X, int64_t ld, int m, int64_t d, const int32_t* rows, int f, int m_sel,
-                           float* out, int32_t* sel, double* scores, void* ws, int* status, cudaStream_t s) {
+                           float* out, int32_t* sel, double* scores, void* ws, int* status, cudaStream_t s,
+                           const VoteFuse* vf = nullptr) {
     KrumWs k = krum_ws(ws, m, d);
     const bool own_status = status == nullptr;
     if (own_status) status = k.status;
@@ -119,7 +131,9 @@ detox_status run_multikrum(const float* X, int64_t ld, int m, int64_t d, const i
         return launch_mean_rows(X, ld, d, rows ? k.mapped : sel_buf, m_sel, out, s);
     }
     if (own_status && cudaMemsetAsync(status, 0, sizeof(int), s) != cudaSuccess) return DETOX_ERR_CUDA;
-    st = launch_sqdist(X, ld, m, d, rows, k.D, k.dist, status, s);
+    st = vf ? launch_sqdist_vote_tc(X, ld, vf->n, d, *vf->members, vf->winner, vf->vote_ws, vf->Z, vf->ldz, k.D, k.dist,
+                                    status, s)
+            : launch_sqdist(X, ld, m, d, rows, k.D, k.dist, status, s);
     if (st != DETOX_OK) return st;
     st = launch_multikrum_select(k.D, m, f, m_sel, sel_buf, scores, k.select, s);
     if (st != DETOX_OK) return st;
@@ -132,7 +146,7 @@ detox_status run_multikrum(const float* X, int64_t ld, int m, int64_t d, const i
 }
 
 detox_status run_bulyan(const float* X, int64_t ld, int m, int64_t d, const int32_t* rows, int f, float* out,
-                        int32_t* sel, void* ws, int* status, cudaStream_t s) {
+                        int32_t* sel, void* ws, int* status, cudaStream_t s, const VoteFuse* vf = nullptr) {
     KrumWs k = krum_ws(ws, m, d);
     const bool own_status = status == nullptr;
     if (own_status) status = k.status;
@@ -148,7 +162,9 @@ detox_status run_bulyan(const float* X, int64_t ld, int m, int64_t d, const int3
         return launch_coord_select(X, ld, theta, d, rows ? k.mapped : sel_buf, beta, out, s);
     }
     if (own_status && cudaMemsetAsync(status, 0, sizeof(int), s) != cudaSuccess) return DETOX_ERR_CUDA;
-    st = launch_sqdist(X, ld, m, d, rows, k.D, k.dist, status, s);
+    st = vf ? launch_sqdist_vote_tc(X, ld, vf->n, d, *vf->members, vf->winner, vf->vote_ws, vf->Z, vf->ldz, k.D, k.dist,
+                                    status, s)
+            : launch_sqdist(X, ld, m, d, rows, k.D, k.dist, status, s);
     if (st != DETOX_OK) return st;
     st = launch_bulyan_select(k.D, m, f, sel_buf, k.select, s);
     if (st != DETOX_OK) return st;
@@ -468,6 +484,8 @@ detox_status detox_aggregate(const detox_pipeline_desc* p, const float* X, int64
     const float* rows = w.Z;
     int64_t row_ld = w.ldz;
     const int32_t* row_list = nullptr;
+    VoteFuse fuse;
+    const VoteFuse* vf = nullptr;
     int m = G;
     if (p->a0 == DETOX_AGG_MEAN) {
         // A_1 that works coordinate by coordinate over at most 16 set means: everything in one pass over X
@@ -528,6 +546,15 @@ detox_status detox_aggregate(const detox_pipeline_desc* p, const float* X, int64
         rows = X;
         row_ld = ld;
         row_list = win;
+    } else if (krum_type(p->a1) && sqdist_vote_tc_supported(X, ld, p->n, p->r, p->d)) {
+        // More than 16 votes of groups of three under a Krum-type A_1: the vote runs inside the tensor-core distance
+        // pass, winner[] comes out of it, and everything after the distances reads the winners' rows of X.
+        if (cudaMemsetAsync(w.status, 0, kStatusBytes + vote_ws_bytes(p->n, p->r), s) != cudaSuccess) return DETOX_ERR_CUDA;
+        fuse = VoteFuse{&groups, p->n, w.vote, w.Z, w.ldz, win};
+        vf = &fuse;
+        rows = X;
+        row_ld = ld;
+        row_list = win;
     } else if ((st = launch_vote(X, ld, p->n, p->r, p->d, groups, w.Z, w.ldz, win, w.vote, s, kStatusBytes)) != DETOX_OK) {
         return st;
     }
@@ -546,12 +573,12 @@ detox_status detox_aggregate(const detox_pipeline_desc* p, const float* X, int64
         case DETOX_AGG_MULTIKRUM:
             cnt = p->m_sel;
             sel_buf = sel ? sel : krum_ws(w.agg, m, p->d).sel;
-            st = run_multikrum(rows, row_ld, m, p->d, row_list, p->f, p->m_sel, out, sel_buf, nullptr, w.agg, w.status, s);
+            st = run_multikrum(rows, row_ld, m, p->d, row_list, p->f, p->m_sel, out, sel_buf, nullptr, w.agg, w.status, s, vf);
             break;
         case DETOX_AGG_BULYAN:
             cnt = m - 2 * p->f;
             sel_buf = sel ? sel : krum_ws(w.agg, m, p->d).sel;
-            st = run_bulyan(rows, row_ld, m, p->d, row_list, p->f, out, sel_buf, w.agg, w.status, s);
+            st = run_bulyan(rows, row_ld, m, p->d, row_list, p->f, out, sel_buf, w.agg, w.status, s, vf);
             break;
         default: st = DETOX_ERR_BAD_ARG;
     }

@@ -35,6 +35,7 @@ int sample_blocks(int64_t d) {
 
 struct CentreWs {
     float* part;        // [nblk][2][m]: per block, every row's squared distance to the first centre, then its squared norm
+    int* agree;         // [nblk][m] votes formed on the fly: which members of the group gave the block's sampled pieces
     float* key;         // [m] scratch of the check after the pass
     unsigned* counter;  // [2] "a row failed the check" / CTAs of the check kernel that have finished; behind them one
                         // float: the typical squared norm of a centred row as the sample predicts it for all d columns
@@ -45,6 +46,8 @@ CentreWs centre_carve(void* ws, int m) {
     char* p = static_cast<char*>(ws);
     w.part = reinterpret_cast<float*>(p);
     p += align_up((size_t)kSampleBlocks * 2 * m * sizeof(float));
+    w.agree = reinterpret_cast<int*>(p);
+    p += align_up((size_t)kSampleBlocks * m * sizeof(int));
     w.key = reinterpret_cast<float*>(p);
     p += align_up((size_t)m * sizeof(float));
     w.counter = reinterpret_cast<unsigned*>(p);
@@ -62,20 +65,61 @@ __device__ __forceinline__ void order2(float& a, float& b) {
 }
 
 // One CTA per sampled block of 64 columns (evenly spaced over d).
+//
+// VOTE: row g of the sample is the vote of the three rows members.id[3g .. 3g + 2] of X, formed piece by piece (four
+// columns) as the distance pass will form it: the value two members agree on bitwise, zeros when all differ.
+// agree[b][g] gets one bit per member: it gave every sampled piece of this block (the pass that follows subtracts
+// rows of X, so the rows listed for centring are handed on as such a member's row).
+template <bool VOTE>
 __global__ void __launch_bounds__(kPickThreads)
 centre_sample_kernel(const float* __restrict__ X, int64_t ld, int m, int64_t d, float* __restrict__ part,
-                     unsigned* __restrict__ counter) {
-    extern __shared__ float tile[];   // [m][kSampleCols + 1], then the first centre [kSampleCols]
+                     unsigned* __restrict__ counter, const __grid_constant__ VoteMembers members,
+                     int* __restrict__ agree) {
+    extern __shared__ float tile[];   // [m][kSampleCols + 1], then the first centre [kSampleCols], then (VOTE) agree bits [m]
     constexpr int pitch = kSampleCols + 1;
     float* first = tile + (size_t)m * pitch;
     const int b = blockIdx.x, nblk = gridDim.x;
     const int64_t nb_all = (d + kSampleCols - 1) / kSampleCols;
     const int64_t c0 = (nb_all * b / nblk) * kSampleCols;
     if (b == 0 && threadIdx.x == 0) counter[0] = counter[1] = 0u;   // for the kernels that follow
-    for (int e = threadIdx.x; e < m * kSampleCols; e += kPickThreads) {
-        const int r = e / kSampleCols, c = e - r * kSampleCols;
-        const int64_t col = c0 + c;
-        tile[r * pitch + c] = col < d ? finite_or_zero(X[(int64_t)r * ld + col]) : 0.f;
+    if (VOTE) {
+        int* ok = reinterpret_cast<int*>(first + kSampleCols);
+        for (int r = threadIdx.x; r < m; r += kPickThreads) ok[r] = 7;
+        __syncthreads();
+        for (int e = threadIdx.x; e < m * (kSampleCols / 4); e += kPickThreads) {
+            const int r = e / (kSampleCols / 4), c = (e - r * (kSampleCols / 4)) * 4;
+            uint32_t v[3][4];
+#pragma unroll
+            for (int k = 0; k < 3; ++k) {
+                const float* row = X + (int64_t)members.id[3 * r + k] * ld;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) v[k][i] = c0 + c + i < d ? __float_as_uint(row[c0 + c + i]) : 0u;
+            }
+            bool ne[3];   // pairs (0,1), (0,2), (1,2)
+#pragma unroll
+            for (int pr = 0; pr < 3; ++pr) {
+                const int a = pr == 2 ? 1 : 0, bb = pr == 0 ? 1 : 2;
+                ne[pr] = ((v[a][0] ^ v[bb][0]) | (v[a][1] ^ v[bb][1]) | (v[a][2] ^ v[bb][2]) | (v[a][3] ^ v[bb][3])) != 0u;
+            }
+            const bool first_wins = !ne[0] || !ne[1], other_wins = !ne[2];
+            int mask = 0;
+            if (first_wins) mask = 1 | (ne[0] ? 0 : 2) | (ne[1] ? 0 : 4);
+            else if (other_wins) mask = 6;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const uint32_t u = first_wins ? v[0][i] : (other_wins ? v[1][i] : 0u);
+                tile[r * pitch + c + i] = finite_or_zero(__uint_as_float(u));
+            }
+            if (mask != 7) atomicAnd(&ok[r], mask);
+        }
+        __syncthreads();
+        for (int r = threadIdx.x; r < m; r += kPickThreads) agree[(size_t)b * m + r] = ok[r];
+    } else {
+        for (int e = threadIdx.x; e < m * kSampleCols; e += kPickThreads) {
+            const int r = e / kSampleCols, c = e - r * kSampleCols;
+            const int64_t col = c0 + c;
+            tile[r * pitch + c] = col < d ? finite_or_zero(X[(int64_t)r * ld + col]) : 0.f;
+        }
     }
     __syncthreads();
     if (threadIdx.x < kSampleCols) {
@@ -114,7 +158,8 @@ centre_sample_kernel(const float* __restrict__ X, int64_t ld, int m, int64_t d, 
 // the row has its typical entry in [2^6, 2^7).  A row whose sample is zero or not finite takes the typical row's scale.
 __global__ void __launch_bounds__(kPickThreads)
 centre_pick_kernel(const float* __restrict__ part, int nblk, int m, float scale, float inv_sampled,
-                   unsigned* __restrict__ counter, int* __restrict__ centre, int* __restrict__ expo) {
+                   unsigned* __restrict__ counter, int* __restrict__ centre, int* __restrict__ expo,
+                   const __grid_constant__ VoteMembers members, const int* __restrict__ agree) {
     extern __shared__ float sh[];   // dist [m], norm [m]
     float* dist = sh;
     float* nrm = sh + m;
@@ -158,6 +203,15 @@ centre_pick_kernel(const float* __restrict__ part, int nblk, int m, float scale,
         *reinterpret_cast<float*>(counter + 2) = med[0] * scale;
     }
     __syncthreads();
+    if (agree != nullptr && threadIdx.x < want) {
+        // votes formed on the fly: listed vote g is handed on as the row of X of a member that gave every sampled piece
+        // (the first member when none did: whatever is subtracted, it is the same for all rows)
+        const int g = centre[2 + threadIdx.x];
+        int mask = 7;
+        for (int b = 0; b < nblk; ++b) mask &= agree[(size_t)b * m + g];
+        const int k = (mask & 1) ? 0 : ((mask & 2) ? 1 : ((mask & 4) ? 2 : 0));
+        centre[2 + kMaxCentreRows + threadIdx.x] = (int)members.id[3 * g + k];
+    }
     const float typical = (centring_on ? med[0] : med[1]) * inv_sampled;
     for (int r = threadIdx.x; r < m; r += kPickThreads) {
         float v = (centring_on ? dist[r] : nrm[r]) * inv_sampled;   // mean square of the sampled entries
@@ -269,24 +323,34 @@ centre_check_kernel(const float* __restrict__ norms, const float* __restrict__ p
 
 size_t centre_ws_bytes(int m, int64_t d) {
     (void)d;
-    return align_up((size_t)kSampleBlocks * 2 * m * sizeof(float)) + align_up((size_t)m * sizeof(float)) + 256;   // counters, float
+    return align_up((size_t)kSampleBlocks * 2 * m * sizeof(float)) + align_up((size_t)kSampleBlocks * m * sizeof(int)) +
+           align_up((size_t)m * sizeof(float)) + 256;   // counters, float
 }
 
+// members != null: the m rows are the votes of the groups of three rows of X listed there.
 detox_status launch_pick_centre(const float* X, int64_t ld, int m, int64_t d, void* ws, int* centre, int* expo,
-                                cudaStream_t s) {
+                                cudaStream_t s, const VoteMembers* members) {
     CentreWs w = centre_carve(ws, m);
     const int nblk = sample_blocks(d);
-    const size_t smem = ((size_t)m * (kSampleCols + 1) + kSampleCols) * sizeof(float);
-    if (cudaFuncSetAttribute(centre_sample_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-        return DETOX_ERR_CUDA;
-    centre_sample_kernel<<<nblk, kPickThreads, smem, s>>>(X, ld, m, d, w.part, w.counter);
+    const size_t smem = ((size_t)m * (kSampleCols + 1) + kSampleCols + (members ? m : 0)) * sizeof(float);
+    const VoteMembers none{};
+    if (members) {
+        if (cudaFuncSetAttribute(centre_sample_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+            return DETOX_ERR_CUDA;
+        centre_sample_kernel<true><<<nblk, kPickThreads, smem, s>>>(X, ld, m, d, w.part, w.counter, *members, w.agree);
+    } else {
+        if (cudaFuncSetAttribute(centre_sample_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+            return DETOX_ERR_CUDA;
+        centre_sample_kernel<false><<<nblk, kPickThreads, smem, s>>>(X, ld, m, d, w.part, w.counter, none, nullptr);
+    }
     detox_status st = launch_status();
     if (st != DETOX_OK) return st;
     // the sample's squared norms are scaled up to all d columns for the check after the pass
     const int64_t sampled = (int64_t)nblk * kSampleCols < d ? (int64_t)nblk * kSampleCols : d;
     const float scale = (float)((double)d / (double)sampled);
     centre_pick_kernel<<<1, kPickThreads, (size_t)2 * m * sizeof(float), s>>>(w.part, nblk, m, scale, 1.f / (float)sampled,
-                                                                            w.counter, centre, expo);
+                                                                            w.counter, centre, expo, members ? *members : none,
+                                                                            members ? w.agree : nullptr);
     return launch_status();
 }
 

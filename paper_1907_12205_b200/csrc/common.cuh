@@ -12,6 +12,8 @@ constexpr int kSMs = 148;            // B200: 2 dies x 74 SMs; grids are sized i
 constexpr int kMaxRows = DETOX_MAX_ROWS;
 constexpr int kMaxR = DETOX_MAX_R;
 
+constexpr int kPairWords = 4;        // "members a and b differed" bits per node group: r <= 15 -> at most 105 pairs
+
 // Small host-side index tables travel as kernel parameters (no copy, no allocation).
 struct IdTable {
     uint16_t id[kMaxRows];
@@ -19,6 +21,10 @@ struct IdTable {
 struct SetTable {
     uint16_t offset[kMaxRows + 1];
     uint16_t member[kMaxRows];
+};
+// The member rows of at most 85 groups of three (the distance pass that votes while it reads).
+struct VoteMembers {
+    uint8_t id[256];
 };
 
 // ---- order-preserving integer key for fp32 bit patterns -------------------------------------
@@ -64,6 +70,14 @@ size_t vote_ws_bytes(int n, int r);
 // uses itself (the pipeline keeps its device status word there)
 detox_status launch_vote(const float* X, int64_t ld, int n, int r, int64_t d, const IdTable& members,
                          float* Z, int64_t ldz, int32_t* winner, void* ws, cudaStream_t s, size_t clear_before = 0);
+
+// the last step of a vote on its own: winners from the "members differed" bits in ws; *none_flag (optional, device) is
+// set to 1 when a group has no majority
+detox_status launch_vote_finalize(int n, int r, const IdTable& members, const void* ws, int32_t* winner, int* none_flag,
+                                  cudaStream_t s);
+// r = 3: the votes as rows of Z (zero rows where winner[g] < 0), written only when *gate (device) is not zero
+detox_status launch_vote_store_gated(const float* X, int64_t ld, int n, int64_t d, const IdTable& members, float* Z,
+                                     int64_t ldz, const int32_t* winner, const int* gate, cudaStream_t s);
 
 // vote + A_0 = mean in one pass: M[s] = mean of the votes of set s; the votes themselves are not stored
 detox_status launch_vote_mean(const float* X, int64_t ld, int n, int r, int64_t d, const IdTable& members,
@@ -117,14 +131,24 @@ detox_status launch_sqdist_partials(const float* X, int64_t ld, int m, int64_t d
                                     int* status, bool clear_status, int* nblocks, cudaStream_t s);
 detox_status launch_sqdist_tc(const float* X, int64_t ld, int m, int64_t d, double* D, void* ws, int* status,
                               cudaStream_t s);
+// The filtering step and the distance pass in one (r = 3, 16 < n / 3 <= 85 groups): the distances between the votes of
+// the groups, formed while the members' rows stream through the tensor-core pass, and winner[]; no vote is stored
+// unless the pass has to be repeated (a group without a majority, an entry outside the fp16 range), in which case
+// the votes go to Z (n / 3 rows of pitch ldz) and the split-TF32 kernels run on them.  vote_ws: the vote's cleared
+// workspace words.  ws as for launch_sqdist_tc with m = n / 3.
+bool sqdist_vote_tc_supported(const float* X, int64_t ld, int n, int r, int64_t d);
+detox_status launch_sqdist_vote_tc(const float* X, int64_t ld, int n, int64_t d, const IdTable& members, int32_t* winner,
+                                   void* vote_ws, float* Z, int64_t ldz, double* D, void* ws, int* status, cudaStream_t s);
 
 // centre.cu: the centring rows for the tensor-core distance pass (m <= 256), chosen on a sample of the columns
 //   centre[0] = how many rows are averaged into the vector that is subtracted from every row (0 when the rows hover
 //   around zero anyway), centre[1] = redo flag (below), centre[2..17] = the rows; expo[m] = every row's power-of-two
 //   scale for the split-fp16 pass
 size_t centre_ws_bytes(int m, int64_t d);
+//   members != null: the m rows are the votes of the groups of three rows of X listed there, formed on the fly;
+//   centre[18..33] = for every listed vote the row of X of a member that gave it
 detox_status launch_pick_centre(const float* X, int64_t ld, int m, int64_t d, void* ws, int* centre, int* expo,
-                                cudaStream_t s);
+                                cudaStream_t s, const VoteMembers* members = nullptr);
 //   after the pass: norms = the rows' exact squared norms after the subtraction (nitems x groups x m), partial = the
 //   slots' sums of products (nitems x m x ncol).  Withdraws the centring (centre[0] = 0) when the typical row came out
 //   far larger than the sample predicted for the rows as they were; expo != null: the split-fp16 pass ran with these

@@ -35,6 +35,7 @@ constexpr int kStageCols = 64;                                  // fp32 columns 
 constexpr int kStagesPerSlab = (int)(kSlabCols / kStageCols);
 constexpr int kMaxStg = 12, kMaxMst = 8;
 constexpr size_t kMaxInFlight = 112 * 1024;   // staging bytes beyond which HBM is no faster (a deeper ring measured no gain)
+constexpr size_t kMaxInFlightVote = 136 * 1024;   // the same with the vote inside the pass (slots come in multiples of boxes x groups)
 constexpr size_t kSmemTail = 4096;   // barriers and the centring ring behind the tiles
 constexpr int kCentreWarps = 1;
 
@@ -52,6 +53,7 @@ namespace {
 struct F16Plan {
     bool wide;                   // more than 128 rows: two boxes per stage, two accumulator halves
     int nbox, box_rows;          // TMA boxes per stage; rows per box (a multiple of 8)
+    int rows_in;                 // rows of the matrix the boxes are cut from (m, or the n members' rows with the vote)
     int ncol;                    // m rounded up to 16
     int mrows;                   // M of the MMA: 64 up to 64 rows, else 128
     int nmma, groups;            // MMA-issuing threads; groups of transform warps
@@ -64,11 +66,14 @@ struct F16Plan {
     size_t smem_bytes;
 };
 
-F16Plan f16_plan(int m, int64_t d) {
+// n_in = 0: the m rows themselves are copied in.  n_in > 0 (the vote inside the pass): the boxes hold the n_in rows of the
+// group members, from which the transform warps form the m votes.
+F16Plan f16_plan(int m, int64_t d, int n_in = 0) {
     F16Plan p;
     p.wide = m > 128;
-    p.nbox = p.wide ? 2 : 1;
-    p.box_rows = p.wide ? ((m + 1) / 2 + 7) / 8 * 8 : (m + 7) / 8 * 8;
+    p.rows_in = n_in > 0 ? n_in : m;
+    p.nbox = p.rows_in > 128 ? 2 : 1;
+    p.box_rows = p.nbox == 2 ? ((p.rows_in + 1) / 2 + 7) / 8 * 8 : (p.rows_in + 7) / 8 * 8;
     p.ncol = (m + 15) / 16 * 16;
     p.mrows = m <= 64 ? 64 : 128;
     p.nmma = m <= 64 ? 4 : 2;
@@ -82,9 +87,21 @@ F16Plan f16_plan(int m, int64_t d) {
     const size_t left = kSmemBudget - kSmemTail - 1024 - (size_t)p.nmst * p.tile_bytes;
     p.nstg = (int)(left / p.stg_bytes);
     if (p.nstg > kMaxStg) p.nstg = kMaxStg;
-    while (p.nstg > 2 && (size_t)p.nstg * p.stg_bytes > kMaxInFlight) --p.nstg;
-    // several transform groups: a staging slot always holds stages of the same group (see the split-TF32 staged kernel)
-    p.nstg -= p.nstg % p.groups;
+    if (n_in > 0) {
+        // a staging slot always holds the same box of the same group's stages: a multiple of boxes x groups, as close
+        // to the byte count that keeps HBM busy as that allows
+        const int unit = p.nbox * p.groups;
+        const size_t ub = (size_t)unit * p.stg_bytes;
+        int k = (int)(kMaxInFlightVote / ub);
+        if (k < 1) k = 1;
+        if ((size_t)k * ub < 96 * 1024 && (size_t)(k + 1) * ub <= 160 * 1024) ++k;
+        while (k > 1 && (k * unit > p.nstg)) --k;
+        p.nstg = k * unit;
+    } else {
+        while (p.nstg > 2 && (size_t)p.nstg * p.stg_bytes > kMaxInFlight) --p.nstg;
+        // several transform groups: a staging slot always holds stages of the same group (see the split-TF32 staged kernel)
+        p.nstg -= p.nstg % p.groups;
+    }
     p.nst_total = (int)ceil_div(d, (int64_t)kStageCols);
     p.grid = p.nst_total < kSMs ? p.nst_total : kSMs;
     const int per_cta = (p.nst_total + p.grid - 1) / p.grid;
@@ -129,13 +146,25 @@ __device__ __forceinline__ uint64_t float2_of(uint32_t h2) {
 // MMA-issuing threads.  Not WIDE: the threads take the stages in turn and own an accumulator of 2 ncol columns each
 // (NMMA a multiple of LX and a divisor of the MMA slots: a thread always serves the same slots and group).  WIDE: both
 // threads work on every stage, each on its half of the rows.
-template <int J, int LX, int NMMA, bool WIDE>
+//
+// VB > 0: the majority vote of DETOX's filtering step (Section 3) runs inside the pass.  The boxes (VB of them per
+// stage) then hold the rows of all n = 3 m group members; for every 16-byte piece of vote row g a transform thread
+// reads the pieces of the group's three members, takes the value two of them agree on bitwise (zeros when all three
+// differ) and carries on with it as if it had been copied in.  A strict majority of the whole rows is also the strict
+// majority of every piece, so whenever the group has a winner the piece is the winner's.  The "members a and b differed
+// somewhere" bits are collected per thread and ORed into the group's word of `pairdiff` at the end, in the format the
+// vote kernels use; the caller finds the winners from them and, should a group have none, repeats the pass on stored
+// votes.  The rows listed for centring are member rows here.
+template <int J, int LX, int NMMA, bool WIDE, int VB>
 __global__ void __launch_bounds__(kProdThreads + 32 * (NMMA + LX + kCentreWarps), 1)
 gram_f16_kernel(const __grid_constant__ CUtensorMap xmap, int m, int box_rows, uint32_t stg_bytes, uint32_t tile_bytes,
                 int lo_row, int mrows, int ncol, int tmem_cols, int nstg, int nmst, int nst_total, int nitems,
                 float* __restrict__ partial, float* __restrict__ norms, const int* __restrict__ centre_ptr,
-                const int* __restrict__ expo, int* __restrict__ status) {
-    constexpr int NBOX = WIDE ? 2 : 1;
+                const int* __restrict__ expo, int* __restrict__ status, const __grid_constant__ VoteMembers members,
+                uint32_t* __restrict__ pairdiff) {
+    constexpr int NBOX = VB > 0 ? VB : (WIDE ? 2 : 1);   // boxes copied in per stage
+    constexpr int NOUT = VB > 0 ? 1 : NBOX;              // blocks of rows a transform thread writes per stage
+    static_assert(VB == 0 || !WIDE, "votes: at most 85 rows come out of at most 255");
     static_assert(!WIDE || (LX == 1 && NMMA == 2), "the wide form has one transform group and one issuing thread per half");
     static_assert(kStagesPerSlab % LX == 0 && (WIDE || kStagesPerSlab % NMMA == 0), "slabs start at every role's own offset");
     static_assert(WIDE || (NMMA % LX == 0 && kMaxMst % NMMA == 0), "an issuing thread serves the same slots and group throughout");
@@ -168,7 +197,7 @@ gram_f16_kernel(const __grid_constant__ CUtensorMap xmap, int m, int box_rows, u
         sm->abort_flag = 0;
         mbar_fence_init();
     }
-    if (tid < ncentre) sm->crow[tid] = centre_ptr[2 + tid];
+    if (tid < ncentre) sm->crow[tid] = centre_ptr[2 + (VB > 0 ? kMaxCentreRows : 0) + tid];
     // rows of the MMA slots that no piece is written to must read as zeros
     for (uint32_t off = (uint32_t)tid * 16u; off < tile_bytes * (uint32_t)nmst; off += kThreads * 16u)
         *reinterpret_cast<uint4*>(mst_base + off) = make_uint4(0u, 0u, 0u, 0u);
@@ -199,21 +228,54 @@ gram_f16_kernel(const __grid_constant__ CUtensorMap xmap, int m, int box_rows, u
         const uint32_t src0 = (uint32_t)row0 * (uint32_t)(kStageCols * 4) + (uint32_t)q * 16u;
         constexpr uint32_t kSrcStep = (uint32_t)R * (uint32_t)(kStageCols * 4);
         constexpr uint32_t kDstStep = (uint32_t)(R / 8) * 1024u;
-        uint32_t dst0[NBOX];
-        float sc[NBOX][J];      // the rows' scales (0: no such row)
-        uint64_t sq[NBOX][J];   // packed pair of partial sums of squares per piece (of the scaled, centred values)
+        uint32_t dst0[NOUT];
+        float sc[NOUT][J];      // the rows' scales (0: no such row)
+        uint64_t sq[NOUT][J];   // packed pair of partial sums of squares per piece (of the scaled, centred values)
+        // votes: where the three members' pieces lie inside the stage's boxes (bit 31: in the second box), and the
+        // "differed" bits of the member pairs (0,1), (0,2), (1,2) of the thread's j-th group at bits 3j .. 3j + 2
+        uint32_t moff[VB > 0 ? J : 1][3];
+        uint32_t differed = 0u;
 #pragma unroll
-        for (int h = 0; h < NBOX; ++h) {
+        for (int h = 0; h < NOUT; ++h) {
             const int g0 = h * box_rows + row0;
             dst0[h] = (uint32_t)(g0 >> 3) * 1024u + (uint32_t)(g0 & 7) * 128u + (uint32_t)(((q >> 1) ^ (g0 & 7)) << 4) +
                       (uint32_t)(q & 1) * 8u;
 #pragma unroll
             for (int j = 0; j < J; ++j) {
                 const int local = row0 + R * j, grow = h * box_rows + local;
-                sc[h][j] = (local < box_rows && grow < m) ? pow2f(expo[grow]) : 0.f;
+                sc[h][j] = ((VB > 0 || local < box_rows) && grow < m) ? pow2f(expo[grow]) : 0.f;
                 sq[h][j] = 0ull;
             }
         }
+        if (VB > 0) {
+#pragma unroll
+            for (int j = 0; j < J; ++j) {
+#pragma unroll
+                for (int k = 0; k < 3; ++k) {
+                    const int g = row0 + R * j;
+                    int xr = g < m ? (int)members.id[g * 3 + k] : 0;
+                    uint32_t second = 0u;
+                    if (VB == 2 && xr >= box_rows) { xr -= box_rows; second = 0x80000000u; }
+                    moff[j][k] = ((uint32_t)xr * (uint32_t)(kStageCols * 4) + (uint32_t)q * 16u) | second;
+                }
+            }
+        }
+
+        // one 16-byte piece (as two packed pairs) -> scaled, centred, added to the row's sum of squares, split into
+        // hi and lo and written to the two operand tiles
+        auto emit = [&](uint64_t a, uint64_t b, const ulonglong2& ck, float scale, uint64_t& sumsq, uint8_t* to) {
+            const uint32_t sb = __float_as_uint(scale);
+            const uint64_t s2 = ((uint64_t)sb << 32) | sb;
+            if (ncentre > 0) { a = sub2(a, ck.x); b = sub2(b, ck.y); }
+            a = mul2(a, s2);
+            b = mul2(b, s2);
+            sumsq = fma2(a, a, fma2(b, b, sumsq));
+            const uint32_t h01 = half2_of(a), h23 = half2_of(b);
+            uint64_t la = sub2(a, float2_of(h01)), lb = sub2(b, float2_of(h23));   // exact
+            if (WIDE) { la = add2(la, la); lb = add2(lb, lb); }   // (not WIDE: the drain doubles the lo part)
+            *reinterpret_cast<uint2*>(to) = make_uint2(h01, h23);
+            *reinterpret_cast<uint2*>(to + lo_off) = make_uint2(half2_of(la), half2_of(lb));
+        };
 
         int ss = group * NBOX, ms = group, cs = group, t = group;
         uint32_t sph = 0, mph = 0, cph = 0;
@@ -226,41 +288,75 @@ gram_f16_kernel(const __grid_constant__ CUtensorMap xmap, int m, int box_rows, u
                     mbar_wait(&sm->c_full[cs], cph, abort_flag, status);
                     ck = *reinterpret_cast<const ulonglong2*>(&sm->cring[cs][q * 4]);
                 }
+                if constexpr (VB > 0) {
+                    // all boxes of the stage must have landed: a group's members may lie in either
+                    const uint8_t* box[2];
+                    int slot[2];
 #pragma unroll
-                for (int h = 0; h < NBOX; ++h) {
-                    mbar_wait(&sm->stg_full[ss], sph, abort_flag, status);
-                    const uint8_t* src = stg_base + (size_t)ss * stg_bytes + src0;
+                    for (int h = 0; h < NBOX; ++h) {
+                        mbar_wait(&sm->stg_full[ss], sph, abort_flag, status);
+                        box[h] = stg_base + (size_t)ss * stg_bytes;
+                        slot[h] = ss;
+                        if (++ss >= nstg) { ss -= nstg; sph ^= 1u; }
+                    }
+                    if (NBOX == 1) { box[1] = box[0]; slot[1] = slot[0]; }
                     ulonglong2 x[J];
 #pragma unroll
-                    for (int j = 0; j < J; ++j)
-                        if (sc[h][j] != 0.f) x[j] = *reinterpret_cast<const ulonglong2*>(src + j * kSrcStep);
-                    // the MMAs that read this slot are done
-                    if (h == 0) mbar_wait(&sm->mst_empty[ms], mph ^ 1u, abort_flag, status);
-                    uint8_t* dst = mst_base + (size_t)ms * tile_bytes + dst0[h];
-#pragma unroll
                     for (int j = 0; j < J; ++j) {
-                        if (sc[h][j] != 0.f) {
-                            const uint32_t sb = __float_as_uint(sc[h][j]);
-                            const uint64_t s2 = ((uint64_t)sb << 32) | sb;
-                            uint64_t a = x[j].x, b = x[j].y;
-                            if (ncentre > 0) { a = sub2(a, ck.x); b = sub2(b, ck.y); }
-                            a = mul2(a, s2);
-                            b = mul2(b, s2);
-                            sq[h][j] = fma2(a, a, fma2(b, b, sq[h][j]));
-                            const uint32_t h01 = half2_of(a), h23 = half2_of(b);
-                            uint64_t la = sub2(a, float2_of(h01)), lb = sub2(b, float2_of(h23));   // exact
-                            if (WIDE) { la = add2(la, la); lb = add2(lb, lb); }   // (not WIDE: the drain doubles the lo part)
-                            *reinterpret_cast<uint2*>(dst + j * kDstStep) = make_uint2(h01, h23);
-                            *reinterpret_cast<uint2*>(dst + lo_off + j * kDstStep) = make_uint2(half2_of(la), half2_of(lb));
+                        if (sc[0][j] != 0.f) {
+                            ulonglong2 v[3];
+#pragma unroll
+                            for (int k = 0; k < 3; ++k)
+                                v[k] = *reinterpret_cast<const ulonglong2*>(((moff[j][k] >> 31) ? box[1] : box[0]) +
+                                                                            (moff[j][k] & 0x7fffffffu));
+                            const bool ne01 = ((v[0].x ^ v[1].x) | (v[0].y ^ v[1].y)) != 0ull;
+                            const bool ne02 = ((v[0].x ^ v[2].x) | (v[0].y ^ v[2].y)) != 0ull;
+                            const bool ne12 = ((v[1].x ^ v[2].x) | (v[1].y ^ v[2].y)) != 0ull;
+                            differed |= ((ne01 ? 1u : 0u) | (ne02 ? 2u : 0u) | (ne12 ? 4u : 0u)) << (3 * j);
+                            // the first member when it agrees with another one, else the second when it agrees with
+                            // the third, else nothing
+                            const bool first = !ne01 || !ne02, other = !ne12;
+                            x[j].x = first ? v[0].x : (other ? v[1].x : 0ull);
+                            x[j].y = first ? v[0].y : (other ? v[1].y : 0ull);
                         }
                     }
-                    if (h == NBOX - 1) fence_proxy_async_smem();   // make the generic-proxy stores visible to the MMA's reads
+                    // the boxes have been read (the values sit in registers)
                     __syncwarp();
                     if (lane == 0) {
-                        mbar_arrive(&sm->stg_empty[ss]);                       // the staging slot has been read
-                        if (h == NBOX - 1) mbar_arrive(&sm->mst_full[ms]);     // one arrival per transform warp of the group
+#pragma unroll
+                        for (int h = 0; h < NBOX; ++h) mbar_arrive(&sm->stg_empty[slot[h]]);
                     }
-                    if (++ss >= nstg) { ss -= nstg; sph ^= 1u; }
+                    mbar_wait(&sm->mst_empty[ms], mph ^ 1u, abort_flag, status);   // the MMAs that read this slot are done
+                    uint8_t* dst = mst_base + (size_t)ms * tile_bytes + dst0[0];
+#pragma unroll
+                    for (int j = 0; j < J; ++j)
+                        if (sc[0][j] != 0.f) emit(x[j].x, x[j].y, ck, sc[0][j], sq[0][j], dst + j * kDstStep);
+                    fence_proxy_async_smem();   // make the generic-proxy stores visible to the MMA's reads
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&sm->mst_full[ms]);   // one arrival per transform warp of the group
+                } else {
+#pragma unroll
+                    for (int h = 0; h < NBOX; ++h) {
+                        mbar_wait(&sm->stg_full[ss], sph, abort_flag, status);
+                        const uint8_t* src = stg_base + (size_t)ss * stg_bytes + src0;
+                        ulonglong2 x[J];
+#pragma unroll
+                        for (int j = 0; j < J; ++j)
+                            if (sc[h][j] != 0.f) x[j] = *reinterpret_cast<const ulonglong2*>(src + j * kSrcStep);
+                        // the MMAs that read this slot are done
+                        if (h == 0) mbar_wait(&sm->mst_empty[ms], mph ^ 1u, abort_flag, status);
+                        uint8_t* dst = mst_base + (size_t)ms * tile_bytes + dst0[h];
+#pragma unroll
+                        for (int j = 0; j < J; ++j)
+                            if (sc[h][j] != 0.f) emit(x[j].x, x[j].y, ck, sc[h][j], sq[h][j], dst + j * kDstStep);
+                        if (h == NBOX - 1) fence_proxy_async_smem();   // make the generic-proxy stores visible to the MMA's reads
+                        __syncwarp();
+                        if (lane == 0) {
+                            mbar_arrive(&sm->stg_empty[ss]);                       // the staging slot has been read
+                            if (h == NBOX - 1) mbar_arrive(&sm->mst_full[ms]);     // one arrival per transform warp of the group
+                        }
+                        if (++ss >= nstg) { ss -= nstg; sph ^= 1u; }
+                    }
                 }
                 if (LX > 1) {
                     ss += (LX - 1) * NBOX;
@@ -278,7 +374,7 @@ gram_f16_kernel(const __grid_constant__ CUtensorMap xmap, int m, int box_rows, u
             // ---- end of a slab: this group's share of the exact squared norms (the 16 lanes that share a row add
             // up; the reduction kernel adds the groups) ...
 #pragma unroll
-            for (int h = 0; h < NBOX; ++h) {
+            for (int h = 0; h < NOUT; ++h) {
 #pragma unroll
                 for (int j = 0; j < J; ++j) {
                     float v = __uint_as_float((uint32_t)sq[h][j]) + __uint_as_float((uint32_t)(sq[h][j] >> 32));
@@ -350,6 +446,20 @@ gram_f16_kernel(const __grid_constant__ CUtensorMap xmap, int m, int box_rows, u
             __syncwarp();
             if (lane == 0) mbar_arrive(&sm->accum_empty);
         }
+        if constexpr (VB > 0) {
+            // the vote's evidence: which member pairs of this thread's groups differed anywhere in this CTA's columns
+            // (the 16 lanes that share a row combine theirs first)
+#pragma unroll
+            for (int j = 0; j < J; ++j) {
+                uint32_t bits = (differed >> (3 * j)) & 7u;
+                bits |= __shfl_xor_sync(0xffffffffu, bits, 1);
+                bits |= __shfl_xor_sync(0xffffffffu, bits, 2);
+                bits |= __shfl_xor_sync(0xffffffffu, bits, 4);
+                bits |= __shfl_xor_sync(0xffffffffu, bits, 8);
+                const int g = row0 + R * j;
+                if (q == 0 && g < m && bits != 0u) atomicOr(pairdiff + (int64_t)g * kPairWords, bits);
+            }
+        }
         // slots of slabs this CTA does not have (it owns one stage fewer than others) read as zero
         for (int l2 = (my_items + kItemSlabs - 1) / kItemSlabs; l2 * (int)gridDim.x < nitems; ++l2) {
             const int64_t item = (int64_t)blockIdx.x + (int64_t)l2 * gridDim.x;
@@ -371,7 +481,7 @@ gram_f16_kernel(const __grid_constant__ CUtensorMap xmap, int m, int box_rows, u
             for (int k = 0; k < kPerHalf; ++k) {
                 const int kk = half * kPerHalf + k;
                 int r = sm->crow[kk < ncentre ? kk : 0];
-                if (WIDE && r >= box_rows) { r -= box_rows; second |= 1u << k; }
+                if (NBOX == 2 && r >= box_rows) { r -= box_rows; second |= 1u << k; }
                 off[k] = (uint32_t)r * (uint32_t)(kStageCols * 4) + (uint32_t)(lane & 15) * 16u;
             }
             const int mine = ncentre - half * kPerHalf;   // listed rows in this half (may be <= 0)
@@ -383,7 +493,7 @@ gram_f16_kernel(const __grid_constant__ CUtensorMap xmap, int m, int box_rows, u
                 const uint8_t* box0 = stg_base + (size_t)s * stg_bytes;
                 const uint8_t* box1 = box0;
                 if (++s == nstg) { s = 0; ph ^= 1u; }
-                if (WIDE) {
+                if (NBOX == 2) {
                     if (!mbar_wait(&sm->stg_full[s], ph, abort_flag, status)) break;
                     box1 = stg_base + (size_t)s * stg_bytes;
                     if (++s == nstg) { s = 0; ph ^= 1u; }
@@ -501,16 +611,17 @@ gram_f16_kernel(const __grid_constant__ CUtensorMap xmap, int m, int box_rows, u
     if (warp == 0) tmem_dealloc(tmem_base, (uint32_t)tmem_cols);
 }
 
-template <int J, int LX, int NMMA, bool WIDE>
+template <int J, int LX, int NMMA, bool WIDE, int VB = 0>
 detox_status launch_f16(const F16Plan& p, const CUtensorMap& xmap, int m, const TcBuffers& b, const int* expo,
-                        cudaStream_t s) {
-    if (cudaFuncSetAttribute(gram_f16_kernel<J, LX, NMMA, WIDE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                        cudaStream_t s, const VoteMembers& members = VoteMembers{}, uint32_t* pairdiff = nullptr) {
+    if (p.smem_bytes > kSmemBudget || p.nstg > kMaxStg || p.nstg < p.nbox * LX) return DETOX_ERR_UNSUPPORTED;
+    if (cudaFuncSetAttribute(gram_f16_kernel<J, LX, NMMA, WIDE, VB>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)p.smem_bytes) != cudaSuccess)
         return DETOX_ERR_CUDA;
     constexpr int kThreads = kProdThreads + 32 * (NMMA + LX + kCentreWarps);
-    gram_f16_kernel<J, LX, NMMA, WIDE><<<p.grid, kThreads, p.smem_bytes, s>>>(
+    gram_f16_kernel<J, LX, NMMA, WIDE, VB><<<p.grid, kThreads, p.smem_bytes, s>>>(
         xmap, m, p.box_rows, p.stg_bytes, p.tile_bytes, p.lo_row, p.mrows, p.ncol, p.tmem_cols, p.nstg, p.nmst, p.nst_total,
-        p.nitems, b.partial, b.norms, b.centre, expo, b.status);
+        p.nitems, b.partial, b.norms, b.centre, expo, b.status, members, pairdiff);
     return launch_status();
 }
 
@@ -541,6 +652,37 @@ detox_status launch_gram_f16(const float* X, int64_t ld, int m, int64_t d, const
     }
     if (per_thread <= 3) return launch_f16<3, 1, 2, false>(p, xmap, m, b, expo, s);
     return launch_f16<4, 1, 2, false>(p, xmap, m, b, expo, s);
+}
+
+// The vote inside the pass: every three consecutive entries of `members` (rows of X) give one vote; 16 < G <= 85.
+bool f16_vote_supported(int n, int r) { return r == 3 && n % 3 == 0 && n / 3 > 16 && n <= 255; }
+
+detox_status launch_gram_f16_vote(const float* X, int64_t ld, int n, int64_t d, const IdTable& groups,
+                                  uint32_t* pairdiff, const TcBuffers& b, const int* expo, cudaStream_t s) {
+    if (!f16_vote_supported(n, 3)) return DETOX_ERR_UNSUPPORTED;
+    const int m = n / 3;
+    VoteMembers members;
+    for (int i = 0; i < 256; ++i) members.id[i] = i < n ? (uint8_t)groups.id[i] : 0;
+    const F16Plan p = f16_plan(m, d, n);
+    CUtensorMap xmap;
+    detox_status st = make_xmap(&xmap, X, ld, n, d, kStageCols, p.box_rows, false);
+    if (st != DETOX_OK) return st;
+    // vote rows per transform thread: one piece of every (threads of a group / 16)-th row
+    const int per_thread = (m * (kStageCols / 4) + kProdThreads / p.groups - 1) / (kProdThreads / p.groups);
+    if (p.groups == 4) {
+        if (per_thread <= 3) return launch_f16<3, 4, 4, false, 1>(p, xmap, m, b, expo, s, members, pairdiff);
+        return launch_f16<4, 4, 4, false, 1>(p, xmap, m, b, expo, s, members, pairdiff);
+    }
+    if (p.groups == 2) {
+        if (p.nbox == 1) {
+            if (per_thread <= 3) return launch_f16<3, 2, 4, false, 1>(p, xmap, m, b, expo, s, members, pairdiff);
+            return launch_f16<4, 2, 4, false, 1>(p, xmap, m, b, expo, s, members, pairdiff);
+        }
+        if (per_thread <= 3) return launch_f16<3, 2, 4, false, 2>(p, xmap, m, b, expo, s, members, pairdiff);
+        return launch_f16<4, 2, 4, false, 2>(p, xmap, m, b, expo, s, members, pairdiff);
+    }
+    if (p.nbox != 2 || per_thread > 3) return DETOX_ERR_UNSUPPORTED;   // 65 .. 85 votes come from 195 .. 255 rows
+    return launch_f16<3, 1, 2, false, 2>(p, xmap, m, b, expo, s, members, pairdiff);
 }
 
 }  // namespace detox

@@ -1061,4 +1061,38 @@ detox_status launch_sqdist_tc(const float* X, int64_t ld, int m, int64_t d, doub
     return launch_status();
 }
 
+bool sqdist_vote_tc_supported(const float* X, int64_t ld, int n, int r, int64_t d) {
+    return f16_vote_supported(n, r) && tc_supported(X, ld, n / 3, d) && g_split_mode.load() == DETOX_SPLIT_AUTO;
+}
+
+// Sequence: sample (votes formed on the fly) and pick -> the split-fp16 pass that votes while it reads -> check ->
+// winners from the vote's bits (a group without a majority also raises the redo flag) -> only if the flag is up: the
+// votes are stored and the split-TF32 pass runs on them -> reduction to distances.
+detox_status launch_sqdist_vote_tc(const float* X, int64_t ld, int n, int64_t d, const IdTable& members, int32_t* winner,
+                                   void* vote_ws, float* Z, int64_t ldz, double* D, void* ws, int* status, cudaStream_t s) {
+    const int m = n / 3;
+    const TcShape o = tc_shape(m, d);
+    const TcWs w = tc_carve(ws, m, d, o);
+    VoteMembers vm;
+    for (int i = 0; i < 256; ++i) vm.id[i] = i < n ? (uint8_t)members.id[i] : 0;
+    detox_status st;
+    if ((st = launch_pick_centre(X, ld, m, d, w.pick, w.centre, w.expo, s, &vm)) != DETOX_OK) return st;
+    TcBuffers b{w.partial, w.norms, w.centre, nullptr, status};
+    if ((st = launch_gram_f16_vote(X, ld, n, d, members, static_cast<uint32_t*>(vote_ws), b, w.expo, s)) != DETOX_OK) return st;
+    st = launch_check_centre(w.norms, w.partial, o.nitems_f16, o.groups_f16, m, o.ncol, w.pick, d, w.centre, w.centre + 1,
+                             w.expo, s);
+    if (st != DETOX_OK) return st;
+    if ((st = launch_vote_finalize(n, 3, members, vote_ws, winner, w.centre + 1, s)) != DETOX_OK) return st;
+    if ((st = launch_vote_store_gated(X, ld, n, d, members, Z, ldz, winner, w.centre + 1, s)) != DETOX_OK) return st;
+    b.redo = w.centre + 1;
+    if ((st = launch_tc_gram(Z, ldz, m, d, o, b, s)) != DETOX_OK) return st;
+    const int nt = (m + kRT - 1) / kRT;
+    const int nchunks = reduce_chunks(m, o.max_items());
+    tc_reduce_kernel<<<dim3((unsigned)(nt * (nt + 1) / 2), (unsigned)nchunks), kRT * 8, 0, s>>>(
+        w.partial, w.norms, o.groups_f16, o.nitems_f16, o.groups, o.nitems, w.expo, w.centre + 1, m, o.ncol, w.dpart);
+    if ((st = launch_status()) != DETOX_OK) return st;
+    tc_dist_kernel<<<(unsigned)ceil_div((int64_t)m * m * 32, 256), 256, 0, s>>>(w.dpart, nchunks, m, status, D);
+    return launch_status();
+}
+
 }  // namespace detox

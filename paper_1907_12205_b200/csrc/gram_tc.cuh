@@ -29,6 +29,11 @@ int f16_nitems(int m, int64_t d);
 int f16_groups(int m);
 detox_status launch_gram_f16(const float* X, int64_t ld, int m, int64_t d, const TcBuffers& b, const int* expo,
                              cudaStream_t s);
+// The same pass over the votes of n / 3 groups of three rows of X, formed inside the pass (Section 3: the filtering
+// step); ORs the "members differed" bits of every group into pairdiff (vote kernels' format), which the caller has cleared.
+bool f16_vote_supported(int n, int r);
+detox_status launch_gram_f16_vote(const float* X, int64_t ld, int n, int64_t d, const IdTable& groups,
+                                  uint32_t* pairdiff, const TcBuffers& b, const int* expo, cudaStream_t s);
 
 // The driver's tensor-map encoder for X as a 2-D fp32 tensor (d columns innermost, m rows, row pitch ld), zero fill
 // outside; swizzle128 = false: rows of a box land one after another.

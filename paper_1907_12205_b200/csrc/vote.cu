@@ -15,7 +15,6 @@ namespace detox {
 namespace {
 
 constexpr int kVoteThreads = 256;
-constexpr int kPairWords = 4;  // r <= 15 -> at most 105 member pairs -> 4 words per group
 
 template <int R>
 struct VoteShape {
@@ -157,8 +156,10 @@ vote_kernel(const float* __restrict__ X, int64_t ld, int64_t d, int64_t tiles_pe
 }
 
 // One thread per group: read the "differs" bits, find the class with more than r/2 members.
+// none_flag (optional): set to 1 when some group has no majority.
 __global__ void vote_finalize_kernel(int G, int r, const __grid_constant__ IdTable members,
-                                     const uint32_t* __restrict__ pairdiff, int32_t* __restrict__ winner) {
+                                     const uint32_t* __restrict__ pairdiff, int32_t* __restrict__ winner,
+                                     int* __restrict__ none_flag = nullptr) {
     int g = blockIdx.x * blockDim.x + threadIdx.x;
     if (g >= G) return;
     const uint32_t* bits = pairdiff + (int64_t)g * kPairWords;
@@ -178,6 +179,33 @@ __global__ void vote_finalize_kernel(int G, int r, const __grid_constant__ IdTab
         if (2 * agree > r) win = lowest;
     }
     winner[g] = win;
+    if (none_flag != nullptr && win < 0) *none_flag = 1;
+}
+
+// The votes of groups of three as rows of Z, written only when *gate is not zero (the distance pass that votes while
+// it reads keeps no votes; when its result cannot be used the pass is repeated on stored ones).  Groups without a
+// majority get their piece-local values here and are cleared by vote_clear_kernel afterwards.
+__global__ void __launch_bounds__(kVoteThreads)
+vote_store_gated_kernel(const float* __restrict__ X, int64_t ld, int64_t d, const __grid_constant__ IdTable members,
+                        float* __restrict__ Z, int64_t ldz, const int* __restrict__ gate) {
+    if (*gate == 0) return;
+    const int g = blockIdx.y;
+    const float* row[3];
+#pragma unroll
+    for (int a = 0; a < 3; ++a) row[a] = X + (int64_t)members.id[g * 3 + a] * ld;
+    for (int64_t col = ((int64_t)blockIdx.x * kVoteThreads + threadIdx.x) * 4; col < d;
+         col += (int64_t)gridDim.x * kVoteThreads * 4) {
+        const int64_t left = d - col;
+        const int valid = left >= 4 ? 4 : (int)left;
+        Piece<4> v[3];
+#pragma unroll
+        for (int a = 0; a < 3; ++a) v[a].load(row[a] + col, valid);
+        Piece<4> pick;
+        pick.clear();
+        if (!v[1].differs(v[2])) pick = v[1];
+        if (!v[0].differs(v[1]) || !v[0].differs(v[2])) pick = v[0];
+        pick.store(Z + (int64_t)g * ldz + col, valid);
+    }
 }
 
 // Clears the vote of every group that turned out to have no majority (rare).
@@ -560,6 +588,28 @@ detox_status launch_vote(const float* X, int64_t ld, int n, int r, int64_t d, co
         st = launch_status();
     }
     return st;
+}
+
+detox_status launch_vote_finalize(int n, int r, const IdTable& members, const void* ws, int32_t* winner, int* none_flag,
+                                  cudaStream_t s) {
+    const int G = n / r;
+    vote_finalize_kernel<<<(G + 127) / 128, 128, 0, s>>>(G, r, members, static_cast<const uint32_t*>(ws), winner, none_flag);
+    return launch_status();
+}
+
+detox_status launch_vote_store_gated(const float* X, int64_t ld, int n, int64_t d, const IdTable& members, float* Z,
+                                     int64_t ldz, const int32_t* winner, const int* gate, cudaStream_t s) {
+    if (!(aligned16(X) && ld % 4 == 0 && aligned16(Z) && ldz % 4 == 0)) return DETOX_ERR_UNSUPPORTED;
+    const int G = n / 3;
+    const int64_t want = ceil_div(d, (int64_t)kVoteThreads * 4 * 4);
+    const unsigned bx = (unsigned)(want < 1 ? 1 : (want > 4096 ? 4096 : want));
+    vote_store_gated_kernel<<<dim3(bx, (unsigned)G), kVoteThreads, 0, s>>>(X, ld, d, members, Z, ldz, gate);
+    detox_status st = launch_status();
+    if (st != DETOX_OK) return st;
+    // (winner[g] < 0 only ever goes with *gate != 0, so the clearing needs no gate of its own)
+    unsigned cx = (unsigned)(ceil_div(d, 256 * 8) < 64 ? ceil_div(d, 256 * 8) : 64);
+    vote_clear_kernel<<<dim3(cx, (unsigned)G), 256, 0, s>>>(winner, Z, ldz, d);
+    return launch_status();
 }
 
 detox_status launch_vote_mean(const float* X, int64_t ld, int n, int r, int64_t d, const IdTable& members,
