@@ -414,8 +414,10 @@ def run_sweep(args):
                 win = torch.empty(G, dtype=torch.int32, device=dev)
                 psel = torch.empty(max(p.n_selected, 1), dtype=torch.int32, device=dev)
                 second = {"coord_median": 0, "multikrum": leg["m_sel"], "bulyan": rows1 - 2 * leg["f"]}[leg["a1"]]
+                # compulsory traffic: every worker's row once, the rows the second sweep averages or sorts, the result
+                # (votes and set means need not travel: the vote runs inside the pass that consumes it)
                 timed(name, lambda: dx.detox_aggregate(p, X, out=out, winner=win, sel=psel, ws=pws),
-                      (n + 2 * rows1 + second + 1) * d * 4)
+                      (n + second + 1) * d * 4)
                 del pws
             elif leg["a1"] == "coord_median":
                 ms = timed(name, lambda: dx.agg_coord_median(X, out=out), (n + 1) * d * 4)

@@ -239,7 +239,11 @@ detox_status agg_bulyan(const float* X, int64_t ld, int m, int64_t d, int f, flo
  * The whole parameter-server step (Algorithm 1, filtering + hierarchical aggregation; Algorithm 2):
  * vote over the node groups, A_0 over each vote group, A_1 over the results.
  *
- *   a0 = DETOX_AGG_NONE : the G votes go to A_1 directly (sets are ignored)
+ *   a0 = DETOX_AGG_NONE : the G votes go to A_1 directly (sets are ignored).  The votes are rows of X, so they are
+ *        read through winner[] and not stored; with a1 = MULTIKRUM or BULYAN over 17 to 85 votes of groups of r = 3
+ *        (16-byte aligned rows) the vote itself runs inside the distance pass, one pass over X for both (the votes are
+ *        stored, and the pass repeated on them, only when a group has no majority or an entry leaves the range of the
+ *        pass's fp16 operands; the results are the same either way)
  *   a0 = DETOX_AGG_MEAN : the S set means go to A_1 (with a1 = MEAN, COORD_MEDIAN or TRIMMED_MEAN over at most 16 sets,
  *        r in {1, 3, 5} and 16-byte aligned rows of X and out, the whole step is one pass over X and the set means
  *        are never stored; the result is bitwise the same either way)

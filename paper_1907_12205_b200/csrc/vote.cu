@@ -601,8 +601,10 @@ detox_status launch_vote_store_gated(const float* X, int64_t ld, int n, int64_t 
                                      int64_t ldz, const int32_t* winner, const int* gate, cudaStream_t s) {
     if (!(aligned16(X) && ld % 4 == 0 && aligned16(Z) && ldz % 4 == 0)) return DETOX_ERR_UNSUPPORTED;
     const int G = n / 3;
-    const int64_t want = ceil_div(d, (int64_t)kVoteThreads * 4 * 4);
-    const unsigned bx = (unsigned)(want < 1 ? 1 : (want > 4096 ? 4096 : want));
+    // a few waves of CTAs that stride over the columns: the launch that finds its gate closed should cost next to nothing
+    const int64_t want = ceil_div(d, (int64_t)kVoteThreads * 4);
+    const int64_t fill = ceil_div((int64_t)kSMs * 16, G);
+    const unsigned bx = (unsigned)(want < fill ? want : fill);
     vote_store_gated_kernel<<<dim3(bx, (unsigned)G), kVoteThreads, 0, s>>>(X, ld, d, members, Z, ldz, gate);
     detox_status st = launch_status();
     if (st != DETOX_OK) return st;
