@@ -304,7 +304,7 @@ def median_alu_roofline(m, d, ms, peaks):
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the tensor-core distance kernel over the algorithmic
 # bytes m d 4, from ncu captures at d = 2.5 M (the kernel reads every row once, so its traffic grows with m d); reset an
 # entry to None when the kernel changes.
-NCU_GRAM_TRAFFIC_RATIO = {45: 1.025, 105: 1.043, 225: 1.096}
+NCU_GRAM_TRAFFIC_RATIO = {45: 1.034, 105: 1.043, 225: 1.095}
 
 
 def gram_roofline(m, d, ms, peaks, peak_kind, ms_tf32=None):
