@@ -674,6 +674,24 @@ def main():
         legs[name] = {"ms": ms2, "GBps": in_bytes / ms2 / 1e6, "f": f, "sets": offsets}
         del ws2
 
+    G_votes = spec.n // spec.r
+    if spec.r == 3 and 16 < G_votes <= 85:
+        # A Krum-type A_1 over all votes: the vote runs inside the tensor-core distance pass (one pass over X for both),
+        # then the kept winners' rows are averaged (Multi-Krum) or go through Bulyan's second stage.  Reported against
+        # the step's compulsory traffic: every row once, the rows of the second sweep, the result.
+        fv = min(2, (G_votes - 3) // 4)
+        for name, a1, second in (("vote_in_distance_pass_multikrum", dx.AGG_MULTIKRUM, G_votes - fv),
+                                 ("vote_in_distance_pass_bulyan", dx.AGG_BULYAN, G_votes - 2 * fv)):
+            p3 = dx.Pipeline(spec.n, spec.r, spec.d, w.members, dx.AGG_NONE, None, None, a1, fv, G_votes - fv)
+            ws3 = torch.empty(p3.workspace_bytes(), dtype=torch.uint8, device=dev)
+            sel3 = torch.empty(max(p3.n_selected, 1), dtype=torch.int32, device=dev)
+            ms3 = time_calls(torch, lambda: dx.detox_aggregate(p3, X, out=out, winner=winner, sel=sel3, ws=ws3), reps, 3)
+            comp = (spec.n + second + 1) * spec.d * 4
+            legs[name] = {"ms": ms3, "GBps": in_bytes / ms3 / 1e6, "f": fv, "votes": G_votes,
+                          "compulsory_bytes": comp, "compulsory_GBps": comp / ms3 / 1e6,
+                          "compulsory_frac_of_hbm": comp / ms3 / 1e6 / peaks["hbm_gbs"], "status_word": dx.read_status(ws3)}
+            del ws3
+
     vote_bytes = (spec.n + dom_rows_out) * spec.d * 4
     achieved = vote_bytes / (vote_ms * 1e-3) / 1e9
     roofline = {"kernel": dom_name, "bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"],
